@@ -1,0 +1,169 @@
+/*
+ * difr.h -- C ABI of the B200 token-scoring library (libdifr.so).
+ *
+ * The library re-scores, on one sm_100a GPU, every claimed output token of a
+ * logged LLM response the way the verification server of "Verifying LLM
+ * Inference to Detect Model Weight Exfiltration" does: the final hidden state
+ * of each position goes through the LM head, and the logits are turned into
+ * the Fixed-Seed Sampling Likelihood estimators of Sec. "Classification using
+ * the Fixed-Seed Sampling Likelihood Policy" with the sampling seed shared with
+ * the inference server.  Logits are never written to memory.
+ *
+ * Conventions
+ *   - Plain C linkage, no exceptions, no global state visible to the caller.
+ *   - Every pointer is a DEVICE pointer owned by the caller unless it says
+ *     "host"; the caller keeps all buffers alive until `stream` has passed the
+ *     call.  The library allocates no device memory and never synchronises
+ *     the stream; all work is enqueued on `stream`.
+ *   - The return value reports what the host can detect (bad arguments,
+ *     alignment, workspace size, wrong architecture, launch failure).  What
+ *     only the device can detect is reported in `row_status` and
+ *     `device_status`.
+ *   - Randomness RO(seed || i) (Sec. "Sampling From Large Language Models") is
+ *     Philox-4x32-10 with key = (seed low word, seed high word) and counter =
+ *     (id >> 2, i, stream, 0); vocabulary id `id` takes output word id & 3.
+ *     stream 0 is the Gumbel noise, stream 1 the single uniform of the
+ *     inverse-probability-transform sampler (id 0).  A 32-bit word x becomes
+ *     u = ((x >> 9) + 1/2) 2^-23 and G = -ln(-ln u) for Gumbel noise, and
+ *     mu = (x + 1/2) 2^-32 for the IPT uniform.
+ */
+#ifndef DIFR_H_
+#define DIFR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* difr_stream_t; /* a cudaStream_t */
+
+typedef enum {
+  DIFR_OK = 0,
+  DIFR_ERR_INVALID_ARG = -1, /* null required pointer, non-positive size, bad scalar  */
+  DIFR_ERR_SHAPE = -2,       /* d not a multiple of 8, V < 2, sizes beyond 2^31 rows  */
+  DIFR_ERR_ALIGN = -3,       /* h, W or workspace not 16-byte aligned                 */
+  DIFR_ERR_WORKSPACE = -4,   /* workspace missing or smaller than difr_workspace_bytes */
+  DIFR_ERR_CUDA = -5,        /* a CUDA runtime/driver call failed                     */
+  DIFR_ERR_ARCH = -6,        /* current device is not compute capability 10.x         */
+  DIFR_ERR_TIMEOUT = -7      /* device_status only: a bounded device-side wait ran out */
+} difr_status;
+
+/* Per-sequence pooled statistics written by difr_detect. */
+typedef struct {
+  int32_t n_flagged; /* rows with score < threshold (or NaN)                      */
+  int32_t n_match;   /* rows whose claimed token is the verifier's own sample      */
+  float sum;         /* sum of the scores (summed log-likelihood)                  */
+  float min;         /* smallest non-NaN score; +inf for an empty sequence         */
+} difr_seq_stats;
+
+/*
+ * Estimator parameters and outputs of one scoring call.  Arrays are device
+ * pointers of T elements; optional ones may be NULL.
+ */
+typedef struct {
+  float sigma; /* width of the Gaussian noise model: raw-logit units for
+                  difr_score_gm, probability (CDF) units for difr_score_ipt; > 0 */
+  float eps;   /* floor inside the logarithm; >= 0 (1e-12 is customary)          */
+  float* score;       /* required. ln(pi + eps) (Token-DiFR) / ln(mass + eps) (IPT)  */
+  float* margin;      /* GM: A = y[t*] - max_{v != t*} y[v], y = l + Temp*G.  A >= +0
+                         means exact match; -0.0 encodes a tie lost to a lower id;
+                         -inf for an out-of-range claim.  Unused by IPT.           */
+  int32_t* argmax;    /* GM: the verifier's own Gumbel-max token (ties: lowest id) */
+  int32_t* runner_up; /* GM: id of the second largest y                            */
+  float* lse;         /* ln sum_v exp(l_v / Temp); NaN when Temp == 0              */
+  float* p_claimed;   /* IPT: softmax probability of the claimed token            */
+  float* cdf_lo;      /* IPT: a = sum_{v < t*} p_v                                 */
+  float* u;           /* IPT: the uniform mu of this row                           */
+  uint32_t* row_status; /* bit0: claimed id outside [0, V); bit1: non-finite logits */
+  void* workspace;      /* >= difr_workspace_bytes(T, d, V) bytes, 16-byte aligned;
+                           contents are scratch, overwritten by every call         */
+  size_t workspace_bytes;
+  int32_t* device_status; /* [1] optional. Sticky: a kernel writes DIFR_ERR_TIMEOUT
+                             here if a bounded wait ran out; never cleared         */
+} difr_out;
+
+/* Scratch bytes a scoring call needs for T rows, hidden size d, vocabulary V.
+ * Returns 0 for sizes the library rejects. */
+size_t difr_workspace_bytes(int64_t T, int64_t d, int64_t V);
+
+/*
+ * Token-DiFR, the Gumbel-max estimator (Alg. "Token-DiFR", with the paper's
+ * default Gaussian noise, one active competitor and no top-k/top-p filter;
+ * Sec. "Gumbel-Max Scoring Function").
+ *
+ * For every row r: logits l = h[r,:] . W^T (bf16 inputs, fp32 accumulation on
+ * the tensor cores), Gumbel noise G regenerated from (seeds[r], positions[r]),
+ * y = l + temperature * G; the claimed token's margin A over its strongest
+ * competitor is re-evaluated in fp64 and scored as
+ * ln(Phi(A / (sigma sqrt 2)) + eps).  The same pass yields the exact-match
+ * replay of Sec. "Sampled-Token Verification via Exact Matching" (argmax,
+ * margin >= 0) and the log-sum-exp of l / temperature.
+ *
+ *   h          bf16 [T, d] row-major; h[r,:] is the hidden state that predicts token r
+ *   W          bf16 [V, d] row-major LM-head matrix
+ *   tokens     int32 [T] claimed ids (any value; out of range => maximally suspicious)
+ *   seeds      uint64 [T], positions uint32 [T]: RO(seed || i) per row
+ *   temperature  >= 0 (0: greedy replay, y = l)
+ *   T >= 0, d > 0 with d % 8 == 0, 2 <= V < 2^31
+ * Errors: see difr_status.  T == 0 returns DIFR_OK without launching.
+ */
+difr_status difr_score_gm(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,
+                          const uint32_t* positions, float temperature, int64_t T, int64_t d, int64_t V,
+                          difr_out* out, difr_stream_t stream);
+
+/*
+ * Token-IPT-DiFR, the inverse-probability-transform estimator (Alg.
+ * "Token-IPT-DiFR"; Sec. "Inverse Probability Transform Scoring Function").
+ *
+ * Same arguments.  Per row: p = softmax(l / temperature), [a, b] the claimed
+ * token's interval of the cumulative distribution in vocabulary-id order, mu the
+ * row's uniform, score = ln(Phi((b - mu)/sigma) - Phi((a - mu)/sigma) + eps).
+ * Requires temperature > 0.  Writes score, lse, p_claimed, cdf_lo, u,
+ * row_status; margin/argmax/runner_up are left untouched.
+ */
+difr_status difr_score_ipt(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,
+                           const uint32_t* positions, float temperature, int64_t T, int64_t d, int64_t V,
+                           difr_out* out, difr_stream_t stream);
+
+/*
+ * Threshold detection and pooling (Sec. "Classification via Thresholding":
+ * flag t iff FSSL(t) < tau; per-sequence match count as in Alg. "Sampled token
+ * verification via prefill").
+ *
+ *   scores      float [T]
+ *   threshold   tau; a score equal to tau is safe, NaN is flagged
+ *   margins     float [T], nullable: rows without a sign bit count as matches
+ *   ranks, rank_cutoff   nullable / ignored when NULL: with raw-logit ranks a flagged row
+ *               whose rank exceeds the cutoff gets flag 2 (Alg. "Per-Token Risk
+ *               Classification")
+ *   seq_offsets int32 [n_seq + 1] ascending row offsets, nullable => one sequence [0, T)
+ *   flags       uint8 [T], nullable: 0 safe, 1 flagged (suspicious), 2 dangerous
+ *   seq_stats   difr_seq_stats [n_seq] (or [1]), nullable
+ */
+difr_status difr_detect(const float* scores, float threshold, const float* margins, const int32_t* ranks,
+                        int32_t rank_cutoff, const int32_t* seq_offsets, int64_t n_seq, int64_t T,
+                        uint8_t* flags, difr_seq_stats* seq_stats, difr_stream_t stream);
+
+/*
+ * Validation aid, not part of the scoring path: writes the fp32 logits
+ * l[r, v] = h[r,:] . W[v,:] computed by the same tensor-core main loop to
+ * `logits` (float [T, V] row-major).  Meant for small shapes.
+ */
+difr_status difr_logits(const void* h, const void* W, int64_t T, int64_t d, int64_t V, float* logits,
+                        int32_t* device_status, difr_stream_t stream);
+
+/*
+ * Validation aid: the library's own Philox-4x32-10 block for n counters.
+ * ctr uint32 [n, 4], key uint32 [n, 2] -> out uint32 [n, 4] (device pointers).
+ */
+difr_status difr_philox(const uint32_t* ctr, const uint32_t* key, int64_t n, uint32_t* out, difr_stream_t stream);
+
+const char* difr_status_string(difr_status status); /* host pointer to a static string */
+int difr_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DIFR_H_ */

@@ -1,0 +1,197 @@
+"""Thin binding of libdifr.so, the B200 token-scoring library.
+
+The functions carry the names of the C entry points in include/difr.h and only
+marshal arguments: torch supplies device memory and streams, every step of the
+scoring path runs in the library's CUDA kernels.  There is no CPU fallback: a
+missing or unloadable library raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "csrc", "libdifr.so")
+
+DIFR_OK = 0
+STATUS_NAMES = {0: "DIFR_OK", -1: "DIFR_ERR_INVALID_ARG", -2: "DIFR_ERR_SHAPE", -3: "DIFR_ERR_ALIGN",
+                -4: "DIFR_ERR_WORKSPACE", -5: "DIFR_ERR_CUDA", -6: "DIFR_ERR_ARCH", -7: "DIFR_ERR_TIMEOUT"}
+
+EXPORTS = ("difr_workspace_bytes", "difr_score_gm", "difr_score_ipt", "difr_detect", "difr_logits", "difr_philox",
+           "difr_status_string", "difr_version")
+
+
+class DifrError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}")
+
+
+class _COut(ctypes.Structure):
+    _fields_ = [
+        ("sigma", ctypes.c_float), ("eps", ctypes.c_float),
+        ("score", ctypes.c_void_p), ("margin", ctypes.c_void_p), ("argmax", ctypes.c_void_p),
+        ("runner_up", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("p_claimed", ctypes.c_void_p),
+        ("cdf_lo", ctypes.c_void_p), ("u", ctypes.c_void_p), ("row_status", ctypes.c_void_p),
+        ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t), ("device_status", ctypes.c_void_p),
+    ]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads csrc/libdifr.so (built by paper_2511_02620_b200.build.build())."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2511_02620_b200.build` "
+                              "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        L.difr_workspace_bytes.restype = ctypes.c_size_t
+        L.difr_workspace_bytes.argtypes = [ctypes.c_int64] * 3
+        score_args = [ctypes.c_void_p] * 5 + [ctypes.c_float] + [ctypes.c_int64] * 3 + [ctypes.POINTER(_COut),
+                                                                                      ctypes.c_void_p]
+        for name in ("difr_score_gm", "difr_score_ipt"):
+            getattr(L, name).restype = ctypes.c_int
+            getattr(L, name).argtypes = score_args
+        L.difr_detect.restype = ctypes.c_int
+        L.difr_detect.argtypes = [ctypes.c_void_p, ctypes.c_float, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32,
+                                  ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p,
+                                  ctypes.c_void_p]
+        L.difr_logits.restype = ctypes.c_int
+        L.difr_logits.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
+                                  ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        L.difr_philox.restype = ctypes.c_int
+        L.difr_philox.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]
+        L.difr_status_string.restype = ctypes.c_char_p
+        L.difr_status_string.argtypes = [ctypes.c_int]
+        L.difr_version.restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    import torch
+
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(t, dtype, shape, name):
+    import torch
+
+    if not isinstance(t, torch.Tensor) or not t.is_cuda or not t.is_contiguous():
+        raise TypeError(f"{name} must be a contiguous CUDA tensor")
+    if t.dtype != dtype or tuple(t.shape) != tuple(shape):
+        raise TypeError(f"{name}: expected {dtype} {tuple(shape)}, got {t.dtype} {tuple(t.shape)}")
+
+
+def difr_workspace_bytes(T: int, d: int, V: int) -> int:
+    return int(lib().difr_workspace_bytes(T, d, V))
+
+
+def difr_version() -> int:
+    return int(lib().difr_version())
+
+
+def difr_status_string(status: int) -> str:
+    return lib().difr_status_string(status).decode()
+
+
+@dataclass
+class DifrOut:
+    """Estimator parameters and output tensors of a scoring call (mirrors `difr_out`)."""
+    sigma: float
+    eps: float
+    score: "object"
+    margin: "object" = None
+    argmax: "object" = None
+    runner_up: "object" = None
+    lse: "object" = None
+    p_claimed: "object" = None
+    cdf_lo: "object" = None
+    u: "object" = None
+    row_status: "object" = None
+    workspace: "object" = None
+    device_status: "object" = None
+
+    @staticmethod
+    def allocate(T: int, d: int, V: int, sigma: float, eps: float = 1e-12, device="cuda"):
+        import torch
+
+        f = lambda: torch.empty(T, dtype=torch.float32, device=device)
+        i = lambda: torch.empty(T, dtype=torch.int32, device=device)
+        nbytes = max(difr_workspace_bytes(T, d, V), 16)
+        return DifrOut(sigma, eps, f(), f(), i(), i(), f(), f(), f(), f(), i(),
+                       torch.empty(nbytes, dtype=torch.uint8, device=device),
+                       torch.zeros(1, dtype=torch.int32, device=device))
+
+    def _c(self) -> _COut:
+        ws = self.workspace
+        return _COut(float(self.sigma), float(self.eps), _ptr(self.score), _ptr(self.margin), _ptr(self.argmax),
+                     _ptr(self.runner_up), _ptr(self.lse), _ptr(self.p_claimed), _ptr(self.cdf_lo), _ptr(self.u),
+                     _ptr(self.row_status), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
+                     _ptr(self.device_status))
+
+
+def _score(fn_name, h, W, tokens, seeds, positions, temperature, out: DifrOut, stream):
+    import torch
+
+    T, d = h.shape
+    V = W.shape[0]
+    _check(h, torch.bfloat16, (T, d), "h")
+    _check(W, torch.bfloat16, (V, d), "W")
+    _check(tokens, torch.int32, (T,), "tokens")
+    _check(seeds, torch.int64, (T,), "seeds")  # uint64 bit patterns carried in int64 storage
+    _check(positions, torch.int32, (T,), "positions")  # uint32 bit patterns
+    c = out._c()
+    rc = getattr(lib(), fn_name)(_ptr(h), _ptr(W), _ptr(tokens), _ptr(seeds), _ptr(positions), float(temperature),
+                                 T, d, V, ctypes.byref(c), _stream(stream))
+    if rc != DIFR_OK:
+        raise DifrError(rc, fn_name)
+    return out
+
+
+def difr_score_gm(h, W, tokens, seeds, positions, temperature, out: DifrOut, stream=None) -> DifrOut:
+    """Token-DiFR (Gumbel-max) scores; see include/difr.h."""
+    return _score("difr_score_gm", h, W, tokens, seeds, positions, temperature, out, stream)
+
+
+def difr_score_ipt(h, W, tokens, seeds, positions, temperature, out: DifrOut, stream=None) -> DifrOut:
+    """Token-IPT-DiFR scores; see include/difr.h."""
+    return _score("difr_score_ipt", h, W, tokens, seeds, positions, temperature, out, stream)
+
+
+def difr_detect(scores, threshold, margins=None, ranks=None, rank_cutoff=0, seq_offsets=None, flags=None,
+                seq_stats=None, stream=None):
+    """Threshold flags and per-sequence statistics; `seq_stats` is an int32 [n_seq, 4] tensor whose rows are
+    (n_flagged, n_match, bits of float sum, bits of float min)."""
+    T = scores.shape[0]
+    n_seq = 1 if seq_offsets is None else seq_offsets.shape[0] - 1
+    rc = lib().difr_detect(_ptr(scores), float(threshold), _ptr(margins), _ptr(ranks), int(rank_cutoff),
+                           _ptr(seq_offsets), n_seq, T, _ptr(flags), _ptr(seq_stats), _stream(stream))
+    if rc != DIFR_OK:
+        raise DifrError(rc, "difr_detect")
+    return flags, seq_stats
+
+
+def difr_logits(h, W, logits, device_status=None, stream=None):
+    T, d = h.shape
+    V = W.shape[0]
+    rc = lib().difr_logits(_ptr(h), _ptr(W), T, d, V, _ptr(logits), _ptr(device_status), _stream(stream))
+    if rc != DIFR_OK:
+        raise DifrError(rc, "difr_logits")
+    return logits
+
+
+def difr_philox(ctr, key, out, stream=None):
+    rc = lib().difr_philox(_ptr(ctr), _ptr(key), ctr.shape[0], _ptr(out), _stream(stream))
+    if rc != DIFR_OK:
+        raise DifrError(rc, "difr_philox")
+    return out

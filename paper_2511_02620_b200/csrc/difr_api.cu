@@ -1,0 +1,199 @@
+// C ABI of libdifr.so: argument validation, work planning, tensor-map encoding
+// and kernel launches.  Nothing here computes; every step of the scoring path
+// runs in the three kernels.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#include "../../include/difr.h"
+#include "difr_kernels.h"
+#include "difr_plan.h"
+
+namespace {
+
+using namespace difr;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(sym);
+  }
+  return fn;
+}
+
+// bf16 [rows, cols] row-major, box = 64 columns (128 bytes, 128-byte swizzle) x box_rows rows.
+bool make_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (fn == nullptr) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct DeviceInfo {
+  int major;
+  int sms;
+};
+
+bool device_info(DeviceInfo* info) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  if (cudaDeviceGetAttribute(&info->major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return false;
+  if (cudaDeviceGetAttribute(&info->sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+  return true;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+difr_status score_common(int ipt, const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,
+                         const uint32_t* positions, float temperature, int64_t T, int64_t d, int64_t V,
+                         difr_out* out, difr_stream_t stream) {
+  if (!h || !W || !tokens || !seeds || !positions || !out || !out->score) return DIFR_ERR_INVALID_ARG;
+  if (T < 0 || d <= 0 || V <= 0) return DIFR_ERR_INVALID_ARG;
+  if (!(out->sigma > 0.f) || !(out->eps >= 0.f) || !isfinite(out->sigma) || !isfinite(out->eps))
+    return DIFR_ERR_INVALID_ARG;
+  if (!(temperature >= 0.f) || !isfinite(temperature) || (ipt && temperature == 0.f)) return DIFR_ERR_INVALID_ARG;
+  if ((d % 8) != 0 || V < 2) return DIFR_ERR_SHAPE;
+  if (T == 0) return DIFR_OK;
+  DeviceInfo info;
+  if (!device_info(&info)) return DIFR_ERR_CUDA;
+  if (info.major != 10) return DIFR_ERR_ARCH;
+  Plan pl;
+  if (!make_plan(T, d, V, info.sms, &pl)) return DIFR_ERR_SHAPE;
+  if (!aligned16(h) || !aligned16(W)) return DIFR_ERR_ALIGN;
+  if (!out->workspace || out->workspace_bytes < pl.workspace_bytes) return DIFR_ERR_WORKSPACE;
+  if (!aligned16(out->workspace)) return DIFR_ERR_ALIGN;
+
+  CUtensorMap tmap_h, tmap_w;
+  if (!make_tmap(&tmap_h, h, T, d, kBM) || !make_tmap(&tmap_w, W, V, d, kBN)) return DIFR_ERR_CUDA;
+
+  K1Params k1;
+  memset(&k1, 0, sizeof k1);
+  k1.tokens = tokens; k1.seeds = seeds; k1.positions = positions;
+  k1.partials = reinterpret_cast<Partial*>(out->workspace);
+  k1.device_status = out->device_status;
+  k1.T = (int)T; k1.d = (int)d; k1.V = (int)V;
+  k1.T_pad = pl.T_pad; k1.m_tiles = pl.m_tiles; k1.n_tiles = pl.n_tiles; k1.k_steps = pl.k_steps;
+  k1.S = pl.S; k1.Gm = pl.Gm; k1.n_units = pl.n_units;
+  k1.c1 = temperature > 0.f ? 1.4426950408889634f / temperature : 0.f;
+  k1.neg_tl2 = -temperature * 0.6931471805599453f;
+  const int grid = pl.n_units < info.sms ? pl.n_units : info.sms;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (launch_k1(ipt ? 1 : 0, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;
+
+  K2Params k2;
+  memset(&k2, 0, sizeof k2);
+  k2.h = reinterpret_cast<const uint16_t*>(h); k2.W = reinterpret_cast<const uint16_t*>(W);
+  k2.tokens = tokens; k2.seeds = seeds; k2.positions = positions;
+  k2.partials = k1.partials; k2.n_slots = pl.n_slots; k2.T_pad = pl.T_pad;
+  k2.T = (int)T; k2.d = (int)d; k2.V = (int)V; k2.ipt = ipt;
+  k2.temperature = temperature; k2.sigma = out->sigma; k2.eps = out->eps; k2.c1 = k1.c1;
+  k2.score = out->score; k2.margin = out->margin; k2.argmax = out->argmax; k2.runner_up = out->runner_up;
+  k2.lse = out->lse; k2.p_claimed = out->p_claimed; k2.cdf_lo = out->cdf_lo; k2.u = out->u;
+  k2.row_status = out->row_status;
+  if (launch_k2(k2, s) != cudaSuccess) return DIFR_ERR_CUDA;
+  return DIFR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t difr_workspace_bytes(int64_t T, int64_t d, int64_t V) {
+  DeviceInfo info;
+  if (!device_info(&info)) info.sms = 148;
+  Plan pl;
+  if (!make_plan(T, d, V, info.sms, &pl)) return 0;
+  return pl.workspace_bytes;
+}
+
+difr_status difr_score_gm(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,
+                          const uint32_t* positions, float temperature, int64_t T, int64_t d, int64_t V,
+                          difr_out* out, difr_stream_t stream) {
+  return score_common(0, h, W, tokens, seeds, positions, temperature, T, d, V, out, stream);
+}
+
+difr_status difr_score_ipt(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,
+                           const uint32_t* positions, float temperature, int64_t T, int64_t d, int64_t V,
+                           difr_out* out, difr_stream_t stream) {
+  return score_common(1, h, W, tokens, seeds, positions, temperature, T, d, V, out, stream);
+}
+
+difr_status difr_detect(const float* scores, float threshold, const float* margins, const int32_t* ranks,
+                        int32_t rank_cutoff, const int32_t* seq_offsets, int64_t n_seq, int64_t T, uint8_t* flags,
+                        difr_seq_stats* seq_stats, difr_stream_t stream) {
+  if (!scores || T < 0 || n_seq < 0) return DIFR_ERR_INVALID_ARG;
+  if (isnan(threshold)) return DIFR_ERR_INVALID_ARG;
+  if (seq_offsets && n_seq == 0) return DIFR_OK;
+  if (!seq_offsets && T == 0 && !seq_stats) return DIFR_OK;
+  K3Params p;
+  memset(&p, 0, sizeof p);
+  p.scores = scores; p.margins = margins; p.ranks = ranks; p.seq_offsets = seq_offsets;
+  p.threshold = threshold; p.rank_cutoff = rank_cutoff; p.n_seq = n_seq; p.T = T;
+  p.flags = flags; p.seq_stats = seq_stats;
+  if (launch_k3(p, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return DIFR_ERR_CUDA;
+  return DIFR_OK;
+}
+
+difr_status difr_logits(const void* h, const void* W, int64_t T, int64_t d, int64_t V, float* logits,
+                        int32_t* device_status, difr_stream_t stream) {
+  if (!h || !W || !logits || T < 0 || d <= 0 || V <= 0) return DIFR_ERR_INVALID_ARG;
+  if ((d % 8) != 0 || V < 2) return DIFR_ERR_SHAPE;
+  if (T == 0) return DIFR_OK;
+  DeviceInfo info;
+  if (!device_info(&info)) return DIFR_ERR_CUDA;
+  if (info.major != 10) return DIFR_ERR_ARCH;
+  Plan pl;
+  if (!make_plan(T, d, V, info.sms, &pl)) return DIFR_ERR_SHAPE;
+  if (!aligned16(h) || !aligned16(W)) return DIFR_ERR_ALIGN;
+  CUtensorMap tmap_h, tmap_w;
+  if (!make_tmap(&tmap_h, h, T, d, kBM) || !make_tmap(&tmap_w, W, V, d, kBN)) return DIFR_ERR_CUDA;
+  K1Params k1;
+  memset(&k1, 0, sizeof k1);
+  k1.logits_out = logits; k1.device_status = device_status;
+  k1.T = (int)T; k1.d = (int)d; k1.V = (int)V;
+  k1.T_pad = pl.T_pad; k1.m_tiles = pl.m_tiles; k1.n_tiles = pl.n_tiles; k1.k_steps = pl.k_steps;
+  k1.S = pl.S; k1.Gm = pl.Gm; k1.n_units = pl.n_units;
+  const int grid = pl.n_units < info.sms ? pl.n_units : info.sms;
+  if (launch_k1(2, tmap_h, tmap_w, k1, grid, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return DIFR_ERR_CUDA;
+  return DIFR_OK;
+}
+
+difr_status difr_philox(const uint32_t* ctr, const uint32_t* key, int64_t n, uint32_t* out, difr_stream_t stream) {
+  if (n < 0 || (n > 0 && (!ctr || !key || !out))) return DIFR_ERR_INVALID_ARG;
+  if (launch_philox(ctr, key, n, out, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess) return DIFR_ERR_CUDA;
+  return DIFR_OK;
+}
+
+const char* difr_status_string(difr_status status) {
+  switch (status) {
+    case DIFR_OK: return "ok";
+    case DIFR_ERR_INVALID_ARG: return "invalid argument";
+    case DIFR_ERR_SHAPE: return "unsupported shape";
+    case DIFR_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case DIFR_ERR_WORKSPACE: return "workspace missing or too small";
+    case DIFR_ERR_CUDA: return "CUDA call failed";
+    case DIFR_ERR_ARCH: return "device is not compute capability 10.x";
+    case DIFR_ERR_TIMEOUT: return "a device-side wait ran out";
+  }
+  return "unknown status";
+}
+
+int difr_version(void) { return 100; }
+
+}  // extern "C"

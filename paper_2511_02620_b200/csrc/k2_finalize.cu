@@ -1,0 +1,245 @@
+// K2: split-V finalize.  One warp per row merges the row's partial records with
+// warp shuffles, re-evaluates in fp64 the few logits the score depends on (the
+// claimed token and the two Gumbel-max candidates: three gathered rows of W
+// against the row of h), re-ranks them, and turns the margin (Token-DiFR) or the
+// CDF interval (Token-IPT-DiFR) into the log-score.
+#include <cuda_runtime.h>
+#include <math_constants.h>
+
+#include "difr_device.cuh"
+#include "difr_kernels.h"
+
+namespace difr {
+
+constexpr int kK2Warps = 8;
+
+struct Merged {
+  float m1, m2;
+  int i1, i2;
+  double lmax, lsum, lpre;  // base-2 log-sum-exp state
+};
+
+__device__ __forceinline__ bool beats(float v, int i, float w, int j) {
+  // candidate (v, i) ranks ahead of (w, j); absent candidates carry id -1
+  if (i < 0) return false;
+  if (j < 0) return true;
+  return v > w || (v == w && i < j);
+}
+
+__device__ __forceinline__ void top2_insert(Merged& a, float v, int i) {
+  if (beats(v, i, a.m1, a.i1)) {
+    a.m2 = a.m1; a.i2 = a.i1;
+    a.m1 = v; a.i1 = i;
+  } else if (beats(v, i, a.m2, a.i2)) {
+    a.m2 = v; a.i2 = i;
+  }
+}
+
+__device__ __forceinline__ void lse_merge(Merged& a, double bmax, double bsum, double bpre) {
+  if (bmax == -CUDART_INF) return;
+  if (a.lmax == -CUDART_INF) {
+    a.lmax = bmax; a.lsum = bsum; a.lpre = bpre;
+    return;
+  }
+  const double m = fmax(a.lmax, bmax);
+  const double fa = exp2(a.lmax - m), fb = exp2(bmax - m);
+  a.lsum = a.lsum * fa + bsum * fb;
+  a.lpre = a.lpre * fa + bpre * fb;
+  a.lmax = m;
+}
+
+__device__ __forceinline__ double shfl_xor_double(double v, int mask) {
+  int lo = __double2loint(v), hi = __double2hiint(v);
+  lo = __shfl_xor_sync(0xffffffffu, lo, mask);
+  hi = __shfl_xor_sync(0xffffffffu, hi, mask);
+  return __hiloint2double(hi, lo);
+}
+
+__device__ __forceinline__ double bf16_to_double(uint32_t bits16) {
+  return (double)__uint_as_float(bits16 << 16);
+}
+
+// fp64 dot product of two bf16 rows of length d (d % 8 == 0, rows 16-byte aligned), whole warp.
+__device__ __forceinline__ double warp_dot(const uint16_t* a, const uint16_t* b, int d, int lane) {
+  double acc = 0.0;
+  for (int k = lane * 8; k < d; k += 32 * 8) {
+    const uint4 va = *reinterpret_cast<const uint4*>(a + k);
+    const uint4 vb = *reinterpret_cast<const uint4*>(b + k);
+    const uint32_t wa[4] = {va.x, va.y, va.z, va.w};
+    const uint32_t wb[4] = {vb.x, vb.y, vb.z, vb.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      acc = fma(bf16_to_double(wa[q] & 0xFFFFu), bf16_to_double(wb[q] & 0xFFFFu), acc);
+      acc = fma(bf16_to_double(wa[q] >> 16), bf16_to_double(wb[q] >> 16), acc);
+    }
+  }
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) acc += shfl_xor_double(acc, m);
+  return acc;
+}
+
+__device__ __forceinline__ double gumbel_exact(uint64_t seed, uint32_t position, uint32_t id) {
+  uint32_t x[4];
+  philox4x32_10(id >> 2, position, 0u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), x);
+  const double u = ((double)(x[id & 3u] >> 9) + 0.5) * (1.0 / 8388608.0);
+  return -log(-log(u));
+}
+
+// Phi(zb) - Phi(za), za <= zb, evaluated in the tail that avoids cancellation.
+__device__ __forceinline__ double normal_interval(double za, double zb) {
+  const double r = 0.70710678118654752440;
+  if (za >= 0.0) return 0.5 * (erfc(za * r) - erfc(zb * r));
+  if (zb <= 0.0) return 0.5 * (erfc(-zb * r) - erfc(-za * r));
+  return 1.0 - 0.5 * erfc(zb * r) - 0.5 * erfc(-za * r);
+}
+
+__global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * kK2Warps + warp;
+  if (row >= p.T) return;  // whole warps leave together
+
+  // ---- merge the row's partial records
+  Merged acc;
+  acc.m1 = acc.m2 = -CUDART_INF_F;
+  acc.i1 = acc.i2 = -1;
+  acc.lmax = -CUDART_INF;
+  acc.lsum = acc.lpre = 0.0;
+  for (int slot = lane; slot < p.n_slots; slot += 32) {
+    const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * (size_t)p.T_pad + row);
+    const float4 a = src[0], b = src[1];
+    top2_insert(acc, a.x, __float_as_int(a.y));
+    top2_insert(acc, a.z, __float_as_int(a.w));
+    lse_merge(acc, (double)b.x, (double)b.y, (double)b.z);
+  }
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) {
+    const float o1 = __shfl_xor_sync(0xffffffffu, acc.m1, m), o2 = __shfl_xor_sync(0xffffffffu, acc.m2, m);
+    const int j1 = __shfl_xor_sync(0xffffffffu, acc.i1, m), j2 = __shfl_xor_sync(0xffffffffu, acc.i2, m);
+    const double om = shfl_xor_double(acc.lmax, m), os = shfl_xor_double(acc.lsum, m),
+                 op = shfl_xor_double(acc.lpre, m);
+    top2_insert(acc, o1, j1);
+    top2_insert(acc, o2, j2);
+    lse_merge(acc, om, os, op);
+  }
+  // (every lane now holds the same merged state up to the order of the lse additions; use lane 0's)
+  acc.lmax = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(acc.lmax), 0),
+                              __shfl_sync(0xffffffffu, __double2loint(acc.lmax), 0));
+  acc.lsum = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(acc.lsum), 0),
+                              __shfl_sync(0xffffffffu, __double2loint(acc.lsum), 0));
+  acc.lpre = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(acc.lpre), 0),
+                              __shfl_sync(0xffffffffu, __double2loint(acc.lpre), 0));
+
+  const int tok = p.tokens[row];
+  const uint64_t seed = p.seeds[row];
+  const uint32_t pos = p.positions[row];
+  const bool tok_ok = tok >= 0 && tok < p.V;
+  const uint16_t* hrow = p.h + (size_t)row * (size_t)p.d;
+  const double temp = (double)p.temperature;
+  const double sigma = (double)p.sigma, eps = (double)p.eps;
+  uint32_t status = tok_ok ? 0u : 1u;
+
+  const double ln2 = 0.69314718055994530942;
+  const bool lse_finite = isfinite(acc.lmax) && isfinite(acc.lsum) && acc.lsum > 0.0;
+  if (!lse_finite) status |= 2u;
+  const double lse = (p.temperature > 0.f) ? (acc.lmax + log2(acc.lsum)) * ln2 : CUDART_NAN;
+
+  double l_tok = 0.0;
+  if (tok_ok) l_tok = warp_dot(hrow, p.W + (size_t)tok * (size_t)p.d, p.d, lane);
+
+  if (!p.ipt) {
+    // ---- Token-DiFR: exact y = l + Temp * G for the claimed token and the two candidates
+    const int c1 = (acc.i1 >= 0 && acc.i1 < p.V) ? acc.i1 : -1;
+    const int c2 = (acc.i2 >= 0 && acc.i2 < p.V) ? acc.i2 : -1;
+    double y1 = -CUDART_INF, y2 = -CUDART_INF, yt = -CUDART_INF;
+    if (c1 >= 0) y1 = warp_dot(hrow, p.W + (size_t)c1 * (size_t)p.d, p.d, lane) + temp * gumbel_exact(seed, pos, c1);
+    if (c2 >= 0) y2 = warp_dot(hrow, p.W + (size_t)c2 * (size_t)p.d, p.d, lane) + temp * gumbel_exact(seed, pos, c2);
+    if (tok_ok) yt = l_tok + temp * gumbel_exact(seed, pos, (uint32_t)tok);
+    if (lane == 0) {
+      // order the two candidates exactly (ties: lowest id)
+      int a = c1, b = c2;
+      double ya = y1, yb = y2;
+      if (b >= 0 && (a < 0 || yb > ya || (yb == ya && b < a))) {
+        int ti = a; a = b; b = ti;
+        double tv = ya; ya = yb; yb = tv;
+      }
+      int best = a, second = b;
+      double A = -CUDART_INF;
+      if (tok_ok) {
+        // strongest competitor: the best candidate that is not the claimed token
+        const int c = (a != tok) ? a : b;
+        const double yc = (a != tok) ? ya : yb;
+        A = (c >= 0) ? yt - yc : CUDART_INF;
+        if (A == 0.0 && tok > c) A = -0.0;
+        const bool tok_first = (c < 0) || (yt > yc) || (yt == yc && tok < c);
+        if (tok != a && tok != b) {
+          // the claimed token was not among the candidates: place it
+          if (tok_first) { second = a; best = tok; }
+          else if (b < 0 || yt > yb || (yt == yb && tok < b)) { second = tok; }
+        }
+      }
+      const double pi = 0.5 * erfc(-A / (2.0 * sigma));  // Phi(A / (sigma sqrt 2))
+      const double score = tok_ok ? log(pi + eps) : log(eps);
+      p.score[row] = (float)score;
+      if (p.margin) p.margin[row] = (float)A;
+      if (p.argmax) p.argmax[row] = best;
+      if (p.runner_up) p.runner_up[row] = second;
+      if (p.lse) p.lse[row] = (float)lse;
+      if (p.row_status) p.row_status[row] = status;
+    }
+  } else {
+    // ---- Token-IPT-DiFR
+    if (lane == 0) {
+      uint32_t x[4];
+      philox4x32_10(0u, pos, 1u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), x);
+      const double mu = ((double)x[0] + 0.5) * (1.0 / 4294967296.0);
+      double score = log(eps), pt = CUDART_NAN, a = CUDART_NAN;
+      if (tok_ok) {
+        const double c1d = (double)p.c1;  // log2(e) / Temp, the very factor the fused kernel scaled its logits by
+        pt = exp2(l_tok * c1d - acc.lmax) / acc.lsum;
+        a = acc.lpre / acc.lsum;
+        const double b = a + pt;
+        const double mass = normal_interval((a - mu) / sigma, (b - mu) / sigma);
+        score = log(mass + eps);
+      }
+      p.score[row] = (float)score;
+      if (p.lse) p.lse[row] = (float)lse;
+      if (p.p_claimed) p.p_claimed[row] = (float)pt;
+      if (p.cdf_lo) p.cdf_lo[row] = (float)a;
+      if (p.u) p.u[row] = (float)mu;
+      if (p.row_status) p.row_status[row] = status;
+    }
+  }
+}
+
+cudaError_t launch_k2(const K2Params& p, cudaStream_t stream) {
+  const int blocks = (p.T + kK2Warps - 1) / kK2Warps;
+  k2_finalize<<<blocks, kK2Warps * 32, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+// --------------------------------------------------------- Philox validation
+__global__ void philox_blocks(const uint32_t* ctr, const uint32_t* key, int64_t n, uint32_t* out) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const uint32_t c0 = ctr[4 * i], c1 = ctr[4 * i + 1], c2 = ctr[4 * i + 2], c3 = ctr[4 * i + 3];
+  const uint32_t k0 = key[2 * i], k1 = key[2 * i + 1];
+  uint32_t x[4];
+  if (c2 == 0u && c3 == 0u) {
+    // the per-row form the scoring epilogue uses
+    RowNoise rn;
+    row_noise_init(rn, ((uint64_t)k1 << 32) | k0, c1);
+    row_noise_block(rn, c0, x);
+  } else {
+    philox4x32_10(c0, c1, c2, c3, k0, k1, x);
+  }
+  out[4 * i] = x[0]; out[4 * i + 1] = x[1]; out[4 * i + 2] = x[2]; out[4 * i + 3] = x[3];
+}
+
+cudaError_t launch_philox(const uint32_t* ctr, const uint32_t* key, int64_t n, uint32_t* out, cudaStream_t stream) {
+  if (n <= 0) return cudaSuccess;
+  const int threads = 128;
+  philox_blocks<<<(unsigned)((n + threads - 1) / threads), threads, 0, stream>>>(ctr, key, n, out);
+  return cudaGetLastError();
+}
+
+}  // namespace difr

