@@ -82,6 +82,9 @@ typedef struct {
   size_t workspace_bytes;
   int32_t* device_status; /* [1] optional. Sticky: a kernel writes DIFR_ERR_TIMEOUT
                              here if a bounded wait ran out; never cleared         */
+  void* event_fused_start; /* optional cudaEvent_t (host handles): recorded on `stream` */
+  void* event_fused_stop;  /* right before / after the fused GEMM+epilogue kernel, so a
+                              caller can time that kernel apart from the finalize pass */
 } difr_out;
 
 /* Scratch bytes a scoring call needs for T rows, hidden size d, vocabulary V.

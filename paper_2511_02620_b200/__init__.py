@@ -35,6 +35,7 @@ class _COut(ctypes.Structure):
         ("runner_up", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("p_claimed", ctypes.c_void_p),
         ("cdf_lo", ctypes.c_void_p), ("u", ctypes.c_void_p), ("row_status", ctypes.c_void_p),
         ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t), ("device_status", ctypes.c_void_p),
+        ("event_fused_start", ctypes.c_void_p), ("event_fused_stop", ctypes.c_void_p),
     ]
 
 
@@ -120,6 +121,8 @@ class DifrOut:
     row_status: "object" = None
     workspace: "object" = None
     device_status: "object" = None
+    event_fused_start: int = 0  # raw cudaEvent_t handles (0: none)
+    event_fused_stop: int = 0
 
     @staticmethod
     def allocate(T: int, d: int, V: int, sigma: float, eps: float = 1e-12, device="cuda"):
@@ -137,7 +140,8 @@ class DifrOut:
         return _COut(float(self.sigma), float(self.eps), _ptr(self.score), _ptr(self.margin), _ptr(self.argmax),
                      _ptr(self.runner_up), _ptr(self.lse), _ptr(self.p_claimed), _ptr(self.cdf_lo), _ptr(self.u),
                      _ptr(self.row_status), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
-                     _ptr(self.device_status))
+                     _ptr(self.device_status), ctypes.c_void_p(self.event_fused_start or None),
+                     ctypes.c_void_p(self.event_fused_stop or None))
 
 
 def _score(fn_name, h, W, tokens, seeds, positions, temperature, out: DifrOut, stream):

@@ -93,7 +93,11 @@ difr_status score_common(int ipt, const void* h, const void* W, const int32_t* t
   k1.neg_tl2 = -temperature * 0.6931471805599453f;
   const int grid = pl.n_units < info.sms ? pl.n_units : info.sms;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (out->event_fused_start && cudaEventRecord(reinterpret_cast<cudaEvent_t>(out->event_fused_start), s) != cudaSuccess)
+    return DIFR_ERR_CUDA;
   if (launch_k1(ipt ? 1 : 0, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;
+  if (out->event_fused_stop && cudaEventRecord(reinterpret_cast<cudaEvent_t>(out->event_fused_stop), s) != cudaSuccess)
+    return DIFR_ERR_CUDA;
 
   K2Params k2;
   memset(&k2, 0, sizeof k2);
