@@ -131,6 +131,39 @@ difr_status difr_score_ipt(const void* h, const void* W, const int32_t* tokens, 
                            difr_out* out, difr_stream_t stream);
 
 /*
+ * difr_score_gm without a workspace: for callers that cannot allocate.
+ * (The paper has no counterpart; this is a property of the library only.)
+ *
+ * Some hosts of this library hand it input and output buffers but have no way
+ * to obtain scratch memory of their own: a plugin running inside another
+ * framework's memory pool that may not call cudaMalloc behind its back, a
+ * process whose device memory was carved up in advance, a caller replaying a
+ * fixed sequence of launches that must not contain an allocation.  For them this
+ * entry point computes exactly what difr_score_gm computes, with the partial
+ * records kept in an array of DIFR_STATIC_SCRATCH_BYTES that is part of the
+ * library's device image.  Every GPU that loads the library holds that array
+ * until the process exits.
+ *
+ *   - out->workspace and out->workspace_bytes are ignored; all other arguments and
+ *     outputs are those of difr_score_gm.
+ *   - Returns DIFR_ERR_WORKSPACE, launching nothing, when
+ *     difr_workspace_bytes(T, d, V) exceeds DIFR_STATIC_SCRATCH_BYTES.
+ *   - Calls no cudaMalloc, cudaFree or other allocating routine.
+ *   - The first call on each device looks up the array's device address (the
+ *     device must be current); make that first call before starting any stream
+ *     capture.
+ *   - All calls on a device share the one array, and it keeps what the last
+ *     call left there.  Nothing in it has to start at zero: each call overwrites
+ *     every record before reading it.  Two calls that overlap on the GPU (different
+ *     streams, no ordering between them) race on it and give wrong scores;
+ *     serialise them, or use difr_score_gm with separate workspaces.
+ */
+#define DIFR_STATIC_SCRATCH_BYTES (16u << 20)
+difr_status difr_score_gm_static(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,
+                                 const uint32_t* positions, float temperature, int64_t T, int64_t d, int64_t V,
+                                 difr_out* out, difr_stream_t stream);
+
+/*
  * Threshold detection and pooling (Sec. "Classification via Thresholding":
  * flag t iff FSSL(t) < tau; per-sequence match count as in Alg. "Sampled token
  * verification via prefill").

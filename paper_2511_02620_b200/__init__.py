@@ -18,8 +18,9 @@ DIFR_OK = 0
 STATUS_NAMES = {0: "DIFR_OK", -1: "DIFR_ERR_INVALID_ARG", -2: "DIFR_ERR_SHAPE", -3: "DIFR_ERR_ALIGN",
                 -4: "DIFR_ERR_WORKSPACE", -5: "DIFR_ERR_CUDA", -6: "DIFR_ERR_ARCH", -7: "DIFR_ERR_TIMEOUT"}
 
-EXPORTS = ("difr_workspace_bytes", "difr_score_gm", "difr_score_ipt", "difr_detect", "difr_logits", "difr_philox",
-           "difr_status_string", "difr_version")
+EXPORTS = ("difr_workspace_bytes", "difr_score_gm", "difr_score_ipt", "difr_score_gm_static", "difr_detect",
+           "difr_logits", "difr_philox", "difr_status_string", "difr_version")
+STATIC_SCRATCH_BYTES = 16 << 20  # DIFR_STATIC_SCRATCH_BYTES
 
 
 class DifrError(RuntimeError):
@@ -54,7 +55,7 @@ def lib() -> ctypes.CDLL:
         L.difr_workspace_bytes.argtypes = [ctypes.c_int64] * 3
         score_args = [ctypes.c_void_p] * 5 + [ctypes.c_float] + [ctypes.c_int64] * 3 + [ctypes.POINTER(_COut),
                                                                                       ctypes.c_void_p]
-        for name in ("difr_score_gm", "difr_score_ipt"):
+        for name in ("difr_score_gm", "difr_score_ipt", "difr_score_gm_static"):
             getattr(L, name).restype = ctypes.c_int
             getattr(L, name).argtypes = score_args
         L.difr_detect.restype = ctypes.c_int
@@ -170,6 +171,13 @@ def difr_score_gm(h, W, tokens, seeds, positions, temperature, out: DifrOut, str
 def difr_score_ipt(h, W, tokens, seeds, positions, temperature, out: DifrOut, stream=None) -> DifrOut:
     """Token-IPT-DiFR scores; see include/difr.h."""
     return _score("difr_score_ipt", h, W, tokens, seeds, positions, temperature, out, stream)
+
+
+def difr_score_gm_static(h, W, tokens, seeds, positions, temperature, out: DifrOut, stream=None) -> DifrOut:
+    """difr_score_gm for callers that cannot allocate scratch memory: `out.workspace` is ignored (it may be
+    None) and the library's built-in 16 MiB array is used instead.  Raises DifrError(DIFR_ERR_WORKSPACE) for
+    problems that need more.  Calls on one device share that array, so do not let two of them overlap."""
+    return _score("difr_score_gm_static", h, W, tokens, seeds, positions, temperature, out, stream)
 
 
 def difr_detect(scores, threshold, margins=None, ranks=None, rank_cutoff=0, seq_offsets=None, flags=None,

@@ -184,6 +184,49 @@ difr_status difr_philox(const uint32_t* ctr, const uint32_t* key, int64_t n, uin
   return DIFR_OK;
 }
 
+// ------------------------------------------------------- allocation-free entry
+// Scratch for difr_score_gm_static: a fixed array inside the library's device
+// image, so the caller never has to obtain workspace memory.
+constexpr size_t kStaticScratchBytes = (size_t)DIFR_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// In host code `g_static_scratch` only names the symbol; the device address has
+// to be asked for, once per device, while that device is current.
+static difr_status static_scratch_address(void** ptr) {
+  constexpr int kMaxDevices = 64;
+  static void* cached[kMaxDevices] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return DIFR_ERR_CUDA;
+  if (dev >= 0 && dev < kMaxDevices && cached[dev] != nullptr) {
+    *ptr = cached[dev];
+    return DIFR_OK;
+  }
+  void* p = nullptr;
+  if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return DIFR_ERR_CUDA;
+  if (dev >= 0 && dev < kMaxDevices) cached[dev] = p;  // same value whichever thread gets here first
+  *ptr = p;
+  return DIFR_OK;
+}
+
+difr_status difr_score_gm_static(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,
+                                 const uint32_t* positions, float temperature, int64_t T, int64_t d, int64_t V,
+                                 difr_out* out, difr_stream_t stream) {
+  if (!out) return DIFR_ERR_INVALID_ARG;
+  if (T > 0 && d > 0 && V > 0) {
+    DeviceInfo info;
+    Plan pl;
+    if (device_info(&info) && make_plan(T, d, V, info.sms, &pl) && pl.workspace_bytes > kStaticScratchBytes)
+      return DIFR_ERR_WORKSPACE;  // problem too large for the built-in scratch: use difr_score_gm
+  }
+  void* scratch = nullptr;
+  const difr_status st = static_scratch_address(&scratch);
+  if (st != DIFR_OK) return st;
+  difr_out local = *out;
+  local.workspace = scratch;
+  local.workspace_bytes = kStaticScratchBytes;
+  return score_common(0, h, W, tokens, seeds, positions, temperature, T, d, V, &local, stream);
+}
+
 const char* difr_status_string(difr_status status) {
   switch (status) {
     case DIFR_OK: return "ok";
