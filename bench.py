@@ -34,7 +34,7 @@ UNIT = "tokens/s"
 L2_BYTES = 126 * 2**20
 # dram__bytes_read.sum + dram__bytes_write.sum of the fused kernel per launch, from the
 # ncu captures summarised under profiles/ (bytes; None until captured for that workload)
-FUSED_TRAFFIC = {}
+FUSED_TRAFFIC = {"llama3b": 953.9e6}  # profiles/k1_fused_score_llama3b.md
 
 
 def load_peaks():
@@ -52,6 +52,28 @@ def pick_workload(args):
     if args.T:
         w = wl.with_T(w, args.T)
     return w
+
+
+# ------------------------------------------------------------------ multi-rank
+def rank_info():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def reduce_max(values, device=None):
+    """Max over ranks of a list of floats (each rank times its own replica; the job is as slow as the slowest)."""
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def whole_job_rate(world, rows_per_rank, steps, elapsed_ms):
+    """Rows are sharded across ranks with no exchange: the job's rate is all ranks' rows over the slowest rank's time."""
+    return world * rows_per_rank * steps / (elapsed_ms * 1e-3)
 
 
 # --------------------------------------------------------------------- clocks
@@ -127,9 +149,8 @@ def oracle_throughput(w, inp, tokens, temperature, sigma, budget_s, rows_overrid
 
 
 def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
-        return
+    if rank_info()[0] != 0:
+        return  # under torchrun rank 0 alone times the oracle
     import oracle
 
     w = pick_workload(args)
@@ -188,9 +209,7 @@ def run_ours(args):
 
     import paper_2511_02620_b200 as difr
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, local_rank, world = rank_info()
     torch.cuda.set_device(local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
@@ -332,16 +351,13 @@ def run_ours(args):
     d2h = score_host.numel() * 4 + flags_host.numel() + stats_host.numel() * 4
     assert torch.equal(flags_host, flags.cpu())
 
-    if world > 1:
-        t = torch.tensor([elapsed_ms, e2e_ms, fused_avg_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms, e2e_ms, fused_avg_ms = (float(x) for x in t.cpu())
+    elapsed_ms, e2e_ms, fused_avg_ms = reduce_max([elapsed_ms, e2e_ms, fused_avg_ms], device="cuda")
 
     if rank == 0:
         peaks = load_peaks()
         flop = 2.0 * T * d * V
         achieved = flop / (fused_avg_ms * 1e-3) / 1e12
-        value = world * T * args.steps / (elapsed_ms * 1e-3)
+        value = whole_job_rate(world, T, args.steps, elapsed_ms)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
@@ -349,7 +365,7 @@ def run_ours(args):
             "config": config_dict(w, args),
             "tflops": world * flop * args.steps / (elapsed_ms * 1e-3) / 1e12,
             "clocks": clocks,
-            "e2e": {"value": world * T * args.steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "e2e": {"value": whole_job_rate(world, T, args.steps, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps,
                     "note": "per-step inputs (h, tokens, seeds, positions) from pinned host memory; W resident"},
             "gpu_launches": 3 * args.steps,
