@@ -46,14 +46,28 @@ bool make_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, i
 
 struct DeviceInfo {
   int major;
-  int sms;
+  int pairs;  // CTA pairs of the fused kernel that are resident at once (0 on other architectures)
 };
 
 bool device_info(DeviceInfo* info) {
+  constexpr int kMaxDevices = 64;
+  static int cached_pairs[kMaxDevices] = {0};  // 0: not asked yet
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return false;
   if (cudaDeviceGetAttribute(&info->major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return false;
-  if (cudaDeviceGetAttribute(&info->sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+  info->pairs = 0;
+  if (info->major != 10) return true;
+  if (dev >= 0 && dev < kMaxDevices && cached_pairs[dev] > 0) {
+    info->pairs = cached_pairs[dev];
+    return true;
+  }
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+  int pairs = k1_max_resident_pairs();
+  if (pairs <= 0) return false;
+  if (pairs > sms / 2) pairs = sms / 2;
+  if (dev >= 0 && dev < kMaxDevices) cached_pairs[dev] = pairs;
+  info->pairs = pairs;
   return true;
 }
 
@@ -73,13 +87,13 @@ difr_status score_common(int ipt, const void* h, const void* W, const int32_t* t
   if (!device_info(&info)) return DIFR_ERR_CUDA;
   if (info.major != 10) return DIFR_ERR_ARCH;
   Plan pl;
-  if (!make_plan(T, d, V, info.sms, &pl)) return DIFR_ERR_SHAPE;
+  if (!make_plan(T, d, V, info.pairs, &pl)) return DIFR_ERR_SHAPE;
   if (!aligned16(h) || !aligned16(W)) return DIFR_ERR_ALIGN;
   if (!out->workspace || out->workspace_bytes < pl.workspace_bytes) return DIFR_ERR_WORKSPACE;
   if (!aligned16(out->workspace)) return DIFR_ERR_ALIGN;
 
   CUtensorMap tmap_h, tmap_w;
-  if (!make_tmap(&tmap_h, h, T, d, kBM) || !make_tmap(&tmap_w, W, V, d, kBN)) return DIFR_ERR_CUDA;
+  if (!make_tmap(&tmap_h, h, T, d, kBM) || !make_tmap(&tmap_w, W, V, d, kBN / 2)) return DIFR_ERR_CUDA;
 
   K1Params k1;
   memset(&k1, 0, sizeof k1);
@@ -91,7 +105,7 @@ difr_status score_common(int ipt, const void* h, const void* W, const int32_t* t
   k1.S = pl.S; k1.Gm = pl.Gm; k1.n_units = pl.n_units;
   k1.c1 = temperature > 0.f ? 1.4426950408889634f / temperature : 0.f;
   k1.neg_tl2 = -temperature * 0.6931471805599453f;
-  const int grid = pl.n_units < info.sms ? pl.n_units : info.sms;
+  const int grid = 2 * (pl.n_units < info.pairs ? pl.n_units : info.pairs);
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   if (out->event_fused_start && cudaEventRecord(reinterpret_cast<cudaEvent_t>(out->event_fused_start), s) != cudaSuccess)
     return DIFR_ERR_CUDA;
@@ -119,9 +133,9 @@ extern "C" {
 
 size_t difr_workspace_bytes(int64_t T, int64_t d, int64_t V) {
   DeviceInfo info;
-  if (!device_info(&info)) info.sms = 148;
+  if (!device_info(&info)) info.pairs = 0;  // no device: plan for a full B200 (74 pairs)
   Plan pl;
-  if (!make_plan(T, d, V, info.sms, &pl)) return 0;
+  if (!make_plan(T, d, V, info.pairs, &pl)) return 0;
   return pl.workspace_bytes;
 }
 
@@ -162,17 +176,17 @@ difr_status difr_logits(const void* h, const void* W, int64_t T, int64_t d, int6
   if (!device_info(&info)) return DIFR_ERR_CUDA;
   if (info.major != 10) return DIFR_ERR_ARCH;
   Plan pl;
-  if (!make_plan(T, d, V, info.sms, &pl)) return DIFR_ERR_SHAPE;
+  if (!make_plan(T, d, V, info.pairs, &pl)) return DIFR_ERR_SHAPE;
   if (!aligned16(h) || !aligned16(W)) return DIFR_ERR_ALIGN;
   CUtensorMap tmap_h, tmap_w;
-  if (!make_tmap(&tmap_h, h, T, d, kBM) || !make_tmap(&tmap_w, W, V, d, kBN)) return DIFR_ERR_CUDA;
+  if (!make_tmap(&tmap_h, h, T, d, kBM) || !make_tmap(&tmap_w, W, V, d, kBN / 2)) return DIFR_ERR_CUDA;
   K1Params k1;
   memset(&k1, 0, sizeof k1);
   k1.logits_out = logits; k1.device_status = device_status;
   k1.T = (int)T; k1.d = (int)d; k1.V = (int)V;
   k1.T_pad = pl.T_pad; k1.m_tiles = pl.m_tiles; k1.n_tiles = pl.n_tiles; k1.k_steps = pl.k_steps;
   k1.S = pl.S; k1.Gm = pl.Gm; k1.n_units = pl.n_units;
-  const int grid = pl.n_units < info.sms ? pl.n_units : info.sms;
+  const int grid = 2 * (pl.n_units < info.pairs ? pl.n_units : info.pairs);
   if (launch_k1(2, tmap_h, tmap_w, k1, grid, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
     return DIFR_ERR_CUDA;
   return DIFR_OK;
@@ -215,7 +229,7 @@ difr_status difr_score_gm_static(const void* h, const void* W, const int32_t* to
   if (T > 0 && d > 0 && V > 0) {
     DeviceInfo info;
     Plan pl;
-    if (device_info(&info) && make_plan(T, d, V, info.sms, &pl) && pl.workspace_bytes > kStaticScratchBytes)
+    if (device_info(&info) && make_plan(T, d, V, info.pairs, &pl) && pl.workspace_bytes > kStaticScratchBytes)
       return DIFR_ERR_WORKSPACE;  // problem too large for the built-in scratch: use difr_score_gm
   }
   void* scratch = nullptr;

@@ -61,7 +61,8 @@ struct K3Params {
 
 // mode: 0 Gumbel-max epilogue, 1 softmax statistics only, 2 logits dump.
 cudaError_t launch_k1(int mode, const CUtensorMap& tmap_h, const CUtensorMap& tmap_w, const K1Params& p, int grid,
-                      cudaStream_t stream);
+                      cudaStream_t stream);  // grid: number of CTAs, two per pair
+int k1_max_resident_pairs();  // CTA pairs of the fused kernel the current device keeps resident at once
 cudaError_t launch_k2(const K2Params& p, cudaStream_t stream);
 cudaError_t launch_k3(const K3Params& p, cudaStream_t stream);
 cudaError_t launch_philox(const uint32_t* ctr, const uint32_t* key, int64_t n, uint32_t* out, cudaStream_t stream);

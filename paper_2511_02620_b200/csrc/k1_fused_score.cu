@@ -8,16 +8,25 @@
 //                                               top-2 of y = l + Temp*G, the running log-sum-exp of
 //                                               l/Temp and the exponential mass below the claimed id
 //
-// A CTA is persistent and warp-specialised: warp 0 issues TMA loads, warp 1
+// CTAs run as persistent pairs (a cluster of two, one CTA per SM).  A pair owns a
+// 256 x 256 logit tile: each CTA loads its own 128 rows of h and its own 128 of
+// the tile's 256 rows of W, and one thread of the pair's first CTA issues
+// tcgen05.mma.cta_group::2, which reads both CTAs' shared memory and writes rows
+// 0..127 of the accumulator to the first CTA's TMEM and rows 128..255 to the
+// second's.  Per 256 x 256 x 64 step each SM therefore fills 32 KB of shared
+// memory instead of the 48 KB a lone 128 x 256 tile needs.
+//
+// Warp roles in each CTA: warp 0 issues the TMA loads, warp 1 (first CTA only)
 // issues the MMAs, warp 2 owns the TMEM allocation, warps 4..11 are the epilogue
-// (two warpgroups, one per 128-column half of the 128 x 256 accumulator tile).
+// (two warpgroups, one per 128-column half of the CTA's 128 x 256 accumulator).
 // Two accumulator stages (all 512 TMEM columns) let the epilogue of tile n
-// overlap the MMAs of tile n + 1.  A work unit is (m tile, vocabulary strip);
-// its running statistics stay in registers across the strip and leave as one
-// 32-byte partial record per (row, strip, column half).
+// overlap the MMAs of tile n + 1.  A work unit is (256-row tile, vocabulary
+// strip); its running statistics stay in registers across the strip and leave
+// as one 32-byte partial record per (row, strip, column half).
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <math_constants.h>
+#include <string.h>
 
 #include "difr_device.cuh"
 #include "difr_kernels.h"
@@ -25,9 +34,9 @@
 
 namespace difr {
 
-constexpr int kStages = 4;
-constexpr int kABytes = kBM * kBK * 2;   // 16 KB
-constexpr int kBBytes = kBN * kBK * 2;   // 32 KB
+constexpr int kStages = 6;
+constexpr int kABytes = kBM * kBK * 2;         // 16 KB: this CTA's 128 rows of h
+constexpr int kBBytes = (kBN / 2) * kBK * 2;   // 16 KB: this CTA's 128 of the tile's 256 rows of W
 constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kAccStages = 2;
 constexpr int kThreads = 384;
@@ -41,7 +50,7 @@ constexpr float kMasked = -3.0e38f;  // stands in for -inf on padded vocabulary 
 enum : int { kModeGm = 0, kModeIpt = 1, kModeDump = 2 };
 
 struct Unit {
-  int m, n0, n1, strip;
+  int m, n0, n1, strip;  // m: 256-row tile of the pair
 };
 
 __device__ __forceinline__ Unit decode_unit(const K1Params& p, int u) {
@@ -181,7 +190,7 @@ __device__ __forceinline__ void process_chunk(uint32_t (&raw)[32], int base, int
 }
 
 template <int MODE>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_w,
                const K1Params p) {
   extern __shared__ uint8_t smem_raw[];
@@ -189,6 +198,11 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
   const uint32_t smem_base = (raw_addr + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (smem_base - raw_addr);
 
+  // Both CTAs of a pair lay out their barriers at the same offsets.
+  //   full[s]      first CTA's copy is used: 1 arrival (its producer) + the bytes of both CTAs' loads
+  //   empty[s]     each CTA's own copy: 1 arrival, the MMA thread's commit delivered to both CTAs
+  //   acc_full[a]  each CTA's own copy: 1 arrival, the commit after a tile's last MMA, delivered to both
+  //   acc_empty[a] first CTA's copy is used: one arrival per epilogue warp of both CTAs
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
   const uint32_t bar0 = smem_base + kStages * kStageBytes;
   auto full_bar = [&](int s) { return bar0 + 8u * (uint32_t)s; };
@@ -200,6 +214,9 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const uint32_t cta = cluster_ctarank();  // 0: the pair's first CTA (issues the MMAs), 1: its partner
+  const int pair = blockIdx.x >> 1;
+  const int n_pairs = gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -208,7 +225,7 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     }
     for (int a = 0; a < kAccStages; ++a) {
       mbar_init(acc_full_bar(a), 1);
-      mbar_init(acc_empty_bar(a), kEpiWarps);
+      mbar_init(acc_empty_bar(a), 2 * kEpiWarps);
     }
     *abort_flag = 0;
     mbar_fence_init();
@@ -216,29 +233,37 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     tma_prefetch_desc(&tmap_w);
   }
   if (warp == 2) {
-    tmem_alloc(smem_u32(tmem_slot), kTmemCols);
-    tmem_relinquish();
+    tmem_alloc_pair(smem_u32(tmem_slot), kTmemCols);
+    tmem_relinquish_pair();
   }
   tc_fence_before();
   __syncthreads();
+  cluster_arrive();  // the partner's barriers are initialised and its TMEM allocated before anyone signals them
+  cluster_wait();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
+      // a CTA re-reads its h tile for every vocabulary tile of the strip: keep it in L2;
+      // a W tile is read by the pairs of one raster group at about the same time, then never again soon
+      const uint64_t keep = l2_policy_evict_last(), stream = l2_policy_evict_first();
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
+      for (int u = pair; u < p.n_units && ok; u += n_pairs) {
         const Unit w = decode_unit(p, u);
+        const int row0 = w.m * kPairM + (int)cta * kBM;
         for (int n = w.n0; n < w.n1 && ok; ++n) {
+          const int wrow0 = n * kBN + (int)cta * (kBN / 2);
           for (int k = 0; k < p.k_steps; ++k) {
             if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
-            mbar_arrive_expect_tx(full_bar(stage), kStageBytes);
+            if (cta == 0) mbar_arrive_expect_tx(full_bar(stage), 2u * kStageBytes);
+            const uint32_t full0 = map_to_cta(full_bar(stage), 0);
             const uint32_t a_dst = smem_base + (uint32_t)stage * kStageBytes;
-            tma_load_2d(a_dst, &tmap_h, k * kBK, w.m * kBM, full_bar(stage));
-            tma_load_2d(a_dst + kABytes, &tmap_w, k * kBK, n * kBN, full_bar(stage));
+            tma_load_2d_pair(a_dst, &tmap_h, k * kBK, row0, full0, keep);
+            tma_load_2d_pair(a_dst + kABytes, &tmap_w, k * kBK, wrow0, full0, stream);
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
         }
@@ -246,12 +271,12 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     }
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(kBM, kBN);
+    if (cta == 0 && lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(kPairM, kBN);
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
+      for (int u = pair; u < p.n_units && ok; u += n_pairs) {
         const Unit w = decode_unit(p, u);
         for (int n = w.n0; n < w.n1 && ok; ++n) {
           if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -266,13 +291,13 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
 #pragma unroll
             for (int kk = 0; kk < kBK / 16; ++kk) {
               // 16 bf16 = 32 bytes further along K inside the 128-byte swizzled row: +2 in 16-byte units
-              umma_bf16(d_tmem, a_desc + (uint64_t)(2 * kk), b_desc + (uint64_t)(2 * kk), idesc,
-                        (uint32_t)((k | kk) != 0));
+              umma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * kk), b_desc + (uint64_t)(2 * kk), idesc,
+                             (uint32_t)((k | kk) != 0));
             }
-            umma_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
+            umma_commit_pair(empty_bar(stage), 3);  // frees the stage in both CTAs once these MMAs have read it
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
-          if (ok) umma_commit(acc_full_bar(acc));
+          if (ok) umma_commit_pair(acc_full_bar(acc), 3);
           if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
         }
       }
@@ -286,9 +311,9 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
+    for (int u = pair; u < p.n_units && ok; u += n_pairs) {
       const Unit w = decode_unit(p, u);
-      const int row = w.m * kBM + quarter * 32 + lane;
+      const int row = w.m * kPairM + (int)cta * kBM + quarter * 32 + lane;
       const bool valid = row < p.T;
       RowNoise rn;
       RowStats st;
@@ -329,7 +354,7 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+        if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(acc), 0));
         if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
       }
       if (MODE != kModeDump && valid && ok) {
@@ -355,9 +380,13 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
   }
   tc_fence_before();
   __syncthreads();
+  // Neither CTA may leave while the other can still signal its barriers or while MMAs
+  // issued by the first CTA can still touch the partner's shared memory and TMEM.
+  cluster_arrive();
+  cluster_wait();
   if (warp == 2) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, kTmemCols);
+    tmem_dealloc_pair(tmem_base, kTmemCols);
   }
   if (threadIdx.x == 0 && *abort_flag && p.device_status != nullptr) *p.device_status = kStatusTimeout;
 }
@@ -368,9 +397,34 @@ static cudaError_t launch_mode(const CUtensorMap& th, const CUtensorMap& tw, con
                                cudaStream_t stream) {
   cudaError_t e = cudaFuncSetAttribute(k1_fused_score<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   if (e != cudaSuccess) return e;
-  k1_fused_score<MODE><<<grid, kThreads, kSmemBytes, stream>>>(th, tw, p);
+  k1_fused_score<MODE><<<grid, kThreads, kSmemBytes, stream>>>(th, tw, p);  // grid: two CTAs per pair
   return cudaGetLastError();
 }
+
+// Number of CTA pairs the device keeps resident at once (one CTA per SM, pairs on adjacent SMs).
+template <int MODE>
+static int max_pairs_mode() {
+  if (cudaFuncSetAttribute(k1_fused_score<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) !=
+      cudaSuccess)
+    return 0;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3(2 * 148, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = 2;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, k1_fused_score<MODE>, &cfg) != cudaSuccess) return 0;
+  return n;
+}
+
+int k1_max_resident_pairs() { return max_pairs_mode<kModeGm>(); }
 
 cudaError_t launch_k1(int mode, const CUtensorMap& tmap_h, const CUtensorMap& tmap_w, const K1Params& p, int grid,
                       cudaStream_t stream) {
