@@ -100,6 +100,7 @@ difr_status score_common(int ipt, const void* h, const void* W, const int32_t* t
   k1.tokens = tokens; k1.seeds = seeds; k1.positions = positions;
   k1.partials = reinterpret_cast<Partial*>(out->workspace);
   k1.device_status = out->device_status;
+  k1.unit_counter = reinterpret_cast<int*>(static_cast<unsigned char*>(out->workspace) + pl.partial_bytes);
   k1.T = (int)T; k1.d = (int)d; k1.V = (int)V;
   k1.T_pad = pl.T_pad; k1.m_tiles = pl.m_tiles; k1.n_tiles = pl.n_tiles; k1.k_steps = pl.k_steps;
   k1.S = pl.S; k1.Gm = pl.Gm; k1.n_units = pl.n_units;
@@ -107,6 +108,7 @@ difr_status score_common(int ipt, const void* h, const void* W, const int32_t* t
   k1.neg_tl2 = -temperature * 0.6931471805599453f;
   const int grid = 2 * (pl.n_units < info.pairs ? pl.n_units : info.pairs);
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
   if (out->event_fused_start && cudaEventRecord(reinterpret_cast<cudaEvent_t>(out->event_fused_start), s) != cudaSuccess)
     return DIFR_ERR_CUDA;
   if (launch_k1(ipt ? 1 : 0, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;

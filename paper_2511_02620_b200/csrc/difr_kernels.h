@@ -17,6 +17,7 @@ struct K1Params {
   Partial* partials;  // [n_slots][T_pad]
   float* logits_out;  // dump mode only
   int32_t* device_status;
+  int* unit_counter;  // zeroed before the launch: units are handed out in order on demand; null: round robin
   int T, d, V;
   int T_pad, m_tiles, n_tiles, k_steps;
   int S, Gm, n_units;

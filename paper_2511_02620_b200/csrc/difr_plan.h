@@ -21,7 +21,7 @@ struct Plan {
   int Gm;        // m tiles per raster group (units of a group run back to back)
   int n_units;   // m_tiles * S
   int T_pad;     // m_tiles * 256
-  int n_slots;   // partial records per row: 2 column halves per strip
+  int n_slots;   // partial records per row: one per strip
   size_t partial_bytes;
   size_t workspace_bytes;
 };
@@ -31,9 +31,14 @@ inline int env_int(const char* name, int fallback) {
   return (v && *v) ? atoi(v) : fallback;
 }
 
-// A unit walks its strip tile by tile keeping running statistics in registers,
-// so more strips mean more partial records but better balance over the SMs.
-// Pick the strip count that minimises the number of tiles on the critical path.
+// A unit walks its strip tile by tile keeping running statistics in registers and
+// leaves one partial record per (row, strip, column half).  Units are handed out in
+// raster order: groups of Gm row tiles, inside a group strip by strip, inside a strip
+// row tile by row tile.  The pairs that run at the same time therefore share Gm row
+// tiles of h (each re-read once per vocabulary tile) and stream the same few strips of
+// W.  Pairs on one strip start within about Gm * len / pairs tiles of one another, so a
+// W tile has to survive in L2 for that long: the strip length `len` and Gm are sized so
+// that the h tiles of a group plus the W tiles in flight stay within a part of L2.
 // `num_pairs` is the number of CTA pairs resident at once (one persistent pair per two SMs).
 inline bool make_plan(int64_t T, int64_t d, int64_t V, int num_pairs, Plan* out) {
   if (T <= 0 || d <= 0 || V < 2 || (d % 8) != 0) return false;
@@ -43,31 +48,45 @@ inline bool make_plan(int64_t T, int64_t d, int64_t V, int num_pairs, Plan* out)
   p.n_tiles = (int)((V + kBN - 1) / kBN);
   p.k_steps = (int)((d + kBK - 1) / kBK);
   if (num_pairs <= 0) num_pairs = 74;
-  int best_S = 1;
-  double best_cost = 1e300;
-  int max_S = p.n_tiles < 64 ? p.n_tiles : 64;
-  for (int S = 1; S <= max_S; ++S) {
-    long long units = (long long)p.m_tiles * S;
-    long long waves = (units + num_pairs - 1) / num_pairs;
-    long long len = (p.n_tiles + S - 1) / S;
-    double cost = (double)waves * (double)len + 0.25 * (double)waves;
-    if (cost < best_cost - 1e-9) {
-      best_cost = cost;
-      best_S = S;
+  // Measured on B200 (126 MB of L2): DRAM traffic is lowest with about 40 MB of h per raster group
+  // and strips of about eight tiles; larger groups push W out of L2 before its strip is done with it.
+  const double tile_bytes = 2.0 * kPairM * (double)d;  // one 256-row tile of h or of W
+  const double group_bytes = (double)env_int("DIFR_DEBUG_L2_MB", 40) * 1048576.0;
+  int gm = (int)(group_bytes / tile_bytes);
+  if (gm < 4) gm = 4;
+  int len_target = 8;
+  if (len_target > p.n_tiles) len_target = p.n_tiles;
+  // strip count: n_tiles / len_target when there are many rounds of units; otherwise the count
+  // near it (or, for small problems, up to one unit per pair) with the fewest tiles on the critical path
+  int best_S = (p.n_tiles + len_target - 1) / len_target;
+  if ((long long)p.m_tiles * best_S < 8LL * num_pairs) {
+    int s_lo = (2 * p.n_tiles + 3 * len_target - 1) / (3 * len_target);
+    int s_hi = (4 * p.n_tiles + 3 * len_target - 1) / (3 * len_target);
+    if (s_hi < num_pairs / p.m_tiles) s_hi = num_pairs / p.m_tiles;
+    if (s_hi > p.n_tiles) s_hi = p.n_tiles;
+    if (s_lo < 1) s_lo = 1;
+    if (s_lo > s_hi) s_lo = s_hi;
+    double best_cost = 1e300;
+    for (int S = s_lo; S <= s_hi; ++S) {
+      long long units = (long long)p.m_tiles * S;
+      long long waves = (units + num_pairs - 1) / num_pairs;
+      long long len = (p.n_tiles + S - 1) / S;
+      double cost = (double)waves * (double)len + 0.25 * (double)waves;
+      if (cost < best_cost - 1e-9) {
+        best_cost = cost;
+        best_S = S;
+      }
     }
   }
   p.S = env_int("DIFR_DEBUG_STRIPS", best_S);
   if (p.S < 1) p.S = 1;
   if (p.S > p.n_tiles) p.S = p.n_tiles;
-  // Units of one raster group share their W tiles through L2 while each keeps
-  // its own h tile resident: bound the group's h footprint to a few tens of MB.
-  int gm = (d <= 2560) ? 37 : 19;
   gm = env_int("DIFR_DEBUG_GROUP", gm);
   if (gm < 1) gm = 1;
   p.Gm = gm < p.m_tiles ? gm : p.m_tiles;
   p.n_units = p.m_tiles * p.S;
   p.T_pad = p.m_tiles * kPairM;
-  p.n_slots = 2 * p.S;
+  p.n_slots = p.S;
   p.partial_bytes = (size_t)p.n_slots * (size_t)p.T_pad * 32;
   p.workspace_bytes = p.partial_bytes + 256;
   *out = p;

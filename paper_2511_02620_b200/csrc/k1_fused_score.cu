@@ -17,12 +17,14 @@
 // memory instead of the 48 KB a lone 128 x 256 tile needs.
 //
 // Warp roles in each CTA: warp 0 issues the TMA loads, warp 1 (first CTA only)
-// issues the MMAs, warp 2 owns the TMEM allocation, warps 4..11 are the epilogue
-// (two warpgroups, one per 128-column half of the CTA's 128 x 256 accumulator).
-// Two accumulator stages (all 512 TMEM columns) let the epilogue of tile n
-// overlap the MMAs of tile n + 1.  A work unit is (256-row tile, vocabulary
-// strip); its running statistics stay in registers across the strip and leave
-// as one 32-byte partial record per (row, strip, column half).
+// issues the MMAs, warp 2 owns the TMEM allocation, warp 3 (first CTA only)
+// hands out work units, warps 4..19 are the epilogue: warp 4 + 4 g + q reads TMEM
+// lanes 32 q .. 32 q + 31 (rows) and columns 64 g .. 64 g + 63 of the CTA's
+// 128 x 256 accumulator.  Two accumulator stages (all 512 TMEM columns) let the
+// epilogue of tile n overlap the MMAs of tile n + 1.  A work unit is (256-row
+// tile, vocabulary strip); its running statistics stay in registers across the
+// strip, the four column groups of a row are merged through shared memory at
+// the end of the unit and leave as one 32-byte partial record per (row, strip).
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <math_constants.h>
@@ -39,13 +41,21 @@ constexpr int kABytes = kBM * kBK * 2;         // 16 KB: this CTA's 128 rows of 
 constexpr int kBBytes = (kBN / 2) * kBK * 2;   // 16 KB: this CTA's 128 of the tile's 256 rows of W
 constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kAccStages = 2;
-constexpr int kThreads = 384;
 constexpr int kEpiWarp0 = 4;
-constexpr int kEpiWarps = 8;
+constexpr int kColGroups = 4;                  // 64-column groups of the CTA's accumulator tile
+constexpr int kEpiWarps = 4 * kColGroups;
+constexpr int kThreads = 32 * (kEpiWarp0 + kEpiWarps);
+constexpr int kSub = 16;                       // vocabulary ids per TMEM load
+constexpr int kSubsPerTile = (kBN / kColGroups) / kSub;
+constexpr int kRoleRegs = 32, kEpiRegs = 112;  // 32 * 128 + 112 * 512 = 96 * 640 registers
 constexpr int kTmemCols = 512;
-constexpr int kBarBytes = 256;
-constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + 1024;  // + slack for 1024-byte alignment
+constexpr int kSchedSlots = 2;                 // unit ids handed out ahead of their use
+constexpr int kSchedReaders = 2 + 1 + 2 * kEpiWarps;  // per pair: two TMA threads, the MMA thread, the epilogue warps
+constexpr int kBarBytes = 512;
+constexpr int kXchBytes = (kColGroups - 1) * kBM * 32;  // statistics of column groups 1..3 on their way to group 0
+constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + kXchBytes + 1024;  // + slack for 1024-byte alignment
 constexpr float kMasked = -3.0e38f;  // stands in for -inf on padded vocabulary columns (keeps keys finite)
+static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one CTA");
 
 enum : int { kModeGm = 0, kModeIpt = 1, kModeDump = 2 };
 
@@ -69,37 +79,44 @@ __device__ __forceinline__ Unit decode_unit(const K1Params& p, int u) {
 
 // ---------------------------------------------------------- running statistics
 struct RowStats {
-  float m1, m2;        // top-2 keys of y' (low 5 mantissa bits carry the column within its chunk)
-  int i1, i2;          // their vocabulary ids
-  float lmax;          // running max of z = l * c1
-  float lsum, lsum_c;  // compensated sum of 2^(z - lmax)
-  float lpre, lpre_c;  // the same restricted to ids below the claimed one
+  float m1, m2;  // top-2 keys of y' (low 4 mantissa bits carry the column within its 16-id group)
+  int i1, i2;    // their vocabulary ids
+  float lmax;    // running max of z = l * c1
+  float lsum;    // sum of 2^(z - lmax)
+  float lpre;    // the same restricted to ids below the claimed one
 };
 
 __device__ __forceinline__ void stats_init(RowStats& s) {
   s.m1 = s.m2 = -CUDART_INF_F;
   s.i1 = s.i2 = -1;
   s.lmax = -CUDART_INF_F;
-  s.lsum = s.lsum_c = s.lpre = s.lpre_c = 0.f;
+  s.lsum = s.lpre = 0.f;
 }
 
-// sum += x with the rounding error carried in comp (Neumaier).
-__device__ __forceinline__ void comp_add(float& sum, float& comp, float x) {
-  float t = sum + x;
-  comp += (fabsf(sum) >= fabsf(x)) ? ((sum - t) + x) : ((x - t) + sum);
-  sum = t;
+// (k1, j1), (k2, j2): the best two of another column group of the same row, k1 >= k2.
+__device__ __forceinline__ void top2_merge(RowStats& s, float k1, int j1, float k2, int j2) {
+  if (k1 > s.m1) {
+    const bool q = k2 > s.m1;
+    s.m2 = q ? k2 : s.m1;
+    s.i2 = q ? j2 : s.i1;
+    s.m1 = k1;
+    s.i1 = j1;
+  } else if (k1 > s.m2) {
+    s.m2 = k1;
+    s.i2 = j1;
+  }
 }
 
-// One chunk of 32 consecutive vocabulary ids [base, base + 32) of one row.
+// 16 consecutive vocabulary ids [base, base + 16) of one row.
 template <int MODE>
-__device__ __forceinline__ void process_chunk(uint32_t (&raw)[32], int base, int V, int tok, float c1,
-                                              float neg_tl2, const RowNoise& rn, RowStats& s) {
-  float l[32];
+__device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base, int V, int tok, float c1,
+                                          float neg_tl2, const RowNoise& rn, RowStats& s) {
+  float l[kSub];
 #pragma unroll
-  for (int j = 0; j < 32; ++j) l[j] = __uint_as_float(raw[j]);
-  if (base + 32 > V) {  // padded columns of the last tile (uniform over the warp)
+  for (int j = 0; j < kSub; ++j) l[j] = __uint_as_float(raw[j]);
+  if (base + kSub > V) {  // padded columns of the last tile (uniform over the warp)
 #pragma unroll
-    for (int j = 0; j < 32; ++j)
+    for (int j = 0; j < kSub; ++j)
       if (base + j >= V) l[j] = kMasked;
   }
 
@@ -107,33 +124,35 @@ __device__ __forceinline__ void process_chunk(uint32_t (&raw)[32], int base, int
   {
     float cm = fmax3(l[0], l[1], l[2]);
 #pragma unroll
-    for (int j = 3; j + 1 < 32; j += 2) cm = fmax3(cm, l[j], l[j + 1]);
-    cm = fmaxf(cm, l[31]);
-    const float new_max = fmaxf(s.lmax, cm * c1);
-    const float scale = ex2_approx(s.lmax - new_max);  // 0 on the first chunk
-    s.lsum *= scale; s.lsum_c *= scale;
-    s.lpre *= scale; s.lpre_c *= scale;
-    s.lmax = new_max;
-    const float shift = -new_max;
+    for (int j = 3; j + 1 < kSub; j += 2) cm = fmax3(cm, l[j], l[j + 1]);
+    cm = fmaxf(cm, l[kSub - 1]);
+    const float zmax = cm * c1;
+    if (zmax > s.lmax) {  // rare after the first few groups of a strip
+      const float scale = ex2_approx(s.lmax - zmax);  // 0 on the first group
+      s.lsum *= scale;
+      s.lpre *= scale;
+      s.lmax = zmax;
+    }
+    const float shift = -s.lmax;
     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-    for (int j = 0; j < 32; j += 4) {
+    for (int j = 0; j < kSub; j += 4) {
       a0 += ex2_approx(fmaf(l[j + 0], c1, shift));
       a1 += ex2_approx(fmaf(l[j + 1], c1, shift));
       a2 += ex2_approx(fmaf(l[j + 2], c1, shift));
       a3 += ex2_approx(fmaf(l[j + 3], c1, shift));
     }
     const float cs = (a0 + a1) + (a2 + a3);
-    comp_add(s.lsum, s.lsum_c, cs);
-    const int tl = tok - base;  // ids below the claimed one: all, none, or the first tl of this chunk
-    if (tl >= 32) {
-      comp_add(s.lpre, s.lpre_c, cs);
+    s.lsum += cs;
+    const int tl = tok - base;  // ids below the claimed one: all, none, or the first tl of this group
+    if (tl >= kSub) {
+      s.lpre += cs;
     } else if (tl > 0) {
       float ps = 0.f;
 #pragma unroll
-      for (int j = 0; j < 32; ++j)
+      for (int j = 0; j < kSub; ++j)
         if (j < tl) ps += ex2_approx(fmaf(l[j], c1, shift));
-      comp_add(s.lpre, s.lpre_c, ps);
+      s.lpre += ps;
     }
   }
 
@@ -141,7 +160,7 @@ __device__ __forceinline__ void process_chunk(uint32_t (&raw)[32], int base, int
   if (MODE == kModeGm) {
     float c1k = -CUDART_INF_F, c2k = -CUDART_INF_F;
 #pragma unroll
-    for (int j = 0; j < 32; j += 4) {
+    for (int j = 0; j < kSub; j += 4) {
       uint32_t x[4];
       row_noise_block(rn, (uint32_t)(base + j) >> 2, x);
       float key[4];
@@ -150,7 +169,7 @@ __device__ __forceinline__ void process_chunk(uint32_t (&raw)[32], int base, int
         const float u = __uint_as_float(0x3F800000u | (x[q] >> 9)) - 0.99999994f;  // ((x>>9) + 1/2) 2^-23, exact
         const float e2 = -lg2_approx(u);                                           // -log2 u = E / ln 2
         const float y = fmaf(lg2_approx(e2), neg_tl2, l[j + q]);
-        key[q] = __uint_as_float((__float_as_uint(y) & ~31u) | (uint32_t)(j + q));
+        key[q] = __uint_as_float((__float_as_uint(y) & ~15u) | (uint32_t)(j + q));
       }
       // u within 2^-11 of one: -log2 u loses relative accuracy, redo those with a series for -ln(1 - w)
       const uint32_t xm = max(max(x[0], x[1]), max(x[2], x[3]));
@@ -161,7 +180,7 @@ __device__ __forceinline__ void process_chunk(uint32_t (&raw)[32], int base, int
             const float w = __uint_as_float(0x3F800000u | ((~x[q]) >> 9)) - 0.99999994f;  // 1 - u, exact
             const float E = w * fmaf(w, fmaf(w, 0.33333334f, 0.5f), 1.0f);
             const float y = fmaf(lg2_approx(E * 1.4426950408889634f), neg_tl2, l[j + q]);
-            key[q] = __uint_as_float((__float_as_uint(y) & ~31u) | (uint32_t)(j + q));
+            key[q] = __uint_as_float((__float_as_uint(y) & ~15u) | (uint32_t)(j + q));
           }
         }
       }
@@ -173,19 +192,8 @@ __device__ __forceinline__ void process_chunk(uint32_t (&raw)[32], int base, int
       c1k = fmaxf(c1k, t1);
       c2k = n2;
     }
-    // merge the chunk's top-2 into the running top-2 (earlier ids win ties)
-    const int g1 = base + (int)(__float_as_uint(c1k) & 31u);
-    const int g2 = base + (int)(__float_as_uint(c2k) & 31u);
-    if (c1k > s.m1) {
-      const bool q = c2k > s.m1;
-      s.m2 = q ? c2k : s.m1;
-      s.i2 = q ? g2 : s.i1;
-      s.m1 = c1k;
-      s.i1 = g1;
-    } else if (c1k > s.m2) {
-      s.m2 = c1k;
-      s.i2 = g1;
-    }
+    // merge the group's top-2 into the running top-2 (earlier ids win ties)
+    top2_merge(s, c1k, base + (int)(__float_as_uint(c1k) & 15u), c2k, base + (int)(__float_as_uint(c2k) & 15u));
   }
 }
 
@@ -199,18 +207,31 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
   uint8_t* smem = smem_raw + (smem_base - raw_addr);
 
   // Both CTAs of a pair lay out their barriers at the same offsets.
-  //   full[s]      first CTA's copy is used: 1 arrival (its producer) + the bytes of both CTAs' loads
-  //   empty[s]     each CTA's own copy: 1 arrival, the MMA thread's commit delivered to both CTAs
-  //   acc_full[a]  each CTA's own copy: 1 arrival, the commit after a tile's last MMA, delivered to both
-  //   acc_empty[a] first CTA's copy is used: one arrival per epilogue warp of both CTAs
+  //   full[s]        first CTA's copy is used: 1 arrival (its producer) + the bytes of both CTAs' loads
+  //   empty[s]       each CTA's own copy: 1 arrival, the MMA thread's commit delivered to both CTAs
+  //   acc_full[a]    each CTA's own copy: 1 arrival, the commit after a tile's last MMA, delivered to both
+  //   acc_empty[a]   first CTA's copy is used: one arrival per epilogue warp of both CTAs
+  //   sched_full[q]  each CTA's own copy: 1 arrival, the scheduler thread's, after it wrote unit id q
+  //   sched_empty[q] first CTA's copy is used: one arrival per reader of the pair
+  //   xch_full[r]    own: column groups 1..3 of lane quarter r have written their statistics (3 arrivals)
+  //   xch_empty[r]   own: column group 0 of lane quarter r has read them (1 arrival)
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
   const uint32_t bar0 = smem_base + kStages * kStageBytes;
+  constexpr int kBarAcc = 2 * kStages, kBarSched = kBarAcc + 2 * kAccStages, kBarXch = kBarSched + 2 * kSchedSlots,
+                kBarEnd = kBarXch + 8;
+  static_assert(kBarEnd * 8 + 16 + 4 * kSchedSlots <= kBarBytes, "barrier block");
   auto full_bar = [&](int s) { return bar0 + 8u * (uint32_t)s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (uint32_t)(kStages + s); };
-  auto acc_full_bar = [&](int a) { return bar0 + 8u * (uint32_t)(2 * kStages + a); };
-  auto acc_empty_bar = [&](int a) { return bar0 + 8u * (uint32_t)(2 * kStages + kAccStages + a); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 2 * kAccStages);
+  auto acc_full_bar = [&](int a) { return bar0 + 8u * (uint32_t)(kBarAcc + a); };
+  auto acc_empty_bar = [&](int a) { return bar0 + 8u * (uint32_t)(kBarAcc + kAccStages + a); };
+  auto sched_full_bar = [&](int q) { return bar0 + 8u * (uint32_t)(kBarSched + q); };
+  auto sched_empty_bar = [&](int q) { return bar0 + 8u * (uint32_t)(kBarSched + kSchedSlots + q); };
+  auto xch_full_bar = [&](int r) { return bar0 + 8u * (uint32_t)(kBarXch + r); };
+  auto xch_empty_bar = [&](int r) { return bar0 + 8u * (uint32_t)(kBarXch + 4 + r); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kBarEnd);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* sched_unit = reinterpret_cast<volatile int*>(tmem_slot + 2);  // [kSchedSlots]
+  float4* xch = reinterpret_cast<float4*>(smem + kStages * kStageBytes + kBarBytes);  // [3][128 rows][2]
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -226,6 +247,14 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     for (int a = 0; a < kAccStages; ++a) {
       mbar_init(acc_full_bar(a), 1);
       mbar_init(acc_empty_bar(a), 2 * kEpiWarps);
+    }
+    for (int q = 0; q < kSchedSlots; ++q) {
+      mbar_init(sched_full_bar(q), 1);
+      mbar_init(sched_empty_bar(q), kSchedReaders);
+    }
+    for (int r = 0; r < 4; ++r) {
+      mbar_init(xch_full_bar(r), kColGroups - 1);
+      mbar_init(xch_empty_bar(r), 1);
     }
     *abort_flag = 0;
     mbar_fence_init();
@@ -243,16 +272,61 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 0) {
+  // Work units reach every role of the pair through a small ring of unit ids that the
+  // scheduler thread (warp 3 of the first CTA) fills in both CTAs.  -1 ends the kernel.
+  auto next_unit = [&](int& slot, uint32_t& phase, bool one_lane_arrives) -> int {
+    if (!mbar_wait(sched_full_bar(slot), phase, abort_flag)) return -1;
+    const int u = sched_unit[slot];
+    if (one_lane_arrives) {
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(sched_empty_bar(slot), 0));
+    } else {
+      mbar_arrive_cluster(map_to_cta(sched_empty_bar(slot), 0));
+    }
+    if (++slot == kSchedSlots) { slot = 0; phase ^= 1u; }
+    return u;
+  };
+
+  // The four single-thread roles need few registers; the rest goes to the epilogue warpgroups.
+  if (warp < kEpiWarp0) {
+  setmaxnreg_dec<kRoleRegs>();
+  if (warp == 3) {
+    // --------------------------------------------------------------- scheduler
+    // Units are taken from a global counter in raster order, so the pairs that run at
+    // the same time work on neighbouring units (the same rows of W at about the same
+    // moment) however far their speeds drift apart.  Without a counter: round robin.
+    if (cta == 0 && lane == 0) {
+      int slot = 0, i = 0;
+      uint32_t phase = 0;
+      while (true) {
+        if (!mbar_wait(sched_empty_bar(slot), phase ^ 1u, abort_flag)) break;
+        int u = (p.unit_counter != nullptr) ? atomicAdd(p.unit_counter, 1) : pair + i * n_pairs;
+        ++i;
+        if (u >= p.n_units) u = -1;
+        sched_unit[slot] = u;
+        st_shared_cluster_u32(map_to_cta(smem_u32(const_cast<int*>(&sched_unit[slot])), 1), (uint32_t)u);
+        mbar_arrive_cluster(map_to_cta(sched_full_bar(slot), 0));
+        mbar_arrive_cluster(map_to_cta(sched_full_bar(slot), 1));
+        if (u < 0) break;
+        if (++slot == kSchedSlots) { slot = 0; phase ^= 1u; }
+      }
+    }
+  } else if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      // a CTA re-reads its h tile for every vocabulary tile of the strip: keep it in L2;
-      // a W tile is read by the pairs of one raster group at about the same time, then never again soon
-      const uint64_t keep = l2_policy_evict_last(), stream = l2_policy_evict_first();
+      // a CTA re-reads its h tile for every vocabulary tile of the strip, and the other strips of the
+      // raster group read it too: ask L2 to keep it.  A W tile is wanted by every pair of its strip within
+      // a few tile times and then not for a long while: ordinary priority (marking it evict-first loses it
+      // before the last pair of the strip has come by).
+      const uint64_t keep = l2_policy_evict_last(), stream = l2_policy_evict_normal();
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int u = pair; u < p.n_units && ok; u += n_pairs) {
+      int uslot = 0;
+      uint32_t uphase = 0;
+      while (ok) {
+        const int u = next_unit(uslot, uphase, false);
+        if (u < 0) break;
         const Unit w = decode_unit(p, u);
         const int row0 = w.m * kPairM + (int)cta * kBM;
         for (int n = w.n0; n < w.n1 && ok; ++n) {
@@ -276,7 +350,11 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int u = pair; u < p.n_units && ok; u += n_pairs) {
+      int uslot = 0;
+      uint32_t uphase = 0;
+      while (ok) {
+        const int u = next_unit(uslot, uphase, false);
+        if (u < 0) break;
         const Unit w = decode_unit(p, u);
         for (int n = w.n0; n < w.n1 && ok; ++n) {
           if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -302,18 +380,25 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
         }
       }
     }
-  } else if (warp >= kEpiWarp0) {
+  }
+  } else {
     // ---------------------------------------------------------------- epilogue
+    setmaxnreg_inc<kEpiRegs>();
     const int ew = warp - kEpiWarp0;
     const int quarter = ew & 3;  // == warp % 4: the TMEM lane quarter this warp may read
-    const int half = ew >> 2;    // which 128 columns of the tile
+    const int colg = ew >> 2;    // which 64 columns of the tile
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    const int row_in_cta = quarter * 32 + lane;
     int acc = 0;
-    uint32_t acc_phase = 0;
+    uint32_t acc_phase = 0, xch_phase = 0;
     bool ok = true;
-    for (int u = pair; u < p.n_units && ok; u += n_pairs) {
+    int uslot = 0;
+    uint32_t uphase = 0;
+    while (ok) {
+      const int u = next_unit(uslot, uphase, true);
+      if (u < 0) break;
       const Unit w = decode_unit(p, u);
-      const int row = w.m * kPairM + (int)cta * kBM + quarter * 32 + lane;
+      const int row = w.m * kPairM + (int)cta * kBM + row_in_cta;
       const bool valid = row < p.T;
       RowNoise rn;
       RowStats st;
@@ -332,24 +417,31 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
       for (int n = w.n0; n < w.n1; ++n) {
         if (!mbar_wait(acc_full_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const int col0 = n * kBN + half * (kBN / 2);
-#pragma unroll 1
-        for (int c = 0; c < (kBN / 2) / 32; ++c) {
-          const int base = col0 + c * 32;
-          if (base >= p.V) break;
-          uint32_t raw[32];
-          __syncwarp();
-          tmem_ld_32x32(tmem_base + lane_addr + (uint32_t)(acc * kBN + half * (kBN / 2) + c * 32), raw);
-          tmem_ld_wait();
-          if (MODE == kModeDump) {
-            if (valid) {
-              float* dst = p.logits_out + (size_t)row * (size_t)p.V + base;
+        const int col0 = n * kBN + colg * (kBN / kColGroups);
+        if (col0 < p.V) {  // uniform over the warp
+          // two register buffers: the load of the next 16 columns is in flight while these are processed
+          const uint32_t t0 = tmem_base + lane_addr + (uint32_t)(acc * kBN + colg * (kBN / kColGroups));
+          uint32_t buf0[kSub], buf1[kSub];
+          tmem_ld_32x16(t0, buf0);
 #pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (base + j < p.V) dst[j] = __uint_as_float(raw[j]);
+          for (int i = 0; i < kSubsPerTile; ++i) {
+            uint32_t (&cur)[kSub] = (i & 1) ? buf1 : buf0;
+            uint32_t (&nxt)[kSub] = (i & 1) ? buf0 : buf1;
+            tmem_ld_wait(cur);
+            const bool more = (i + 1 < kSubsPerTile) && (col0 + (i + 1) * kSub < p.V);
+            if (more) tmem_ld_32x16(t0 + (uint32_t)((i + 1) * kSub), nxt);
+            const int base = col0 + i * kSub;
+            if (MODE == kModeDump) {
+              if (valid) {
+                float* dst = p.logits_out + (size_t)row * (size_t)p.V + base;
+#pragma unroll
+                for (int j = 0; j < kSub; ++j)
+                  if (base + j < p.V) dst[j] = __uint_as_float(cur[j]);
+              }
+            } else {
+              process16<MODE>(cur, base, p.V, tok, p.c1, p.neg_tl2, rn, st);
             }
-          } else {
-            process_chunk<MODE>(raw, base, p.V, tok, p.c1, p.neg_tl2, rn, st);
+            if (!more) break;
           }
         }
         tc_fence_before();
@@ -357,17 +449,39 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
         if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(acc), 0));
         if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
       }
-      if (MODE != kModeDump && valid && ok) {
-        Partial out;
-        out.m1 = st.m1; out.i1 = st.i1; out.m2 = st.m2; out.i2 = st.i2;
-        out.lse2_max = st.lmax;
-        out.lse2_sum = st.lsum + st.lsum_c;
-        out.prefix2 = st.lpre + st.lpre_c;
-        out.reserved = 0.f;
-        Partial* dst = p.partials + (size_t)(w.strip * 2 + half) * (size_t)p.T_pad + row;
-        const float4* src = reinterpret_cast<const float4*>(&out);
-        reinterpret_cast<float4*>(dst)[0] = src[0];
-        reinterpret_cast<float4*>(dst)[1] = src[1];
+      if (MODE != kModeDump && ok) {
+        // the four column groups of a row meet in shared memory; group 0 merges and writes the record
+        if (colg != 0) {
+          if (!mbar_wait(xch_empty_bar(quarter), xch_phase ^ 1u, abort_flag)) { ok = false; break; }
+          float4* dst = xch + ((size_t)(colg - 1) * kBM + row_in_cta) * 2;
+          dst[0] = make_float4(st.m1, __int_as_float(st.i1), st.m2, __int_as_float(st.i2));
+          dst[1] = make_float4(st.lmax, st.lsum, st.lpre, 0.f);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(xch_full_bar(quarter));
+        } else {
+          if (!mbar_wait(xch_full_bar(quarter), xch_phase, abort_flag)) { ok = false; break; }
+#pragma unroll
+          for (int g = 0; g < kColGroups - 1; ++g) {
+            const float4* src = xch + ((size_t)g * kBM + row_in_cta) * 2;
+            const float4 a = src[0], b = src[1];
+            top2_merge(st, a.x, __float_as_int(a.y), a.z, __float_as_int(a.w));
+            if (b.x > -CUDART_INF_F) {  // that group saw columns
+              const float m = fmaxf(st.lmax, b.x);
+              const float fa = ex2_approx(st.lmax - m), fb = ex2_approx(b.x - m);
+              st.lsum = st.lsum * fa + b.y * fb;
+              st.lpre = st.lpre * fa + b.z * fb;
+              st.lmax = m;
+            }
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(xch_empty_bar(quarter));
+          if (valid) {
+            float4* dst = reinterpret_cast<float4*>(p.partials + (size_t)w.strip * (size_t)p.T_pad + row);
+            dst[0] = make_float4(st.m1, __int_as_float(st.i1), st.m2, __int_as_float(st.i2));
+            dst[1] = make_float4(st.lmax, st.lsum, st.lpre, 0.f);
+          }
+        }
+        xch_phase ^= 1u;
       }
     }
   }

@@ -30,9 +30,10 @@ def test_host_only_entry_points():
     assert difr.difr_status_string(0) == "ok"
     assert "workspace" in difr.difr_status_string(-4)
     assert difr.difr_status_string(-7)
-    # plan-derived sizes: 32-byte records, two column halves per strip, rows padded to 128
+    # plan-derived sizes: one 32-byte record per (row, strip), rows padded to 256, plus a 256-byte tail
     nbytes = difr.difr_workspace_bytes(4096, 3072, 128256)
-    assert nbytes > 0 and (nbytes - 256) % (32 * 2 * 4096) == 0
+    assert nbytes > 0 and (nbytes - 256) % (32 * 4096) == 0
+    assert (difr.difr_workspace_bytes(4097, 3072, 128256) - 256) % (32 * (4096 + 256)) == 0
     assert difr.difr_workspace_bytes(4096, 3076, 128256) == 0  # d not a multiple of 8
     assert difr.difr_workspace_bytes(4096, 3072, 1) == 0
     assert difr.difr_workspace_bytes(0, 3072, 128256) == 0
