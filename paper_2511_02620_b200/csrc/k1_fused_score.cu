@@ -319,6 +319,7 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
       // a few tile times and then not for a long while: ordinary priority (marking it evict-first loses it
       // before the last pair of the strip has come by).
       const uint64_t keep = l2_policy_evict_last(), stream = l2_policy_evict_normal();
+      const uint32_t full0_base = map_to_cta(full_bar(0), 0);  // the first CTA's full[0] as seen from either CTA
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -334,7 +335,7 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
           for (int k = 0; k < p.k_steps; ++k) {
             if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
             if (cta == 0) mbar_arrive_expect_tx(full_bar(stage), 2u * kStageBytes);
-            const uint32_t full0 = map_to_cta(full_bar(stage), 0);
+            const uint32_t full0 = full0_base + 8u * (uint32_t)stage;
             const uint32_t a_dst = smem_base + (uint32_t)stage * kStageBytes;
             tma_load_2d_pair(a_dst, &tmap_h, k * kBK, row0, full0, keep);
             tma_load_2d_pair(a_dst + kABytes, &tmap_w, k * kBK, wrow0, full0, stream);
@@ -347,6 +348,10 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     // -------------------------------------------------------------- MMA issuer
     if (cta == 0 && lane == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16(kPairM, kBN);
+      // The descriptors of a stage differ from those of stage 0 only in the 14-bit address field
+      // (units of 16 bytes), which never carries out of the field: shared memory ends below 256 KB.
+      const uint64_t desc0 = umma_desc_k_major_sw128(smem_base);
+      const uint32_t desc_hi = (uint32_t)(desc0 >> 32), desc_lo0 = (uint32_t)desc0;
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
@@ -360,17 +365,18 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
           if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kBN);
+          uint32_t accumulate = 0;
           for (int k = 0; k < p.k_steps; ++k) {
             if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t a_src = smem_base + (uint32_t)stage * kStageBytes;
-            const uint64_t a_desc = umma_desc_k_major_sw128(a_src);
-            const uint64_t b_desc = umma_desc_k_major_sw128(a_src + kABytes);
+            const uint32_t a_lo = desc_lo0 + (uint32_t)stage * (kStageBytes >> 4);
 #pragma unroll
             for (int kk = 0; kk < kBK / 16; ++kk) {
               // 16 bf16 = 32 bytes further along K inside the 128-byte swizzled row: +2 in 16-byte units
-              umma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * kk), b_desc + (uint64_t)(2 * kk), idesc,
-                             (uint32_t)((k | kk) != 0));
+              const uint64_t a_desc = ((uint64_t)desc_hi << 32) | (a_lo + 2u * kk);
+              const uint64_t b_desc = ((uint64_t)desc_hi << 32) | (a_lo + (kABytes >> 4) + 2u * kk);
+              umma_bf16_pair(d_tmem, a_desc, b_desc, idesc, accumulate);
+              accumulate = 1;
             }
             umma_commit_pair(empty_bar(stage), 3);  // frees the stage in both CTAs once these MMAs have read it
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
