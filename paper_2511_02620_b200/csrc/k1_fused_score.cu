@@ -134,15 +134,17 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
       s.lmax = zmax;
     }
     const float shift = -s.lmax;
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    const float2 c1_2 = make_float2(c1, c1), shift2 = make_float2(shift, shift);
+    float2 a01 = make_float2(0.f, 0.f), a23 = make_float2(0.f, 0.f);
 #pragma unroll
     for (int j = 0; j < kSub; j += 4) {
-      a0 += ex2_approx(fmaf(l[j + 0], c1, shift));
-      a1 += ex2_approx(fmaf(l[j + 1], c1, shift));
-      a2 += ex2_approx(fmaf(l[j + 2], c1, shift));
-      a3 += ex2_approx(fmaf(l[j + 3], c1, shift));
+      const float2 z01 = ffma2(make_float2(l[j + 0], l[j + 1]), c1_2, shift2);
+      const float2 z23 = ffma2(make_float2(l[j + 2], l[j + 3]), c1_2, shift2);
+      a01 = fadd2(a01, make_float2(ex2_approx(z01.x), ex2_approx(z01.y)));
+      a23 = fadd2(a23, make_float2(ex2_approx(z23.x), ex2_approx(z23.y)));
     }
-    const float cs = (a0 + a1) + (a2 + a3);
+    const float2 a = fadd2(a01, a23);
+    const float cs = a.x + a.y;
     s.lsum += cs;
     const int tl = tok - base;  // ids below the claimed one: all, none, or the first tl of this group
     if (tl >= kSub) {
@@ -164,12 +166,16 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
       uint32_t x[4];
       row_noise_block(rn, (uint32_t)(base + j) >> 2, x);
       float key[4];
+      const float2 minus1 = make_float2(-0.99999994f, -0.99999994f), ntl2 = make_float2(neg_tl2, neg_tl2);
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const float u = __uint_as_float(0x3F800000u | (x[q] >> 9)) - 0.99999994f;  // ((x>>9) + 1/2) 2^-23, exact
-        const float e2 = -lg2_approx(u);                                           // -log2 u = E / ln 2
-        const float y = fmaf(lg2_approx(e2), neg_tl2, l[j + q]);
-        key[q] = __uint_as_float((__float_as_uint(y) & ~15u) | (uint32_t)(j + q));
+      for (int q = 0; q < 4; q += 2) {
+        // u = ((x >> 9) + 1/2) 2^-23, exact;  -log2 u = E / ln 2;  y' = l - Temp ln2 log2(E / ln 2)
+        const float2 u = fadd2(make_float2(__uint_as_float(0x3F800000u | (x[q] >> 9)),
+                                           __uint_as_float(0x3F800000u | (x[q + 1] >> 9))), minus1);
+        const float2 g = make_float2(lg2_approx(-lg2_approx(u.x)), lg2_approx(-lg2_approx(u.y)));
+        const float2 y = ffma2(g, ntl2, make_float2(l[j + q], l[j + q + 1]));
+        key[q] = __uint_as_float((__float_as_uint(y.x) & ~15u) | (uint32_t)(j + q));
+        key[q + 1] = __uint_as_float((__float_as_uint(y.y) & ~15u) | (uint32_t)(j + q + 1));
       }
       // u within 2^-11 of one: -log2 u loses relative accuracy, redo those with a series for -ln(1 - w)
       const uint32_t xm = max(max(x[0], x[1]), max(x[2], x[3]));
@@ -279,9 +285,9 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     const int u = sched_unit[slot];
     if (one_lane_arrives) {
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(map_to_cta(sched_empty_bar(slot), 0));
+      if (lane == 0) mbar_arrive_cluster_nofence(map_to_cta(sched_empty_bar(slot), 0));
     } else {
-      mbar_arrive_cluster(map_to_cta(sched_empty_bar(slot), 0));
+      mbar_arrive_cluster_nofence(map_to_cta(sched_empty_bar(slot), 0));
     }
     if (++slot == kSchedSlots) { slot = 0; phase ^= 1u; }
     return u;
@@ -452,7 +458,7 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(acc), 0));
+        if (lane == 0) mbar_arrive_cluster_nofence(map_to_cta(acc_empty_bar(acc), 0));
         if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
       }
       if (MODE != kModeDump && ok) {
