@@ -34,7 +34,7 @@ UNIT = "tokens/s"
 L2_BYTES = 126 * 2**20
 # dram__bytes_read.sum + dram__bytes_write.sum of the fused kernel per launch, from the
 # ncu captures summarised under profiles/ (bytes; None until captured for that workload)
-FUSED_TRAFFIC = {"llama3b": 953.9e6}  # profiles/k1_fused_score_llama3b.md
+FUSED_TRAFFIC = {"llama3b": 893.6e6}  # profiles/k1_fused_score_llama3b.md
 
 
 def load_peaks():
@@ -395,11 +395,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama3b", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--T", type=int, default=0, help="override the number of rows (whole sequences)")
-    ap.add_argument("--temperature", type=float, default=1.0)
+    ap.add_argument("--temperature", type=float, default=None,
+                    help="sampling temperature (default: the workload's own, its last listed one)")
     ap.add_argument("--sigma", type=float, default=0.05)
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.temperature is None:
+        args.temperature = float(wl.WORKLOADS[args.workload].temperatures[-1])
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
