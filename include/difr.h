@@ -153,8 +153,9 @@ difr_status difr_score_ipt(const void* h, const void* W, const int32_t* tokens, 
  *     device must be current); make that first call before starting any stream
  *     capture.
  *   - All calls on a device share the one array, and it keeps what the last
- *     call left there.  Nothing in it has to start at zero: each call overwrites
- *     every record before reading it.  Two calls that overlap on the GPU (different
+ *     call left there.  The one word that has to start at zero (the work counter
+ *     behind the records) is cleared on the stream by every call; the records
+ *     themselves are overwritten before they are read.  Two calls that overlap on the GPU (different
  *     streams, no ordering between them) race on it and give wrong scores;
  *     serialise them, or use difr_score_gm with separate workspaces.
  */
