@@ -25,12 +25,20 @@
  *   IPT sampler     : min{ v : C_v > u }                      (Alg. "IPT Sampler")
  *   detection       : flag iff score < tau                    (Sec. "Classification via
  *                     Thresholding"); per-sequence match count (Alg. prefill verification)
+ *   risk classes    : safe / suspicious / dangerous from the score and the raw-logit rank
+ *                     (Alg. "Per-Token Risk Classification via GLS and Rank")
+ *   admissible set  : A_t(tau) = { i : FSSL_t(i) >= tau }, the score each vocabulary id
+ *                     would get if it were the claim          (Sec. "Empirical Results")
+ *   exfiltratable information : log2 |A_t| / log2 R / log2 |V| by class, summed per
+ *                     sequence                               (Sec. "Problems with FSSL
+ *                     Estimators and Logit-Rank as a Solution", displayed cases)
  *
  * Parity pins (tests, -m "not gpu"): Philox against the cuRAND host generator;
  * Gumbel-max sampler against softmax frequencies (chi-square); honest tokens
  * give margin >= 0; closed form against a literal Monte-Carlo of the fixed-seed
  * posterior; lse against scipy; IPT mass against mpmath quadrature and the
- * telescoping identity.  Absolute score values on realistic model data are
+ * telescoping identity; the admissible set against re-scoring every id as the
+ * claim; the information formula against hand-worked cases.  Absolute score values on realistic model data are
  * "parity unpinned": the paper prints no worked numeric example.
  */
 #include <math.h>
@@ -369,6 +377,107 @@ int oracle_detect(const double* scores, double threshold, const double* margins,
       if (scores[r] < st.min) st.min = scores[r]; /* NaN never compares below */
     }
     stats[s] = st;
+  }
+  return ORACLE_OK;
+}
+
+/* ------------------------------------------------------- risk classes */
+/* Alg. "Per-Token Risk Classification via GLS and Rank": 0 safe if score >= tau;
+ * otherwise 2 (dangerous) if the raw-logit rank exceeds R, else 1 (suspicious).
+ * A NaN score is not >= tau.  ranks nullable => classes 0/1 only. */
+int oracle_classify(const double* scores, double threshold, const int32_t* ranks, int32_t rank_cutoff, int64_t T,
+                    uint8_t* classes) {
+  if (!scores || !classes || T < 0) return ORACLE_ERR_ARG;
+  for (int64_t r = 0; r < T; ++r) {
+    if (scores[r] >= threshold) {
+      classes[r] = 0;
+    } else if (ranks && ranks[r] > rank_cutoff) {
+      classes[r] = 2;
+    } else {
+      classes[r] = 1;
+    }
+  }
+  return ORACLE_OK;
+}
+
+/* ----------------------------------------------------- admissible sets */
+/* |A_t(tau)| for every row: each vocabulary id i is scored as if it were the
+ * claimed token (Token-DiFR, one competitor: the best other id under the row's
+ * regenerated noise) and counted when that score is >= tau. */
+int oracle_admissible_count(const uint16_t* h, const uint16_t* W, const uint64_t* seeds, const uint32_t* positions,
+                            double temperature, double sigma, double eps, double tau, int64_t T, int64_t d,
+                            int64_t V, int32_t* counts) {
+  if (!h || !W || !seeds || !positions || !counts || T < 0 || d <= 0 || V < 2) return ORACLE_ERR_ARG;
+  if (!(sigma > 0.0) || !(eps >= 0.0) || !(temperature >= 0.0)) return ORACLE_ERR_ARG;
+  int err = 0;
+#pragma omp parallel
+  {
+    double* hd = (double*)malloc((size_t)d * sizeof(double));
+    double* logit = (double*)malloc((size_t)V * sizeof(double));
+    double* y = (double*)malloc((size_t)V * sizeof(double));
+    if (!hd || !logit || !y) {
+#pragma omp atomic write
+      err = 1;
+    }
+#pragma omp barrier
+    if (!err) {
+#pragma omp for schedule(dynamic, 1)
+      for (int64_t r = 0; r < T; ++r) {
+        row_logits(h + r * d, W, d, V, hd, logit);
+        for (int64_t v = 0; v < V; ++v) y[v] = logit[v] + temperature * oracle_gumbel_noise(seeds[r], positions[r], (uint32_t)v);
+        int64_t i1 = -1, i2 = -1;
+        for (int64_t v = 0; v < V; ++v) {
+          if (i1 < 0 || y[v] > y[i1]) {
+            i2 = i1;
+            i1 = v;
+          } else if (i2 < 0 || y[v] > y[i2]) {
+            i2 = v;
+          }
+        }
+        int32_t n = 0;
+        for (int64_t i = 0; i < V; ++i) {
+          int64_t c = (i == i1) ? i2 : i1;
+          double A = y[i] - y[c];
+          if (oracle_gm_score(A, sigma, eps) >= tau) ++n;
+        }
+        counts[r] = n;
+      }
+    }
+    free(hd);
+    free(logit);
+    free(y);
+  }
+  return err ? ORACLE_ERR_MEM : ORACLE_OK;
+}
+
+/* ------------------------------------------- exfiltratable information */
+/* Per token: log2 |A_t| if safe, log2 R if suspicious, log2 |V| if dangerous
+ * (the displayed cases of Sec. "Problems with FSSL Estimators ..."); bits[r]
+ * nullable, seq_bits[s] = sum over the sequence's rows.  An empty admissible set
+ * (count 0) carries no information: 0 bits. */
+int oracle_exfiltratable_bits(const uint8_t* classes, const int32_t* counts, int32_t rank_cutoff, int64_t V,
+                              const int32_t* seq_offsets, int64_t n_seq, int64_t T, double* bits,
+                              double* seq_bits) {
+  if (!classes || !counts || T < 0 || n_seq < 0 || V < 1 || rank_cutoff < 1) return ORACLE_ERR_ARG;
+  int64_t ns = seq_offsets ? n_seq : 1;
+  for (int64_t s = 0; s < ns; ++s) {
+    int64_t lo = seq_offsets ? seq_offsets[s] : 0;
+    int64_t hi = seq_offsets ? seq_offsets[s + 1] : T;
+    if (lo < 0 || hi > T || lo > hi) return ORACLE_ERR_ARG;
+    double total = 0.0;
+    for (int64_t r = lo; r < hi; ++r) {
+      double b;
+      if (classes[r] == 0) {
+        b = counts[r] > 0 ? log2((double)counts[r]) : 0.0;
+      } else if (classes[r] == 1) {
+        b = log2((double)rank_cutoff);
+      } else {
+        b = log2((double)V);
+      }
+      if (bits) bits[r] = b;
+      total += b;
+    }
+    if (seq_bits) seq_bits[s] = total;
   }
   return ORACLE_OK;
 }
