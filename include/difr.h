@@ -85,6 +85,17 @@ typedef struct {
   void* event_fused_start; /* optional cudaEvent_t (host handles): recorded on `stream` */
   void* event_fused_stop;  /* right before / after the fused GEMM+epilogue kernel, so a
                               caller can time that kernel apart from the finalize pass */
+  /* -- members added in version 200; zero them when unused -- */
+  int32_t* rank;     /* GM, optional: raw-logit rank of the claimed token, #{v != t* : l_v > l_t*}
+                        (0 = largest logit; V for an out-of-range claim), Sec. "Problems with FSSL
+                        Estimators and Logit-Rank as a Solution".  Counted on the tensor cores' fp32
+                        logits against l_t* rounded to fp32, so ids whose logit lies within fp32
+                        rounding of l_t* may fall on either side.  Asking for it adds one gather pass
+                        and a compare per logit.                                              */
+  float* y_max;      /* GM, optional: y = l + Temp*G of the verifier's own sample (the largest) */
+  float* y_second;   /* GM, optional: the second largest y                                     */
+  float sigma_ipt;   /* difr_score_both only: noise width of the IPT estimator (CDF units), > 0 */
+  float* score_ipt;  /* difr_score_both only, required there: ln(mass + eps)                   */
 } difr_out;
 
 /* Scratch bytes a scoring call needs for T rows, hidden size d, vocabulary V.
@@ -165,6 +176,56 @@ difr_status difr_score_gm_static(const void* h, const void* W, const int32_t* to
                                  difr_out* out, difr_stream_t stream);
 
 /*
+ * Both estimators from one pass over the logits (the fused kernel keeps the
+ * statistics of both anyway): everything difr_score_gm writes, with sigma in
+ * raw-logit units, plus score_ipt / p_claimed / cdf_lo / u of difr_score_ipt
+ * with out->sigma_ipt.  Requires temperature > 0 and out->score_ipt.
+ */
+difr_status difr_score_both(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,
+                            const uint32_t* positions, float temperature, int64_t T, int64_t d, int64_t V,
+                            difr_out* out, difr_stream_t stream);
+
+/*
+ * Sizes of the admissible sets A_t(tau) = { i : FSSL_t(i) >= tau } (Sec.
+ * "Empirical Results"), the quantity behind the paper's information bound
+ * sum_t log2 |A_t(tau)|, for the Token-DiFR score with one competitor.
+ *
+ * For id i != the verifier's own sample the score is ln(Phi((y_i - y_max) /
+ * (sigma sqrt 2)) + eps), so i is admissible iff y_i >= y_max + A(tau) with
+ * A(tau) = sigma sqrt 2 Phi^-1(e^tau - eps); the sample itself is admissible iff
+ * y_max - y_second >= A(tau).  The call makes a second pass over the logits
+ * (same tensor-core main loop, noise regenerated, one compare per logit and
+ * threshold) and needs the outputs of a difr_score_gm call on the same h, W,
+ * seeds, positions and temperature: argmax, y_max, y_second.
+ *
+ *   taus      host pointer, n_tau thresholds, 1 <= n_tau <= 4
+ *   counts    int32 [n_tau, T] (device): |A_t(taus[j])| in counts[j*T + t]
+ *   workspace >= difr_workspace_bytes(T, d, V), scratch
+ * y is evaluated in fp32 here (the scoring calls re-evaluate their few
+ * candidates in fp64), so an id whose y lies within about 1e-3 * max(1, Temp)
+ * of the bound may fall on either side.
+ */
+difr_status difr_admissible(const void* h, const void* W, const uint64_t* seeds, const uint32_t* positions,
+                            float temperature, int64_t T, int64_t d, int64_t V, const int32_t* argmax,
+                            const float* y_max, const float* y_second, float sigma, float eps, const float* taus,
+                            int32_t n_tau, int32_t* counts, void* workspace, size_t workspace_bytes,
+                            int32_t* device_status, difr_stream_t stream);
+
+/*
+ * Per-token exfiltratable information (displayed cases of Sec. "Problems with
+ * FSSL Estimators and Logit-Rank as a Solution"): log2 |A_t| for a safe token,
+ * log2 R for a suspicious one, log2 V for a dangerous one, summed per sequence.
+ *
+ *   classes     uint8 [T]: 0 safe, 1 suspicious, 2 dangerous (the flags of difr_detect)
+ *   counts      int32 [T]: |A_t(tau)| from difr_admissible (0 counts as no information)
+ *   rank_cutoff R >= 1, V >= 1
+ *   bits        float [T], nullable; seq_bits float [n_seq] (or [1]), nullable
+ */
+difr_status difr_exfiltratable_bits(const uint8_t* classes, const int32_t* counts, int32_t rank_cutoff, int64_t V,
+                                    const int32_t* seq_offsets, int64_t n_seq, int64_t T, float* bits,
+                                    float* seq_bits, difr_stream_t stream);
+
+/*
  * Threshold detection and pooling (Sec. "Classification via Thresholding":
  * flag t iff FSSL(t) < tau; per-sequence match count as in Alg. "Sampled token
  * verification via prefill").
@@ -172,9 +233,9 @@ difr_status difr_score_gm_static(const void* h, const void* W, const int32_t* to
  *   scores      float [T]
  *   threshold   tau; a score equal to tau is safe, NaN is flagged
  *   margins     float [T], nullable: rows without a sign bit count as matches
- *   ranks, rank_cutoff   nullable / ignored when NULL: with raw-logit ranks a flagged row
- *               whose rank exceeds the cutoff gets flag 2 (Alg. "Per-Token Risk
- *               Classification")
+ *   ranks, rank_cutoff   nullable / ignored when NULL: with raw-logit ranks (difr_out.rank) a
+ *               flagged row whose rank exceeds the cutoff gets flag 2 (Alg. "Per-Token Risk
+ *               Classification via GLS and Rank": 0 safe, 1 suspicious, 2 dangerous)
  *   seq_offsets int32 [n_seq + 1] ascending row offsets, nullable => one sequence [0, T)
  *   flags       uint8 [T], nullable: 0 safe, 1 flagged (suspicious), 2 dangerous
  *   seq_stats   difr_seq_stats [n_seq] (or [1]), nullable

@@ -18,8 +18,9 @@ DIFR_OK = 0
 STATUS_NAMES = {0: "DIFR_OK", -1: "DIFR_ERR_INVALID_ARG", -2: "DIFR_ERR_SHAPE", -3: "DIFR_ERR_ALIGN",
                 -4: "DIFR_ERR_WORKSPACE", -5: "DIFR_ERR_CUDA", -6: "DIFR_ERR_ARCH", -7: "DIFR_ERR_TIMEOUT"}
 
-EXPORTS = ("difr_workspace_bytes", "difr_score_gm", "difr_score_ipt", "difr_score_gm_static", "difr_detect",
-           "difr_logits", "difr_philox", "difr_status_string", "difr_version")
+EXPORTS = ("difr_workspace_bytes", "difr_score_gm", "difr_score_ipt", "difr_score_both", "difr_score_gm_static",
+           "difr_admissible", "difr_exfiltratable_bits", "difr_detect", "difr_logits", "difr_philox",
+           "difr_status_string", "difr_version")
 STATIC_SCRATCH_BYTES = 16 << 20  # DIFR_STATIC_SCRATCH_BYTES
 
 
@@ -37,6 +38,8 @@ class _COut(ctypes.Structure):
         ("cdf_lo", ctypes.c_void_p), ("u", ctypes.c_void_p), ("row_status", ctypes.c_void_p),
         ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t), ("device_status", ctypes.c_void_p),
         ("event_fused_start", ctypes.c_void_p), ("event_fused_stop", ctypes.c_void_p),
+        ("rank", ctypes.c_void_p), ("y_max", ctypes.c_void_p), ("y_second", ctypes.c_void_p),
+        ("sigma_ipt", ctypes.c_float), ("score_ipt", ctypes.c_void_p),
     ]
 
 
@@ -55,13 +58,22 @@ def lib() -> ctypes.CDLL:
         L.difr_workspace_bytes.argtypes = [ctypes.c_int64] * 3
         score_args = [ctypes.c_void_p] * 5 + [ctypes.c_float] + [ctypes.c_int64] * 3 + [ctypes.POINTER(_COut),
                                                                                       ctypes.c_void_p]
-        for name in ("difr_score_gm", "difr_score_ipt", "difr_score_gm_static"):
+        for name in ("difr_score_gm", "difr_score_ipt", "difr_score_both", "difr_score_gm_static"):
             getattr(L, name).restype = ctypes.c_int
             getattr(L, name).argtypes = score_args
         L.difr_detect.restype = ctypes.c_int
         L.difr_detect.argtypes = [ctypes.c_void_p, ctypes.c_float, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32,
                                   ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p,
                                   ctypes.c_void_p]
+        L.difr_admissible.restype = ctypes.c_int
+        L.difr_admissible.argtypes = ([ctypes.c_void_p] * 4 + [ctypes.c_float] + [ctypes.c_int64] * 3
+                                      + [ctypes.c_void_p] * 3 + [ctypes.c_float] * 2
+                                      + [ctypes.POINTER(ctypes.c_float), ctypes.c_int32, ctypes.c_void_p,
+                                         ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p])
+        L.difr_exfiltratable_bits.restype = ctypes.c_int
+        L.difr_exfiltratable_bits.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64,
+                                              ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p,
+                                              ctypes.c_void_p, ctypes.c_void_p]
         L.difr_logits.restype = ctypes.c_int
         L.difr_logits.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
@@ -124,6 +136,11 @@ class DifrOut:
     device_status: "object" = None
     event_fused_start: int = 0  # raw cudaEvent_t handles (0: none)
     event_fused_stop: int = 0
+    rank: "object" = None       # int32 [T]: ask for the raw-logit rank of the claimed token (GM calls)
+    y_max: "object" = None      # float [T]: largest / second largest l + Temp*G (GM calls); difr_admissible needs them
+    y_second: "object" = None
+    sigma_ipt: float = 0.0      # difr_score_both: width of the IPT estimator
+    score_ipt: "object" = None  # difr_score_both: float [T]
 
     @staticmethod
     def allocate(T: int, d: int, V: int, sigma: float, eps: float = 1e-12, device="cuda"):
@@ -142,7 +159,8 @@ class DifrOut:
                      _ptr(self.runner_up), _ptr(self.lse), _ptr(self.p_claimed), _ptr(self.cdf_lo), _ptr(self.u),
                      _ptr(self.row_status), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
                      _ptr(self.device_status), ctypes.c_void_p(self.event_fused_start or None),
-                     ctypes.c_void_p(self.event_fused_stop or None))
+                     ctypes.c_void_p(self.event_fused_stop or None), _ptr(self.rank), _ptr(self.y_max),
+                     _ptr(self.y_second), float(self.sigma_ipt), _ptr(self.score_ipt))
 
 
 def _score(fn_name, h, W, tokens, seeds, positions, temperature, out: DifrOut, stream):
@@ -171,6 +189,42 @@ def difr_score_gm(h, W, tokens, seeds, positions, temperature, out: DifrOut, str
 def difr_score_ipt(h, W, tokens, seeds, positions, temperature, out: DifrOut, stream=None) -> DifrOut:
     """Token-IPT-DiFR scores; see include/difr.h."""
     return _score("difr_score_ipt", h, W, tokens, seeds, positions, temperature, out, stream)
+
+
+def difr_score_both(h, W, tokens, seeds, positions, temperature, out: DifrOut, stream=None) -> DifrOut:
+    """Token-DiFR and Token-IPT-DiFR scores from one pass (`out.sigma_ipt`, `out.score_ipt`); see include/difr.h."""
+    return _score("difr_score_both", h, W, tokens, seeds, positions, temperature, out, stream)
+
+
+def difr_admissible(h, W, seeds, positions, temperature, scored: DifrOut, taus, counts, stream=None):
+    """Admissible-set sizes |A_t(tau)| for up to four thresholds; `scored` holds argmax, y_max, y_second, sigma,
+    eps and the workspace of a difr_score_gm call on the same inputs; `counts` is int32 [len(taus), T]."""
+    import torch
+
+    T, d = h.shape
+    V = W.shape[0]
+    taus = [float(t) for t in taus]
+    _check(counts, torch.int32, (len(taus), T), "counts")
+    arr = (ctypes.c_float * len(taus))(*taus)
+    ws = scored.workspace
+    rc = lib().difr_admissible(_ptr(h), _ptr(W), _ptr(seeds), _ptr(positions), float(temperature), T, d, V,
+                               _ptr(scored.argmax), _ptr(scored.y_max), _ptr(scored.y_second), float(scored.sigma),
+                               float(scored.eps), arr, len(taus), _ptr(counts), _ptr(ws),
+                               ws.numel() * ws.element_size(), _ptr(scored.device_status), _stream(stream))
+    if rc != DIFR_OK:
+        raise DifrError(rc, "difr_admissible")
+    return counts
+
+
+def difr_exfiltratable_bits(classes, counts, rank_cutoff, V, seq_offsets=None, bits=None, seq_bits=None, stream=None):
+    """Per-token / per-sequence information bound from the risk classes and admissible-set sizes."""
+    T = classes.shape[0]
+    n_seq = 1 if seq_offsets is None else seq_offsets.shape[0] - 1
+    rc = lib().difr_exfiltratable_bits(_ptr(classes), _ptr(counts), int(rank_cutoff), int(V), _ptr(seq_offsets), n_seq,
+                                       T, _ptr(bits), _ptr(seq_bits), _stream(stream))
+    if rc != DIFR_OK:
+        raise DifrError(rc, "difr_exfiltratable_bits")
+    return bits, seq_bits
 
 
 def difr_score_gm_static(h, W, tokens, seeds, positions, temperature, out: DifrOut, stream=None) -> DifrOut:

@@ -19,7 +19,7 @@ struct __align__(16) Partial {
   float lse2_max;  // max_v z_v, -inf if the strip is empty
   float lse2_sum;
   float prefix2;   // sum over v < claimed id of 2^(z_v - lse2_max)
-  float reserved;
+  int32_t larger;  // ids of the strip (claimed id left out) whose logit exceeds the claimed one; rank mode only
 };
 static_assert(sizeof(Partial) == 32, "partial record is 32 bytes");
 

@@ -14,6 +14,7 @@ struct K1Params {
   const int32_t* tokens;
   const uint64_t* seeds;
   const uint32_t* positions;
+  const float* bounds;  // [1 or 4][T_pad]: claimed logits (rank mode) or bounds on y' (counting modes)
   Partial* partials;  // [n_slots][T_pad]
   float* logits_out;  // dump mode only
   int32_t* device_status;
@@ -34,7 +35,12 @@ struct K2Params {
   const Partial* partials;
   int n_slots, T_pad;
   int T, d, V;
-  int ipt;  // 0: Token-DiFR (Gumbel-max), 1: Token-IPT-DiFR
+  int ipt;  // 0: Token-DiFR (Gumbel-max), 1: Token-IPT-DiFR, 2: both (IPT score to score_ipt with sigma_ipt)
+  float sigma_ipt;
+  float* score_ipt;
+  int32_t* rank;
+  float* y_max;
+  float* y_second;
   float temperature, sigma, eps;
   float c1;  // log2(e) / Temp as used by the fused kernel
   float* score;
@@ -60,12 +66,43 @@ struct K3Params {
   void* seq_stats;
 };
 
-// mode: 0 Gumbel-max epilogue, 1 softmax statistics only, 2 logits dump.
+// mode: 0 Gumbel-max epilogue, 1 softmax statistics only, 2 logits dump, 3 Gumbel-max + raw-logit rank,
+// 4 / 5 count the ids whose noisy logit reaches one / four per-row bounds.
 cudaError_t launch_k1(int mode, const CUtensorMap& tmap_h, const CUtensorMap& tmap_w, const K1Params& p, int grid,
                       cudaStream_t stream);  // grid: number of CTAs, two per pair
 int k1_max_resident_pairs();  // CTA pairs of the fused kernel the current device keeps resident at once
 cudaError_t launch_k2(const K2Params& p, cudaStream_t stream);
 cudaError_t launch_k3(const K3Params& p, cudaStream_t stream);
+
+// Claimed logits l[r, tokens[r]] rounded to fp32 into out[r] (+inf for an id outside [0, V)): one warp per row.
+cudaError_t launch_claimed_logits(const uint16_t* h, const uint16_t* W, const int32_t* tokens, int T, int d, int V,
+                                  float* out, cudaStream_t stream);
+
+// Counting pass of the admissible sets.
+struct CountParams {
+  const Partial* partials;  // records of the counting modes: four int32 counts each
+  int n_slots, T_pad, T, V, n_tau;
+  const int32_t* argmax;
+  const float* y_max;
+  const float* y_second;
+  float a_tau[4];   // A(tau_j): id i != argmax is admissible iff y_i - y_max >= A(tau_j)
+  float y_shift;    // the fused kernel ranks y' = y + y_shift
+  float* bounds;    // [4][T_pad] out: bounds on y'
+  int32_t* counts;  // [n_tau][T] out
+};
+cudaError_t launch_count_bounds(const CountParams& p, cudaStream_t stream);
+cudaError_t launch_count_finalize(const CountParams& p, cudaStream_t stream);
+
+struct BitsParams {
+  const uint8_t* classes;
+  const int32_t* counts;
+  const int32_t* seq_offsets;
+  int64_t n_seq, T;
+  float log2_r, log2_v;
+  float* bits;
+  float* seq_bits;
+};
+cudaError_t launch_bits(const BitsParams& p, cudaStream_t stream);
 cudaError_t launch_philox(const uint32_t* ctr, const uint32_t* key, int64_t n, uint32_t* out, cudaStream_t stream);
 
 }  // namespace difr

@@ -23,6 +23,7 @@ struct Plan {
   int T_pad;     // m_tiles * 256
   int n_slots;   // partial records per row: one per strip
   size_t partial_bytes;
+  size_t bounds_offset;  // [4][T_pad] floats behind the records and the 256-byte tail (unit counter)
   size_t workspace_bytes;
 };
 
@@ -88,7 +89,8 @@ inline bool make_plan(int64_t T, int64_t d, int64_t V, int num_pairs, Plan* out)
   p.T_pad = p.m_tiles * kPairM;
   p.n_slots = p.S;
   p.partial_bytes = (size_t)p.n_slots * (size_t)p.T_pad * 32;
-  p.workspace_bytes = p.partial_bytes + 256;
+  p.bounds_offset = p.partial_bytes + 256;
+  p.workspace_bytes = p.bounds_offset + (size_t)4 * (size_t)p.T_pad * sizeof(float);
   *out = p;
   return true;
 }

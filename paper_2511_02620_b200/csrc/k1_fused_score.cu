@@ -57,7 +57,19 @@ constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + kXchBytes + 1024;
 constexpr float kMasked = -3.0e38f;  // stands in for -inf on padded vocabulary columns (keeps keys finite)
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one CTA");
 
-enum : int { kModeGm = 0, kModeIpt = 1, kModeDump = 2 };
+// Epilogue variants.  GmRank adds the raw-logit rank of the claimed token; Count1 / Count4 regenerate the
+// noise only to count the ids whose y reaches one / four per-row bounds (admissible-set sizes).
+enum : int { kModeGm = 0, kModeIpt = 1, kModeDump = 2, kModeGmRank = 3, kModeCount1 = 4, kModeCount4 = 5 };
+
+template <int MODE>
+struct Mode {
+  static constexpr bool gm = MODE == kModeGm || MODE == kModeGmRank;
+  static constexpr bool softmax = gm || MODE == kModeIpt;
+  static constexpr bool rank = MODE == kModeGmRank;
+  static constexpr int ng = MODE == kModeCount1 ? 1 : (MODE == kModeCount4 ? 4 : 0);  // bounds per row
+  static constexpr bool noise = gm || ng > 0;
+  static constexpr int ncnt = rank ? 1 : (ng > 0 ? ng : 1);
+};
 
 struct Unit {
   int m, n0, n1, strip;  // m: 256-row tile of the pair
@@ -84,6 +96,8 @@ struct RowStats {
   float lmax;    // running max of z = l * c1
   float lsum;    // sum of 2^(z - lmax)
   float lpre;    // the same restricted to ids below the claimed one
+  int cnt[4];    // GmRank: cnt[0] = ids whose logit exceeds the claimed one; Count: ids at or above bound g
+  float bound[4];  // GmRank: bound[0] = claimed logit; Count: the row's bounds on y'
 };
 
 __device__ __forceinline__ void stats_init(RowStats& s) {
@@ -91,6 +105,7 @@ __device__ __forceinline__ void stats_init(RowStats& s) {
   s.i1 = s.i2 = -1;
   s.lmax = -CUDART_INF_F;
   s.lsum = s.lpre = 0.f;
+  s.cnt[0] = s.cnt[1] = s.cnt[2] = s.cnt[3] = 0;
 }
 
 // (k1, j1), (k2, j2): the best two of another column group of the same row, k1 >= k2.
@@ -107,10 +122,42 @@ __device__ __forceinline__ void top2_merge(RowStats& s, float k1, int j1, float 
   }
 }
 
-// 16 consecutive vocabulary ids [base, base + 16) of one row.
+// y' = l - Temp ln2 log2(-log2 u) = l + Temp G + Temp ln(ln 2) for ids [id0, id0 + 4) of one row (id0 % 4 == 0).
+__device__ __forceinline__ void noisy4(const RowNoise& rn, int id0, const float (&l)[4], float neg_tl2,
+                                       float (&y)[4]) {
+  uint32_t x[4];
+  row_noise_block(rn, (uint32_t)id0 >> 2, x);
+  const float2 minus1 = make_float2(-0.99999994f, -0.99999994f), ntl2 = make_float2(neg_tl2, neg_tl2);
+#pragma unroll
+  for (int q = 0; q < 4; q += 2) {
+    // u = ((x >> 9) + 1/2) 2^-23, exact;  -log2 u = E / ln 2
+    const float2 u = fadd2(make_float2(__uint_as_float(0x3F800000u | (x[q] >> 9)),
+                                       __uint_as_float(0x3F800000u | (x[q + 1] >> 9))), minus1);
+    const float2 g = make_float2(lg2_approx(-lg2_approx(u.x)), lg2_approx(-lg2_approx(u.y)));
+    const float2 yy = ffma2(g, ntl2, make_float2(l[q], l[q + 1]));
+    y[q] = yy.x;
+    y[q + 1] = yy.y;
+  }
+  // u within 2^-11 of one: -log2 u loses relative accuracy, redo those with a series for -ln(1 - w)
+  const uint32_t xm = max(max(x[0], x[1]), max(x[2], x[3]));
+  if (xm >= 0xFFE00000u) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      if (x[q] >= 0xFFE00000u) {
+        const float w = __uint_as_float(0x3F800000u | ((~x[q]) >> 9)) - 0.99999994f;  // 1 - u, exact
+        const float E = w * fmaf(w, fmaf(w, 0.33333334f, 0.5f), 1.0f);
+        y[q] = fmaf(lg2_approx(E * 1.4426950408889634f), neg_tl2, l[q]);
+      }
+    }
+  }
+}
+
+// 16 consecutive vocabulary ids [base, base + 16) of one row.  `tok` is the id the row singles out: the
+// claimed token (scoring modes) or the id left out of the count (counting modes).
 template <int MODE>
 __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base, int V, int tok, float c1,
                                           float neg_tl2, const RowNoise& rn, RowStats& s) {
+  using M = Mode<MODE>;
   float l[kSub];
 #pragma unroll
   for (int j = 0; j < kSub; ++j) l[j] = __uint_as_float(raw[j]);
@@ -119,9 +166,10 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
     for (int j = 0; j < kSub; ++j)
       if (base + j >= V) l[j] = kMasked;
   }
+  const int tl = tok - base;  // position of the singled-out id relative to this group
 
   // ---- softmax statistics (online log-sum-exp in base 2)
-  {
+  if (M::softmax) {
     float cm = fmax3(l[0], l[1], l[2]);
 #pragma unroll
     for (int j = 3; j + 1 < kSub; j += 2) cm = fmax3(cm, l[j], l[j + 1]);
@@ -146,7 +194,7 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
     const float2 a = fadd2(a01, a23);
     const float cs = a.x + a.y;
     s.lsum += cs;
-    const int tl = tok - base;  // ids below the claimed one: all, none, or the first tl of this group
+    // ids below the claimed one: all, none, or the first tl of this group
     if (tl >= kSub) {
       s.lpre += cs;
     } else if (tl > 0) {
@@ -158,48 +206,90 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
     }
   }
 
-  // ---- Gumbel-max replay: top-2 of y' = l - Temp*ln2 * log2(-log2 u)
-  if (MODE == kModeGm) {
+  // ---- raw-logit rank of the claimed token: ids whose logit is larger (the claimed id itself left out)
+  if (M::rank) {
+    const float lt = s.bound[0];
+    int c = 0;
+#pragma unroll
+    for (int j = 0; j < kSub; ++j) c += (l[j] > lt) ? 1 : 0;
+    if (tl >= 0 && tl < kSub) {
+#pragma unroll
+      for (int j = 0; j < kSub; ++j)
+        if (j == tl && l[j] > lt) --c;
+    }
+    s.cnt[0] += c;
+  }
+
+  // ---- Gumbel-max replay: top-2 of y' = l - Temp*ln2 * log2(-log2 u), or counts of y' against the row's bounds
+  if (M::noise) {
     float c1k = -CUDART_INF_F, c2k = -CUDART_INF_F;
 #pragma unroll
     for (int j = 0; j < kSub; j += 4) {
-      uint32_t x[4];
-      row_noise_block(rn, (uint32_t)(base + j) >> 2, x);
-      float key[4];
-      const float2 minus1 = make_float2(-0.99999994f, -0.99999994f), ntl2 = make_float2(neg_tl2, neg_tl2);
+      const float l4[4] = {l[j], l[j + 1], l[j + 2], l[j + 3]};
+      float y[4];
+      noisy4(rn, base + j, l4, neg_tl2, y);
+      if (M::gm) {
+        float key[4];
 #pragma unroll
-      for (int q = 0; q < 4; q += 2) {
-        // u = ((x >> 9) + 1/2) 2^-23, exact;  -log2 u = E / ln 2;  y' = l - Temp ln2 log2(E / ln 2)
-        const float2 u = fadd2(make_float2(__uint_as_float(0x3F800000u | (x[q] >> 9)),
-                                           __uint_as_float(0x3F800000u | (x[q + 1] >> 9))), minus1);
-        const float2 g = make_float2(lg2_approx(-lg2_approx(u.x)), lg2_approx(-lg2_approx(u.y)));
-        const float2 y = ffma2(g, ntl2, make_float2(l[j + q], l[j + q + 1]));
-        key[q] = __uint_as_float((__float_as_uint(y.x) & ~15u) | (uint32_t)(j + q));
-        key[q + 1] = __uint_as_float((__float_as_uint(y.y) & ~15u) | (uint32_t)(j + q + 1));
+        for (int q = 0; q < 4; ++q) key[q] = __uint_as_float((__float_as_uint(y[q]) & ~15u) | (uint32_t)(j + q));
+        const float h1 = fmaxf(key[0], key[1]), l1 = fminf(key[0], key[1]);
+        const float h2 = fmaxf(key[2], key[3]), l2 = fminf(key[2], key[3]);
+        const float t1 = fmaxf(h1, h2);
+        const float t2 = fmax3(fminf(h1, h2), l1, l2);
+        const float n2 = fmax3(fminf(c1k, t1), c2k, t2);
+        c1k = fmaxf(c1k, t1);
+        c2k = n2;
       }
-      // u within 2^-11 of one: -log2 u loses relative accuracy, redo those with a series for -ln(1 - w)
-      const uint32_t xm = max(max(x[0], x[1]), max(x[2], x[3]));
-      if (xm >= 0xFFE00000u) {
+      if (M::ng > 0) {
+        if (tl >= j && tl < j + 4) {  // the id left out never counts
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          if (x[q] >= 0xFFE00000u) {
-            const float w = __uint_as_float(0x3F800000u | ((~x[q]) >> 9)) - 0.99999994f;  // 1 - u, exact
-            const float E = w * fmaf(w, fmaf(w, 0.33333334f, 0.5f), 1.0f);
-            const float y = fmaf(lg2_approx(E * 1.4426950408889634f), neg_tl2, l[j + q]);
-            key[q] = __uint_as_float((__float_as_uint(y) & ~15u) | (uint32_t)(j + q));
-          }
+          for (int q = 0; q < 4; ++q)
+            if (j + q == tl) y[q] = kMasked;
+        }
+#pragma unroll
+        for (int g = 0; g < M::ng; ++g) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) s.cnt[g] += (y[q] >= s.bound[g]) ? 1 : 0;
         }
       }
-      const float h1 = fmaxf(key[0], key[1]), l1 = fminf(key[0], key[1]);
-      const float h2 = fmaxf(key[2], key[3]), l2 = fminf(key[2], key[3]);
-      const float t1 = fmaxf(h1, h2);
-      const float t2 = fmax3(fminf(h1, h2), l1, l2);
-      const float n2 = fmax3(fminf(c1k, t1), c2k, t2);
-      c1k = fmaxf(c1k, t1);
-      c2k = n2;
     }
     // merge the group's top-2 into the running top-2 (earlier ids win ties)
-    top2_merge(s, c1k, base + (int)(__float_as_uint(c1k) & 15u), c2k, base + (int)(__float_as_uint(c2k) & 15u));
+    if (M::gm)
+      top2_merge(s, c1k, base + (int)(__float_as_uint(c1k) & 15u), c2k, base + (int)(__float_as_uint(c2k) & 15u));
+  }
+}
+
+// The 32-byte record of a row: what leaves a column group for shared memory and a unit for the workspace.
+//   scoring modes:  {m1, i1, m2, i2, lse2_max, lse2_sum, prefix2, count of larger logits}
+//   counting modes: {count at bound 0..3, -, -, -, -}
+template <int MODE>
+__device__ __forceinline__ void record_pack(const RowStats& st, float4& a, float4& b) {
+  if (Mode<MODE>::ng > 0) {
+    a = make_float4(__int_as_float(st.cnt[0]), __int_as_float(st.cnt[1]), __int_as_float(st.cnt[2]),
+                    __int_as_float(st.cnt[3]));
+    b = make_float4(0.f, 0.f, 0.f, 0.f);
+  } else {
+    a = make_float4(st.m1, __int_as_float(st.i1), st.m2, __int_as_float(st.i2));
+    b = make_float4(st.lmax, st.lsum, st.lpre, __int_as_float(st.cnt[0]));
+  }
+}
+template <int MODE>
+__device__ __forceinline__ void record_merge(RowStats& st, const float4& a, const float4& b) {
+  if (Mode<MODE>::ng > 0) {
+    st.cnt[0] += __float_as_int(a.x);
+    st.cnt[1] += __float_as_int(a.y);
+    st.cnt[2] += __float_as_int(a.z);
+    st.cnt[3] += __float_as_int(a.w);
+  } else {
+    top2_merge(st, a.x, __float_as_int(a.y), a.z, __float_as_int(a.w));
+    if (b.x > -CUDART_INF_F) {  // that group saw columns
+      const float m = fmaxf(st.lmax, b.x);
+      const float fa = ex2_approx(st.lmax - m), fb = ex2_approx(b.x - m);
+      st.lsum = st.lsum * fa + b.y * fb;
+      st.lpre = st.lpre * fa + b.z * fb;
+      st.lmax = m;
+    }
+    st.cnt[0] += __float_as_int(b.w);
   }
 }
 
@@ -424,7 +514,13 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
           seed = p.seeds[row];
           pos = p.positions[row];
         }
-        if (MODE == kModeGm) row_noise_init(rn, seed, pos);
+        if (Mode<MODE>::noise) row_noise_init(rn, seed, pos);
+        // per-row bounds: the claimed logit (rank) or the bounds on y' (counting); rows beyond T count nothing
+        if (Mode<MODE>::rank || Mode<MODE>::ng > 0) {
+#pragma unroll
+          for (int g = 0; g < Mode<MODE>::ncnt; ++g)
+            st.bound[g] = valid ? p.bounds[(size_t)g * (size_t)p.T_pad + row] : CUDART_INF_F;
+        }
       }
       for (int n = w.n0; n < w.n1; ++n) {
         if (!mbar_wait(acc_full_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
@@ -466,8 +562,7 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
         if (colg != 0) {
           if (!mbar_wait(xch_empty_bar(quarter), xch_phase ^ 1u, abort_flag)) { ok = false; break; }
           float4* dst = xch + ((size_t)(colg - 1) * kBM + row_in_cta) * 2;
-          dst[0] = make_float4(st.m1, __int_as_float(st.i1), st.m2, __int_as_float(st.i2));
-          dst[1] = make_float4(st.lmax, st.lsum, st.lpre, 0.f);
+          record_pack<MODE>(st, dst[0], dst[1]);
           __syncwarp();
           if (lane == 0) mbar_arrive(xch_full_bar(quarter));
         } else {
@@ -475,22 +570,13 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
 #pragma unroll
           for (int g = 0; g < kColGroups - 1; ++g) {
             const float4* src = xch + ((size_t)g * kBM + row_in_cta) * 2;
-            const float4 a = src[0], b = src[1];
-            top2_merge(st, a.x, __float_as_int(a.y), a.z, __float_as_int(a.w));
-            if (b.x > -CUDART_INF_F) {  // that group saw columns
-              const float m = fmaxf(st.lmax, b.x);
-              const float fa = ex2_approx(st.lmax - m), fb = ex2_approx(b.x - m);
-              st.lsum = st.lsum * fa + b.y * fb;
-              st.lpre = st.lpre * fa + b.z * fb;
-              st.lmax = m;
-            }
+            record_merge<MODE>(st, src[0], src[1]);
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(xch_empty_bar(quarter));
           if (valid) {
             float4* dst = reinterpret_cast<float4*>(p.partials + (size_t)w.strip * (size_t)p.T_pad + row);
-            dst[0] = make_float4(st.m1, __int_as_float(st.i1), st.m2, __int_as_float(st.i2));
-            dst[1] = make_float4(st.lmax, st.lsum, st.lpre, 0.f);
+            record_pack<MODE>(st, dst[0], dst[1]);
           }
         }
         xch_phase ^= 1u;
@@ -558,6 +644,9 @@ cudaError_t launch_k1(int mode, const CUtensorMap& tmap_h, const CUtensorMap& tm
     case kModeGm: return launch_mode<kModeGm>(tmap_h, tmap_w, p, grid, stream);
     case kModeIpt: return launch_mode<kModeIpt>(tmap_h, tmap_w, p, grid, stream);
     case kModeDump: return launch_mode<kModeDump>(tmap_h, tmap_w, p, grid, stream);
+    case kModeGmRank: return launch_mode<kModeGmRank>(tmap_h, tmap_w, p, grid, stream);
+    case kModeCount1: return launch_mode<kModeCount1>(tmap_h, tmap_w, p, grid, stream);
+    case kModeCount4: return launch_mode<kModeCount4>(tmap_h, tmap_w, p, grid, stream);
   }
   return cudaErrorInvalidValue;
 }

@@ -17,6 +17,7 @@ struct Merged {
   float m1, m2;
   int i1, i2;
   double lmax, lsum, lpre;  // base-2 log-sum-exp state
+  int larger;               // ids whose logit exceeds the claimed one (rank mode)
 };
 
 __device__ __forceinline__ bool beats(float v, int i, float w, int j) {
@@ -104,12 +105,14 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
   acc.i1 = acc.i2 = -1;
   acc.lmax = -CUDART_INF;
   acc.lsum = acc.lpre = 0.0;
+  acc.larger = 0;
   for (int slot = lane; slot < p.n_slots; slot += 32) {
     const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * (size_t)p.T_pad + row);
     const float4 a = src[0], b = src[1];
     top2_insert(acc, a.x, __float_as_int(a.y));
     top2_insert(acc, a.z, __float_as_int(a.w));
     lse_merge(acc, (double)b.x, (double)b.y, (double)b.z);
+    acc.larger += __float_as_int(b.w);
   }
 #pragma unroll
   for (int m = 16; m >= 1; m >>= 1) {
@@ -120,6 +123,7 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
     top2_insert(acc, o1, j1);
     top2_insert(acc, o2, j2);
     lse_merge(acc, om, os, op);
+    acc.larger += __shfl_xor_sync(0xffffffffu, acc.larger, m);
   }
   // (every lane now holds the same merged state up to the order of the lse additions; use lane 0's)
   acc.lmax = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(acc.lmax), 0),
@@ -146,7 +150,7 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
   double l_tok = 0.0;
   if (tok_ok) l_tok = warp_dot(hrow, p.W + (size_t)tok * (size_t)p.d, p.d, lane);
 
-  if (!p.ipt) {
+  if (p.ipt != 1) {
     // ---- Token-DiFR: exact y = l + Temp * G for the claimed token and the two candidates
     const int c1 = (acc.i1 >= 0 && acc.i1 < p.V) ? acc.i1 : -1;
     const int c2 = (acc.i2 >= 0 && acc.i2 < p.V) ? acc.i2 : -1;
@@ -163,6 +167,7 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
         double tv = ya; ya = yb; yb = tv;
       }
       int best = a, second = b;
+      double ybest = ya, ysecond = yb;
       double A = -CUDART_INF;
       if (tok_ok) {
         // strongest competitor: the best candidate that is not the claimed token
@@ -173,8 +178,8 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
         const bool tok_first = (c < 0) || (yt > yc) || (yt == yc && tok < c);
         if (tok != a && tok != b) {
           // the claimed token was not among the candidates: place it
-          if (tok_first) { second = a; best = tok; }
-          else if (b < 0 || yt > yb || (yt == yb && tok < b)) { second = tok; }
+          if (tok_first) { second = a; ysecond = ya; best = tok; ybest = yt; }
+          else if (b < 0 || yt > yb || (yt == yb && tok < b)) { second = tok; ysecond = yt; }
         }
       }
       const double pi = 0.5 * erfc(-A / (2.0 * sigma));  // Phi(A / (sigma sqrt 2))
@@ -185,8 +190,12 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
       if (p.runner_up) p.runner_up[row] = second;
       if (p.lse) p.lse[row] = (float)lse;
       if (p.row_status) p.row_status[row] = status;
+      if (p.rank) p.rank[row] = tok_ok ? acc.larger : p.V;
+      if (p.y_max) p.y_max[row] = (float)ybest;
+      if (p.y_second) p.y_second[row] = (float)ysecond;
     }
-  } else {
+  }
+  if (p.ipt != 0) {
     // ---- Token-IPT-DiFR
     if (lane == 0) {
       uint32_t x[4];
@@ -198,10 +207,11 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
         pt = exp2(l_tok * c1d - acc.lmax) / acc.lsum;
         a = acc.lpre / acc.lsum;
         const double b = a + pt;
-        const double mass = normal_interval((a - mu) / sigma, (b - mu) / sigma);
+        const double sg = (p.ipt == 2) ? (double)p.sigma_ipt : sigma;
+        const double mass = normal_interval((a - mu) / sg, (b - mu) / sg);
         score = log(mass + eps);
       }
-      p.score[row] = (float)score;
+      (p.ipt == 2 ? p.score_ipt : p.score)[row] = (float)score;
       if (p.lse) p.lse[row] = (float)lse;
       if (p.p_claimed) p.p_claimed[row] = (float)pt;
       if (p.cdf_lo) p.cdf_lo[row] = (float)a;
@@ -214,6 +224,77 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
 cudaError_t launch_k2(const K2Params& p, cudaStream_t stream) {
   const int blocks = (p.T + kK2Warps - 1) / kK2Warps;
   k2_finalize<<<blocks, kK2Warps * 32, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+// --------------------------------------------------------- claimed logits
+// l[r, tokens[r]] in fp64, rounded to fp32: what the fused kernel's rank mode compares every logit with.
+__global__ void __launch_bounds__(kK2Warps * 32)
+claimed_logits(const uint16_t* h, const uint16_t* W, const int32_t* tokens, int T, int d, int V, float* out) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * kK2Warps + warp;
+  if (row >= T) return;
+  const int tok = tokens[row];
+  float v = CUDART_INF_F;
+  if (tok >= 0 && tok < V) v = (float)warp_dot(h + (size_t)row * (size_t)d, W + (size_t)tok * (size_t)d, d, lane);
+  if (lane == 0) out[row] = v;
+}
+
+cudaError_t launch_claimed_logits(const uint16_t* h, const uint16_t* W, const int32_t* tokens, int T, int d, int V,
+                                  float* out, cudaStream_t stream) {
+  const int blocks = (T + kK2Warps - 1) / kK2Warps;
+  claimed_logits<<<blocks, kK2Warps * 32, 0, stream>>>(h, W, tokens, T, d, V, out);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------- admissible sets
+// Bounds of the counting pass: id i != argmax is admissible at threshold j iff y_i >= y_max + A(tau_j); the
+// fused kernel sees y' = y + y_shift.  Unused thresholds get +inf (nothing counts).
+__global__ void count_bounds(const CountParams p) {
+  const int row = blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= p.T) return;
+  const float ymax = p.y_max[row];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    float b = CUDART_INF_F;
+    if (j < p.n_tau) {
+      // -inf (everything admissible) must stay above the value that masks padded vocabulary columns
+      b = fmaxf(ymax + p.a_tau[j] + p.y_shift, -1.0e38f);
+      if (isnan(b)) b = CUDART_INF_F;
+    }
+    p.bounds[(size_t)j * (size_t)p.T_pad + row] = b;
+  }
+}
+
+// One warp per row: sums the strips' counts and adds the verifier's own sample, which the counting pass
+// leaves out and which is admissible iff y_max - y_second >= A(tau_j).
+__global__ void __launch_bounds__(kK2Warps * 32) count_finalize(const CountParams p) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * kK2Warps + warp;
+  if (row >= p.T) return;
+  int c[4] = {0, 0, 0, 0};
+  for (int slot = lane; slot < p.n_slots; slot += 32) {
+    const int4 a = *reinterpret_cast<const int4*>(p.partials + (size_t)slot * (size_t)p.T_pad + row);
+    c[0] += a.x; c[1] += a.y; c[2] += a.z; c[3] += a.w;
+  }
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) c[j] += __shfl_xor_sync(0xffffffffu, c[j], m);
+  }
+  if (lane == 0) {
+    const float top_margin = p.y_max[row] - p.y_second[row];
+    for (int j = 0; j < p.n_tau; ++j)
+      p.counts[(size_t)j * (size_t)p.T + row] = c[j] + ((top_margin >= p.a_tau[j]) ? 1 : 0);
+  }
+}
+
+cudaError_t launch_count_bounds(const CountParams& p, cudaStream_t stream) {
+  count_bounds<<<(p.T + 255) / 256, 256, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+cudaError_t launch_count_finalize(const CountParams& p, cudaStream_t stream) {
+  count_finalize<<<(p.T + kK2Warps - 1) / kK2Warps, kK2Warps * 32, 0, stream>>>(p);
   return cudaGetLastError();
 }
 

@@ -81,4 +81,43 @@ cudaError_t launch_k3(const K3Params& p, cudaStream_t stream) {
   return cudaGetLastError();
 }
 
+// ------------------------------------------------ exfiltratable information
+// Per token log2 |A_t| (safe), log2 R (suspicious) or log2 V (dangerous); one CTA per sequence sums them.
+__global__ void __launch_bounds__(kK3Threads) k3_bits(const BitsParams p) {
+  const int64_t seq = blockIdx.x;
+  const int64_t lo = p.seq_offsets ? (int64_t)p.seq_offsets[seq] : 0;
+  const int64_t hi = p.seq_offsets ? (int64_t)p.seq_offsets[seq + 1] : p.T;
+  float sum = 0.f;
+  for (int64_t r = lo + threadIdx.x; r < hi; r += kK3Threads) {
+    const uint8_t c = p.classes[r];
+    float b;
+    if (c == 0) {
+      const int32_t n = p.counts[r];
+      b = n > 0 ? log2f((float)n) : 0.f;
+    } else {
+      b = (c == 1) ? p.log2_r : p.log2_v;
+    }
+    if (p.bits) p.bits[r] = b;
+    sum += b;
+  }
+  if (p.seq_bits == nullptr) return;
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, m);
+  __shared__ float part[kK3Threads / 32];
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = sum;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int w = 0; w < kK3Threads / 32; ++w) t += part[w];
+    p.seq_bits[seq] = t;
+  }
+}
+
+cudaError_t launch_bits(const BitsParams& p, cudaStream_t stream) {
+  const int64_t blocks = p.seq_offsets ? p.n_seq : 1;
+  if (blocks <= 0) return cudaSuccess;
+  k3_bits<<<(unsigned)blocks, kK3Threads, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
 }  // namespace difr

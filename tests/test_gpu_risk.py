@@ -1,0 +1,176 @@
+"""GPU-vs-oracle parity of the widened path: raw-logit rank and the three risk
+classes, both estimators from one pass, admissible-set sizes and the
+information bound.  Where floating point decides an integer (a rank, a set
+size) the kernel decides on its fp32 values, so the test accepts any integer
+the oracle reaches when the deciding quantity moves by the kernel's rounding
+error, and asks for equality with the oracle on almost every row."""
+import math
+
+import numpy as np
+import pytest
+import torch
+from scipy.special import ndtr
+
+import oracle
+import workloads as wl
+from gpu_util import Device, f32, to_dev
+
+import paper_2511_02620_b200 as difr
+
+pytestmark = pytest.mark.gpu
+
+EPS = 1e-12
+SCORE_TOL = 2e-3
+LOGIT_DELTA = 2e-5   # fp32 accumulation error of a tensor-core logit of unit scale (measured: ~2e-6)
+Y_DELTA = 1e-3       # error of the kernel's fp32 noisy logit (two lg2.approx): ~2.4e-4 * Temp
+
+
+def _small(T, d, V, seed):
+    g = np.random.default_rng(seed)
+    h = wl.f32_to_bf16_bits(g.standard_normal((T, d)).astype(np.float32))
+    W = wl.f32_to_bf16_bits((g.standard_normal((V, d)) / math.sqrt(d)).astype(np.float32))
+    seeds = np.array([wl.splitmix64(seed * 1000 + r // 64) for r in range(T)], dtype=np.uint64)
+    positions = (np.arange(T) % 64 + 1).astype(np.uint32)
+    return h, W, seeds, positions
+
+
+def _claims(h, W, seeds, positions, temperature, seed):
+    honest, runner = oracle.sample_gm(h, W, seeds, positions, temperature)
+    g = np.random.default_rng(seed)
+    T, V = h.shape[0], W.shape[0]
+    tokens = honest.copy()
+    k = np.arange(T)
+    tokens[k % 5 == 1] = runner[k % 5 == 1]
+    rnd = g.integers(0, V, size=T)
+    tokens[k % 5 == 3] = rnd[k % 5 == 3]
+    return tokens.astype(np.int32)
+
+
+def _score(dev, fn, tokens, temperature, sigma, want_rank=False, sigma_ipt=0.0):
+    out = difr.DifrOut.allocate(dev.T, dev.d, dev.V, sigma, EPS)
+    f = lambda: torch.full((dev.T,), float("nan"), dtype=torch.float32, device="cuda")
+    out.y_max, out.y_second = f(), f()
+    if want_rank:
+        out.rank = torch.full((dev.T,), -7, dtype=torch.int32, device="cuda")
+    if sigma_ipt:
+        out.sigma_ipt, out.score_ipt = sigma_ipt, f()
+    fn(dev.h, dev.W, to_dev(np.asarray(tokens, dtype=np.int32)), dev.seeds, dev.positions, f32(temperature), out)
+    torch.cuda.synchronize()
+    assert int(out.device_status.item()) == 0
+    return out
+
+
+@pytest.mark.parametrize("T,d,V,temperature", [(300, 128, 3000, 1.0), (130, 72, 777, 0.7)])
+def test_rank_and_three_classes(T, d, V, temperature):
+    h, W, seeds, positions = _small(T, d, V, 21)
+    tokens = _claims(h, W, seeds, positions, f32(temperature), 22)
+    tokens[7] = V + 5  # an id outside the vocabulary
+    dev = Device(h, W, seeds, positions)
+    sigma = 0.3
+    out = _score(dev, difr.difr_score_gm, tokens, temperature, sigma, want_rank=True)
+    plain = _score(dev, difr.difr_score_gm, tokens, temperature, sigma)
+    assert torch.equal(out.score, plain.score) and torch.equal(out.argmax, plain.argmax)  # asking for ranks changes nothing else
+    ref = oracle.score_gm(h, W, tokens, seeds, positions, f32(temperature), f32(sigma), f32(EPS))
+    got = out.rank.cpu().numpy()
+    logits = oracle.logits(h, W)
+    ok = (tokens >= 0) & (tokens < V)
+    lt = logits[np.arange(T), np.where(ok, tokens, 0)][:, None]
+    others = np.ones((T, V), dtype=bool)
+    others[np.arange(T)[ok], tokens[ok]] = False
+    lo = ((logits > lt + LOGIT_DELTA) & others).sum(axis=1)
+    hi = ((logits > lt - LOGIT_DELTA) & others).sum(axis=1)
+    assert np.all(got[ok] >= lo[ok]) and np.all(got[ok] <= hi[ok])
+    assert np.all(got[~ok] == V) and np.all(ref.rank[~ok] == V)
+    assert (got == ref.rank).mean() >= 0.98
+    assert got[ok].max() > V // 2 and got[ok].min() < 10  # both ends of the range are exercised
+
+    # three classes: decided where neither the score nor the rank sits on its boundary
+    score = out.score.cpu().numpy()
+    np.testing.assert_allclose(score, ref.score, rtol=0, atol=SCORE_TOL)
+    tau, R = -1.5, 200
+    want = oracle.classify(ref.score, tau, ref.rank, R)
+    flags = torch.full((T,), 9, dtype=torch.uint8, device="cuda")
+    difr.difr_detect(out.score, tau, out.margin, out.rank, R, None, flags, None)
+    torch.cuda.synchronize()
+    decided = (np.abs(ref.score - tau) > 2 * SCORE_TOL) & (lo == hi)
+    assert decided.mean() > 0.9
+    assert np.array_equal(flags.cpu().numpy()[decided], want[decided])
+    assert set(np.unique(want[decided])) == {0, 1, 2}
+
+
+def test_both_scores_from_one_pass_equal_the_two_separate_calls():
+    T, d, V = 260, 136, 2100
+    h, W, seeds, positions = _small(T, d, V, 31)
+    tokens = _claims(h, W, seeds, positions, f32(0.7), 32)
+    dev = Device(h, W, seeds, positions)
+    both = _score(dev, difr.difr_score_both, tokens, 0.7, 0.3, sigma_ipt=0.05)
+    gm = _score(dev, difr.difr_score_gm, tokens, 0.7, 0.3)
+    ipt = _score(dev, difr.difr_score_ipt, tokens, 0.7, 0.05)
+    for name in ("score", "margin", "argmax", "runner_up", "y_max", "y_second"):
+        assert torch.equal(getattr(both, name), getattr(gm, name)), name
+    assert torch.equal(both.score_ipt, ipt.score)
+    for name in ("p_claimed", "cdf_lo", "u", "lse"):
+        assert torch.equal(getattr(both, name), getattr(ipt, name)), name
+    ref_gm = oracle.score_gm(h, W, tokens, seeds, positions, f32(0.7), f32(0.3), f32(EPS))
+    ref_ipt = oracle.score_ipt(h, W, tokens, seeds, positions, f32(0.7), f32(0.05), f32(EPS))
+    np.testing.assert_allclose(both.score.cpu().numpy(), ref_gm.score, rtol=0, atol=SCORE_TOL)
+    np.testing.assert_allclose(both.score_ipt.cpu().numpy(), ref_ipt.score, rtol=0, atol=SCORE_TOL)
+    # y_max / y_second are the two largest noisy logits
+    np.testing.assert_allclose(both.y_max.cpu().numpy() - both.y_second.cpu().numpy(), ref_gm.top2_margin, atol=1e-4)
+
+
+def _noisy_logits(h, W, seeds, positions, temperature):
+    T, V = h.shape[0], W.shape[0]
+    y = oracle.logits(h, W)
+    for r in range(T):
+        y[r] += temperature * oracle.gumbel_noise_row(int(seeds[r]), int(positions[r]), V)
+    return y
+
+
+@pytest.mark.parametrize("T,d,V,temperature,sigma", [(150, 64, 1200, 1.0, 1.0), (140, 72, 520, 0.7, 0.3)])
+def test_admissible_set_sizes_and_information_bound(T, d, V, temperature, sigma):
+    h, W, seeds, positions = _small(T, d, V, 41)
+    dev = Device(h, W, seeds, positions)
+    tokens = _claims(h, W, seeds, positions, f32(temperature), 42)
+    scored = _score(dev, difr.difr_score_gm, tokens, temperature, sigma, want_rank=True)
+    taus = [f32(-0.9), f32(-3.0), f32(-9.0), f32(math.log(EPS))]  # the last: every id is admissible
+    counts = torch.full((len(taus), T), -1, dtype=torch.int32, device="cuda")
+    difr.difr_admissible(dev.h, dev.W, dev.seeds, dev.positions, f32(temperature), scored, taus, counts)
+    one = torch.full((1, T), -1, dtype=torch.int32, device="cuda")
+    difr.difr_admissible(dev.h, dev.W, dev.seeds, dev.positions, f32(temperature), scored, taus[1:2], one)
+    torch.cuda.synchronize()
+    assert int(scored.device_status.item()) == 0
+    got = counts.cpu().numpy()
+    assert np.array_equal(one.cpu().numpy()[0], got[1])  # one bound or four: the same count
+
+    # the oracle's sets, and the sets reachable when every margin moves by the kernel's rounding error
+    y = _noisy_logits(h, W, seeds, positions, f32(temperature))
+    order = np.sort(y, axis=1)
+    ymax, ysec = order[:, -1:], order[:, -2:-1]
+    A = np.where(y == ymax, ymax - ysec, y - ymax)
+
+    def size(shift, tau):
+        return (np.log(ndtr((A + shift) / (f32(sigma) * math.sqrt(2.0))) + f32(EPS)) >= tau).sum(axis=1)
+
+    exact = 0
+    for j, tau in enumerate(taus):
+        want = oracle.admissible_count(h, W, seeds, positions, f32(temperature), f32(sigma), tau, f32(EPS))
+        assert np.array_equal(size(0.0, tau), want)
+        assert np.all(got[j] >= size(-Y_DELTA, tau)) and np.all(got[j] <= size(+Y_DELTA, tau)), j
+        exact += (got[j] == want).sum()
+    assert exact >= 0.97 * len(taus) * T
+    assert np.all(got[3] == V) and got[0].max() < V and got[2].max() > got[0].max()
+
+    # information bound per token and per sequence
+    tau, R = taus[1], 8
+    flags = torch.empty(T, dtype=torch.uint8, device="cuda")
+    difr.difr_detect(scored.score, tau, scored.margin, scored.rank, R, None, flags, None)
+    seq_offsets = np.array([0, T // 3, T // 3, T], dtype=np.int32)  # one empty sequence
+    bits = torch.full((T,), float("nan"), dtype=torch.float32, device="cuda")
+    seq_bits = torch.full((3,), float("nan"), dtype=torch.float32, device="cuda")
+    difr.difr_exfiltratable_bits(flags, counts[1], R, V, to_dev(seq_offsets), bits, seq_bits)
+    torch.cuda.synchronize()
+    want_bits, want_seq = oracle.exfiltratable_bits(flags.cpu().numpy(), got[1], R, V, seq_offsets)
+    np.testing.assert_allclose(bits.cpu().numpy(), want_bits, rtol=1e-6, atol=1e-6)
+    np.testing.assert_allclose(seq_bits.cpu().numpy(), want_seq, rtol=1e-5)
+    assert seq_bits.cpu().numpy()[1] == 0.0
