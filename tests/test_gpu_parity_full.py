@@ -131,3 +131,61 @@ def test_full_size_ipt(name, T, temperature, sigma):
     assert np.all(got["row_status"] == 0)
     assert np.all((got["cdf_lo"] >= -1e-6) & (got["cdf_lo"] <= 1 + 1e-6))
     assert np.all((got["u"] > 0) & (got["u"] < 1))
+
+
+@pytest.mark.parametrize("name,T,temperature,sigma", [("llama3b", 0, 1.0, 1.0), ("moe30b", 0, 0.7, 0.3)])
+def test_full_size_rank_both_and_admissible_sets(name, T, temperature, sigma):
+    """The widened calls at full size: ranks, both scores and admissible-set sizes on sampled rows against the
+    oracle (integers within the reach of the kernel's fp32 rounding, equal on almost every row), and
+    size-independent properties on all rows."""
+    from scipy.special import ndtr
+
+    w, inp, dev = _inputs(name, T)
+    rows = wl.sample_rows(w, 24, salt=2)
+    g = np.random.default_rng(wl.stream_seed(w, 9))
+    tokens = g.integers(0, w.V, size=w.T).astype(np.int32)
+    tokens[rows] = _sampled_claims(w, inp, rows, f32(temperature), "gm")
+    out = difr.DifrOut.allocate(w.T, w.d, w.V, sigma, EPS)
+    f = lambda: torch.full((w.T,), float("nan"), dtype=torch.float32, device="cuda")
+    out.y_max, out.y_second, out.score_ipt, out.sigma_ipt = f(), f(), f(), 0.05
+    out.rank = torch.full((w.T,), -7, dtype=torch.int32, device="cuda")
+    difr.difr_score_both(dev.h, dev.W, to_dev(tokens), dev.seeds, dev.positions, f32(temperature), out)
+    taus = [f32(-0.9), f32(-3.0)]
+    counts = torch.full((2, w.T), -1, dtype=torch.int32, device="cuda")
+    difr.difr_admissible(dev.h, dev.W, dev.seeds, dev.positions, f32(temperature), out, taus, counts)
+    torch.cuda.synchronize()
+    assert int(out.device_status.item()) == 0
+
+    hs, Ws = np.ascontiguousarray(inp.h[rows]), inp.W
+    ref = oracle.score_gm(hs, Ws, tokens[rows], inp.seeds[rows], inp.positions[rows], f32(temperature), f32(sigma),
+                          f32(EPS))
+    ref_ipt = oracle.score_ipt(hs, Ws, tokens[rows], inp.seeds[rows], inp.positions[rows], f32(temperature),
+                               f32(0.05), f32(EPS))
+    np.testing.assert_allclose(out.score.cpu().numpy()[rows], ref.score, rtol=0, atol=SCORE_TOL)
+    np.testing.assert_allclose(out.score_ipt.cpu().numpy()[rows], ref_ipt.score, rtol=0, atol=SCORE_TOL)
+    # ranks
+    logits = oracle.logits(hs, Ws)
+    lt = logits[np.arange(len(rows)), tokens[rows]][:, None]
+    others = np.ones_like(logits, dtype=bool)
+    others[np.arange(len(rows)), tokens[rows]] = False
+    lo = ((logits > lt + 2e-5) & others).sum(axis=1)
+    hi = ((logits > lt - 2e-5) & others).sum(axis=1)
+    rank = out.rank.cpu().numpy()
+    assert np.all(rank[rows] >= lo) and np.all(rank[rows] <= hi)
+    assert (rank[rows] == ref.rank).mean() >= 0.9
+    assert np.all((rank >= 0) & (rank < w.V))
+    # admissible sets
+    y = logits.copy()
+    for i, r in enumerate(rows):
+        y[i] += f32(temperature) * oracle.gumbel_noise_row(int(inp.seeds[r]), int(inp.positions[r]), w.V)
+    order = np.sort(y, axis=1)
+    ymax, ysec = order[:, -1:], order[:, -2:-1]
+    A = np.where(y == ymax, ymax - ysec, y - ymax)
+    got = counts.cpu().numpy()
+    for j, tau in enumerate(taus):
+        size = lambda shift: (np.log(ndtr((A + shift) / (f32(sigma) * np.sqrt(2.0))) + f32(EPS)) >= tau).sum(axis=1)
+        want = oracle.admissible_count(hs, Ws, inp.seeds[rows], inp.positions[rows], f32(temperature), f32(sigma),
+                                       tau, f32(EPS))
+        assert np.array_equal(size(0.0), want)
+        assert np.all(got[j][rows] >= size(-1e-3)) and np.all(got[j][rows] <= size(1e-3))
+    assert np.all(got[0] <= got[1]) and np.all(got[1] >= 1) and np.all(got[1] <= w.V)
