@@ -6,6 +6,10 @@
 #include <stdint.h>
 #include <stdlib.h>
 
+#include <functional>
+#include <queue>
+#include <vector>
+
 namespace difr {
 
 constexpr int kBM = 128;        // rows (tokens) per CTA tile
@@ -30,6 +34,27 @@ struct Plan {
 inline int env_int(const char* name, int fallback) {
   const char* v = getenv(name);
   return (v && *v) ? atoi(v) : fallback;
+}
+
+// Tile times until the last pair is done when the units (in raster order, each as long as its strip, plus
+// a small fixed cost per unit) are taken on demand by `num_pairs` pairs that all start together.
+inline double makespan_tiles(int m_tiles, int n_tiles, int S, int gm, int num_pairs) {
+  std::priority_queue<double, std::vector<double>, std::greater<double>> free_at;
+  for (int i = 0; i < num_pairs; ++i) free_at.push(0.0);
+  double last = 0.0;
+  for (int m0 = 0; m0 < m_tiles; m0 += gm) {
+    const int cnt = (m_tiles - m0 < gm) ? m_tiles - m0 : gm;
+    for (int strip = 0; strip < S; ++strip) {
+      const int n0 = (int)(((long long)strip * n_tiles) / S), n1 = (int)(((long long)(strip + 1) * n_tiles) / S);
+      for (int i = 0; i < cnt; ++i) {
+        const double t = free_at.top() + (double)(n1 - n0) + 0.05;
+        free_at.pop();
+        free_at.push(t);
+        if (t > last) last = t;
+      }
+    }
+  }
+  return last;
 }
 
 // A unit walks its strip tile by tile keeping running statistics in registers and
@@ -57,10 +82,10 @@ inline bool make_plan(int64_t T, int64_t d, int64_t V, int num_pairs, Plan* out)
   if (gm < 4) gm = 4;
   int len_target = 8;
   if (len_target > p.n_tiles) len_target = p.n_tiles;
-  // strip count: n_tiles / len_target when there are many rounds of units; otherwise the count
-  // near it (or, for small problems, up to one unit per pair) with the fewest tiles on the critical path
+  // strip count: n_tiles / len_target when there are many rounds of units; otherwise the count near it
+  // (or, for small problems, up to one unit per pair) whose on-demand schedule finishes first
   int best_S = (p.n_tiles + len_target - 1) / len_target;
-  if ((long long)p.m_tiles * best_S < 8LL * num_pairs) {
+  if ((long long)p.m_tiles * best_S < 64LL * num_pairs) {
     int s_lo = (2 * p.n_tiles + 3 * len_target - 1) / (3 * len_target);
     int s_hi = (4 * p.n_tiles + 3 * len_target - 1) / (3 * len_target);
     if (s_hi < num_pairs / p.m_tiles) s_hi = num_pairs / p.m_tiles;
@@ -69,10 +94,7 @@ inline bool make_plan(int64_t T, int64_t d, int64_t V, int num_pairs, Plan* out)
     if (s_lo > s_hi) s_lo = s_hi;
     double best_cost = 1e300;
     for (int S = s_lo; S <= s_hi; ++S) {
-      long long units = (long long)p.m_tiles * S;
-      long long waves = (units + num_pairs - 1) / num_pairs;
-      long long len = (p.n_tiles + S - 1) / S;
-      double cost = (double)waves * (double)len + 0.25 * (double)waves;
+      const double cost = makespan_tiles(p.m_tiles, p.n_tiles, S, gm, num_pairs) + 0.02 * S;
       if (cost < best_cost - 1e-9) {
         best_cost = cost;
         best_S = S;
