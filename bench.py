@@ -323,28 +323,52 @@ def run_ours(args):
     score_host = torch.empty(T, dtype=torch.float32).pin_memory()
     flags_host = torch.empty(T, dtype=torch.uint8).pin_memory()
     stats_host = torch.empty((n_seq, 4), dtype=torch.int32).pin_memory()
-    h_in = torch.empty_like(h_dev)
-    tok_in, seed_in, pos_in = torch.empty_like(tokens_dev), torch.empty_like(seeds_dev), torch.empty_like(pos_dev)
+    # Two input buffers: a copy stream uploads step i + 1 while the kernels of step i run (what a serving
+    # loop does); every step's upload, kernels and read-back lie inside the timed region.
+    copy_stream, run_stream = torch.cuda.Stream(), torch.cuda.current_stream()
+    bufs = [(torch.empty_like(h_dev), torch.empty_like(tokens_dev), torch.empty_like(seeds_dev),
+             torch.empty_like(pos_dev)) for _ in range(2)]
+    uploaded = [torch.cuda.Event() for _ in range(2)]
+    consumed = [torch.cuda.Event() for _ in range(2)]
 
-    def e2e_step():
-        h_in.view(torch.int16).copy_(h_host, non_blocking=True)
-        tok_in.copy_(tokens_host, non_blocking=True)
-        seed_in.copy_(seeds_host, non_blocking=True)
-        pos_in.copy_(pos_host, non_blocking=True)
+    def upload(i):
+        h_in, tok_in, seed_in, pos_in = bufs[i % 2]
+        with torch.cuda.stream(copy_stream):
+            copy_stream.wait_event(consumed[i % 2])  # the kernels that last read this buffer are done
+            h_in.view(torch.int16).copy_(h_host, non_blocking=True)
+            tok_in.copy_(tokens_host, non_blocking=True)
+            seed_in.copy_(seeds_host, non_blocking=True)
+            pos_in.copy_(pos_host, non_blocking=True)
+            uploaded[i % 2].record(copy_stream)
+
+    def run(i):
+        h_in, tok_in, seed_in, pos_in = bufs[i % 2]
+        run_stream.wait_event(uploaded[i % 2])
         difr.difr_score_gm(h_in, W_dev, tok_in, seed_in, pos_in, temperature, out)
         difr.difr_detect(out.score, tau, out.margin, None, 0, seq_dev, flags, stats)
+        consumed[i % 2].record(run_stream)
         score_host.copy_(out.score, non_blocking=True)
         flags_host.copy_(flags, non_blocking=True)
         stats_host.copy_(stats, non_blocking=True)
 
-    for _ in range(min(args.warmup, 3)):
-        e2e_step()
+    def e2e_loop(n):
+        upload(0)
+        for i in range(n):
+            if i + 1 < n:
+                upload(i + 1)
+            run(i)
+
+    for ev in consumed:
+        ev.record(run_stream)
+    e2e_loop(min(args.warmup, 3))
     barrier()
     e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e_begin.record()
-    for _ in range(args.steps):
-        e2e_step()
-    e_end.record()
+    for ev in consumed:
+        ev.record(run_stream)
+    e_begin.record(run_stream)
+    copy_stream.wait_event(e_begin)  # the first upload starts inside the timed region
+    e2e_loop(args.steps)
+    e_end.record(run_stream)
     barrier()
     e2e_ms = e_begin.elapsed_time(e_end)
     h2d = h_host.numel() * 2 + tokens_host.numel() * 4 + seeds_host.numel() * 8 + pos_host.numel() * 4
@@ -367,7 +391,8 @@ def run_ours(args):
             "clocks": clocks,
             "e2e": {"value": whole_job_rate(world, T, args.steps, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps,
-                    "note": "per-step inputs (h, tokens, seeds, positions) from pinned host memory; W resident"},
+                    "note": "per-step inputs (h, tokens, seeds, positions) from pinned host memory, uploaded on a copy "
+                            "stream one step ahead of the kernels; scores, flags and statistics read back; W resident"},
             "gpu_launches": 3 * args.steps,
             "roofline": {"kernel": "k1_fused_score", "bound": "tensor", "achieved": achieved,
                          "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
