@@ -61,6 +61,8 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).argtypes = [ctypes.c_uint32]
         L.oracle_gumbel_noise.restype = ctypes.c_double
         L.oracle_gumbel_noise.argtypes = [ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint32]
+        L.oracle_gumbel_row.restype = None
+        L.oracle_gumbel_row.argtypes = [ctypes.c_uint64, ctypes.c_uint32, ctypes.c_int64, ctypes.c_void_p]
         L.oracle_ipt_uniform.restype = ctypes.c_double
         L.oracle_ipt_uniform.argtypes = [ctypes.c_uint64, ctypes.c_uint32]
         L.oracle_normal_cdf.restype = ctypes.c_double
@@ -143,7 +145,9 @@ def gumbel_noise(seed: int, position: int, idx: int) -> float:
 
 
 def gumbel_noise_row(seed: int, position: int, V: int) -> np.ndarray:
-    return np.array([gumbel_noise(seed, position, v) for v in range(V)], dtype=np.float64)
+    out = np.zeros(V, dtype=np.float64)
+    lib().oracle_gumbel_row(int(seed), int(position), int(V), _p(out))
+    return out
 
 
 def ipt_uniform(seed: int, position: int) -> float:

@@ -106,6 +106,11 @@ double oracle_gumbel_noise(uint64_t seed, uint32_t position, uint32_t id) {
   return oracle_gumbel(oracle_ro_word(seed, position, 0u, id));
 }
 
+/* The whole row of Gumbel noise, ids 0..V-1. */
+void oracle_gumbel_row(uint64_t seed, uint32_t position, int64_t V, double* out) {
+  for (int64_t v = 0; v < V; ++v) out[v] = oracle_gumbel_noise(seed, position, (uint32_t)v);
+}
+
 double oracle_ipt_uniform(uint64_t seed, uint32_t position) {
   return oracle_uniform32(oracle_ro_word(seed, position, 1u, 0u));
 }

@@ -1,0 +1,110 @@
+"""Alg. Token-DiFR in full: top-k / top-p cutoff, the B_i terms and an active
+subset of s competitors -- TEST INFRASTRUCTURE, plain numpy / scipy.
+
+    pi = E_{x ~ N(0, sigma^2)} [ 1{l_t* + x > cutoff} * prod_{i in S} Phi(max(x + A_i, B_i) / sigma) ]
+
+with S the top-s ids by y = l + Temp*G (the claimed token left out),
+A_i = y_t* - y_i, B_i = cutoff - l_i, and `cutoff` the smallest logit that
+survives the sampling filter (the reading of the algorithm's garbled cutoff
+line): keep the top_k largest logits, then, among those, the shortest prefix in
+descending order whose renormalised temperature-softmax mass reaches top_p.
+The expectation is evaluated by adaptive quadrature (a library routine) split at
+the kinks of the integrand; the algorithm's own Monte-Carlo loop is in
+`posterior.token_difr_monte_carlo`.
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+from scipy.integrate import quad
+from scipy.special import log_ndtr
+
+from . import posterior
+
+
+def filter_cutoff(logits: np.ndarray, temperature: float, top_k: int, top_p: float) -> float:
+    """Smallest logit that survives top-k followed by top-p (-inf when neither is set)."""
+    logits = np.asarray(logits, dtype=np.float64)
+    V = logits.shape[0]
+    k_on = 0 < top_k < V
+    p_on = top_p < 1.0
+    if not k_on and not p_on:
+        return -math.inf
+    order = np.argsort(-logits, kind="stable")  # descending, ties: lowest id first
+    kept = order[:top_k] if k_on else order
+    if p_on:
+        if temperature > 0.0:
+            z = logits[kept] / temperature
+            p = np.exp(z - z.max())
+            c = np.cumsum(p) / p.sum()
+            n = int(np.searchsorted(c, top_p, side="left")) + 1  # first prefix whose mass is >= top_p
+        else:
+            n = 1  # a greedy sampler's nucleus is the largest logit
+        kept = kept[: min(n, len(kept))]
+    return float(logits[kept[-1]])
+
+
+def token_difr_filtered(logits, gumbel, temperature, claimed, s, sigma, cutoff=-math.inf) -> float:
+    """The expectation above, by adaptive quadrature."""
+    logits = np.asarray(logits, dtype=np.float64)
+    gumbel = np.asarray(gumbel, dtype=np.float64)
+    y = logits + temperature * gumbel
+    S = posterior.active_subset(y, claimed, s)
+    A = posterior.margins(logits, gumbel, temperature, claimed, S)
+    B = cutoff - logits[S]
+
+    def integrand(x):
+        t = np.maximum(x + A, B) / sigma
+        return math.exp(-0.5 * (x / sigma) ** 2 + float(np.sum(log_ndtr(t)))) / (sigma * math.sqrt(2.0 * math.pi))
+
+    lo = max(cutoff - logits[claimed], -14.0 * sigma)
+    hi = max(14.0 * sigma, float(np.max(-A, initial=0.0)) + 14.0 * sigma)
+    if lo >= hi:
+        return 0.0
+    kinks = [float(b - a) for a, b in zip(A, B) if np.isfinite(b) and lo < b - a < hi]
+    # break the range where the integrand peaks as well: the peak is narrow (about sigma) in a wide range
+    grid = np.linspace(lo, hi, 2001)
+    peak = float(grid[int(np.argmax([integrand(x) for x in grid]))])
+    pts = sorted(set(kinks + [p for p in (peak - sigma, peak, peak + sigma) if lo < p < hi]))
+    val, _ = quad(integrand, lo, hi, points=pts or None, epsabs=1e-18, epsrel=1e-11, limit=400)
+    return float(min(max(val, 0.0), 1.0))
+
+
+def model_posterior_mc(logits, gumbel, temperature, claimed, sigma, cutoff, n_draws, rng) -> float:
+    """The event the expectation measures, simulated literally with every id a competitor: each logit gets an
+    independent N(0, sigma^2) perturbation; an id takes part iff its perturbed logit exceeds the (fixed) cutoff;
+    the claimed token comes out iff it takes part and beats every other participant under the fixed noise."""
+    logits = np.asarray(logits, dtype=np.float64)
+    gumbel = np.asarray(gumbel, dtype=np.float64)
+    V = logits.shape[0]
+    hits = done = 0
+    while done < n_draws:
+        n = min(200_000, n_draws - done)
+        pert = logits[None, :] + sigma * rng.standard_normal((n, V))
+        alive = pert > cutoff
+        yy = np.where(alive, pert + temperature * gumbel[None, :], -np.inf)
+        others = np.delete(yy, claimed, axis=1).max(axis=1)
+        hits += int(np.sum(alive[:, claimed] & (yy[:, claimed] > others)))
+        done += n
+    return hits / n_draws
+
+
+def score_gm_filtered(h_bits, W_bits, tokens, seeds, positions, temperature, sigma, eps=1e-12, top_k=0, top_p=1.0,
+                      s=1):
+    """Per row: (score = ln(pi + eps), pi, cutoff).  Out-of-range claims score ln(eps)."""
+    from . import gumbel_noise_row, logits as all_logits
+
+    L = all_logits(h_bits, W_bits)
+    T, V = L.shape
+    score = np.empty(T)
+    pi = np.zeros(T)
+    cut = np.empty(T)
+    for r in range(T):
+        cut[r] = filter_cutoff(L[r], temperature, top_k, top_p)
+        t = int(tokens[r])
+        if 0 <= t < V:
+            G = gumbel_noise_row(int(seeds[r]), int(positions[r]), V)
+            pi[r] = token_difr_filtered(L[r], G, temperature, t, s, sigma, cut[r])
+        score[r] = math.log(pi[r] + eps)
+    return score, pi, cut
