@@ -76,7 +76,8 @@ typedef struct {
   float* p_claimed;   /* IPT: softmax probability of the claimed token            */
   float* cdf_lo;      /* IPT: a = sum_{v < t*} p_v                                 */
   float* u;           /* IPT: the uniform mu of this row                           */
-  uint32_t* row_status; /* bit0: claimed id outside [0, V); bit1: non-finite logits */
+  uint32_t* row_status; /* bit0: claimed id outside [0, V); bit1: non-finite logits;
+                           bit2: candidate list overflow (difr_score_gm_filtered)         */
   void* workspace;      /* >= difr_workspace_bytes(T, d, V) bytes, 16-byte aligned;
                            contents are scratch, overwritten by every call         */
   size_t workspace_bytes;
@@ -96,6 +97,7 @@ typedef struct {
   float* y_second;   /* GM, optional: the second largest y                                     */
   float sigma_ipt;   /* difr_score_both only: noise width of the IPT estimator (CDF units), > 0 */
   float* score_ipt;  /* difr_score_both only, required there: ln(mass + eps)                   */
+  float* cutoff;     /* difr_score_gm_filtered only, optional: the filter's cutoff per row     */
 } difr_out;
 
 /* Scratch bytes a scoring call needs for T rows, hidden size d, vocabulary V.
@@ -184,6 +186,45 @@ difr_status difr_score_gm_static(const void* h, const void* W, const int32_t* to
 difr_status difr_score_both(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,
                             const uint32_t* positions, float temperature, int64_t T, int64_t d, int64_t V,
                             difr_out* out, difr_stream_t stream);
+
+/*
+ * Token-DiFR in full (Alg. "Token-DiFR"): the sampling filter's cutoff, the
+ * B_i terms and an active subset of s competitors,
+ *
+ *   pi = E_{x ~ N(0, sigma^2)} [ 1{l_t* + x > cutoff} prod_{i in S} Phi(max(x + A_i, B_i) / sigma) ],
+ *
+ * S = the s ids with the largest y = l + Temp*G other than t*, A_i = y_t* - y_i,
+ * B_i = cutoff - l_i, score = ln(pi + eps).  `cutoff` is the smallest logit that
+ * survives the filter: the top_k largest logits are kept, then, among those,
+ * the shortest prefix in descending order whose renormalised softmax(l / Temp)
+ * mass reaches top_p.  The expectation is evaluated by Gauss-Legendre quadrature
+ * (512 nodes over the range that carries the mass), not by sampling.
+ *
+ *   filter->top_k  0: no top-k; otherwise 1..64 (a top_k >= V filters nothing)
+ *   filter->top_p  in (0, 1]; 1: no nucleus; < 1 requires top_k >= 1
+ *   filter->s      1..8
+ *   temperature > 0
+ *   out->workspace needs difr_filtered_workspace_bytes(T, d, V) bytes
+ *
+ * Everything difr_score_gm writes is written as there (margin, argmax, runner_up,
+ * lse, y_max, y_second; `rank` is not available in this call); `score` holds
+ * the full estimator and out->cutoff, if given, the cutoff per row (-inf: no
+ * filter).  Two passes over the logits: the scoring pass, then a pass that
+ * collects, per row, the ids that can be among the s + 2 best or among the top_k
+ * logits (about 3 KB of list per row; row_status bit 2 marks a row whose list
+ * overflowed, which takes hundreds of logits within rounding of the top_k-th).
+ * With s = 1 and no filter the result equals difr_score_gm's up to quadrature
+ * error (< 1e-6 in the score).
+ */
+typedef struct {
+  int32_t top_k;
+  float top_p;
+  int32_t s;
+} difr_filter;
+size_t difr_filtered_workspace_bytes(int64_t T, int64_t d, int64_t V);
+difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,
+                                   const uint32_t* positions, float temperature, int64_t T, int64_t d, int64_t V,
+                                   const difr_filter* filter, difr_out* out, difr_stream_t stream);
 
 /*
  * Sizes of the admissible sets A_t(tau) = { i : FSSL_t(i) >= tau } (Sec.

@@ -18,7 +18,8 @@ DIFR_OK = 0
 STATUS_NAMES = {0: "DIFR_OK", -1: "DIFR_ERR_INVALID_ARG", -2: "DIFR_ERR_SHAPE", -3: "DIFR_ERR_ALIGN",
                 -4: "DIFR_ERR_WORKSPACE", -5: "DIFR_ERR_CUDA", -6: "DIFR_ERR_ARCH", -7: "DIFR_ERR_TIMEOUT"}
 
-EXPORTS = ("difr_workspace_bytes", "difr_score_gm", "difr_score_ipt", "difr_score_both", "difr_score_gm_static",
+EXPORTS = ("difr_workspace_bytes", "difr_filtered_workspace_bytes", "difr_score_gm", "difr_score_ipt",
+           "difr_score_both", "difr_score_gm_filtered", "difr_score_gm_static",
            "difr_admissible", "difr_exfiltratable_bits", "difr_detect", "difr_logits", "difr_philox",
            "difr_status_string", "difr_version")
 STATIC_SCRATCH_BYTES = 16 << 20  # DIFR_STATIC_SCRATCH_BYTES
@@ -39,8 +40,12 @@ class _COut(ctypes.Structure):
         ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t), ("device_status", ctypes.c_void_p),
         ("event_fused_start", ctypes.c_void_p), ("event_fused_stop", ctypes.c_void_p),
         ("rank", ctypes.c_void_p), ("y_max", ctypes.c_void_p), ("y_second", ctypes.c_void_p),
-        ("sigma_ipt", ctypes.c_float), ("score_ipt", ctypes.c_void_p),
+        ("sigma_ipt", ctypes.c_float), ("score_ipt", ctypes.c_void_p), ("cutoff", ctypes.c_void_p),
     ]
+
+
+class _CFilter(ctypes.Structure):
+    _fields_ = [("top_k", ctypes.c_int32), ("top_p", ctypes.c_float), ("s", ctypes.c_int32)]
 
 
 _lib = None
@@ -65,6 +70,11 @@ def lib() -> ctypes.CDLL:
         L.difr_detect.argtypes = [ctypes.c_void_p, ctypes.c_float, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32,
                                   ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p,
                                   ctypes.c_void_p]
+        L.difr_filtered_workspace_bytes.restype = ctypes.c_size_t
+        L.difr_filtered_workspace_bytes.argtypes = [ctypes.c_int64] * 3
+        L.difr_score_gm_filtered.restype = ctypes.c_int
+        L.difr_score_gm_filtered.argtypes = ([ctypes.c_void_p] * 5 + [ctypes.c_float] + [ctypes.c_int64] * 3
+                                             + [ctypes.POINTER(_CFilter), ctypes.POINTER(_COut), ctypes.c_void_p])
         L.difr_admissible.restype = ctypes.c_int
         L.difr_admissible.argtypes = ([ctypes.c_void_p] * 4 + [ctypes.c_float] + [ctypes.c_int64] * 3
                                       + [ctypes.c_void_p] * 3 + [ctypes.c_float] * 2
@@ -141,6 +151,7 @@ class DifrOut:
     y_second: "object" = None
     sigma_ipt: float = 0.0      # difr_score_both: width of the IPT estimator
     score_ipt: "object" = None  # difr_score_both: float [T]
+    cutoff: "object" = None     # difr_score_gm_filtered: float [T], the filter's cutoff per row
 
     @staticmethod
     def allocate(T: int, d: int, V: int, sigma: float, eps: float = 1e-12, device="cuda"):
@@ -160,7 +171,7 @@ class DifrOut:
                      _ptr(self.row_status), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
                      _ptr(self.device_status), ctypes.c_void_p(self.event_fused_start or None),
                      ctypes.c_void_p(self.event_fused_stop or None), _ptr(self.rank), _ptr(self.y_max),
-                     _ptr(self.y_second), float(self.sigma_ipt), _ptr(self.score_ipt))
+                     _ptr(self.y_second), float(self.sigma_ipt), _ptr(self.score_ipt), _ptr(self.cutoff))
 
 
 def _score(fn_name, h, W, tokens, seeds, positions, temperature, out: DifrOut, stream):
@@ -194,6 +205,31 @@ def difr_score_ipt(h, W, tokens, seeds, positions, temperature, out: DifrOut, st
 def difr_score_both(h, W, tokens, seeds, positions, temperature, out: DifrOut, stream=None) -> DifrOut:
     """Token-DiFR and Token-IPT-DiFR scores from one pass (`out.sigma_ipt`, `out.score_ipt`); see include/difr.h."""
     return _score("difr_score_both", h, W, tokens, seeds, positions, temperature, out, stream)
+
+
+def difr_filtered_workspace_bytes(T: int, d: int, V: int) -> int:
+    return int(lib().difr_filtered_workspace_bytes(T, d, V))
+
+
+def difr_score_gm_filtered(h, W, tokens, seeds, positions, temperature, top_k, top_p, s, out: DifrOut, stream=None):
+    """Alg. Token-DiFR in full: top-k / top-p cutoff, B_i terms, s competitors; `out.workspace` must hold
+    difr_filtered_workspace_bytes(T, d, V) bytes.  See include/difr.h."""
+    import torch
+
+    T, d = h.shape
+    V = W.shape[0]
+    _check(h, torch.bfloat16, (T, d), "h")
+    _check(W, torch.bfloat16, (V, d), "W")
+    _check(tokens, torch.int32, (T,), "tokens")
+    _check(seeds, torch.int64, (T,), "seeds")
+    _check(positions, torch.int32, (T,), "positions")
+    c = out._c()
+    f = _CFilter(int(top_k), float(top_p), int(s))
+    rc = lib().difr_score_gm_filtered(_ptr(h), _ptr(W), _ptr(tokens), _ptr(seeds), _ptr(positions),
+                                      float(temperature), T, d, V, ctypes.byref(f), ctypes.byref(c), _stream(stream))
+    if rc != DIFR_OK:
+        raise DifrError(rc, "difr_score_gm_filtered")
+    return out
 
 
 def difr_admissible(h, W, seeds, positions, temperature, scored: DifrOut, taus, counts, stream=None):

@@ -243,6 +243,154 @@ difr_status difr_admissible(const void* h, const void* W, const uint64_t* seeds,
   return DIFR_OK;
 }
 
+// ------------------------------------------------- full Token-DiFR estimator
+constexpr int kCandCap = 256;      // candidates kept per row when the vocabulary has at least 32 tiles
+constexpr int kFilterMinStrips = 32;
+
+// Layout behind the ordinary workspace: per-row candidate counters, then the candidate lists.
+static bool filtered_layout(int64_t T, int64_t d, int64_t V, int pairs, Plan* pl, int* cap, size_t* count_off,
+                            size_t* list_off, size_t* total) {
+  if (!make_plan(T, d, V, pairs, pl, kFilterMinStrips)) return false;
+  // with fewer than 32 vocabulary tiles the strips' maxima cannot bound the top_k-th logit: keep every id
+  *cap = (pl->n_tiles < kFilterMinStrips) ? (int)V : kCandCap;
+  *count_off = (pl->workspace_bytes + 255) & ~(size_t)255;
+  *list_off = *count_off + (((size_t)pl->T_pad * sizeof(int) + 255) & ~(size_t)255);
+  *total = *list_off + (size_t)T * (size_t)*cap * sizeof(Candidate);
+  return true;
+}
+
+// Nodes and weights of the n-point Gauss-Legendre rule on [-1, 1]: Newton's iteration on the Legendre
+// polynomial from the Chebyshev-like starting points, weights 2 / ((1 - x^2) P_n'(x)^2).
+static void gauss_legendre(int n, double* x, double* w) {
+  const double pi = 3.14159265358979323846;
+  for (int i = 0; i < n; ++i) {
+    double z = cos(pi * (i + 0.75) / (n + 0.5)), dp = 1.0;
+    for (int it = 0; it < 100; ++it) {
+      double p0 = 1.0, p1 = z;
+      for (int k = 2; k <= n; ++k) {
+        const double pk = ((2.0 * k - 1.0) * z * p1 - (k - 1.0) * p0) / k;
+        p0 = p1;
+        p1 = pk;
+      }
+      dp = n * (z * p1 - p0) / (z * z - 1.0);
+      const double dz = p1 / dp;
+      z -= dz;
+      if (fabs(dz) < 1e-16) break;
+    }
+    x[i] = z;
+    w[i] = 2.0 / ((1.0 - z * z) * dp * dp);
+  }
+}
+
+static difr_status ensure_quadrature_tables() {
+  constexpr int kMaxDevices = 64;
+  static bool done[kMaxDevices] = {false};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return DIFR_ERR_CUDA;
+  if (dev >= 0 && dev < kMaxDevices && done[dev]) return DIFR_OK;
+  double x[16], w[16];
+  gauss_legendre(16, x, w);
+  if (set_gauss_legendre(x, w) != cudaSuccess) return DIFR_ERR_CUDA;
+  if (dev >= 0 && dev < kMaxDevices) done[dev] = true;
+  return DIFR_OK;
+}
+
+size_t difr_filtered_workspace_bytes(int64_t T, int64_t d, int64_t V) {
+  DeviceInfo info;
+  if (!device_info(&info)) info.pairs = 0;
+  Plan pl;
+  int cap;
+  size_t count_off, list_off, total;
+  if (!filtered_layout(T, d, V, info.pairs, &pl, &cap, &count_off, &list_off, &total)) return 0;
+  return total;
+}
+
+difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,
+                                   const uint32_t* positions, float temperature, int64_t T, int64_t d, int64_t V,
+                                   const difr_filter* filter, difr_out* out, difr_stream_t stream) {
+  if (!h || !W || !tokens || !seeds || !positions || !out || !out->score || !filter) return DIFR_ERR_INVALID_ARG;
+  if (T < 0 || d <= 0 || V <= 0) return DIFR_ERR_INVALID_ARG;
+  if (!(out->sigma > 0.f) || !(out->eps >= 0.f) || !isfinite(out->sigma) || !isfinite(out->eps))
+    return DIFR_ERR_INVALID_ARG;
+  if (!(temperature > 0.f) || !isfinite(temperature)) return DIFR_ERR_INVALID_ARG;
+  int top_k = filter->top_k;
+  const float top_p = filter->top_p;
+  if (top_k < 0 || !(top_p > 0.f) || !(top_p <= 1.f) || filter->s < 1 || filter->s > 8) return DIFR_ERR_INVALID_ARG;
+  if (top_k >= V && top_p >= 1.f) top_k = 0;  // keeps the whole vocabulary: no filter
+  if (top_k > 64 && top_k < V) return DIFR_ERR_INVALID_ARG;
+  if (top_p < 1.f && (top_k < 1 || (top_k > 64 && V > 64))) return DIFR_ERR_INVALID_ARG;
+  if (top_k > V) top_k = (int)V;
+  if ((d % 8) != 0 || V < 2) return DIFR_ERR_SHAPE;
+  if (T == 0) return DIFR_OK;
+  DeviceInfo info;
+  if (!device_info(&info)) return DIFR_ERR_CUDA;
+  if (info.major != 10) return DIFR_ERR_ARCH;
+  Plan pl;
+  int cap;
+  size_t count_off, list_off, total;
+  if (!filtered_layout(T, d, V, info.pairs, &pl, &cap, &count_off, &list_off, &total)) return DIFR_ERR_SHAPE;
+  if (!aligned16(h) || !aligned16(W)) return DIFR_ERR_ALIGN;
+  if (!out->workspace || out->workspace_bytes < total) return DIFR_ERR_WORKSPACE;
+  if (!aligned16(out->workspace)) return DIFR_ERR_ALIGN;
+  const difr_status qs = ensure_quadrature_tables();
+  if (qs != DIFR_OK) return qs;
+  CUtensorMap tmap_h, tmap_w;
+  if (!make_tmap(&tmap_h, h, T, d, kBM) || !make_tmap(&tmap_w, W, V, d, kBN / 2)) return DIFR_ERR_CUDA;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  unsigned char* ws = static_cast<unsigned char*>(out->workspace);
+  const int grid = 2 * (pl.n_units < info.pairs ? pl.n_units : info.pairs);
+
+  // ---- first pass: the ordinary scoring pass, which also leaves each strip's two largest group maxima
+  K1Params k1;
+  memset(&k1, 0, sizeof k1);
+  k1.tokens = tokens; k1.seeds = seeds; k1.positions = positions;
+  k1.partials = reinterpret_cast<Partial*>(ws);
+  k1.device_status = out->device_status;
+  k1.unit_counter = reinterpret_cast<int*>(ws + pl.partial_bytes);
+  k1.T = (int)T; k1.d = (int)d; k1.V = (int)V;
+  k1.T_pad = pl.T_pad; k1.m_tiles = pl.m_tiles; k1.n_tiles = pl.n_tiles; k1.k_steps = pl.k_steps;
+  k1.S = pl.S; k1.Gm = pl.Gm; k1.n_units = pl.n_units;
+  k1.c1 = 1.4426950408889634f / temperature;
+  k1.neg_tl2 = -temperature * 0.6931471805599453f;
+  if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
+  if (launch_k1(6, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;
+
+  K2Params k2;
+  memset(&k2, 0, sizeof k2);
+  k2.h = reinterpret_cast<const uint16_t*>(h); k2.W = reinterpret_cast<const uint16_t*>(W);
+  k2.tokens = tokens; k2.seeds = seeds; k2.positions = positions;
+  k2.partials = k1.partials; k2.n_slots = pl.n_slots; k2.T_pad = pl.T_pad;
+  k2.T = (int)T; k2.d = (int)d; k2.V = (int)V; k2.ipt = 0;
+  k2.temperature = temperature; k2.sigma = out->sigma; k2.eps = out->eps; k2.c1 = k1.c1;
+  k2.score = out->score; k2.margin = out->margin; k2.argmax = out->argmax; k2.runner_up = out->runner_up;
+  k2.lse = out->lse; k2.row_status = out->row_status; k2.y_max = out->y_max; k2.y_second = out->y_second;
+  if (launch_k2(k2, s) != cudaSuccess) return DIFR_ERR_CUDA;
+
+  // ---- bounds, collecting pass, finalize
+  FilterParams fp;
+  memset(&fp, 0, sizeof fp);
+  fp.h = k2.h; fp.W = k2.W; fp.tokens = tokens; fp.seeds = seeds; fp.positions = positions;
+  fp.partials = k1.partials; fp.n_slots = pl.n_slots; fp.T_pad = pl.T_pad; fp.T = (int)T; fp.d = (int)d; fp.V = (int)V;
+  fp.temperature = temperature; fp.sigma = out->sigma; fp.eps = out->eps; fp.c1 = k1.c1;
+  fp.top_k = top_k; fp.top_p = top_p; fp.s = filter->s;
+  fp.bounds = reinterpret_cast<float*>(ws + pl.bounds_offset);
+  fp.cand_list = reinterpret_cast<const Candidate*>(ws + list_off);
+  fp.cand_count = reinterpret_cast<const int*>(ws + count_off);
+  fp.cand_cap = cap;
+  fp.score = out->score; fp.cutoff = out->cutoff; fp.row_status = out->row_status;
+  if (launch_filter_bounds(fp, s) != cudaSuccess) return DIFR_ERR_CUDA;
+
+  if (cudaMemsetAsync(ws + count_off, 0, (size_t)pl.T_pad * sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
+  if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
+  k1.bounds = fp.bounds;
+  k1.cand_list = ws + list_off;
+  k1.cand_count = reinterpret_cast<int*>(ws + count_off);
+  k1.cand_cap = cap;
+  if (launch_k1(7, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;
+  if (launch_filtered_finalize(fp, s) != cudaSuccess) return DIFR_ERR_CUDA;
+  return DIFR_OK;
+}
+
 difr_status difr_exfiltratable_bits(const uint8_t* classes, const int32_t* counts, int32_t rank_cutoff, int64_t V,
                                     const int32_t* seq_offsets, int64_t n_seq, int64_t T, float* bits,
                                     float* seq_bits, difr_stream_t stream) {

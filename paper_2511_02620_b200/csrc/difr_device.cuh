@@ -23,6 +23,12 @@ struct __align__(16) Partial {
 };
 static_assert(sizeof(Partial) == 32, "partial record is 32 bytes");
 
+// One entry of a row's candidate list (collecting pass of the full Token-DiFR estimator).
+struct Candidate {
+  int32_t id;
+  float l, y;  // fp32 logit and y' = y + Temp ln ln 2 as the fused kernel computes them
+};
+
 // -------------------------------------------------------------------- Philox
 constexpr uint32_t kPhiloxM0 = 0xD2511F53u;
 constexpr uint32_t kPhiloxM1 = 0xCD9E8D57u;

@@ -15,6 +15,9 @@ struct K1Params {
   const uint64_t* seeds;
   const uint32_t* positions;
   const float* bounds;  // [1 or 4][T_pad]: claimed logits (rank mode) or bounds on y' (counting modes)
+  void* cand_list;      // collect mode: [T][cand_cap] records {int32 id, float l, float y'}
+  int* cand_count;      // collect mode: [T], zeroed before the launch; may end above cand_cap (overflow)
+  int cand_cap;
   Partial* partials;  // [n_slots][T_pad]
   float* logits_out;  // dump mode only
   int32_t* device_status;
@@ -67,7 +70,8 @@ struct K3Params {
 };
 
 // mode: 0 Gumbel-max epilogue, 1 softmax statistics only, 2 logits dump, 3 Gumbel-max + raw-logit rank,
-// 4 / 5 count the ids whose noisy logit reaches one / four per-row bounds.
+// 4 / 5 count the ids whose noisy logit reaches one / four per-row bounds, 6 Gumbel-max + the strips' two
+// largest 16-id group maxima (word 7 of the record), 7 collect the ids that reach the row's bounds on y' / l.
 cudaError_t launch_k1(int mode, const CUtensorMap& tmap_h, const CUtensorMap& tmap_w, const K1Params& p, int grid,
                       cudaStream_t stream);  // grid: number of CTAs, two per pair
 int k1_max_resident_pairs();  // CTA pairs of the fused kernel the current device keeps resident at once
@@ -92,6 +96,31 @@ struct CountParams {
 };
 cudaError_t launch_count_bounds(const CountParams& p, cudaStream_t stream);
 cudaError_t launch_count_finalize(const CountParams& p, cudaStream_t stream);
+
+// Full Token-DiFR estimator: bounds for the collecting pass and the finalize over the candidate lists.
+struct FilterParams {
+  const uint16_t* h;
+  const uint16_t* W;
+  const int32_t* tokens;
+  const uint64_t* seeds;
+  const uint32_t* positions;
+  const Partial* partials;  // records of the first pass (mode GmFilter)
+  int n_slots, T_pad, T, d, V;
+  float temperature, sigma, eps, c1;
+  int top_k;    // 0: no top-k
+  float top_p;  // 1: no nucleus
+  int s;        // competitors in the active subset
+  float* bounds;  // [2][T_pad]: on y', on the raw logit
+  const Candidate* cand_list;
+  const int* cand_count;
+  int cand_cap;
+  float* score;
+  float* cutoff;  // nullable
+  uint32_t* row_status;
+};
+cudaError_t set_gauss_legendre(const double* x, const double* w);  // 16 nodes / weights on [-1, 1]
+cudaError_t launch_filter_bounds(const FilterParams& p, cudaStream_t stream);
+cudaError_t launch_filtered_finalize(const FilterParams& p, cudaStream_t stream);
 
 struct BitsParams {
   const uint8_t* classes;

@@ -59,16 +59,24 @@ static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one CTA");
 
 // Epilogue variants.  GmRank adds the raw-logit rank of the claimed token; Count1 / Count4 regenerate the
 // noise only to count the ids whose y reaches one / four per-row bounds (admissible-set sizes).
-enum : int { kModeGm = 0, kModeIpt = 1, kModeDump = 2, kModeGmRank = 3, kModeCount1 = 4, kModeCount4 = 5 };
+// GmFilter is Gm that also keeps each strip's two largest 16-id group maxima of the raw logits (the bound of
+// the filter's cutoff comes from them); Collect appends every id whose y' or raw logit reaches the row's
+// bounds to the row's candidate list.
+enum : int { kModeGm = 0, kModeIpt = 1, kModeDump = 2, kModeGmRank = 3, kModeCount1 = 4, kModeCount4 = 5,
+             kModeGmFilter = 6, kModeCollect = 7 };
 
 template <int MODE>
 struct Mode {
-  static constexpr bool gm = MODE == kModeGm || MODE == kModeGmRank;
+  static constexpr bool gm = MODE == kModeGm || MODE == kModeGmRank || MODE == kModeGmFilter;
   static constexpr bool softmax = gm || MODE == kModeIpt;
   static constexpr bool rank = MODE == kModeGmRank;
+  static constexpr bool groupmax = MODE == kModeGmFilter;
+  static constexpr bool collect = MODE == kModeCollect;
   static constexpr int ng = MODE == kModeCount1 ? 1 : (MODE == kModeCount4 ? 4 : 0);  // bounds per row
-  static constexpr bool noise = gm || ng > 0;
-  static constexpr int ncnt = rank ? 1 : (ng > 0 ? ng : 1);
+  static constexpr bool noise = gm || ng > 0 || collect;
+  static constexpr int ncnt = rank ? 1 : (collect ? 2 : (ng > 0 ? ng : 1));
+  static constexpr bool bounds = rank || collect || ng > 0;
+  static constexpr bool record = !collect && MODE != kModeDump;
 };
 
 struct Unit {
@@ -97,7 +105,8 @@ struct RowStats {
   float lsum;    // sum of 2^(z - lmax)
   float lpre;    // the same restricted to ids below the claimed one
   int cnt[4];    // GmRank: cnt[0] = ids whose logit exceeds the claimed one; Count: ids at or above bound g
-  float bound[4];  // GmRank: bound[0] = claimed logit; Count: the row's bounds on y'
+  float bound[4];  // GmRank: bound[0] = claimed logit; Count: the row's bounds on y'; Collect: bounds on y', on l
+  float gm2;     // GmFilter: the second largest 16-id group maximum of z (lmax is the largest)
 };
 
 __device__ __forceinline__ void stats_init(RowStats& s) {
@@ -106,6 +115,7 @@ __device__ __forceinline__ void stats_init(RowStats& s) {
   s.lmax = -CUDART_INF_F;
   s.lsum = s.lpre = 0.f;
   s.cnt[0] = s.cnt[1] = s.cnt[2] = s.cnt[3] = 0;
+  s.gm2 = -CUDART_INF_F;
 }
 
 // (k1, j1), (k2, j2): the best two of another column group of the same row, k1 >= k2.
@@ -156,7 +166,8 @@ __device__ __forceinline__ void noisy4(const RowNoise& rn, int id0, const float 
 // claimed token (scoring modes) or the id left out of the count (counting modes).
 template <int MODE>
 __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base, int V, int tok, float c1,
-                                          float neg_tl2, const RowNoise& rn, RowStats& s) {
+                                          float neg_tl2, const RowNoise& rn, RowStats& s, Candidate* cand_list,
+                                          int* cand_count, int cand_cap) {
   using M = Mode<MODE>;
   float l[kSub];
 #pragma unroll
@@ -175,6 +186,7 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
     for (int j = 3; j + 1 < kSub; j += 2) cm = fmax3(cm, l[j], l[j + 1]);
     cm = fmaxf(cm, l[kSub - 1]);
     const float zmax = cm * c1;
+    if (M::groupmax) s.gm2 = fmaxf(s.gm2, fminf(s.lmax, zmax));
     if (zmax > s.lmax) {  // rare after the first few groups of a strip
       const float scale = ex2_approx(s.lmax - zmax);  // 0 on the first group
       s.lsum *= scale;
@@ -240,6 +252,23 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
         c1k = fmaxf(c1k, t1);
         c2k = n2;
       }
+      if (M::collect) {
+        const float ym = fmaxf(fmaxf(y[0], y[1]), fmaxf(y[2], y[3]));
+        const float lm = fmaxf(fmaxf(l4[0], l4[1]), fmaxf(l4[2], l4[3]));
+        if (ym >= s.bound[0] || lm >= s.bound[1]) {  // rare
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            if ((y[q] >= s.bound[0] || l4[q] >= s.bound[1]) && base + j + q < V) {
+              const int pos = atomicAdd(cand_count, 1);
+              if (pos < cand_cap) {
+                Candidate c;
+                c.id = base + j + q; c.l = l4[q]; c.y = y[q];
+                cand_list[pos] = c;
+              }
+            }
+          }
+        }
+      }
       if (M::ng > 0) {
         if (tl >= j && tl < j + 4) {  // the id left out never counts
 #pragma unroll
@@ -270,7 +299,7 @@ __device__ __forceinline__ void record_pack(const RowStats& st, float4& a, float
     b = make_float4(0.f, 0.f, 0.f, 0.f);
   } else {
     a = make_float4(st.m1, __int_as_float(st.i1), st.m2, __int_as_float(st.i2));
-    b = make_float4(st.lmax, st.lsum, st.lpre, __int_as_float(st.cnt[0]));
+    b = make_float4(st.lmax, st.lsum, st.lpre, Mode<MODE>::groupmax ? st.gm2 : __int_as_float(st.cnt[0]));
   }
 }
 template <int MODE>
@@ -282,6 +311,7 @@ __device__ __forceinline__ void record_merge(RowStats& st, const float4& a, cons
     st.cnt[3] += __float_as_int(a.w);
   } else {
     top2_merge(st, a.x, __float_as_int(a.y), a.z, __float_as_int(a.w));
+    if (Mode<MODE>::groupmax) st.gm2 = fmax3(st.gm2, b.w, fminf(st.lmax, b.x));  // (b.x, b.w): its two largest
     if (b.x > -CUDART_INF_F) {  // that group saw columns
       const float m = fmaxf(st.lmax, b.x);
       const float fa = ex2_approx(st.lmax - m), fb = ex2_approx(b.x - m);
@@ -289,7 +319,7 @@ __device__ __forceinline__ void record_merge(RowStats& st, const float4& a, cons
       st.lpre = st.lpre * fa + b.z * fb;
       st.lmax = m;
     }
-    st.cnt[0] += __float_as_int(b.w);
+    if (!Mode<MODE>::groupmax) st.cnt[0] += __float_as_int(b.w);
   }
 }
 
@@ -516,11 +546,17 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
         }
         if (Mode<MODE>::noise) row_noise_init(rn, seed, pos);
         // per-row bounds: the claimed logit (rank) or the bounds on y' (counting); rows beyond T count nothing
-        if (Mode<MODE>::rank || Mode<MODE>::ng > 0) {
+        if (Mode<MODE>::bounds) {
 #pragma unroll
           for (int g = 0; g < Mode<MODE>::ncnt; ++g)
             st.bound[g] = valid ? p.bounds[(size_t)g * (size_t)p.T_pad + row] : CUDART_INF_F;
         }
+      }
+      Candidate* cand_list = nullptr;
+      int* cand_count = nullptr;
+      if (Mode<MODE>::collect && valid) {
+        cand_list = reinterpret_cast<Candidate*>(p.cand_list) + (size_t)row * (size_t)p.cand_cap;
+        cand_count = p.cand_count + row;
       }
       for (int n = w.n0; n < w.n1; ++n) {
         if (!mbar_wait(acc_full_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
@@ -547,7 +583,7 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
                   if (base + j < p.V) dst[j] = __uint_as_float(cur[j]);
               }
             } else {
-              process16<MODE>(cur, base, p.V, tok, p.c1, p.neg_tl2, rn, st);
+              process16<MODE>(cur, base, p.V, tok, p.c1, p.neg_tl2, rn, st, cand_list, cand_count, p.cand_cap);
             }
             if (!more) break;
           }
@@ -557,7 +593,7 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
         if (lane == 0) mbar_arrive_cluster_nofence(map_to_cta(acc_empty_bar(acc), 0));
         if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
       }
-      if (MODE != kModeDump && ok) {
+      if (Mode<MODE>::record && ok) {
         // the four column groups of a row meet in shared memory; group 0 merges and writes the record
         if (colg != 0) {
           if (!mbar_wait(xch_empty_bar(quarter), xch_phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -647,6 +683,8 @@ cudaError_t launch_k1(int mode, const CUtensorMap& tmap_h, const CUtensorMap& tm
     case kModeGmRank: return launch_mode<kModeGmRank>(tmap_h, tmap_w, p, grid, stream);
     case kModeCount1: return launch_mode<kModeCount1>(tmap_h, tmap_w, p, grid, stream);
     case kModeCount4: return launch_mode<kModeCount4>(tmap_h, tmap_w, p, grid, stream);
+    case kModeGmFilter: return launch_mode<kModeGmFilter>(tmap_h, tmap_w, p, grid, stream);
+    case kModeCollect: return launch_mode<kModeCollect>(tmap_h, tmap_w, p, grid, stream);
   }
   return cudaErrorInvalidValue;
 }

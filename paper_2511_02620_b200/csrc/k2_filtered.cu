@@ -1,0 +1,301 @@
+// Finalize kernels of the full Token-DiFR estimator (Alg. Token-DiFR with the top-k / top-p cutoff, the B_i
+// terms and an active subset of s competitors):
+//   filter_bounds      from the first pass's partial records, per row: a lower bound of the (s+3)-th largest
+//                      y' and of the top_k-th largest raw logit -- what the collecting pass compares against
+//   filtered_finalize  from the row's candidate list: the cutoff (top-k, then the nucleus inside it), the
+//                      s + 2 best competitors by y', their exact logits and noise in fp64, and the expectation
+//                      E_x[ 1{l_t + x > cutoff} prod_i Phi(max(x + A_i, B_i) / sigma) ] by composite
+//                      Gauss-Legendre quadrature (one panel per lane).
+#include <cuda_runtime.h>
+#include <math_constants.h>
+
+#include "difr_device.cuh"
+#include "difr_kernels.h"
+
+namespace difr {
+
+constexpr int kFWarps = 4;
+constexpr int kMaxK = 64;        // top_k limit (the nucleus is resolved inside the top k)
+constexpr int kMaxCand = 10;     // s + 2 with s <= 8
+constexpr int kGlOrder = 16;
+
+__constant__ double c_gl_x[kGlOrder];
+__constant__ double c_gl_w[kGlOrder];
+
+__device__ __forceinline__ double shfl_xor_f64(double v, int mask) {
+  int lo = __double2loint(v), hi = __double2hiint(v);
+  lo = __shfl_xor_sync(0xffffffffu, lo, mask);
+  hi = __shfl_xor_sync(0xffffffffu, hi, mask);
+  return __hiloint2double(hi, lo);
+}
+
+__device__ __forceinline__ double bf16_f64(uint32_t bits16) { return (double)__uint_as_float(bits16 << 16); }
+
+__device__ __forceinline__ double warp_dot64(const uint16_t* a, const uint16_t* b, int d, int lane) {
+  double acc = 0.0;
+  for (int k = lane * 8; k < d; k += 32 * 8) {
+    const uint4 va = *reinterpret_cast<const uint4*>(a + k);
+    const uint4 vb = *reinterpret_cast<const uint4*>(b + k);
+    const uint32_t wa[4] = {va.x, va.y, va.z, va.w};
+    const uint32_t wb[4] = {vb.x, vb.y, vb.z, vb.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      acc = fma(bf16_f64(wa[q] & 0xFFFFu), bf16_f64(wb[q] & 0xFFFFu), acc);
+      acc = fma(bf16_f64(wa[q] >> 16), bf16_f64(wb[q] >> 16), acc);
+    }
+  }
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) acc += shfl_xor_f64(acc, m);
+  return acc;
+}
+
+__device__ __forceinline__ double gumbel_f64(uint64_t seed, uint32_t position, uint32_t id) {
+  uint32_t x[4];
+  philox4x32_10(id >> 2, position, 0u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), x);
+  const double u = ((double)(x[id & 3u] >> 9) + 0.5) * (1.0 / 8388608.0);
+  return -log(-log(u));
+}
+
+// n-th largest (n >= 1) of the values the warp holds, eight per lane; -inf when there are fewer than n.
+__device__ __forceinline__ float warp_nth_largest(float (&v)[8], int n, int lane) {
+  float result = -CUDART_INF_F;
+  for (int it = 0; it < n; ++it) {
+    float lm = v[0];
+#pragma unroll
+    for (int e = 1; e < 8; ++e) lm = fmaxf(lm, v[e]);
+    float wm = lm;
+#pragma unroll
+    for (int m = 16; m >= 1; m >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, m));
+    result = wm;
+    if (wm == -CUDART_INF_F) break;
+    const unsigned holders = __ballot_sync(0xffffffffu, lm == wm);
+    if (lane == __ffs(holders) - 1) {  // one instance leaves
+      bool gone = false;
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        if (!gone && v[e] == wm) { v[e] = -CUDART_INF_F; gone = true; }
+    }
+  }
+  return result;
+}
+
+__global__ void __launch_bounds__(kFWarps * 32) filter_bounds(const FilterParams p) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * kFWarps + warp;
+  if (row >= p.T) return;
+  // up to 128 strips: four records per lane, two values of each kind per record
+  float yk[8], zk[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) yk[e] = zk[e] = -CUDART_INF_F;
+#pragma unroll
+  for (int t = 0; t < 4; ++t) {
+    const int slot = lane + 32 * t;
+    if (slot < p.n_slots) {
+      const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * (size_t)p.T_pad + row);
+      const float4 a = src[0], b = src[1];
+      if (__float_as_int(a.y) >= 0) yk[2 * t] = a.x;
+      if (__float_as_int(a.w) >= 0) yk[2 * t + 1] = a.z;
+      zk[2 * t] = b.x;
+      zk[2 * t + 1] = b.w;
+    }
+  }
+  // Any subset's n-th largest is a lower bound of the whole row's n-th largest.  s competitors are refined out of
+  // s + 2, and the claimed token may sit among them: s + 3.  A little is taken off for the index bits stored in
+  // the keys and for the rounding of z = l * c1.
+  float by = -CUDART_INF_F, bl = CUDART_INF_F;
+  if (p.n_slots <= 128) {
+    const float ky = warp_nth_largest(yk, p.s + 3, lane);
+    if (ky > -CUDART_INF_F) by = ky - 1e-4f * fmaxf(1.f, fabsf(ky));
+    if (p.top_k > 0) {
+      const float kz = warp_nth_largest(zk, p.top_k, lane);
+      bl = -CUDART_INF_F;
+      if (kz > -CUDART_INF_F) {
+        const float l = kz / p.c1;
+        bl = l - 1e-5f * fmaxf(1.f, fabsf(l));
+      }
+    }
+  } else if (p.top_k > 0) {
+    bl = -CUDART_INF_F;
+  }
+  if (lane == 0) {
+    p.bounds[row] = by;
+    p.bounds[(size_t)p.T_pad + row] = bl;
+  }
+}
+
+__global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterParams p) {
+  __shared__ float sm_l[kFWarps][kMaxK];
+  __shared__ int sm_id[kFWarps][kMaxK];
+  __shared__ int sm_cand[kFWarps][kMaxCand];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * kFWarps + warp;
+  if (row >= p.T) return;
+  const int tok = p.tokens[row];
+  const bool tok_ok = tok >= 0 && tok < p.V;
+  const Candidate* list = p.cand_list + (size_t)row * (size_t)p.cand_cap;
+  const int n_found = p.cand_count[row];
+  const int n = n_found < p.cand_cap ? n_found : p.cand_cap;
+  uint32_t status_bits = (n_found > p.cand_cap) ? 4u : 0u;
+
+  const int k_eff = (p.top_k > 0) ? (p.top_k < n ? p.top_k : n) : 0;
+  int n_others = 0;  // entries that are not the claimed token
+  for (int i = lane; i < n; i += 32) n_others += (list[i].id != tok) ? 1 : 0;
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) n_others += __shfl_xor_sync(0xffffffffu, n_others, m);
+  const int want = p.s + 2;
+  const int n_cand = n_others < want ? n_others : want;
+
+  // ---- order statistics of the list: rank by raw logit (the filter) and by y' (the competitors)
+  double cutoff = -CUDART_INF;
+  int cut_rank = -1;
+  for (int j = 0; j < n; ++j) {
+    const Candidate cj = list[j];
+    int rl = 0, ry = 0;
+    for (int i = lane; i < n; i += 32) {
+      const Candidate ci = list[i];
+      rl += (ci.l > cj.l || (ci.l == cj.l && ci.id < cj.id)) ? 1 : 0;
+      ry += (ci.id != tok && (ci.y > cj.y || (ci.y == cj.y && ci.id < cj.id))) ? 1 : 0;
+    }
+#pragma unroll
+    for (int m = 16; m >= 1; m >>= 1) {
+      rl += __shfl_xor_sync(0xffffffffu, rl, m);
+      ry += __shfl_xor_sync(0xffffffffu, ry, m);
+    }
+    if (lane == 0) {
+      if (rl < k_eff) { sm_l[warp][rl] = cj.l; sm_id[warp][rl] = cj.id; }
+      if (cj.id != tok && ry < n_cand) sm_cand[warp][ry] = cj.id;
+    }
+  }
+  __syncwarp();
+  if (k_eff > 0) {
+    cut_rank = k_eff - 1;  // the top_k-th largest logit
+    if (p.top_p < 1.f) {
+      // nucleus inside the top k: shortest prefix (descending) whose renormalised softmax mass reaches top_p
+      double e0 = 0.0, e1 = 0.0;
+      const double c1 = (double)p.c1, l0 = (double)sm_l[warp][0];
+      if (lane < k_eff) e0 = exp2(((double)sm_l[warp][lane] - l0) * c1);
+      if (lane + 32 < k_eff) e1 = exp2(((double)sm_l[warp][lane + 32] - l0) * c1);
+      double c0 = e0, c1s = e1;  // inclusive scans of both halves
+#pragma unroll
+      for (int m = 1; m < 32; m <<= 1) {
+        int lo0 = __shfl_up_sync(0xffffffffu, __double2loint(c0), m), hi0 = __shfl_up_sync(0xffffffffu, __double2hiint(c0), m);
+        int lo1 = __shfl_up_sync(0xffffffffu, __double2loint(c1s), m), hi1 = __shfl_up_sync(0xffffffffu, __double2hiint(c1s), m);
+        if (lane >= m) {
+          c0 += __hiloint2double(hi0, lo0);
+          c1s += __hiloint2double(hi1, lo1);
+        }
+      }
+      const double half = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(c0), 31),
+                                           __shfl_sync(0xffffffffu, __double2loint(c0), 31));
+      c1s += half;
+      const double total = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(c1s), 31),
+                                            __shfl_sync(0xffffffffu, __double2loint(c1s), 31));
+      const double need = (double)p.top_p * total;
+      const unsigned m0 = __ballot_sync(0xffffffffu, lane < k_eff && c0 >= need);
+      const unsigned m1 = __ballot_sync(0xffffffffu, lane + 32 < k_eff && c1s >= need);
+      int last = k_eff - 1;
+      if (m0) last = __ffs(m0) - 1;
+      else if (m1) last = 32 + __ffs(m1) - 1;
+      cut_rank = last;
+    }
+    // the cutoff is that id's logit: re-evaluated in fp64 like every other logit the score depends on
+    cutoff = warp_dot64(p.h + (size_t)row * (size_t)p.d, p.W + (size_t)sm_id[warp][cut_rank] * (size_t)p.d, p.d, lane);
+  }
+
+  double score = log((double)p.eps);
+  if (tok_ok) {
+    const uint64_t seed = p.seeds[row];
+    const uint32_t pos = p.positions[row];
+    const uint16_t* hrow = p.h + (size_t)row * (size_t)p.d;
+    const double temp = (double)p.temperature, sigma = (double)p.sigma;
+    const double l_t = warp_dot64(hrow, p.W + (size_t)tok * (size_t)p.d, p.d, lane);
+    const double y_t = l_t + temp * gumbel_f64(seed, pos, (uint32_t)tok);
+    // exact logits and noisy logits of the s + 2 candidates; then the s best of them
+    double cl[kMaxCand], cy[kMaxCand];
+    int cid[kMaxCand];
+#pragma unroll
+    for (int c = 0; c < kMaxCand; ++c) {
+      cl[c] = 0.0; cy[c] = -CUDART_INF; cid[c] = 0x7fffffff;
+      if (c < n_cand) {
+        const int id = sm_cand[warp][c];
+        cid[c] = id;
+        cl[c] = warp_dot64(hrow, p.W + (size_t)id * (size_t)p.d, p.d, lane);
+        cy[c] = cl[c] + temp * gumbel_f64(seed, pos, (uint32_t)id);
+      }
+    }
+    // selection sort, descending y, ties to the lower id (kMaxCand is tiny; every lane does the same)
+#pragma unroll
+    for (int a = 0; a < kMaxCand - 1; ++a) {
+#pragma unroll
+      for (int b = a + 1; b < kMaxCand; ++b) {
+        const bool swap = cy[b] > cy[a] || (cy[b] == cy[a] && cid[b] < cid[a]);
+        if (swap) {
+          const double ty = cy[a]; cy[a] = cy[b]; cy[b] = ty;
+          const double tl = cl[a]; cl[a] = cl[b]; cl[b] = tl;
+          const int ti = cid[a]; cid[a] = cid[b]; cid[b] = ti;
+        }
+      }
+    }
+    const int s_eff = p.s < n_cand ? p.s : n_cand;
+    double A[kMaxCand], B[kMaxCand];
+    double max_neg_a = 0.0;
+#pragma unroll
+    for (int c = 0; c < kMaxCand; ++c) {
+      A[c] = y_t - cy[c];
+      B[c] = cutoff - cl[c];
+      if (c < s_eff && -A[c] > max_neg_a) max_neg_a = -A[c];
+    }
+    // ---- the expectation over x ~ N(0, sigma^2), x > cutoff - l_t
+    const double x0 = cutoff - l_t;
+    const double lo = fmax(x0, -14.0 * sigma);
+    const double hi = 14.0 * sigma + fmin(max_neg_a, 60.0 * sigma);
+    double pi_hat = 0.0;
+    if (lo < hi) {
+      const double w = (hi - lo) / 32.0, mid = lo + ((double)lane + 0.5) * w;
+      const double inv_sigma = 1.0 / sigma, r2 = 0.70710678118654752440;
+      double acc = 0.0;
+#pragma unroll 1
+      for (int q = 0; q < kGlOrder; ++q) {
+        const double x = mid + 0.5 * w * c_gl_x[q];
+        const double xs = x * inv_sigma;
+        double f = exp(-0.5 * xs * xs);
+#pragma unroll
+        for (int c = 0; c < kMaxCand; ++c) {
+          if (c < s_eff) {
+            const double t = fmax(x + A[c], B[c]) * inv_sigma;
+            f *= 0.5 * erfc(-t * r2);
+          }
+        }
+        acc += c_gl_w[q] * f;
+      }
+      acc *= 0.5 * w * inv_sigma * 0.39894228040143267794;  // 1 / (sigma sqrt(2 pi))
+#pragma unroll
+      for (int m = 16; m >= 1; m >>= 1) acc += shfl_xor_f64(acc, m);
+      pi_hat = fmin(fmax(acc, 0.0), 1.0);
+    }
+    score = log(pi_hat + (double)p.eps);
+  }
+  if (lane == 0) {
+    p.score[row] = (float)score;
+    if (p.cutoff) p.cutoff[row] = (float)cutoff;
+    if (p.row_status && status_bits) p.row_status[row] |= status_bits;
+  }
+}
+
+cudaError_t set_gauss_legendre(const double* x, const double* w) {
+  cudaError_t e = cudaMemcpyToSymbol(c_gl_x, x, sizeof(double) * kGlOrder);
+  if (e != cudaSuccess) return e;
+  return cudaMemcpyToSymbol(c_gl_w, w, sizeof(double) * kGlOrder);
+}
+
+cudaError_t launch_filter_bounds(const FilterParams& p, cudaStream_t stream) {
+  filter_bounds<<<(p.T + kFWarps - 1) / kFWarps, kFWarps * 32, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_filtered_finalize(const FilterParams& p, cudaStream_t stream) {
+  filtered_finalize<<<(p.T + kFWarps - 1) / kFWarps, kFWarps * 32, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace difr

@@ -1,0 +1,117 @@
+"""GPU-vs-oracle parity of the full Token-DiFR estimator (top-k / top-p cutoff, B_i terms, s competitors)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads as wl
+from gpu_util import Device, f32, to_dev
+from oracle import filtered
+
+import paper_2511_02620_b200 as difr
+
+pytestmark = pytest.mark.gpu
+
+EPS = 1e-12
+SCORE_TOL = 2e-3
+
+
+def _small(T, d, V, seed, scale=1.0):
+    g = np.random.default_rng(seed)
+    h = wl.f32_to_bf16_bits(g.standard_normal((T, d)).astype(np.float32))
+    W = wl.f32_to_bf16_bits((scale * g.standard_normal((V, d)) / math.sqrt(d)).astype(np.float32))
+    seeds = np.array([wl.splitmix64(seed * 1000 + r // 64) for r in range(T)], dtype=np.uint64)
+    positions = (np.arange(T) % 64 + 1).astype(np.uint32)
+    return h, W, seeds, positions
+
+
+def _claims(h, W, seeds, positions, temperature, seed):
+    honest, runner = oracle.sample_gm(h, W, seeds, positions, temperature)
+    L = oracle.logits(h, W)
+    g = np.random.default_rng(seed)
+    T, V = h.shape[0], W.shape[0]
+    tokens = honest.copy()
+    k = np.arange(T)
+    tokens[k % 6 == 1] = runner[k % 6 == 1]
+    tokens[k % 6 == 3] = g.integers(0, V, size=T)[k % 6 == 3]
+    third = np.argsort(-L, axis=1)[:, 2]  # a high-logit id that was not sampled
+    tokens[k % 6 == 5] = third[k % 6 == 5]
+    return tokens.astype(np.int32)
+
+
+def _run(dev, tokens, temperature, sigma, top_k, top_p, s):
+    out = difr.DifrOut.allocate(dev.T, dev.d, dev.V, sigma, EPS)
+    out.workspace = torch.empty(difr.difr_filtered_workspace_bytes(dev.T, dev.d, dev.V), dtype=torch.uint8, device="cuda")
+    out.cutoff = torch.full((dev.T,), float("nan"), dtype=torch.float32, device="cuda")
+    out.score.fill_(float("nan"))
+    difr.difr_score_gm_filtered(dev.h, dev.W, to_dev(np.asarray(tokens, dtype=np.int32)), dev.seeds, dev.positions,
+                                f32(temperature), top_k, top_p, s, out)
+    torch.cuda.synchronize()
+    assert int(out.device_status.item()) == 0
+    return out
+
+
+def test_one_competitor_and_no_filter_is_the_plain_estimator():
+    T, d, V = 200, 64, 3000
+    h, W, seeds, positions = _small(T, d, V, 51)
+    tokens = _claims(h, W, seeds, positions, f32(1.0), 52)
+    tokens[9] = -3
+    dev = Device(h, W, seeds, positions)
+    for sigma in (0.5, 0.05):
+        plain = dev.score("gm", tokens, 1.0, sigma, EPS)
+        out = _run(dev, tokens, 1.0, sigma, 0, 1.0, 1)
+        np.testing.assert_allclose(out.score.cpu().numpy(), plain["score"], rtol=0, atol=2e-5)
+        assert np.all(np.isneginf(out.cutoff.cpu().numpy()))
+        assert np.array_equal(out.argmax.cpu().numpy(), plain["argmax"])
+        assert np.array_equal(out.row_status.cpu().numpy(), plain["row_status"])
+
+
+@pytest.mark.parametrize("T,d,V,scale,temperature,sigma,top_k,top_p,s", [
+    (96, 64, 3000, 2.0, 1.0, 0.3, 50, 0.95, 4),     # the paper's sampling setting; every id is a candidate (V < 8192)
+    (96, 64, 3000, 2.0, 0.7, 0.05, 8, 1.0, 2),      # top-k only, narrow noise
+    (64, 72, 9000, 3.0, 1.0, 0.5, 20, 0.9, 8),      # candidate lists bounded from the first pass (V >= 8192)
+    (64, 72, 9000, 1.0, 1.0, 1.0, 0, 1.0, 8),       # no filter, many competitors, flat logits
+    (40, 64, 40, 2.0, 1.0, 0.4, 64, 0.8, 3),        # top_k beyond the vocabulary: the nucleus acts on all of it
+])
+def test_full_estimator_matches_the_oracle(T, d, V, scale, temperature, sigma, top_k, top_p, s):
+    h, W, seeds, positions = _small(T, d, V, 61, scale)
+    tokens = _claims(h, W, seeds, positions, f32(temperature), 62)
+    tokens[5] = V + 1
+    dev = Device(h, W, seeds, positions)
+    out = _run(dev, tokens, temperature, sigma, top_k, top_p, s)
+    want, pi, cut = filtered.score_gm_filtered(h, W, tokens, seeds, positions, f32(temperature), f32(sigma), f32(EPS),
+                                               top_k, f32(top_p), s)
+    got, got_cut = out.score.cpu().numpy(), out.cutoff.cpu().numpy().astype(np.float64)
+    assert np.all(out.row_status.cpu().numpy() & 4 == 0)  # no candidate list overflowed
+    # the cutoff is one of the row's logits: equal up to fp32 rounding, except where two prefixes of the nucleus
+    # differ by less than rounding (then the neighbouring logit is as good an answer)
+    same_cut = np.isclose(got_cut, cut, rtol=0, atol=1e-5) | (np.isneginf(got_cut) & np.isneginf(cut))
+    assert same_cut.mean() >= 0.97
+    np.testing.assert_allclose(got[same_cut], want[same_cut], rtol=0, atol=SCORE_TOL)
+    assert got[5] == pytest.approx(math.log(EPS), abs=1e-5)
+    # the estimate is not degenerate: the filter and the extra competitors move it
+    if top_k or s > 1:
+        plain = dev.score("gm", tokens, temperature, sigma, EPS)["score"]
+        assert np.abs(got - plain).max() > 0.05
+
+
+def test_full_estimator_at_full_size_on_sampled_rows():
+    w = wl.WORKLOADS["llama3b"]
+    inp = wl.make_inputs(w)
+    dev = Device(inp.h, inp.W, inp.seeds, inp.positions)
+    rows = wl.sample_rows(w, 12, salt=3)
+    temperature, sigma, top_k, top_p, s = 1.0, 0.3, 50, 0.95, 4
+    g = np.random.default_rng(5)
+    tokens = g.integers(0, w.V, size=w.T).astype(np.int32)
+    hs = np.ascontiguousarray(inp.h[rows])
+    tokens[rows] = _claims(hs, inp.W, inp.seeds[rows], inp.positions[rows], f32(temperature), 6)
+    out = _run(dev, tokens, temperature, sigma, top_k, top_p, s)
+    want, _, cut = filtered.score_gm_filtered(hs, inp.W, tokens[rows], inp.seeds[rows], inp.positions[rows],
+                                              f32(temperature), f32(sigma), f32(EPS), top_k, f32(top_p), s)
+    got, got_cut = out.score.cpu().numpy(), out.cutoff.cpu().numpy()
+    np.testing.assert_allclose(got_cut[rows], cut, rtol=0, atol=1e-5)
+    np.testing.assert_allclose(got[rows], want, rtol=0, atol=SCORE_TOL)
+    assert np.all(out.row_status.cpu().numpy() == 0)
+    assert np.all(np.isfinite(got)) and np.all(got <= 1e-6)
