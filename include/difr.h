@@ -77,7 +77,8 @@ typedef struct {
   float* cdf_lo;      /* IPT: a = sum_{v < t*} p_v                                 */
   float* u;           /* IPT: the uniform mu of this row                           */
   uint32_t* row_status; /* bit0: claimed id outside [0, V); bit1: non-finite logits;
-                           bit2: candidate list overflow (difr_score_gm_filtered)         */
+                           bit2: candidate list overflow (difr_score_gm_filtered);
+                           bit3: unusable per-row temperature                             */
   void* workspace;      /* >= difr_workspace_bytes(T, d, V) bytes, 16-byte aligned;
                            contents are scratch, overwritten by every call         */
   size_t workspace_bytes;
@@ -98,6 +99,11 @@ typedef struct {
   float sigma_ipt;   /* difr_score_both only: noise width of the IPT estimator (CDF units), > 0 */
   float* score_ipt;  /* difr_score_both only, required there: ln(mass + eps)                   */
   float* cutoff;     /* difr_score_gm_filtered only, optional: the filter's cutoff per row     */
+  const float* temperatures; /* difr_score_gm / _ipt / _both, optional: [T] one sampling temperature per
+                        row (requests with their own sampling parameters in one batch); when given, the
+                        `temperature` argument is ignored.  A row whose value is negative, not finite, or
+                        zero where the IPT score is asked for gets a NaN score and row_status bit 3.
+                        Must be NULL for difr_score_gm_filtered.                                */
 } difr_out;
 
 /* Scratch bytes a scoring call needs for T rows, hidden size d, vocabulary V.

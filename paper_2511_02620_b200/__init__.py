@@ -41,6 +41,7 @@ class _COut(ctypes.Structure):
         ("event_fused_start", ctypes.c_void_p), ("event_fused_stop", ctypes.c_void_p),
         ("rank", ctypes.c_void_p), ("y_max", ctypes.c_void_p), ("y_second", ctypes.c_void_p),
         ("sigma_ipt", ctypes.c_float), ("score_ipt", ctypes.c_void_p), ("cutoff", ctypes.c_void_p),
+        ("temperatures", ctypes.c_void_p),
     ]
 
 
@@ -152,6 +153,7 @@ class DifrOut:
     sigma_ipt: float = 0.0      # difr_score_both: width of the IPT estimator
     score_ipt: "object" = None  # difr_score_both: float [T]
     cutoff: "object" = None     # difr_score_gm_filtered: float [T], the filter's cutoff per row
+    temperatures: "object" = None  # float [T]: one temperature per row instead of the call's scalar
 
     @staticmethod
     def allocate(T: int, d: int, V: int, sigma: float, eps: float = 1e-12, device="cuda"):
@@ -171,7 +173,8 @@ class DifrOut:
                      _ptr(self.row_status), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
                      _ptr(self.device_status), ctypes.c_void_p(self.event_fused_start or None),
                      ctypes.c_void_p(self.event_fused_stop or None), _ptr(self.rank), _ptr(self.y_max),
-                     _ptr(self.y_second), float(self.sigma_ipt), _ptr(self.score_ipt), _ptr(self.cutoff))
+                     _ptr(self.y_second), float(self.sigma_ipt), _ptr(self.score_ipt), _ptr(self.cutoff),
+                     _ptr(self.temperatures))
 
 
 def _score(fn_name, h, W, tokens, seeds, positions, temperature, out: DifrOut, stream):

@@ -81,7 +81,10 @@ difr_status score_common(int ipt, const void* h, const void* W, const int32_t* t
   if (T < 0 || d <= 0 || V <= 0) return DIFR_ERR_INVALID_ARG;
   if (!(out->sigma > 0.f) || !(out->eps >= 0.f) || !isfinite(out->sigma) || !isfinite(out->eps))
     return DIFR_ERR_INVALID_ARG;
-  if (!(temperature >= 0.f) || !isfinite(temperature) || (ipt && temperature == 0.f)) return DIFR_ERR_INVALID_ARG;
+  if (out->temperatures == nullptr &&
+      (!(temperature >= 0.f) || !isfinite(temperature) || (ipt && temperature == 0.f)))
+    return DIFR_ERR_INVALID_ARG;
+  if (out->temperatures != nullptr) temperature = 1.f;  // unused: every row brings its own
   if (ipt == 2 && (!out->score_ipt || !(out->sigma_ipt > 0.f) || !isfinite(out->sigma_ipt))) return DIFR_ERR_INVALID_ARG;
   if ((d % 8) != 0 || V < 2) return DIFR_ERR_SHAPE;
   if (T == 0) return DIFR_OK;
@@ -102,6 +105,7 @@ difr_status score_common(int ipt, const void* h, const void* W, const int32_t* t
   k1.tokens = tokens; k1.seeds = seeds; k1.positions = positions;
   k1.partials = reinterpret_cast<Partial*>(out->workspace);
   k1.device_status = out->device_status;
+  k1.temperatures = out->temperatures;
   k1.unit_counter = reinterpret_cast<int*>(static_cast<unsigned char*>(out->workspace) + pl.partial_bytes);
   k1.T = (int)T; k1.d = (int)d; k1.V = (int)V;
   k1.T_pad = pl.T_pad; k1.m_tiles = pl.m_tiles; k1.n_tiles = pl.n_tiles; k1.k_steps = pl.k_steps;
@@ -136,6 +140,7 @@ difr_status score_common(int ipt, const void* h, const void* W, const int32_t* t
   k2.score = out->score; k2.margin = out->margin; k2.argmax = out->argmax; k2.runner_up = out->runner_up;
   k2.lse = out->lse; k2.p_claimed = out->p_claimed; k2.cdf_lo = out->cdf_lo; k2.u = out->u;
   k2.row_status = out->row_status;
+  k2.temperatures = out->temperatures;
   k2.sigma_ipt = out->sigma_ipt; k2.score_ipt = out->score_ipt;
   k2.rank = want_rank ? out->rank : nullptr; k2.y_max = out->y_max; k2.y_second = out->y_second;
   if (launch_k2(k2, s) != cudaSuccess) return DIFR_ERR_CUDA;
@@ -312,7 +317,7 @@ difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* 
   if (T < 0 || d <= 0 || V <= 0) return DIFR_ERR_INVALID_ARG;
   if (!(out->sigma > 0.f) || !(out->eps >= 0.f) || !isfinite(out->sigma) || !isfinite(out->eps))
     return DIFR_ERR_INVALID_ARG;
-  if (!(temperature > 0.f) || !isfinite(temperature)) return DIFR_ERR_INVALID_ARG;
+  if (!(temperature > 0.f) || !isfinite(temperature) || out->temperatures != nullptr) return DIFR_ERR_INVALID_ARG;
   int top_k = filter->top_k;
   const float top_p = filter->top_p;
   if (top_k < 0 || !(top_p > 0.f) || !(top_p <= 1.f) || filter->s < 1 || filter->s > 8) return DIFR_ERR_INVALID_ARG;

@@ -14,6 +14,7 @@ struct K1Params {
   const int32_t* tokens;
   const uint64_t* seeds;
   const uint32_t* positions;
+  const float* temperatures;  // [T], nullable: per-row temperature in place of c1 / neg_tl2
   const float* bounds;  // [1 or 4][T_pad]: claimed logits (rank mode) or bounds on y' (counting modes)
   void* cand_list;      // collect mode: [T][cand_cap] records {int32 id, float l, float y'}
   int* cand_count;      // collect mode: [T], zeroed before the launch; may end above cand_cap (overflow)
@@ -38,6 +39,7 @@ struct K2Params {
   const Partial* partials;
   int n_slots, T_pad;
   int T, d, V;
+  const float* temperatures;  // [T], nullable: per-row temperature in place of `temperature` / `c1`
   int ipt;  // 0: Token-DiFR (Gumbel-max), 1: Token-IPT-DiFR, 2: both (IPT score to score_ipt with sigma_ipt)
   float sigma_ipt;
   float* score_ipt;

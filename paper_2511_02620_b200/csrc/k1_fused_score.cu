@@ -552,6 +552,13 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
             st.bound[g] = valid ? p.bounds[(size_t)g * (size_t)p.T_pad + row] : CUDART_INF_F;
         }
       }
+      // the temperature is the call's, or the row's own when the caller passes one per row
+      float c1 = p.c1, neg_tl2 = p.neg_tl2;
+      if (p.temperatures != nullptr && MODE != kModeDump) {
+        const float temp = valid ? p.temperatures[row] : 1.f;
+        c1 = temp > 0.f ? 1.4426950408889634f / temp : 0.f;
+        neg_tl2 = -temp * 0.6931471805599453f;
+      }
       Candidate* cand_list = nullptr;
       int* cand_count = nullptr;
       if (Mode<MODE>::collect && valid) {
@@ -583,7 +590,7 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
                   if (base + j < p.V) dst[j] = __uint_as_float(cur[j]);
               }
             } else {
-              process16<MODE>(cur, base, p.V, tok, p.c1, p.neg_tl2, rn, st, cand_list, cand_count, p.cand_cap);
+              process16<MODE>(cur, base, p.V, tok, c1, neg_tl2, rn, st, cand_list, cand_count, p.cand_cap);
             }
             if (!more) break;
           }

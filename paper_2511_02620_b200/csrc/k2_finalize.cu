@@ -138,14 +138,22 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
   const uint32_t pos = p.positions[row];
   const bool tok_ok = tok >= 0 && tok < p.V;
   const uint16_t* hrow = p.h + (size_t)row * (size_t)p.d;
-  const double temp = (double)p.temperature;
+  // the call's temperature, or the row's own (then c1 is rebuilt exactly as the fused kernel built it)
+  float temp_f = p.temperature, c1_f = p.c1;
+  if (p.temperatures != nullptr) {
+    temp_f = p.temperatures[row];
+    c1_f = temp_f > 0.f ? 1.4426950408889634f / temp_f : 0.f;
+  }
+  const double temp = (double)temp_f;
   const double sigma = (double)p.sigma, eps = (double)p.eps;
   uint32_t status = tok_ok ? 0u : 1u;
 
   const double ln2 = 0.69314718055994530942;
   const bool lse_finite = isfinite(acc.lmax) && isfinite(acc.lsum) && acc.lsum > 0.0;
   if (!lse_finite) status |= 2u;
-  const double lse = (p.temperature > 0.f) ? (acc.lmax + log2(acc.lsum)) * ln2 : CUDART_NAN;
+  const bool temp_bad = !(temp_f >= 0.f) || isinf(temp_f) || (p.ipt != 0 && temp_f == 0.f);
+  if (temp_bad) status |= 8u;
+  const double lse = (temp_f > 0.f) ? (acc.lmax + log2(acc.lsum)) * ln2 : CUDART_NAN;
 
   double l_tok = 0.0;
   if (tok_ok) l_tok = warp_dot(hrow, p.W + (size_t)tok * (size_t)p.d, p.d, lane);
@@ -183,7 +191,8 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
         }
       }
       const double pi = 0.5 * erfc(-A / (2.0 * sigma));  // Phi(A / (sigma sqrt 2))
-      const double score = tok_ok ? log(pi + eps) : log(eps);
+      double score = tok_ok ? log(pi + eps) : log(eps);
+      if (temp_bad) score = CUDART_NAN;
       p.score[row] = (float)score;
       if (p.margin) p.margin[row] = (float)A;
       if (p.argmax) p.argmax[row] = best;
@@ -203,7 +212,7 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
       const double mu = ((double)x[0] + 0.5) * (1.0 / 4294967296.0);
       double score = log(eps), pt = CUDART_NAN, a = CUDART_NAN;
       if (tok_ok) {
-        const double c1d = (double)p.c1;  // log2(e) / Temp, the very factor the fused kernel scaled its logits by
+        const double c1d = (double)c1_f;  // log2(e) / Temp, the very factor the fused kernel scaled its logits by
         pt = exp2(l_tok * c1d - acc.lmax) / acc.lsum;
         a = acc.lpre / acc.lsum;
         const double b = a + pt;
@@ -211,6 +220,7 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
         const double mass = normal_interval((a - mu) / sg, (b - mu) / sg);
         score = log(mass + eps);
       }
+      if (temp_bad) score = CUDART_NAN;
       (p.ipt == 2 ? p.score_ipt : p.score)[row] = (float)score;
       if (p.lse) p.lse[row] = (float)lse;
       if (p.p_claimed) p.p_claimed[row] = (float)pt;

@@ -174,3 +174,39 @@ def test_admissible_set_sizes_and_information_bound(T, d, V, temperature, sigma)
     np.testing.assert_allclose(bits.cpu().numpy(), want_bits, rtol=1e-6, atol=1e-6)
     np.testing.assert_allclose(seq_bits.cpu().numpy(), want_seq, rtol=1e-5)
     assert seq_bits.cpu().numpy()[1] == 0.0
+
+
+def test_per_row_temperatures_equal_one_call_per_temperature():
+    """Requests with their own sampling temperature in one batch: every row must come out exactly as in a call
+    that uses its temperature for the whole batch."""
+    T, d, V = 300, 128, 2600
+    h, W, seeds, positions = _small(T, d, V, 71)
+    temps = np.where(np.arange(T) % 3 == 0, 0.7, 1.0).astype(np.float32)
+    temps[T // 2:] = np.where(np.arange(T - T // 2) % 4 == 0, 1.3, temps[T // 2:])
+    tokens = np.empty(T, dtype=np.int32)
+    for t in np.unique(temps):
+        sel = temps == t
+        tokens[sel] = _claims(h[sel], W, seeds[sel], positions[sel], float(t), 72)
+    dev = Device(h, W, seeds, positions)
+    bad = temps.copy()
+    bad[11], bad[12] = -1.0, np.nan
+    out = difr.DifrOut.allocate(T, d, V, 0.3, EPS)
+    f = lambda: torch.full((T,), float("nan"), dtype=torch.float32, device="cuda")
+    out.score_ipt, out.sigma_ipt, out.y_max, out.y_second = f(), 0.05, f(), f()
+    out.temperatures = to_dev(bad)
+    difr.difr_score_both(dev.h, dev.W, to_dev(tokens), dev.seeds, dev.positions, 123.0, out)  # the scalar is ignored
+    torch.cuda.synchronize()
+    assert int(out.device_status.item()) == 0
+    good = np.ones(T, dtype=bool)
+    good[[11, 12]] = False
+    status = out.row_status.cpu().numpy()
+    assert np.all(status[~good] & 8) and np.all(status[good] == 0)
+    assert np.all(np.isnan(out.score.cpu().numpy()[~good])) and np.all(np.isnan(out.score_ipt.cpu().numpy()[~good]))
+    for t in np.unique(temps):
+        sel = (temps == t) & good
+        one = _score(dev, difr.difr_score_both, tokens, float(t), 0.3, sigma_ipt=0.05)
+        for name in ("score", "score_ipt", "margin", "argmax", "lse", "cdf_lo", "y_max"):
+            a, b = getattr(out, name).cpu().numpy()[sel], getattr(one, name).cpu().numpy()[sel]
+            assert np.array_equal(a, b), (t, name)
+        ref = oracle.score_gm(h[sel], W, tokens[sel], seeds[sel], positions[sel], float(t), f32(0.3), f32(EPS))
+        np.testing.assert_allclose(out.score.cpu().numpy()[sel], ref.score, rtol=0, atol=SCORE_TOL)
