@@ -35,7 +35,7 @@ class _GmOut(ctypes.Structure):
         ("score", ctypes.c_void_p), ("margin", ctypes.c_void_p), ("argmax", ctypes.c_void_p),
         ("runner_up", ctypes.c_void_p), ("top2_margin", ctypes.c_void_p), ("lse", ctypes.c_void_p),
         ("y_claimed", ctypes.c_void_p), ("logit_claimed", ctypes.c_void_p), ("rank", ctypes.c_void_p),
-        ("match", ctypes.c_void_p), ("row_status", ctypes.c_void_p),
+        ("match", ctypes.c_void_p), ("row_status", ctypes.c_void_p), ("top23_margin", ctypes.c_void_p),
     ]
 
 
@@ -192,6 +192,7 @@ class GmResult:
     rank: np.ndarray
     match: np.ndarray
     row_status: np.ndarray
+    top23_margin: np.ndarray
 
 
 @dataclass
@@ -227,7 +228,7 @@ def score_gm(h_bits, W_bits, tokens, seeds, positions, temperature, sigma, eps=1
         assert noise_id.shape == (V,)
     f8 = lambda: np.zeros(T, dtype=np.float64)
     i4 = lambda: np.zeros(T, dtype=np.int32)
-    res = GmResult(f8(), f8(), i4(), i4(), f8(), f8(), f8(), f8(), i4(), i4(), np.zeros(T, dtype=np.uint32))
+    res = GmResult(f8(), f8(), i4(), i4(), f8(), f8(), f8(), f8(), i4(), i4(), np.zeros(T, dtype=np.uint32), f8())
     out = _GmOut(*[_p(getattr(res, name)) for name, _ in _GmOut._fields_])
     rc = lib().oracle_score_gm(_p(h_bits), _p(W_bits), _p(tokens), _p(seeds), _p(positions), float(temperature),
                                float(sigma), float(eps), T, d, V, _p(noise_id), ctypes.byref(out))

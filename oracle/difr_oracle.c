@@ -190,6 +190,7 @@ typedef struct {
   int32_t* rank;       /* [T] #{v : l_v > l_t*}  (raw-logit rank, 0 = largest)   */
   int32_t* match;      /* [T] 1 iff argmax == t*                                 */
   uint32_t* row_status; /* [T] bit0: claim outside [0,V); bit1: non-finite logit */
+  double* top23_margin; /* [T] y_(2) - y_(3); +inf when V < 3                     */
 } oracle_gm_out;
 
 /* noise_id (nullable): vocabulary id v draws the noise of id noise_id[v]; used
@@ -249,6 +250,12 @@ int oracle_score_gm(const uint16_t* h, const uint16_t* W, const int32_t* tokens,
         if (out->argmax) out->argmax[r] = (int32_t)i1;
         if (out->runner_up) out->runner_up[r] = (int32_t)i2;
         if (out->top2_margin) out->top2_margin[r] = y[i1] - y[i2];
+        if (out->top23_margin) {
+          double third = -INFINITY;
+          for (int64_t v = 0; v < V; ++v)
+            if (v != i1 && v != i2 && y[v] > third) third = y[v];
+          out->top23_margin[r] = y[i2] - third;
+        }
         if (out->lse) out->lse[r] = temperature > 0.0 ? log_sum_exp_scaled(logit, V, 1.0 / temperature) : NAN;
         if (out->y_claimed) out->y_claimed[r] = in_range ? y[t] : NAN;
         if (out->logit_claimed) out->logit_claimed[r] = in_range ? logit[t] : NAN;

@@ -85,7 +85,8 @@ def test_full_size_gm(name, T, temperature, sigma):
     np.testing.assert_allclose(got["margin"][rows], ref.margin, rtol=0, atol=1e-4)
     clear = ref.top2_margin >= ARGMAX_MARGIN
     assert np.array_equal(got["argmax"][rows][clear], ref.argmax[clear])
-    assert np.array_equal(got["runner_up"][rows][clear], ref.runner_up[clear])
+    clear2 = clear & (ref.top23_margin >= ARGMAX_MARGIN)
+    assert np.array_equal(got["runner_up"][rows][clear2], ref.runner_up[clear2])
     np.testing.assert_allclose(got["lse"][rows], ref.lse, rtol=LSE_RTOL)
     # every row: well-formed outputs and the exact-match bookkeeping
     assert np.all(got["row_status"] == 0)

@@ -51,7 +51,9 @@ def check_gm(got, ref, tol=SCORE_TOL):
     assert np.array_equal(got["margin"][~fin], ref.margin[~fin])
     clear = ref.top2_margin >= ARGMAX_MARGIN
     assert np.array_equal(got["argmax"][clear], ref.argmax[clear])
-    assert np.array_equal(got["runner_up"][clear], ref.runner_up[clear]) or True
+    clear2 = clear & (ref.top23_margin >= ARGMAX_MARGIN)  # the runner-up is unique where the third is clearly behind
+    assert np.array_equal(got["runner_up"][clear2], ref.runner_up[clear2])
+    assert clear2.mean() > 0.9
     np.testing.assert_allclose(got["lse"], ref.lse, rtol=LSE_RTOL, atol=1e-3)
     assert np.array_equal(got["row_status"], ref.row_status)
 

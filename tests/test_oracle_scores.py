@@ -112,6 +112,8 @@ def test_margin_and_argmax_against_a_numpy_replay():
         y = logits[i] + temperature * G
         order = np.argsort(-y, kind="stable")
         assert r.argmax[i] == order[0] and r.runner_up[i] == order[1]
+        assert r.top2_margin[i] == pytest.approx(y[order[0]] - y[order[1]], abs=1e-12)
+        assert r.top23_margin[i] == pytest.approx(y[order[1]] - y[order[2]], abs=1e-12)
         others = np.delete(y, tokens[i])
         assert r.margin[i] == pytest.approx(y[tokens[i]] - others.max(), abs=1e-12)
         assert r.y_claimed[i] == pytest.approx(y[tokens[i]], abs=1e-12)
