@@ -40,3 +40,63 @@ def test_host_only_entry_points():
     assert difr.difr_workspace_bytes(0, 3072, 128256) == 0
     small = difr.difr_workspace_bytes(100, 64, 300)  # 100 rows pad to 256; 300 ids are two tiles: at most two strips
     assert small in (256 + 16 * 256 + 32 * 256 * s for s in (1, 2))
+
+
+def test_bad_arguments_are_refused_on_the_host():
+    """Everything the host can check is checked before the device is touched: these calls run without a GPU and
+    never dereference the (fake) pointers."""
+    import ctypes
+
+    L = difr.lib()
+    p = ctypes.c_void_p(0x10000)  # non-null, 16-byte aligned, never read
+    INVALID, SHAPE, OK = -1, -2, 0
+
+    def out(**kw):
+        c = difr._COut()
+        c.sigma, c.eps, c.score = 0.3, 1e-12, 0x10000
+        for k, v in kw.items():
+            setattr(c, k, v)
+        return c
+
+    def score(fn, h=p, tokens=p, temperature=1.0, T=128, d=64, V=1000, o=None):
+        o = o if o is not None else out()
+        return getattr(L, fn)(h, p, tokens, p, p, temperature, T, d, V, ctypes.byref(o), None)
+
+    for fn in ("difr_score_gm", "difr_score_ipt", "difr_score_both"):
+        assert score(fn, h=None) == INVALID
+        assert score(fn, tokens=None) == INVALID
+        assert score(fn, T=-1) == INVALID
+        assert score(fn, o=out(sigma=0.0)) == INVALID
+        assert score(fn, o=out(eps=-1.0)) == INVALID
+        assert score(fn, o=out(score=None)) == INVALID
+        assert score(fn, temperature=-0.5) == INVALID
+        assert score(fn, temperature=float("nan")) == INVALID
+    assert score("difr_score_ipt", temperature=0.0) == INVALID   # the IPT sampler needs a distribution
+    assert score("difr_score_both", temperature=0.0) == INVALID
+    assert score("difr_score_both") == INVALID                   # no score_ipt / sigma_ipt given
+    assert score("difr_score_gm", d=60, o=out()) == SHAPE        # d must be a multiple of 8
+    assert score("difr_score_gm", V=1) == SHAPE
+    assert score("difr_score_gm", T=0) == OK                     # nothing to do
+    assert difr.difr_filtered_workspace_bytes(128, 60, 1000) == 0
+    assert difr.difr_filtered_workspace_bytes(128, 64, 1000) > difr.difr_workspace_bytes(128, 64, 1000)
+
+    def filtered(top_k, top_p, s, temperature=1.0, o=None):
+        f = difr._CFilter(top_k, top_p, s)
+        o = o if o is not None else out()
+        return L.difr_score_gm_filtered(p, p, p, p, p, temperature, 128, 64, 1000, ctypes.byref(f), ctypes.byref(o), None)
+
+    assert filtered(50, 0.95, 0) == INVALID and filtered(50, 0.95, 9) == INVALID   # 1 <= s <= 8
+    assert filtered(65, 1.0, 1) == INVALID                                         # top_k <= 64
+    assert filtered(0, 0.9, 1) == INVALID                                          # a nucleus needs a top_k in front
+    assert filtered(50, 0.0, 1) == INVALID and filtered(50, 1.5, 1) == INVALID
+    assert filtered(50, 0.95, 4, temperature=0.0) == INVALID
+    assert filtered(50, 0.95, 4, o=out(temperatures=0x10000)) == INVALID
+
+    taus = (ctypes.c_float * 5)(-1.0, -2.0, -3.0, -4.0, -5.0)
+    adm = lambda n, sigma=0.3: L.difr_admissible(p, p, p, p, 1.0, 128, 64, 1000, p, p, p, sigma, 1e-12, taus, n, p, p,
+                                                 1 << 30, None, None)
+    assert adm(0) == INVALID and adm(5) == INVALID and adm(2, sigma=0.0) == INVALID
+    assert L.difr_exfiltratable_bits(p, p, 0, 1000, None, 1, 128, None, None, None) == INVALID  # R >= 1
+    assert L.difr_exfiltratable_bits(None, p, 8, 1000, None, 1, 128, None, None, None) == INVALID
+    assert L.difr_detect(None, -1.0, None, None, 0, None, 1, 128, None, None, None) == INVALID
+    assert L.difr_detect(p, float("nan"), None, None, 0, None, 1, 128, None, None, None) == INVALID
