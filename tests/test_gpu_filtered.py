@@ -115,3 +115,25 @@ def test_full_estimator_at_full_size_on_sampled_rows():
     np.testing.assert_allclose(got[rows], want, rtol=0, atol=SCORE_TOL)
     assert np.all(out.row_status.cpu().numpy() == 0)
     assert np.all(np.isfinite(got)) and np.all(got <= 1e-6)
+
+
+def test_results_do_not_depend_on_the_order_work_is_handed_out():
+    """Work units are taken on demand and candidates are appended with atomics, so the order of work differs from
+    launch to launch; the results must not."""
+    T, d, V = 700, 128, 9000
+    h, W, seeds, positions = _small(T, d, V, 81, 2.0)
+    tokens = _claims(h, W, seeds, positions, f32(1.0), 82)
+    dev = Device(h, W, seeds, positions)
+    first = _run(dev, tokens, 1.0, 0.3, 50, 0.95, 4)
+    keep = {k: getattr(first, k).clone() for k in ("score", "cutoff", "margin", "argmax", "runner_up", "lse")}
+    for _ in range(3):
+        again = _run(dev, tokens, 1.0, 0.3, 50, 0.95, 4)
+        for k, v in keep.items():
+            assert torch.equal(getattr(again, k), v, ) or (k in ("score", "cutoff", "margin", "lse")
+                                                            and torch.equal(torch.isnan(getattr(again, k)), torch.isnan(v))
+                                                            and torch.equal(torch.nan_to_num(getattr(again, k)), torch.nan_to_num(v))), k
+    plain = [dev.score("gm", tokens, 1.0, 0.3, EPS) for _ in range(3)]
+    for other in plain[1:]:
+        for k in ("score", "margin", "argmax", "runner_up", "lse"):
+            assert np.array_equal(plain[0][k], other[k], equal_nan=True) if plain[0][k].dtype.kind == "f" else \
+                np.array_equal(plain[0][k], other[k]), k
