@@ -193,3 +193,35 @@ def test_detect_matches_oracle():
     one = stats1.cpu().numpy().view(SEQ_STATS_DTYPE).reshape(-1)
     _, ref1 = oracle.detect(scores.astype(np.float64), f32(tau), margins.astype(np.float64), None)
     assert one["n_flagged"][0] == ref1["n_flagged"][0] and one["n_match"][0] == ref1["n_match"][0]
+
+
+@pytest.mark.parametrize("temperature,sigma", [(1.0, 0.05), (0.7, 1.0)])
+def test_peaked_large_logits(temperature, sigma):
+    """Logits as a trained head produces them: spread over tens of units with a common offset, one or two ids far
+    ahead of the rest, rather than the unit-variance logits of the synthetic workloads."""
+    T, d, V = 260, 256, 6000
+    g = np.random.default_rng(12)
+    hf = g.standard_normal((T, d)).astype(np.float32)
+    Wf = (6.0 * g.standard_normal((V, d)) / math.sqrt(d)).astype(np.float32)
+    bias_dir = g.standard_normal(d).astype(np.float32) / math.sqrt(d)
+    hf += 4.0 * math.sqrt(d) * bias_dir            # every row carries the same strong component ...
+    Wf += 7.0 * bias_dir / math.sqrt(d)            # ... that every id responds to: a common offset of about +28
+    Wf[g.integers(0, V, size=40)] *= 1.8           # a few ids with much larger logits
+    h, W = wl.f32_to_bf16_bits(hf), wl.f32_to_bf16_bits(Wf)
+    seeds = np.array([wl.splitmix64(900 + r // 32) for r in range(T)], dtype=np.uint64)
+    positions = (np.arange(T) % 32 + 1).astype(np.uint32)
+    L = oracle.logits(h, W)
+    assert L.mean() > 15 and L.std() > 4 and L.max() > 50
+    tokens = _claims(h, W, seeds, positions, f32(temperature), 13)
+    dev = Device(h, W, seeds, positions)
+    ref = oracle.score_gm(h, W, tokens, seeds, positions, f32(temperature), f32(sigma), f32(EPS))
+    check_gm(dev.score("gm", tokens, temperature, sigma, EPS), ref)
+    itok = oracle.sample_ipt(h, W, seeds, positions, f32(temperature)).astype(np.int32)
+    itok[::5] = tokens[::5]
+    iref = oracle.score_ipt(h, W, itok, seeds, positions, f32(temperature), f32(0.05), f32(EPS))
+    got = dev.score("ipt", itok, temperature, 0.05, EPS)
+    np.testing.assert_allclose(got["score"], iref.score, rtol=0, atol=SCORE_TOL)
+    np.testing.assert_allclose(got["lse"], iref.lse, rtol=LSE_RTOL)
+    # logits of magnitude 50 carry about 5e-5 of fp32 accumulation error from the tensor cores, which the softmax
+    # turns into a relative error of that size in every probability
+    np.testing.assert_allclose(got["cdf_lo"], iref.cdf_lo, rtol=1e-4, atol=2e-6)
