@@ -305,6 +305,14 @@ difr_status difr_logits(const void* h, const void* W, int64_t T, int64_t d, int6
  */
 difr_status difr_philox(const uint32_t* ctr, const uint32_t* key, int64_t n, uint32_t* out, difr_stream_t stream);
 
+/*
+ * Validation aid: exercises the bounded wait every kernel of the library uses.  One warp waits on a barrier
+ * that nothing arrives at; after `limit_cycles` SM clocks (1 .. 1e9, i.e. well under a second) the wait must
+ * give up.  status2 (device, int32 [2]) receives {DIFR_ERR_TIMEOUT, 1} when it did; the kernel ends normally
+ * either way and the context stays usable.
+ */
+difr_status difr_selftest_wait(int32_t* status2, int64_t limit_cycles, difr_stream_t stream);
+
 const char* difr_status_string(difr_status status); /* host pointer to a static string */
 int difr_version(void);
 

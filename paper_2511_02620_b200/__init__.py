@@ -21,7 +21,7 @@ STATUS_NAMES = {0: "DIFR_OK", -1: "DIFR_ERR_INVALID_ARG", -2: "DIFR_ERR_SHAPE", 
 EXPORTS = ("difr_workspace_bytes", "difr_filtered_workspace_bytes", "difr_score_gm", "difr_score_ipt",
            "difr_score_both", "difr_score_gm_filtered", "difr_score_gm_static",
            "difr_admissible", "difr_exfiltratable_bits", "difr_detect", "difr_logits", "difr_philox",
-           "difr_status_string", "difr_version")
+           "difr_selftest_wait", "difr_status_string", "difr_version")
 STATIC_SCRATCH_BYTES = 16 << 20  # DIFR_STATIC_SCRATCH_BYTES
 
 
@@ -90,6 +90,8 @@ def lib() -> ctypes.CDLL:
                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         L.difr_philox.restype = ctypes.c_int
         L.difr_philox.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]
+        L.difr_selftest_wait.restype = ctypes.c_int
+        L.difr_selftest_wait.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p]
         L.difr_status_string.restype = ctypes.c_char_p
         L.difr_status_string.argtypes = [ctypes.c_int]
         L.difr_version.restype = ctypes.c_int
@@ -293,6 +295,14 @@ def difr_logits(h, W, logits, device_status=None, stream=None):
     if rc != DIFR_OK:
         raise DifrError(rc, "difr_logits")
     return logits
+
+
+def difr_selftest_wait(status2, limit_cycles, stream=None):
+    """Runs the bounded-wait self-test; `status2` is an int32 [2] CUDA tensor."""
+    rc = lib().difr_selftest_wait(_ptr(status2), int(limit_cycles), _stream(stream))
+    if rc != DIFR_OK:
+        raise DifrError(rc, "difr_selftest_wait")
+    return status2
 
 
 def difr_philox(ctr, key, out, stream=None):

@@ -500,6 +500,13 @@ difr_status difr_score_gm_static(const void* h, const void* W, const int32_t* to
   return score_common(0, h, W, tokens, seeds, positions, temperature, T, d, V, &local, stream);
 }
 
+difr_status difr_selftest_wait(int32_t* status2, int64_t limit_cycles, difr_stream_t stream) {
+  if (!status2 || limit_cycles < 1 || limit_cycles > 1000000000LL) return DIFR_ERR_INVALID_ARG;
+  if (launch_wait_selftest(status2, (long long)limit_cycles, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return DIFR_ERR_CUDA;
+  return DIFR_OK;
+}
+
 const char* difr_status_string(difr_status status) {
   switch (status) {
     case DIFR_OK: return "ok";

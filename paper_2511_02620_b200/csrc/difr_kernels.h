@@ -134,6 +134,7 @@ struct BitsParams {
   float* seq_bits;
 };
 cudaError_t launch_bits(const BitsParams& p, cudaStream_t stream);
+cudaError_t launch_wait_selftest(int32_t* status, long long limit_cycles, cudaStream_t stream);
 cudaError_t launch_philox(const uint32_t* ctr, const uint32_t* key, int64_t n, uint32_t* out, cudaStream_t stream);
 
 }  // namespace difr

@@ -308,6 +308,31 @@ cudaError_t launch_count_finalize(const CountParams& p, cudaStream_t stream) {
   return cudaGetLastError();
 }
 
+// --------------------------------------------------- bounded-wait self-test
+// One warp waits on a barrier that nothing ever arrives at, with a short limit: the wait must give up, raise the
+// abort flag and let the kernel end normally.  status[0] = kStatusTimeout if it did, status[1] = the abort flag.
+__global__ void wait_selftest(int32_t* status, long long limit_cycles) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    mbar_fence_init();
+  }
+  __syncthreads();
+  const bool completed = mbar_wait(smem_u32(&bar), 0u, &abort_flag, limit_cycles);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    status[0] = completed ? 0 : kStatusTimeout;
+    status[1] = abort_flag;
+  }
+}
+
+cudaError_t launch_wait_selftest(int32_t* status, long long limit_cycles, cudaStream_t stream) {
+  wait_selftest<<<1, 32, 0, stream>>>(status, limit_cycles);
+  return cudaGetLastError();
+}
+
 // --------------------------------------------------------- Philox validation
 __global__ void philox_blocks(const uint32_t* ctr, const uint32_t* key, int64_t n, uint32_t* out) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;

@@ -225,3 +225,18 @@ def test_peaked_large_logits(temperature, sigma):
     # logits of magnitude 50 carry about 5e-5 of fp32 accumulation error from the tensor cores, which the softmax
     # turns into a relative error of that size in every probability
     np.testing.assert_allclose(got["cdf_lo"], iref.cdf_lo, rtol=1e-4, atol=2e-6)
+
+
+def test_a_wait_that_cannot_complete_gives_up_and_reports_it():
+    """Every device-side wait of the library is bounded; here the bound is a millisecond and nothing ever arrives."""
+    status = torch.zeros(2, dtype=torch.int32, device="cuda")
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    difr.difr_selftest_wait(status, 2_000_000)
+    t1.record()
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [-7, 1]  # DIFR_ERR_TIMEOUT, abort flag raised
+    assert t0.elapsed_time(t1) < 100.0       # milliseconds: it really was bounded
+    # the context is still usable
+    assert int(torch.ones(4, device="cuda").sum().item()) == 4
