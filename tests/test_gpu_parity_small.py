@@ -240,3 +240,28 @@ def test_a_wait_that_cannot_complete_gives_up_and_reports_it():
     assert t0.elapsed_time(t1) < 100.0       # milliseconds: it really was bounded
     # the context is still usable
     assert int(torch.ones(4, device="cuda").sum().item()) == 4
+
+
+def test_scores_do_not_depend_on_how_the_vocabulary_is_split(monkeypatch):
+    """The number of vocabulary strips (and with it the partial records that are merged) is a planning choice:
+    argmax, runner-up and margins must not move at all (they are re-evaluated exactly), the log-sum-exp and the
+    IPT statistics only by the rounding of a differently ordered sum."""
+    T, d, V = 300, 128, 5000
+    h, W, seeds, positions = _small(T, d, V, 14)
+    tokens = _claims(h, W, seeds, positions, 1.0, 15)
+    dev = Device(h, W, seeds, positions)
+    results = []
+    for strips, group in ((1, 1), (3, 2), (20, 1)):
+        monkeypatch.setenv("DIFR_DEBUG_STRIPS", str(strips))
+        monkeypatch.setenv("DIFR_DEBUG_GROUP", str(group))
+        results.append((dev.score("gm", tokens, 1.0, 0.3, EPS), dev.score("ipt", tokens, 1.0, 0.1, EPS)))
+    monkeypatch.delenv("DIFR_DEBUG_STRIPS")
+    monkeypatch.delenv("DIFR_DEBUG_GROUP")
+    results.append((dev.score("gm", tokens, 1.0, 0.3, EPS), dev.score("ipt", tokens, 1.0, 0.1, EPS)))
+    gm0, ipt0 = results[0]
+    for gm, ipt in results[1:]:
+        for k in ("score", "margin", "argmax", "runner_up"):
+            assert np.array_equal(gm[k], gm0[k]), k
+        np.testing.assert_allclose(gm["lse"], gm0["lse"], rtol=2e-6)
+        np.testing.assert_allclose(ipt["cdf_lo"], ipt0["cdf_lo"], rtol=2e-5, atol=1e-7)
+        np.testing.assert_allclose(ipt["score"], ipt0["score"], rtol=0, atol=2e-4)
