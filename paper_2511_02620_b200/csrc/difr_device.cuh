@@ -167,8 +167,8 @@ __device__ __forceinline__ void tma_prefetch_desc(const void* tmap) {
 
 // The same load issued by either CTA of a pair: the data lands in the issuing
 // CTA's shared memory, the byte count is credited to `bar`, a shared::cluster
-// address that may name the partner's barrier.  (No multicast: each CTA fetches
-// its own tile.)
+// address that may name the partner's barrier.  Each CTA fetches its own tile;
+// no load is delivered to more than one CTA.
 // `policy` is an L2 eviction policy made by l2_policy_*().
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst_smem, const void* tmap, int x, int y, uint32_t bar,
                                                  uint64_t policy) {
