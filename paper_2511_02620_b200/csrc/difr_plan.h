@@ -58,7 +58,7 @@ inline double makespan_tiles(int m_tiles, int n_tiles, int S, int gm, int num_pa
 }
 
 // A unit walks its strip tile by tile keeping running statistics in registers and
-// leaves one partial record per (row, strip, column half).  Units are handed out in
+// leaves one partial record per (row, strip).  Units are handed out in
 // raster order: groups of Gm row tiles, inside a group strip by strip, inside a strip
 // row tile by row tile.  The pairs that run at the same time therefore share Gm row
 // tiles of h (each re-read once per vocabulary tile) and stream the same few strips of
