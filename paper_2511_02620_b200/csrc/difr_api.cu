@@ -71,6 +71,25 @@ bool device_info(DeviceInfo* info) {
   return true;
 }
 
+// Shape, plan and temperature fields of the fused kernel's parameters; `ws` (nullable) is the workspace that
+// holds the partial records and, behind them, the unit counter.
+K1Params k1_params(const Plan& pl, int64_t T, int64_t d, int64_t V, float temperature, void* ws) {
+  K1Params k1;
+  memset(&k1, 0, sizeof k1);
+  k1.T = (int)T; k1.d = (int)d; k1.V = (int)V;
+  k1.T_pad = pl.T_pad; k1.m_tiles = pl.m_tiles; k1.n_tiles = pl.n_tiles; k1.k_steps = pl.k_steps;
+  k1.S = pl.S; k1.Gm = pl.Gm; k1.n_units = pl.n_units;
+  k1.c1 = temperature > 0.f ? 1.4426950408889634f / temperature : 0.f;
+  k1.neg_tl2 = -temperature * 0.6931471805599453f;
+  if (ws != nullptr) {
+    k1.partials = reinterpret_cast<Partial*>(ws);
+    k1.unit_counter = reinterpret_cast<int*>(static_cast<unsigned char*>(ws) + pl.partial_bytes);
+  }
+  return k1;
+}
+
+int k1_grid(const Plan& pl, int pairs) { return 2 * (pl.n_units < pairs ? pl.n_units : pairs); }
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // kind: 0 Token-DiFR, 1 Token-IPT-DiFR, 2 both.
@@ -100,19 +119,11 @@ difr_status score_common(int ipt, const void* h, const void* W, const int32_t* t
   CUtensorMap tmap_h, tmap_w;
   if (!make_tmap(&tmap_h, h, T, d, kBM) || !make_tmap(&tmap_w, W, V, d, kBN / 2)) return DIFR_ERR_CUDA;
 
-  K1Params k1;
-  memset(&k1, 0, sizeof k1);
+  K1Params k1 = k1_params(pl, T, d, V, temperature, out->workspace);
   k1.tokens = tokens; k1.seeds = seeds; k1.positions = positions;
-  k1.partials = reinterpret_cast<Partial*>(out->workspace);
   k1.device_status = out->device_status;
   k1.temperatures = out->temperatures;
-  k1.unit_counter = reinterpret_cast<int*>(static_cast<unsigned char*>(out->workspace) + pl.partial_bytes);
-  k1.T = (int)T; k1.d = (int)d; k1.V = (int)V;
-  k1.T_pad = pl.T_pad; k1.m_tiles = pl.m_tiles; k1.n_tiles = pl.n_tiles; k1.k_steps = pl.k_steps;
-  k1.S = pl.S; k1.Gm = pl.Gm; k1.n_units = pl.n_units;
-  k1.c1 = temperature > 0.f ? 1.4426950408889634f / temperature : 0.f;
-  k1.neg_tl2 = -temperature * 0.6931471805599453f;
-  const int grid = 2 * (pl.n_units < info.pairs ? pl.n_units : info.pairs);
+  const int grid = k1_grid(pl, info.pairs);
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
   const bool want_rank = (ipt != 1) && out->rank != nullptr;
@@ -228,21 +239,13 @@ difr_status difr_admissible(const void* h, const void* W, const uint64_t* seeds,
   cp.counts = counts;
   if (launch_count_bounds(cp, s) != cudaSuccess) return DIFR_ERR_CUDA;
 
-  K1Params k1;
-  memset(&k1, 0, sizeof k1);
+  K1Params k1 = k1_params(pl, T, d, V, temperature, ws);
   k1.tokens = argmax;  // the id the count leaves out
   k1.seeds = seeds; k1.positions = positions;
-  k1.partials = reinterpret_cast<Partial*>(ws);
   k1.bounds = cp.bounds;
   k1.device_status = device_status;
-  k1.unit_counter = reinterpret_cast<int*>(ws + pl.partial_bytes);
-  k1.T = (int)T; k1.d = (int)d; k1.V = (int)V;
-  k1.T_pad = pl.T_pad; k1.m_tiles = pl.m_tiles; k1.n_tiles = pl.n_tiles; k1.k_steps = pl.k_steps;
-  k1.S = pl.S; k1.Gm = pl.Gm; k1.n_units = pl.n_units;
-  k1.c1 = 0.f;
-  k1.neg_tl2 = -temperature * 0.6931471805599453f;
   if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
-  const int grid = 2 * (pl.n_units < info.pairs ? pl.n_units : info.pairs);
+  const int grid = k1_grid(pl, info.pairs);
   if (launch_k1(n_tau == 1 ? 4 : 5, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;
   if (launch_count_finalize(cp, s) != cudaSuccess) return DIFR_ERR_CUDA;
   return DIFR_OK;
@@ -343,20 +346,12 @@ difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* 
   if (!make_tmap(&tmap_h, h, T, d, kBM) || !make_tmap(&tmap_w, W, V, d, kBN / 2)) return DIFR_ERR_CUDA;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   unsigned char* ws = static_cast<unsigned char*>(out->workspace);
-  const int grid = 2 * (pl.n_units < info.pairs ? pl.n_units : info.pairs);
+  const int grid = k1_grid(pl, info.pairs);
 
   // ---- first pass: the ordinary scoring pass, which also leaves each strip's two largest group maxima
-  K1Params k1;
-  memset(&k1, 0, sizeof k1);
+  K1Params k1 = k1_params(pl, T, d, V, temperature, ws);
   k1.tokens = tokens; k1.seeds = seeds; k1.positions = positions;
-  k1.partials = reinterpret_cast<Partial*>(ws);
   k1.device_status = out->device_status;
-  k1.unit_counter = reinterpret_cast<int*>(ws + pl.partial_bytes);
-  k1.T = (int)T; k1.d = (int)d; k1.V = (int)V;
-  k1.T_pad = pl.T_pad; k1.m_tiles = pl.m_tiles; k1.n_tiles = pl.n_tiles; k1.k_steps = pl.k_steps;
-  k1.S = pl.S; k1.Gm = pl.Gm; k1.n_units = pl.n_units;
-  k1.c1 = 1.4426950408889634f / temperature;
-  k1.neg_tl2 = -temperature * 0.6931471805599453f;
   if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
   if (launch_k1(6, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;
 
@@ -439,13 +434,9 @@ difr_status difr_logits(const void* h, const void* W, int64_t T, int64_t d, int6
   if (!aligned16(h) || !aligned16(W)) return DIFR_ERR_ALIGN;
   CUtensorMap tmap_h, tmap_w;
   if (!make_tmap(&tmap_h, h, T, d, kBM) || !make_tmap(&tmap_w, W, V, d, kBN / 2)) return DIFR_ERR_CUDA;
-  K1Params k1;
-  memset(&k1, 0, sizeof k1);
+  K1Params k1 = k1_params(pl, T, d, V, 1.f, nullptr);  // no counter: units go round robin
   k1.logits_out = logits; k1.device_status = device_status;
-  k1.T = (int)T; k1.d = (int)d; k1.V = (int)V;
-  k1.T_pad = pl.T_pad; k1.m_tiles = pl.m_tiles; k1.n_tiles = pl.n_tiles; k1.k_steps = pl.k_steps;
-  k1.S = pl.S; k1.Gm = pl.Gm; k1.n_units = pl.n_units;
-  const int grid = 2 * (pl.n_units < info.pairs ? pl.n_units : info.pairs);
+  const int grid = k1_grid(pl, info.pairs);
   if (launch_k1(2, tmap_h, tmap_w, k1, grid, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
     return DIFR_ERR_CUDA;
   return DIFR_OK;
