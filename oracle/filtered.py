@@ -108,3 +108,66 @@ def score_gm_filtered(h_bits, W_bits, tokens, seeds, positions, temperature, sig
             pi[r] = token_difr_filtered(L[r], G, temperature, t, s, sigma, cut[r])
         score[r] = math.log(pi[r] + eps)
     return score, pi, cut
+
+
+# ---------------------------------------------------------------- Token-IPT-DiFR under the sampling filter
+def filter_kept(logits: np.ndarray, temperature: float, top_k: int, top_p: float) -> np.ndarray:
+    """Ids that survive top-k followed by top-p (all ids when neither is set), in descending logit order."""
+    logits = np.asarray(logits, dtype=np.float64)
+    V = logits.shape[0]
+    order = np.argsort(-logits, kind="stable")
+    kept = order[:top_k] if 0 < top_k < V else order
+    if top_p < 1.0:
+        if temperature > 0.0:
+            z = logits[kept] / temperature
+            p = np.exp(z - z.max())
+            c = np.cumsum(p) / p.sum()
+            n = int(np.searchsorted(c, top_p, side="left")) + 1
+        else:
+            n = 1
+        kept = kept[: min(n, len(kept))]
+    return kept
+
+
+def filtered_probs(logits: np.ndarray, temperature: float, top_k: int, top_p: float) -> np.ndarray:
+    """The distribution the filtered sampler draws from: softmax(l / Temp) restricted to the surviving ids and
+    renormalised (Alg. Token-IPT-DiFR: the same temperature / top-k / nucleus policy as generation)."""
+    logits = np.asarray(logits, dtype=np.float64)
+    kept = filter_kept(logits, temperature, top_k, top_p)
+    p = np.zeros_like(logits)
+    z = logits[kept] / temperature
+    e = np.exp(z - z.max())
+    p[kept] = e / e.sum()
+    return p
+
+
+def ipt_sample_filtered(logits, temperature, top_k, top_p, mu: float) -> int:
+    """Alg. IPT Sampler on the filtered distribution: min{v : C_v > mu}."""
+    c = np.cumsum(filtered_probs(logits, temperature, top_k, top_p))
+    hit = np.nonzero(c > mu)[0]
+    return int(hit[0]) if len(hit) else int(np.nonzero(filtered_probs(logits, temperature, top_k, top_p))[0][-1])
+
+
+def score_ipt_filtered(h_bits, W_bits, tokens, seeds, positions, temperature, sigma, eps=1e-12, top_k=0, top_p=1.0):
+    """Per row: (score, p_claimed, cdf_lo, mu, cutoff) of Token-IPT-DiFR with the filtered distribution."""
+    from . import ipt_uniform, logits as all_logits, normal_interval_mass
+
+    L = all_logits(h_bits, W_bits)
+    T, V = L.shape
+    score = np.empty(T)
+    pt = np.full(T, np.nan)
+    a = np.full(T, np.nan)
+    mu = np.empty(T)
+    cut = np.empty(T)
+    for r in range(T):
+        mu[r] = ipt_uniform(int(seeds[r]), int(positions[r]))
+        cut[r] = filter_cutoff(L[r], temperature, top_k, top_p)
+        t = int(tokens[r])
+        mass = 0.0
+        if 0 <= t < V:
+            p = filtered_probs(L[r], temperature, top_k, top_p)
+            a[r] = float(np.sum(p[:t]))
+            pt[r] = float(p[t])
+            mass = normal_interval_mass((a[r] - mu[r]) / sigma, (a[r] + pt[r] - mu[r]) / sigma)
+        score[r] = math.log(mass + eps)
+    return score, pt, a, mu, cut

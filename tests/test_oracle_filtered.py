@@ -129,3 +129,57 @@ def test_score_rows_wrap_the_pieces():
     score_f, _, cut_f = filtered.score_gm_filtered(h, W, tokens, seeds, positions, 1.0, 0.3, 1e-12, 5, 0.9, 3)
     L = oracle.logits(h, W)
     assert np.all(cut_f >= np.sort(L, axis=1)[:, -5]) and np.all(np.isfinite(score_f))
+
+
+# ------------------------------------------------------------- Token-IPT-DiFR under the filter
+def test_filtered_distribution_on_a_hand_worked_example():
+    l = np.array([0.0, 3.0, 1.0, 2.0])
+    p = filtered.filtered_probs(l, 1.0, 3, 0.90)      # top 3 = ids 1, 3, 2; nucleus 0.9 keeps ids 1 and 3
+    e3, e2 = math.exp(3.0), math.exp(2.0)
+    np.testing.assert_allclose(p, [0.0, e3 / (e3 + e2), 0.0, e2 / (e3 + e2)], rtol=1e-14)
+    assert filtered.filter_kept(l, 1.0, 0, 1.0).tolist() == [1, 3, 2, 0]
+    full = filtered.filtered_probs(l, 1.0, 0, 1.0)
+    np.testing.assert_allclose(full, np.exp(l) / np.exp(l).sum(), rtol=1e-14)
+    # the cutoff is the smallest kept logit
+    for k, pp in ((3, 0.9), (2, 1.0), (0, 0.65)):
+        kept = filtered.filter_kept(l, 1.0, k, pp)
+        assert filtered.filter_cutoff(l, 1.0, k, pp) == l[kept].min()
+
+
+def test_ipt_score_without_filter_is_the_plain_one_and_with_filter_obeys_the_identities():
+    g = np.random.default_rng(21)
+    T, d, V = 40, 16, 60
+    h = wl.f32_to_bf16_bits(g.standard_normal((T, d)).astype(np.float32))
+    W = wl.f32_to_bf16_bits((2.0 * g.standard_normal((V, d)) / 4).astype(np.float32))
+    seeds = g.integers(1, 2**62, size=T).astype(np.uint64)
+    positions = np.arange(1, T + 1, dtype=np.uint32)
+    tokens = g.integers(0, V, size=T).astype(np.int32)
+    plain = oracle.score_ipt(h, W, tokens, seeds, positions, 0.8, 0.1, 1e-12)
+    s0, pt0, a0, mu0, cut0 = filtered.score_ipt_filtered(h, W, tokens, seeds, positions, 0.8, 0.1, 1e-12, 0, 1.0)
+    np.testing.assert_allclose(s0, plain.score, rtol=0, atol=1e-9)
+    np.testing.assert_allclose(a0, plain.cdf_lo, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(mu0, plain.u, rtol=0, atol=0)
+    assert np.all(np.isneginf(cut0))
+
+    L = oracle.logits(h, W)
+    sigma = 0.07
+    for top_k, top_p in ((8, 1.0), (12, 0.9)):
+        # honest claims of the filtered sampler contain mu in their CDF interval
+        honest = np.array([filtered.ipt_sample_filtered(L[r], 0.8, top_k, top_p, mu0[r]) for r in range(T)], dtype=np.int32)
+        s, pt, a, mu, cut = filtered.score_ipt_filtered(h, W, honest, seeds, positions, 0.8, sigma, 1e-12, top_k, top_p)
+        assert np.all(a <= mu) and np.all(mu < a + pt)
+        assert np.all(L[np.arange(T), honest] >= cut)                      # a sampled id survived the filter
+        assert np.all(s >= np.log(ndtr(pt / sigma) - 0.5 + 1e-12) - 1e-9)   # mu inside [a, b): at worst at an end
+        # an id the filter removed has probability zero: floor score
+        removed = np.array([int(np.argmin(L[r])) for r in range(T)], dtype=np.int32)
+        sr, ptr, _, _, _ = filtered.score_ipt_filtered(h, W, removed, seeds, positions, 0.8, sigma, 1e-12, top_k, top_p)
+        assert np.all(ptr == 0.0) and np.allclose(sr, math.log(1e-12))
+        # telescoping: the masses of all claims add up to the Gaussian mass of [0, 1]
+        r = 3
+        total = 0.0
+        for t in range(V):
+            st, _, _, _, _ = filtered.score_ipt_filtered(h[r:r + 1], W, np.array([t], dtype=np.int32), seeds[r:r + 1],
+                                                         positions[r:r + 1], 0.8, sigma, 1e-300, top_k, top_p)
+            total += math.exp(st[0])
+        want = oracle.normal_interval_mass((0.0 - mu0[r]) / sigma, (1.0 - mu0[r]) / sigma)
+        assert total == pytest.approx(want, rel=1e-9)
