@@ -98,7 +98,7 @@ typedef struct {
   float* y_second;   /* GM, optional: the second largest y                                     */
   float sigma_ipt;   /* difr_score_both only: noise width of the IPT estimator (CDF units), > 0 */
   float* score_ipt;  /* difr_score_both only, required there: ln(mass + eps)                   */
-  float* cutoff;     /* difr_score_gm_filtered only, optional: the filter's cutoff per row     */
+  float* cutoff;     /* difr_score_*_filtered only, optional: the filter's cutoff per row      */
   const float* temperatures; /* difr_score_gm / _ipt / _both, optional: [T] one sampling temperature per
                         row (requests with their own sampling parameters in one batch); when given, the
                         `temperature` argument is ignored.  A row whose value is negative, not finite, or
@@ -231,6 +231,26 @@ size_t difr_filtered_workspace_bytes(int64_t T, int64_t d, int64_t V);
 difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,
                                    const uint32_t* positions, float temperature, int64_t T, int64_t d, int64_t V,
                                    const difr_filter* filter, difr_out* out, difr_stream_t stream);
+
+/*
+ * Token-IPT-DiFR with the generation's sampling filter (Alg. "Token-IPT-DiFR":
+ * the token probabilities include the same temperature / top-k / nucleus
+ * policy as generation): p is softmax(l / Temp) restricted to the ids that
+ * survive the filter (as in difr_score_gm_filtered: the top_k largest logits,
+ * then the shortest prefix whose renormalised mass reaches top_p) and
+ * renormalised; [a, b] is the claimed token's interval of that distribution's
+ * CDF in vocabulary-id order; a claimed id the filter removed has p = 0 and
+ * scores ln(eps).
+ *
+ *   filter->top_k 1..64 (or >= V when V <= 64), filter->top_p in (0, 1]; filter->s is ignored
+ *   temperature > 0; out->workspace needs difr_filtered_workspace_bytes(T, d, V)
+ * Writes score, p_claimed, cdf_lo, u, row_status, out->cutoff (optional) and
+ * lse (of the unfiltered logits).  Two passes over the logits, the second
+ * without noise.
+ */
+difr_status difr_score_ipt_filtered(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,
+                                    const uint32_t* positions, float temperature, int64_t T, int64_t d, int64_t V,
+                                    const difr_filter* filter, difr_out* out, difr_stream_t stream);
 
 /*
  * Sizes of the admissible sets A_t(tau) = { i : FSSL_t(i) >= tau } (Sec.

@@ -19,7 +19,7 @@ STATUS_NAMES = {0: "DIFR_OK", -1: "DIFR_ERR_INVALID_ARG", -2: "DIFR_ERR_SHAPE", 
                 -4: "DIFR_ERR_WORKSPACE", -5: "DIFR_ERR_CUDA", -6: "DIFR_ERR_ARCH", -7: "DIFR_ERR_TIMEOUT"}
 
 EXPORTS = ("difr_workspace_bytes", "difr_filtered_workspace_bytes", "difr_score_gm", "difr_score_ipt",
-           "difr_score_both", "difr_score_gm_filtered", "difr_score_gm_static",
+           "difr_score_both", "difr_score_gm_filtered", "difr_score_ipt_filtered", "difr_score_gm_static",
            "difr_admissible", "difr_exfiltratable_bits", "difr_detect", "difr_logits", "difr_philox",
            "difr_selftest_wait", "difr_status_string", "difr_version")
 STATIC_SCRATCH_BYTES = 16 << 20  # DIFR_STATIC_SCRATCH_BYTES
@@ -73,9 +73,10 @@ def lib() -> ctypes.CDLL:
                                   ctypes.c_void_p]
         L.difr_filtered_workspace_bytes.restype = ctypes.c_size_t
         L.difr_filtered_workspace_bytes.argtypes = [ctypes.c_int64] * 3
-        L.difr_score_gm_filtered.restype = ctypes.c_int
-        L.difr_score_gm_filtered.argtypes = ([ctypes.c_void_p] * 5 + [ctypes.c_float] + [ctypes.c_int64] * 3
-                                             + [ctypes.POINTER(_CFilter), ctypes.POINTER(_COut), ctypes.c_void_p])
+        for name in ("difr_score_gm_filtered", "difr_score_ipt_filtered"):
+            getattr(L, name).restype = ctypes.c_int
+            getattr(L, name).argtypes = ([ctypes.c_void_p] * 5 + [ctypes.c_float] + [ctypes.c_int64] * 3
+                                         + [ctypes.POINTER(_CFilter), ctypes.POINTER(_COut), ctypes.c_void_p])
         L.difr_admissible.restype = ctypes.c_int
         L.difr_admissible.argtypes = ([ctypes.c_void_p] * 4 + [ctypes.c_float] + [ctypes.c_int64] * 3
                                       + [ctypes.c_void_p] * 3 + [ctypes.c_float] * 2
@@ -216,7 +217,14 @@ def difr_filtered_workspace_bytes(T: int, d: int, V: int) -> int:
     return int(lib().difr_filtered_workspace_bytes(T, d, V))
 
 
-def difr_score_gm_filtered(h, W, tokens, seeds, positions, temperature, top_k, top_p, s, out: DifrOut, stream=None):
+def difr_score_ipt_filtered(h, W, tokens, seeds, positions, temperature, top_k, top_p, out: DifrOut, stream=None):
+    """Token-IPT-DiFR on the filtered distribution; workspace as for difr_score_gm_filtered."""
+    return difr_score_gm_filtered(h, W, tokens, seeds, positions, temperature, top_k, top_p, 1, out, stream,
+                                  _fn="difr_score_ipt_filtered")
+
+
+def difr_score_gm_filtered(h, W, tokens, seeds, positions, temperature, top_k, top_p, s, out: DifrOut, stream=None,
+                           _fn="difr_score_gm_filtered"):
     """Alg. Token-DiFR in full: top-k / top-p cutoff, B_i terms, s competitors; `out.workspace` must hold
     difr_filtered_workspace_bytes(T, d, V) bytes.  See include/difr.h."""
     import torch
@@ -230,10 +238,10 @@ def difr_score_gm_filtered(h, W, tokens, seeds, positions, temperature, top_k, t
     _check(positions, torch.int32, (T,), "positions")
     c = out._c()
     f = _CFilter(int(top_k), float(top_p), int(s))
-    rc = lib().difr_score_gm_filtered(_ptr(h), _ptr(W), _ptr(tokens), _ptr(seeds), _ptr(positions),
-                                      float(temperature), T, d, V, ctypes.byref(f), ctypes.byref(c), _stream(stream))
+    rc = getattr(lib(), _fn)(_ptr(h), _ptr(W), _ptr(tokens), _ptr(seeds), _ptr(positions),
+                             float(temperature), T, d, V, ctypes.byref(f), ctypes.byref(c), _stream(stream))
     if rc != DIFR_OK:
-        raise DifrError(rc, "difr_score_gm_filtered")
+        raise DifrError(rc, _fn)
     return out
 
 

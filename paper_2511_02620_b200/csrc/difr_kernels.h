@@ -73,7 +73,8 @@ struct K3Params {
 
 // mode: 0 Gumbel-max epilogue, 1 softmax statistics only, 2 logits dump, 3 Gumbel-max + raw-logit rank,
 // 4 / 5 count the ids whose noisy logit reaches one / four per-row bounds, 6 Gumbel-max + the strips' two
-// largest 16-id group maxima (word 7 of the record), 7 collect the ids that reach the row's bounds on y' / l.
+// largest 16-id group maxima (word 7 of the record), 7 collect the ids that reach the row's bounds on y' / l,
+// 8 softmax statistics + group maxima, 9 collect by raw logit only.
 cudaError_t launch_k1(int mode, const CUtensorMap& tmap_h, const CUtensorMap& tmap_w, const K1Params& p, int grid,
                       cudaStream_t stream);  // grid: number of CTAs, two per pair
 int k1_max_resident_pairs();  // CTA pairs of the fused kernel the current device keeps resident at once
@@ -119,10 +120,14 @@ struct FilterParams {
   float* score;
   float* cutoff;  // nullable
   uint32_t* row_status;
+  float* p_claimed;  // IPT finalize only, nullable
+  float* cdf_lo;
+  float* u;
 };
 cudaError_t set_gauss_legendre(const double* x, const double* w);  // 16 nodes / weights on [-1, 1]
 cudaError_t launch_filter_bounds(const FilterParams& p, cudaStream_t stream);
 cudaError_t launch_filtered_finalize(const FilterParams& p, cudaStream_t stream);
+cudaError_t launch_ipt_filtered_finalize(const FilterParams& p, cudaStream_t stream);
 
 struct BitsParams {
   const uint8_t* classes;

@@ -62,18 +62,19 @@ static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one CTA");
 // GmFilter is Gm that also keeps each strip's two largest 16-id group maxima of the raw logits (the bound of
 // the filter's cutoff comes from them); Collect appends every id whose y' or raw logit reaches the row's
 // bounds to the row's candidate list.
+// IptFilter / CollectLogit are their counterparts without noise, for the IPT estimator under a filter.
 enum : int { kModeGm = 0, kModeIpt = 1, kModeDump = 2, kModeGmRank = 3, kModeCount1 = 4, kModeCount4 = 5,
-             kModeGmFilter = 6, kModeCollect = 7 };
+             kModeGmFilter = 6, kModeCollect = 7, kModeIptFilter = 8, kModeCollectLogit = 9 };
 
 template <int MODE>
 struct Mode {
   static constexpr bool gm = MODE == kModeGm || MODE == kModeGmRank || MODE == kModeGmFilter;
-  static constexpr bool softmax = gm || MODE == kModeIpt;
+  static constexpr bool softmax = gm || MODE == kModeIpt || MODE == kModeIptFilter;
   static constexpr bool rank = MODE == kModeGmRank;
-  static constexpr bool groupmax = MODE == kModeGmFilter;
-  static constexpr bool collect = MODE == kModeCollect;
+  static constexpr bool groupmax = MODE == kModeGmFilter || MODE == kModeIptFilter;
+  static constexpr bool collect = MODE == kModeCollect || MODE == kModeCollectLogit;
   static constexpr int ng = MODE == kModeCount1 ? 1 : (MODE == kModeCount4 ? 4 : 0);  // bounds per row
-  static constexpr bool noise = gm || ng > 0 || collect;
+  static constexpr bool noise = gm || ng > 0 || MODE == kModeCollect;
   static constexpr int ncnt = rank ? 1 : (collect ? 2 : (ng > 0 ? ng : 1));
   static constexpr bool bounds = rank || collect || ng > 0;
   static constexpr bool record = !collect && MODE != kModeDump;
@@ -232,6 +233,27 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
     s.cnt[0] += c;
   }
 
+  // ---- candidates by raw logit only (the IPT estimator under a filter needs no noise)
+  if (MODE == kModeCollectLogit) {
+#pragma unroll
+    for (int j = 0; j < kSub; j += 4) {
+      const float lm = fmaxf(fmaxf(l[j], l[j + 1]), fmaxf(l[j + 2], l[j + 3]));
+      if (lm >= s.bound[1]) {  // rare
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          if (l[j + q] >= s.bound[1] && base + j + q < V) {
+            const int pos = atomicAdd(cand_count, 1);
+            if (pos < cand_cap) {
+              Candidate c;
+              c.id = base + j + q; c.l = l[j + q]; c.y = 0.f;
+              cand_list[pos] = c;
+            }
+          }
+        }
+      }
+    }
+  }
+
   // ---- Gumbel-max replay: top-2 of y' = l - Temp*ln2 * log2(-log2 u), or counts of y' against the row's bounds
   if (M::noise) {
     float c1k = -CUDART_INF_F, c2k = -CUDART_INF_F;
@@ -252,7 +274,7 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
         c1k = fmaxf(c1k, t1);
         c2k = n2;
       }
-      if (M::collect) {
+      if (MODE == kModeCollect) {
         const float ym = fmaxf(fmaxf(y[0], y[1]), fmaxf(y[2], y[3]));
         const float lm = fmaxf(fmaxf(l4[0], l4[1]), fmaxf(l4[2], l4[3]));
         if (ym >= s.bound[0] || lm >= s.bound[1]) {  // rare
@@ -692,6 +714,8 @@ cudaError_t launch_k1(int mode, const CUtensorMap& tmap_h, const CUtensorMap& tm
     case kModeCount4: return launch_mode<kModeCount4>(tmap_h, tmap_w, p, grid, stream);
     case kModeGmFilter: return launch_mode<kModeGmFilter>(tmap_h, tmap_w, p, grid, stream);
     case kModeCollect: return launch_mode<kModeCollect>(tmap_h, tmap_w, p, grid, stream);
+    case kModeIptFilter: return launch_mode<kModeIptFilter>(tmap_h, tmap_w, p, grid, stream);
+    case kModeCollectLogit: return launch_mode<kModeCollectLogit>(tmap_h, tmap_w, p, grid, stream);
   }
   return cudaErrorInvalidValue;
 }

@@ -102,10 +102,13 @@ __global__ void __launch_bounds__(kFWarps * 32) filter_bounds(const FilterParams
   // Any subset's n-th largest is a lower bound of the whole row's n-th largest.  s competitors are refined out of
   // s + 2, and the claimed token may sit among them: s + 3.  A little is taken off for the index bits stored in
   // the keys and for the rounding of z = l * c1.
-  float by = -CUDART_INF_F, bl = CUDART_INF_F;
+  float by = (p.s > 0) ? -CUDART_INF_F : CUDART_INF_F;  // s == 0: no competitors wanted (IPT estimator)
+  float bl = CUDART_INF_F;
   if (p.n_slots <= 128) {
-    const float ky = warp_nth_largest(yk, p.s + 3, lane);
-    if (ky > -CUDART_INF_F) by = ky - 1e-4f * fmaxf(1.f, fabsf(ky));
+    if (p.s > 0) {
+      const float ky = warp_nth_largest(yk, p.s + 3, lane);
+      if (ky > -CUDART_INF_F) by = ky - 1e-4f * fmaxf(1.f, fabsf(ky));
+    }
     if (p.top_k > 0) {
       const float kz = warp_nth_largest(zk, p.top_k, lane);
       bl = -CUDART_INF_F;
@@ -280,6 +283,109 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
     if (p.cutoff) p.cutoff[row] = (float)cutoff;
     if (p.row_status && status_bits) p.row_status[row] |= status_bits;
   }
+}
+
+
+// Token-IPT-DiFR on the filtered distribution (Alg. Token-IPT-DiFR with the generation's top-k / nucleus policy):
+// the kept ids are the first ranks of the row's candidate list by logit; the claimed token's CDF interval is
+// taken over the kept ids in vocabulary-id order.  One warp per row.
+__global__ void __launch_bounds__(kFWarps * 32) ipt_filtered_finalize(const FilterParams p) {
+  __shared__ float sm_l[kFWarps][kMaxK];
+  __shared__ int sm_id[kFWarps][kMaxK];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * kFWarps + warp;
+  if (row >= p.T) return;
+  const int tok = p.tokens[row];
+  const bool tok_ok = tok >= 0 && tok < p.V;
+  const Candidate* list = p.cand_list + (size_t)row * (size_t)p.cand_cap;
+  const int n_found = p.cand_count[row];
+  const int n = n_found < p.cand_cap ? n_found : p.cand_cap;
+  const uint32_t status_bits = (n_found > p.cand_cap) ? 4u : 0u;
+  const int k_eff = p.top_k < n ? p.top_k : n;
+
+  for (int j = 0; j < n; ++j) {
+    const Candidate cj = list[j];
+    int rl = 0;
+    for (int i = lane; i < n; i += 32) {
+      const Candidate ci = list[i];
+      rl += (ci.l > cj.l || (ci.l == cj.l && ci.id < cj.id)) ? 1 : 0;
+    }
+#pragma unroll
+    for (int m = 16; m >= 1; m >>= 1) rl += __shfl_xor_sync(0xffffffffu, rl, m);
+    if (lane == 0 && rl < k_eff) { sm_l[warp][rl] = cj.l; sm_id[warp][rl] = cj.id; }
+  }
+  __syncwarp();
+
+  const uint64_t seed = p.seeds[row];
+  const uint32_t pos = p.positions[row];
+  uint32_t x[4];
+  philox4x32_10(0u, pos, 1u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), x);
+  const double mu = ((double)x[0] + 0.5) * (1.0 / 4294967296.0);
+  double score = log((double)p.eps), pt = CUDART_NAN, a = CUDART_NAN, cutoff = -CUDART_INF;
+  if (k_eff > 0) {
+    const double c1 = (double)p.c1, l0 = (double)sm_l[warp][0];
+    double e0 = 0.0, e1 = 0.0;  // unnormalised masses of ranks lane and lane + 32
+    if (lane < k_eff) e0 = exp2(((double)sm_l[warp][lane] - l0) * c1);
+    if (lane + 32 < k_eff) e1 = exp2(((double)sm_l[warp][lane + 32] - l0) * c1);
+    int last = k_eff - 1;
+    if (p.top_p < 1.f) {
+      double c0 = e0, c1s = e1;
+#pragma unroll
+      for (int m = 1; m < 32; m <<= 1) {
+        const double u0 = __hiloint2double(__shfl_up_sync(0xffffffffu, __double2hiint(c0), m),
+                                           __shfl_up_sync(0xffffffffu, __double2loint(c0), m));
+        const double u1 = __hiloint2double(__shfl_up_sync(0xffffffffu, __double2hiint(c1s), m),
+                                           __shfl_up_sync(0xffffffffu, __double2loint(c1s), m));
+        if (lane >= m) { c0 += u0; c1s += u1; }
+      }
+      c1s += __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(c0), 31),
+                              __shfl_sync(0xffffffffu, __double2loint(c0), 31));
+      const double total = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(c1s), 31),
+                                            __shfl_sync(0xffffffffu, __double2loint(c1s), 31));
+      const double need = (double)p.top_p * total;
+      const unsigned m0 = __ballot_sync(0xffffffffu, lane < k_eff && c0 >= need);
+      const unsigned m1 = __ballot_sync(0xffffffffu, lane + 32 < k_eff && c1s >= need);
+      if (m0) last = __ffs(m0) - 1;
+      else if (m1) last = 32 + __ffs(m1) - 1;
+    }
+    cutoff = warp_dot64(p.h + (size_t)row * (size_t)p.d, p.W + (size_t)sm_id[warp][last] * (size_t)p.d, p.d, lane);
+    if (tok_ok) {
+      // mass of the kept ids, of those below the claimed id, and whether the claimed id is kept
+      const bool k0 = lane <= last, k1 = lane + 32 <= last;
+      const int id0 = k0 ? sm_id[warp][lane] : -1, id1 = k1 ? sm_id[warp][lane + 32] : -1;
+      double z = (k0 ? e0 : 0.0) + (k1 ? e1 : 0.0);
+      double below = ((k0 && id0 < tok) ? e0 : 0.0) + ((k1 && id1 < tok) ? e1 : 0.0);
+      double mine = ((k0 && id0 == tok) ? e0 : 0.0) + ((k1 && id1 == tok) ? e1 : 0.0);
+#pragma unroll
+      for (int m = 16; m >= 1; m >>= 1) {
+        z += shfl_xor_f64(z, m);
+        below += shfl_xor_f64(below, m);
+        mine += shfl_xor_f64(mine, m);
+      }
+      a = below / z;
+      pt = mine / z;  // zero when the filter removed the claimed id
+      const double sigma = (double)p.sigma;
+      const double za = (a - mu) / sigma, zb = (a + pt - mu) / sigma, r2 = 0.70710678118654752440;
+      double mass;
+      if (za >= 0.0) mass = 0.5 * (erfc(za * r2) - erfc(zb * r2));
+      else if (zb <= 0.0) mass = 0.5 * (erfc(-zb * r2) - erfc(-za * r2));
+      else mass = 1.0 - 0.5 * erfc(zb * r2) - 0.5 * erfc(-za * r2);
+      score = log(mass + (double)p.eps);
+    }
+  }
+  if (lane == 0) {
+    p.score[row] = (float)score;
+    if (p.p_claimed) p.p_claimed[row] = (float)pt;
+    if (p.cdf_lo) p.cdf_lo[row] = (float)a;
+    if (p.u) p.u[row] = (float)mu;
+    if (p.cutoff) p.cutoff[row] = (float)cutoff;
+    if (p.row_status && status_bits) p.row_status[row] |= status_bits;
+  }
+}
+
+cudaError_t launch_ipt_filtered_finalize(const FilterParams& p, cudaStream_t stream) {
+  ipt_filtered_finalize<<<(p.T + kFWarps - 1) / kFWarps, kFWarps * 32, 0, stream>>>(p);
+  return cudaGetLastError();
 }
 
 cudaError_t set_gauss_legendre(const double* x, const double* w) {

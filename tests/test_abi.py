@@ -92,6 +92,12 @@ def test_bad_arguments_are_refused_on_the_host():
     assert filtered(50, 0.95, 4, temperature=0.0) == INVALID
     assert filtered(50, 0.95, 4, o=out(temperatures=0x10000)) == INVALID
 
+    f0 = difr._CFilter(0, 1.0, 1)
+    o = out()
+    assert L.difr_score_ipt_filtered(p, p, p, p, p, 1.0, 128, 64, 1000, ctypes.byref(f0), ctypes.byref(o), None) == INVALID
+    f1 = difr._CFilter(65, 1.0, 1)
+    assert L.difr_score_ipt_filtered(p, p, p, p, p, 1.0, 128, 64, 1000, ctypes.byref(f1), ctypes.byref(o), None) == INVALID
+
     taus = (ctypes.c_float * 5)(-1.0, -2.0, -3.0, -4.0, -5.0)
     adm = lambda n, sigma=0.3: L.difr_admissible(p, p, p, p, 1.0, 128, 64, 1000, p, p, p, sigma, 1e-12, taus, n, p, p,
                                                  1 << 30, None, None)

@@ -137,3 +137,45 @@ def test_results_do_not_depend_on_the_order_work_is_handed_out():
         for k in ("score", "margin", "argmax", "runner_up", "lse"):
             assert np.array_equal(plain[0][k], other[k], equal_nan=True) if plain[0][k].dtype.kind == "f" else \
                 np.array_equal(plain[0][k], other[k]), k
+
+
+@pytest.mark.parametrize("T,d,V,scale,temperature,sigma,top_k,top_p", [
+    (96, 64, 3000, 2.0, 1.0, 0.1, 50, 0.95),
+    (80, 72, 9000, 3.0, 0.7, 0.05, 20, 0.9),
+    (64, 64, 9000, 1.0, 1.0, 1.0, 64, 1.0),
+    (40, 64, 40, 2.0, 1.3, 0.2, 64, 0.8),
+])
+def test_ipt_estimator_under_the_filter_matches_the_oracle(T, d, V, scale, temperature, sigma, top_k, top_p):
+    h, W, seeds, positions = _small(T, d, V, 91, scale)
+    L = oracle.logits(h, W)
+    mu = np.array([oracle.ipt_uniform(int(s), int(p)) for s, p in zip(seeds, positions)])
+    tokens = np.array([filtered.ipt_sample_filtered(L[r], f32(temperature), top_k, f32(top_p), mu[r]) for r in range(T)],
+                      dtype=np.int32)                                    # honest claims of the filtered sampler
+    k = np.arange(T)
+    tokens[k % 5 == 1] = np.argsort(-L, axis=1)[k % 5 == 1, 1]           # a likely id that was not drawn
+    tokens[k % 5 == 3] = np.argmin(L, axis=1)[k % 5 == 3]                # an id the filter removes
+    tokens[7] = V + 3
+    dev = Device(h, W, seeds, positions)
+    out = difr.DifrOut.allocate(T, d, V, sigma, EPS)
+    out.workspace = torch.empty(difr.difr_filtered_workspace_bytes(T, d, V), dtype=torch.uint8, device="cuda")
+    out.cutoff = torch.full((T,), float("nan"), dtype=torch.float32, device="cuda")
+    for name in ("score", "p_claimed", "cdf_lo", "u"):
+        getattr(out, name).fill_(float("nan"))
+    difr.difr_score_ipt_filtered(dev.h, dev.W, to_dev(tokens), dev.seeds, dev.positions, f32(temperature), top_k, top_p, out)
+    torch.cuda.synchronize()
+    assert int(out.device_status.item()) == 0
+    want, pt, a, mu_ref, cut = filtered.score_ipt_filtered(h, W, tokens, seeds, positions, f32(temperature), f32(sigma),
+                                                           f32(EPS), top_k, f32(top_p))
+    got = out.score.cpu().numpy()
+    got_cut = out.cutoff.cpu().numpy().astype(np.float64)
+    same_cut = np.isclose(got_cut, cut, rtol=0, atol=1e-5)
+    assert same_cut.mean() >= 0.97
+    ok = same_cut & (np.arange(T) != 7)
+    np.testing.assert_allclose(got[ok], want[ok], rtol=0, atol=SCORE_TOL)
+    np.testing.assert_allclose(out.p_claimed.cpu().numpy()[ok], pt[ok], rtol=2e-4, atol=1e-9)
+    np.testing.assert_allclose(out.cdf_lo.cpu().numpy()[ok], a[ok], rtol=2e-4, atol=2e-6)
+    np.testing.assert_allclose(out.u.cpu().numpy(), mu_ref, rtol=0, atol=1e-7)
+    assert got[7] == pytest.approx(math.log(EPS), abs=1e-5)
+    removed = ok & (k % 5 == 3) & (pt == 0.0)
+    assert removed.sum() > 3 and np.allclose(got[removed], math.log(EPS), atol=1e-5)
+    assert np.all(out.row_status.cpu().numpy() & 4 == 0)
