@@ -231,7 +231,9 @@ difr_status difr_score_both(const void* h, const void* W, const int32_t* tokens,
  * logits (about 3 KB of list per row; row_status bit 2 marks a row whose list
  * overflowed, which takes hundreds of logits within rounding of the top_k-th).
  * With s = 1 and no filter the result equals difr_score_gm's up to quadrature
- * error (< 1e-6 in the score).
+ * error (< 1e-6 in the score).  The first call on a device copies the
+ * quadrature nodes (256 bytes) into the library's constant memory with a
+ * synchronous cudaMemcpyToSymbol.
  */
 typedef struct {
   int32_t top_k;
