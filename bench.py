@@ -403,6 +403,9 @@ def run_ours(args):
             "detect": {"threshold": tau, "n_flagged": n_flagged, "n_tampered": int(tampered.sum()),
                        "n_match": int(stats_np[:, 1].sum())},
         }
+        if args.variants:
+            line["variants_ms"] = time_variants(difr, h_dev, W_dev, tokens_dev, seeds_dev, pos_dev, temperature, sigma,
+                                                T, d, V)
         if world == 1 and not args.no_cpu_baseline:
             val, n, dt, cores = oracle_throughput(w, inp, tokens_np, temperature, sigma, args.cpu_seconds)
             line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
@@ -410,6 +413,50 @@ def run_ours(args):
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def time_variants(difr, h, W, tokens, seeds, pos, temperature, sigma, T, d, V, iters=3):
+    """Milliseconds per call of the other entry points on the same resident inputs (context for the headline)."""
+    import torch
+
+    out = difr.DifrOut.allocate(T, d, V, sigma, 1e-12)
+    out.workspace = torch.empty(difr.difr_filtered_workspace_bytes(T, d, V), dtype=torch.uint8, device="cuda")
+    f = lambda: torch.empty(T, dtype=torch.float32, device="cuda")
+    out.y_max, out.y_second, out.score_ipt, out.sigma_ipt, out.cutoff = f(), f(), f(), 0.05, f()
+    rank = torch.empty(T, dtype=torch.int32, device="cuda")
+    counts = torch.empty((4, T), dtype=torch.int32, device="cuda")
+
+    def gm_rank():
+        out.rank = rank
+        difr.difr_score_gm(h, W, tokens, seeds, pos, temperature, out)
+        out.rank = None
+
+    calls = {
+        "score_gm": lambda: difr.difr_score_gm(h, W, tokens, seeds, pos, temperature, out),
+        "score_gm_with_rank": gm_rank,
+        "score_ipt": lambda: difr.difr_score_ipt(h, W, tokens, seeds, pos, temperature, out),
+        "score_both": lambda: difr.difr_score_both(h, W, tokens, seeds, pos, temperature, out),
+        "admissible_4_thresholds": lambda: difr.difr_admissible(h, W, seeds, pos, temperature, out,
+                                                                [-1.0, -3.0, -6.0, -9.0], counts),
+        "score_gm_filtered_k50_p095_s4": lambda: difr.difr_score_gm_filtered(h, W, tokens, seeds, pos, temperature,
+                                                                             50, 0.95, 4, out),
+        "score_ipt_filtered_k50_p095": lambda: difr.difr_score_ipt_filtered(h, W, tokens, seeds, pos, temperature,
+                                                                           50, 0.95, out),
+    }
+    res = {}
+    calls["score_gm"]()
+    for name, fn in calls.items():
+        fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(iters):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        res[name] = a.elapsed_time(b) / iters
+    assert int(out.device_status.item()) == 0
+    return res
 
 
 def main():
@@ -425,6 +472,7 @@ def main():
     ap.add_argument("--sigma", type=float, default=0.05)
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--variants", action="store_true", help="also time the other entry points (extra JSON key)")
     args = ap.parse_args()
     if args.temperature is None:
         args.temperature = float(wl.WORKLOADS[args.workload].temperatures[-1])
