@@ -106,3 +106,17 @@ def test_bad_arguments_are_refused_on_the_host():
     assert L.difr_exfiltratable_bits(None, p, 8, 1000, None, 1, 128, None, None, None) == INVALID
     assert L.difr_detect(None, -1.0, None, None, 0, None, 1, 128, None, None, None) == INVALID
     assert L.difr_detect(p, float("nan"), None, None, 0, None, 1, 128, None, None, None) == INVALID
+
+
+def test_header_is_plain_c():
+    """include/difr.h is the boundary: it must compile as C99 and as C++ on its own."""
+    import subprocess
+    import tempfile
+
+    src = '#include "difr.h"\nint main(void) { difr_out o; difr_filter f; (void)o; (void)f; return (int)sizeof(difr_seq_stats) - 16; }\n'
+    with tempfile.TemporaryDirectory() as tmp:
+        path = os.path.join(tmp, "t.c")
+        open(path, "w").write(src)
+        inc = os.path.join(ROOT, "include")
+        subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-I", inc, path])
+        subprocess.check_call(["g++", "-std=c++17", "-Wall", "-Werror", "-fsyntax-only", "-x", "c++", "-I", inc, path])
