@@ -494,7 +494,11 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     }
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
-    if (cta == 0 && lane == 0) {
+    // The whole warp walks the loop and one elected lane issues: with a warp-uniform loop the descriptors and
+    // barrier addresses live in uniform registers, and an MMA costs the issuing warp a fraction of the
+    // instructions it costs a lone lane.  (As a single-lane loop this thread was the bottleneck: competing for
+    // issue slots with the epilogue warps of its scheduler it needed about 590 clocks per 512-clock step.)
+    if (cta == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16(kPairM, kBN);
       // The descriptors of a stage differ from those of stage 0 only in the 14-bit address field
       // (units of 16 bytes), which never carries out of the field: shared memory ends below 256 KB.
@@ -506,30 +510,33 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
       int uslot = 0;
       uint32_t uphase = 0;
       while (ok) {
-        const int u = next_unit(uslot, uphase, false);
+        const int u = next_unit(uslot, uphase, true);
         if (u < 0) break;
         const Unit w = decode_unit(p, u);
         for (int n = w.n0; n < w.n1 && ok; ++n) {
-          if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+          if (!__all_sync(0xffffffffu, mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag))) { ok = false; break; }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kBN);
           uint32_t accumulate = 0;
           for (int k = 0; k < p.k_steps; ++k) {
-            if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait(full_bar(stage), phase, abort_flag))) { ok = false; break; }
             tc_fence_after();
             const uint32_t a_lo = desc_lo0 + (uint32_t)stage * (kStageBytes >> 4);
+            if (elect_one()) {
 #pragma unroll
-            for (int kk = 0; kk < kBK / 16; ++kk) {
-              // 16 bf16 = 32 bytes further along K inside the 128-byte swizzled row: +2 in 16-byte units
-              const uint64_t a_desc = ((uint64_t)desc_hi << 32) | (a_lo + 2u * kk);
-              const uint64_t b_desc = ((uint64_t)desc_hi << 32) | (a_lo + (kABytes >> 4) + 2u * kk);
-              umma_bf16_pair(d_tmem, a_desc, b_desc, idesc, accumulate);
-              accumulate = 1;
+              for (int kk = 0; kk < kBK / 16; ++kk) {
+                const uint64_t a_desc = ((uint64_t)desc_hi << 32) | (a_lo + 2u * kk);
+                const uint64_t b_desc = ((uint64_t)desc_hi << 32) | (a_lo + (kABytes >> 4) + 2u * kk);
+                umma_bf16_pair(d_tmem, a_desc, b_desc, idesc, (kk == 0) ? accumulate : 1u);
+              }
+              umma_commit_pair(empty_bar(stage), 3);
             }
-            umma_commit_pair(empty_bar(stage), 3);  // frees the stage in both CTAs once these MMAs have read it
+            __syncwarp();
+            accumulate = 1;
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
-          if (ok) umma_commit_pair(acc_full_bar(acc), 3);
+          if (ok && elect_one()) umma_commit_pair(acc_full_bar(acc), 3);
+          __syncwarp();
           if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
         }
       }
