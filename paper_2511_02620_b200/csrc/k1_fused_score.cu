@@ -461,7 +461,8 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     }
   } else if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    // (the whole warp walks the loop, one elected lane issues: see the MMA issuer)
+    {
       // a CTA re-reads its h tile for every vocabulary tile of the strip, and the other strips of the
       // raster group read it too: ask L2 to keep it.  A W tile is wanted by every pair of its strip within
       // a few tile times and then not for a long while: ordinary priority (marking it evict-first loses it
@@ -474,19 +475,22 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
       int uslot = 0;
       uint32_t uphase = 0;
       while (ok) {
-        const int u = next_unit(uslot, uphase, false);
+        const int u = next_unit(uslot, uphase, true);
         if (u < 0) break;
         const Unit w = decode_unit(p, u);
         const int row0 = w.m * kPairM + (int)cta * kBM;
         for (int n = w.n0; n < w.n1 && ok; ++n) {
           const int wrow0 = n * kBN + (int)cta * (kBN / 2);
           for (int k = 0; k < p.k_steps; ++k) {
-            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
-            if (cta == 0) mbar_arrive_expect_tx(full_bar(stage), 2u * kStageBytes);
-            const uint32_t full0 = full0_base + 8u * (uint32_t)stage;
-            const uint32_t a_dst = smem_base + (uint32_t)stage * kStageBytes;
-            tma_load_2d_pair(a_dst, &tmap_h, k * kBK, row0, full0, keep);
-            tma_load_2d_pair(a_dst + kABytes, &tmap_w, k * kBK, wrow0, full0, stream);
+            if (!__all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag))) { ok = false; break; }
+            if (elect_one()) {
+              if (cta == 0) mbar_arrive_expect_tx(full_bar(stage), 2u * kStageBytes);
+              const uint32_t full0 = full0_base + 8u * (uint32_t)stage;
+              const uint32_t a_dst = smem_base + (uint32_t)stage * kStageBytes;
+              tma_load_2d_pair(a_dst, &tmap_h, k * kBK, row0, full0, keep);
+              tma_load_2d_pair(a_dst + kABytes, &tmap_w, k * kBK, wrow0, full0, stream);
+            }
+            __syncwarp();
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
         }
