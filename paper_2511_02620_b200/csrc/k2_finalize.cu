@@ -79,6 +79,38 @@ __device__ __forceinline__ double warp_dot(const uint16_t* a, const uint16_t* b,
   return acc;
 }
 
+// Three such dot products against the same row a, their loads in flight together; a null row gives 0.
+// Each sum is taken in warp_dot's order, so the values are the same as three separate calls.
+__device__ __forceinline__ void warp_dot3(const uint16_t* a, const uint16_t* b0, const uint16_t* b1,
+                                          const uint16_t* b2, int d, int lane, double out[3]) {
+  const uint16_t* b[3] = {b0, b1, b2};
+  double acc[3] = {0.0, 0.0, 0.0};
+  for (int k = lane * 8; k < d; k += 32 * 8) {
+    const uint4 va = *reinterpret_cast<const uint4*>(a + k);
+    uint4 vb[3];
+#pragma unroll
+    for (int j = 0; j < 3; ++j)
+      vb[j] = b[j] != nullptr ? *reinterpret_cast<const uint4*>(b[j] + k) : make_uint4(0u, 0u, 0u, 0u);
+    const uint32_t wa[4] = {va.x, va.y, va.z, va.w};
+#pragma unroll
+    for (int j = 0; j < 3; ++j) {
+      const uint32_t wb[4] = {vb[j].x, vb[j].y, vb[j].z, vb[j].w};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        acc[j] = fma(bf16_to_double(wa[q] & 0xFFFFu), bf16_to_double(wb[q] & 0xFFFFu), acc[j]);
+        acc[j] = fma(bf16_to_double(wa[q] >> 16), bf16_to_double(wb[q] >> 16), acc[j]);
+      }
+    }
+  }
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) {
+#pragma unroll
+    for (int j = 0; j < 3; ++j) acc[j] += shfl_xor_double(acc[j], m);
+  }
+#pragma unroll
+  for (int j = 0; j < 3; ++j) out[j] = acc[j];
+}
+
 __device__ __forceinline__ double gumbel_exact(uint64_t seed, uint32_t position, uint32_t id) {
   uint32_t x[4];
   philox4x32_10(id >> 2, position, 0u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), x);
@@ -155,16 +187,20 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
   if (temp_bad) status |= 8u;
   const double lse = (temp_f > 0.f) ? (acc.lmax + log2(acc.lsum)) * ln2 : CUDART_NAN;
 
-  double l_tok = 0.0;
-  if (tok_ok) l_tok = warp_dot(hrow, p.W + (size_t)tok * (size_t)p.d, p.d, lane);
+  // the exact logits of the claimed token and (Token-DiFR) of the two candidates, in one pass over h's row
+  const int c1 = (p.ipt != 1 && acc.i1 >= 0 && acc.i1 < p.V) ? acc.i1 : -1;
+  const int c2 = (p.ipt != 1 && acc.i2 >= 0 && acc.i2 < p.V) ? acc.i2 : -1;
+  double l_exact[3];
+  warp_dot3(hrow, tok_ok ? p.W + (size_t)tok * (size_t)p.d : nullptr,
+            c1 >= 0 ? p.W + (size_t)c1 * (size_t)p.d : nullptr,
+            c2 >= 0 ? p.W + (size_t)c2 * (size_t)p.d : nullptr, p.d, lane, l_exact);
+  const double l_tok = l_exact[0];
 
   if (p.ipt != 1) {
     // ---- Token-DiFR: exact y = l + Temp * G for the claimed token and the two candidates
-    const int c1 = (acc.i1 >= 0 && acc.i1 < p.V) ? acc.i1 : -1;
-    const int c2 = (acc.i2 >= 0 && acc.i2 < p.V) ? acc.i2 : -1;
     double y1 = -CUDART_INF, y2 = -CUDART_INF, yt = -CUDART_INF;
-    if (c1 >= 0) y1 = warp_dot(hrow, p.W + (size_t)c1 * (size_t)p.d, p.d, lane) + temp * gumbel_exact(seed, pos, c1);
-    if (c2 >= 0) y2 = warp_dot(hrow, p.W + (size_t)c2 * (size_t)p.d, p.d, lane) + temp * gumbel_exact(seed, pos, c2);
+    if (c1 >= 0) y1 = l_exact[1] + temp * gumbel_exact(seed, pos, c1);
+    if (c2 >= 0) y2 = l_exact[2] + temp * gumbel_exact(seed, pos, c2);
     if (tok_ok) yt = l_tok + temp * gumbel_exact(seed, pos, (uint32_t)tok);
     if (lane == 0) {
       // order the two candidates exactly (ties: lowest id)
