@@ -3,6 +3,7 @@ uniform mapping and the Gumbel transform."""
 import ctypes
 import ctypes.util
 import math
+import os
 
 import mpmath
 import numpy as np
@@ -56,6 +57,19 @@ def test_philox_matches_curand_host_generator():
             counter, sub = divmod(first + j, 65536)
             mine = oracle.philox4x32_10([counter & 0xFFFFFFFF, counter >> 32, sub, 0], key)
             assert np.array_equal(mine, words[j]), (hex(seed), first, j)
+
+
+def test_philox_known_answer_vectors():
+    """The published known-answer vectors of the algorithm (all-zero, all-one and
+    pi-digit inputs); unlike the cuRAND comparison this needs no library."""
+    path = os.path.join(os.path.dirname(__file__), "golden", "philox4x32_10_kat.txt")
+    rows = [ln.split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 3
+    for words in rows:
+        w = [int(x, 16) for x in words]
+        assert len(w) == 10
+        out = oracle.philox4x32_10(w[0:4], w[4:6])
+        assert [int(x) for x in out] == w[6:10]
 
 
 def test_philox_is_a_bijection_of_the_counter_low_bits():

@@ -1,6 +1,7 @@
 """Pins for the oracle's risk classes, admissible sets and information bound
 (Sec. "Empirical Results"; Alg. "Per-Token Risk Classification via GLS and Rank")."""
 import math
+import os
 
 import numpy as np
 import pytest
@@ -83,3 +84,15 @@ def test_exfiltratable_information_worked_cases():
     assert one.tolist() == [18.0]
     # a suspicious token never carries more than a dangerous one, nor a safe one more than log2 |V|
     assert math.log2(R) <= math.log2(V)
+
+
+def test_exfiltratable_information_caps_the_paper_states():
+    """Suspicious tokens carry log2(rank cutoff) bits (2 at cutoff 4, 3 at cutoff 8), dangerous ones
+    log2 |V|: the figures the paper prints, read from the fixture."""
+    path = os.path.join(os.path.dirname(__file__), "golden", "risk_class_bits.txt")
+    rows = [ln.split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 4
+    for cls, R, V, want in rows:
+        bits, _ = oracle.exfiltratable_bits(np.array([int(cls)], dtype=np.uint8), np.array([7], dtype=np.int32),
+                                            int(R), int(V))
+        assert bits.tolist() == [float(want)]
