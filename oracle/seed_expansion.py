@@ -16,8 +16,9 @@ library takes, one plain loop per definition:
                             precede row r, each bound to its place, plus the caller's hash of the prompt
   expanded seed           s'_r = words 0,1 of Philox-4x32-10(counter (c_r low, c_r high, 0, 2), key seed_r)
 
-and s'_r then takes the place of seed_r in RO(seed || i).  Nothing here is
-printed by the paper, so only properties pin it (tests/test_oracle_seed_expansion.py).
+and s'_r then takes the place of seed_r in RO(seed || i).  Parity unpinned:
+nothing here is printed by the paper, so only properties pin it
+(tests/test_oracle_seed_expansion.py).
 """
 from __future__ import annotations
 

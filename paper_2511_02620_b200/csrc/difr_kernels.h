@@ -140,6 +140,9 @@ struct BitsParams {
 };
 cudaError_t launch_bits(const BitsParams& p, cudaStream_t stream);
 cudaError_t launch_wait_selftest(int32_t* status, long long limit_cycles, cudaStream_t stream);
+cudaError_t launch_expand_seeds(const uint64_t* seeds, const int32_t* tokens, const int32_t* seq_offsets,
+                                const uint64_t* prompt_hashes, long long n_seq, long long T, uint64_t* expanded,
+                                cudaStream_t stream);
 cudaError_t launch_philox(const uint32_t* ctr, const uint32_t* key, int64_t n, uint32_t* out, cudaStream_t stream);
 
 }  // namespace difr

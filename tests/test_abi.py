@@ -106,6 +106,11 @@ def test_bad_arguments_are_refused_on_the_host():
     assert L.difr_exfiltratable_bits(None, p, 8, 1000, None, 1, 128, None, None, None) == INVALID
     assert L.difr_detect(None, -1.0, None, None, 0, None, 1, 128, None, None, None) == INVALID
     assert L.difr_detect(p, float("nan"), None, None, 0, None, 1, 128, None, None, None) == INVALID
+    assert L.difr_expand_seeds(None, p, None, 1, None, 128, p, None) == INVALID
+    assert L.difr_expand_seeds(p, None, None, 1, None, 128, p, None) == INVALID
+    assert L.difr_expand_seeds(p, p, None, 1, None, 128, None, None) == INVALID
+    assert L.difr_expand_seeds(p, p, None, 1, None, -1, p, None) == INVALID
+    assert L.difr_expand_seeds(p, p, None, 1, None, 0, p, None) == OK
 
 
 def test_header_is_plain_c():
