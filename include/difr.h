@@ -90,7 +90,8 @@ typedef struct {
   float* u;           /* IPT: the uniform mu of this row                           */
   uint32_t* row_status; /* bit0: claimed id outside [0, V); bit1: non-finite logits;
                            bit2: candidate list overflow (difr_score_gm_filtered);
-                           bit3: unusable per-row temperature                             */
+                           bit3: unusable per-row temperature; bit4: the nucleus holds more
+                           ids than the filtered calls resolve (64)                        */
   void* workspace;      /* >= difr_workspace_bytes(T, d, V) bytes, 16-byte aligned;
                            contents are scratch, overwritten by every call         */
   size_t workspace_bytes;
@@ -219,7 +220,10 @@ difr_status difr_score_both(const void* h, const void* W, const int32_t* tokens,
  * (512 nodes over the range that carries the mass), not by sampling.
  *
  *   filter->top_k  0: no top-k; otherwise 1..64 (a top_k >= V filters nothing)
- *   filter->top_p  in (0, 1]; 1: no nucleus; < 1 requires top_k >= 1
+ *   filter->top_p  in (0, 1]; 1: no nucleus.  With no top-k in front of it the nucleus is the
+ *                  shortest prefix that holds top_p of the whole row's softmax mass, and it is
+ *                  resolved among the 64 largest logits: a row whose 64 largest logits hold
+ *                  less than that gets row_status bit 4 and the 64th largest logit as cutoff
  *   filter->s      1..8
  *   temperature > 0
  *   out->workspace needs difr_filtered_workspace_bytes(T, d, V) bytes
@@ -256,7 +260,9 @@ difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* 
  * CDF in vocabulary-id order; a claimed id the filter removed has p = 0 and
  * scores ln(eps).
  *
- *   filter->top_k 1..64 (or >= V when V <= 64), filter->top_p in (0, 1]; filter->s is ignored
+ *   filter->top_k 1..64 (or >= V when V <= 64), or 0 with top_p < 1: a nucleus over the whole
+ *   vocabulary as in difr_score_gm_filtered (row_status bit 4 when it holds more than 64 ids);
+ *   filter->top_p in (0, 1]; filter->s is ignored
  *   temperature > 0; out->workspace needs difr_filtered_workspace_bytes(T, d, V)
  * Writes score, p_claimed, cdf_lo, u, row_status, out->cutoff (optional) and
  * lse (of the unfiltered logits).  Two passes over the logits, the second

@@ -326,7 +326,10 @@ difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* 
   if (top_k < 0 || !(top_p > 0.f) || !(top_p <= 1.f) || filter->s < 1 || filter->s > 8) return DIFR_ERR_INVALID_ARG;
   if (top_k >= V && top_p >= 1.f) top_k = 0;  // keeps the whole vocabulary: no filter
   if (top_k > 64 && top_k < V) return DIFR_ERR_INVALID_ARG;
-  if (top_p < 1.f && (top_k < 1 || (top_k > 64 && V > 64))) return DIFR_ERR_INVALID_ARG;
+  // a nucleus with no top-k in front of it (or one that keeps everything) is taken over the whole
+  // vocabulary's mass and resolved among the 64 largest logits
+  const int nucleus_full = (top_p < 1.f && (top_k < 1 || top_k >= V)) ? 1 : 0;
+  if (nucleus_full) top_k = 64;
   if (top_k > V) top_k = (int)V;
   if ((d % 8) != 0 || V < 2) return DIFR_ERR_SHAPE;
   if (T == 0) return DIFR_OK;
@@ -372,7 +375,7 @@ difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* 
   fp.h = k2.h; fp.W = k2.W; fp.tokens = tokens; fp.seeds = seeds; fp.positions = positions;
   fp.partials = k1.partials; fp.n_slots = pl.n_slots; fp.T_pad = pl.T_pad; fp.T = (int)T; fp.d = (int)d; fp.V = (int)V;
   fp.temperature = temperature; fp.sigma = out->sigma; fp.eps = out->eps; fp.c1 = k1.c1;
-  fp.top_k = top_k; fp.top_p = top_p; fp.s = filter->s;
+  fp.top_k = top_k; fp.top_p = top_p; fp.s = filter->s; fp.nucleus_full = nucleus_full;
   fp.bounds = reinterpret_cast<float*>(ws + pl.bounds_offset);
   fp.cand_list = reinterpret_cast<const Candidate*>(ws + list_off);
   fp.cand_count = reinterpret_cast<const int*>(ws + count_off);
@@ -401,9 +404,13 @@ difr_status difr_score_ipt_filtered(const void* h, const void* W, const int32_t*
   if (!(temperature > 0.f) || !isfinite(temperature) || out->temperatures != nullptr) return DIFR_ERR_INVALID_ARG;
   int top_k = filter->top_k;
   const float top_p = filter->top_p;
-  if (top_k < 1 || !(top_p > 0.f) || !(top_p <= 1.f)) return DIFR_ERR_INVALID_ARG;  // no filter: difr_score_ipt
-  if (top_k > 64 && top_k < V) return DIFR_ERR_INVALID_ARG;
+  if (top_k < 0 || !(top_p > 0.f) || !(top_p <= 1.f)) return DIFR_ERR_INVALID_ARG;
   if (top_k > V) top_k = (int)V;
+  if ((top_k < 1 || top_k >= V) && top_p >= 1.f && V > 64) return DIFR_ERR_INVALID_ARG;  // no filter: difr_score_ipt
+  if (top_k > 64 && top_k < V) return DIFR_ERR_INVALID_ARG;
+  // a nucleus with no top-k in front of it: over the whole vocabulary's mass, resolved among the 64 largest logits
+  const int nucleus_full = (top_p < 1.f && (top_k < 1 || top_k >= V)) ? 1 : 0;
+  if (nucleus_full || top_k < 1) top_k = V < 64 ? (int)V : 64;
   if (top_k > 64) return DIFR_ERR_INVALID_ARG;  // the kept set is held in 64 slots
   if ((d % 8) != 0 || V < 2) return DIFR_ERR_SHAPE;
   if (T == 0) return DIFR_OK;
@@ -447,7 +454,7 @@ difr_status difr_score_ipt_filtered(const void* h, const void* W, const int32_t*
   fp.h = k2.h; fp.W = k2.W; fp.tokens = tokens; fp.seeds = seeds; fp.positions = positions;
   fp.partials = k1.partials; fp.n_slots = pl.n_slots; fp.T_pad = pl.T_pad; fp.T = (int)T; fp.d = (int)d; fp.V = (int)V;
   fp.temperature = temperature; fp.sigma = out->sigma; fp.eps = out->eps; fp.c1 = k1.c1;
-  fp.top_k = top_k; fp.top_p = top_p; fp.s = 0;
+  fp.top_k = top_k; fp.top_p = top_p; fp.s = 0; fp.nucleus_full = nucleus_full;
   fp.bounds = reinterpret_cast<float*>(ws + pl.bounds_offset);
   fp.cand_list = reinterpret_cast<const Candidate*>(ws + list_off);
   fp.cand_count = reinterpret_cast<const int*>(ws + count_off);

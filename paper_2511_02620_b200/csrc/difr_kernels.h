@@ -112,6 +112,8 @@ struct FilterParams {
   float temperature, sigma, eps, c1;
   int top_k;    // 0: no top-k
   float top_p;  // 1: no nucleus
+  int nucleus_full;  // the nucleus is taken over the whole vocabulary (its mass from the first pass), resolved
+                     // among the top_k largest logits
   int s;        // competitors in the active subset
   float* bounds;  // [2][T_pad]: on y', on the raw logit
   const Candidate* cand_list;

@@ -10,7 +10,7 @@
 //
 // CTAs run as persistent pairs (a cluster of two, one CTA per SM).  A pair owns a
 // 256 x 256 logit tile: each CTA loads its own 128 rows of h and its own 128 of
-// the tile's 256 rows of W, and one thread of the pair's first CTA issues
+// the tile's 256 rows of W, and one elected lane of the pair's first CTA issues
 // tcgen05.mma.cta_group::2, which reads both CTAs' shared memory and writes rows
 // 0..127 of the accumulator to the first CTA's TMEM and rows 128..255 to the
 // second's.  Per 256 x 256 x 64 step each SM therefore fills 32 KB of shared
@@ -50,7 +50,7 @@ constexpr int kSubsPerTile = (kBN / kColGroups) / kSub;
 constexpr int kRoleRegs = 32, kEpiRegs = 112;  // 32 * 128 + 112 * 512 = 96 * 640 registers
 constexpr int kTmemCols = 512;
 constexpr int kSchedSlots = 2;                 // unit ids handed out ahead of their use
-constexpr int kSchedReaders = 2 + 1 + 2 * kEpiWarps;  // per pair: two TMA threads, the MMA thread, the epilogue warps
+constexpr int kSchedReaders = 2 + 1 + 2 * kEpiWarps;  // per pair, one arrival each: two TMA warps, the MMA warp, the epilogue warps
 constexpr int kBarBytes = 512;
 constexpr int kXchBytes = (kColGroups - 1) * kBM * 32;  // statistics of column groups 1..3 on their way to group 0
 constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + kXchBytes + 1024;  // + slack for 1024-byte alignment
@@ -435,7 +435,7 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     return u;
   };
 
-  // The four single-thread roles need few registers; the rest goes to the epilogue warpgroups.
+  // The four role warps need few registers; the rest goes to the epilogue warpgroups.
   if (warp < kEpiWarp0) {
   setmaxnreg_dec<kRoleRegs>();
   if (warp == 3) {

@@ -79,6 +79,29 @@ __device__ __forceinline__ float warp_nth_largest(float (&v)[8], int n, int lane
   return result;
 }
 
+// Softmax mass of the whole row in units of 2^(c1 * l0), from the first pass's records: sum_v 2^(c1 (l_v - l0)).
+// The same value in every lane.
+__device__ __forceinline__ double row_mass_relative(const FilterParams& p, int row, int lane, double l0) {
+  double lmax = -CUDART_INF, lsum = 0.0;
+  for (int slot = lane; slot < p.n_slots; slot += 32) {
+    const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * (size_t)p.T_pad + row);
+    const float4 b = src[1];
+    const double bm = (double)b.x, bs = (double)b.y;
+    if (bm == -CUDART_INF) continue;
+    if (bm > lmax) { lsum = lsum * exp2(lmax - bm) + bs; lmax = bm; }
+    else lsum += bs * exp2(bm - lmax);
+  }
+  double wmax = lmax;
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) wmax = fmax(wmax, shfl_xor_f64(wmax, m));
+  double part = (lmax == -CUDART_INF) ? 0.0 : lsum * exp2(lmax - wmax);
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) part += shfl_xor_f64(part, m);
+  part = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(part), 0),
+                          __shfl_sync(0xffffffffu, __double2loint(part), 0));
+  return part * exp2(wmax - l0 * (double)p.c1);
+}
+
 __global__ void __launch_bounds__(kFWarps * 32) filter_bounds(const FilterParams p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = blockIdx.x * kFWarps + warp;
@@ -193,12 +216,14 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
       c1s += half;
       const double total = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(c1s), 31),
                                             __shfl_sync(0xffffffffu, __double2loint(c1s), 31));
-      const double need = (double)p.top_p * total;
+      // (a nucleus over the whole vocabulary: the mass it must reach is a share of the whole row's)
+      const double need = (double)p.top_p * (p.nucleus_full ? row_mass_relative(p, row, lane, l0) : total);
       const unsigned m0 = __ballot_sync(0xffffffffu, lane < k_eff && c0 >= need);
       const unsigned m1 = __ballot_sync(0xffffffffu, lane + 32 < k_eff && c1s >= need);
       int last = k_eff - 1;
       if (m0) last = __ffs(m0) - 1;
       else if (m1) last = 32 + __ffs(m1) - 1;
+      else if (p.nucleus_full && k_eff < p.V) status_bits |= 16u;  // the nucleus holds more ids than were resolved
       cut_rank = last;
     }
     // the cutoff is that id's logit: re-evaluated in fp64 like every other logit the score depends on
@@ -300,7 +325,7 @@ __global__ void __launch_bounds__(kFWarps * 32) ipt_filtered_finalize(const Filt
   const Candidate* list = p.cand_list + (size_t)row * (size_t)p.cand_cap;
   const int n_found = p.cand_count[row];
   const int n = n_found < p.cand_cap ? n_found : p.cand_cap;
-  const uint32_t status_bits = (n_found > p.cand_cap) ? 4u : 0u;
+  uint32_t status_bits = (n_found > p.cand_cap) ? 4u : 0u;
   const int k_eff = p.top_k < n ? p.top_k : n;
 
   for (int j = 0; j < n; ++j) {
@@ -342,11 +367,12 @@ __global__ void __launch_bounds__(kFWarps * 32) ipt_filtered_finalize(const Filt
                               __shfl_sync(0xffffffffu, __double2loint(c0), 31));
       const double total = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(c1s), 31),
                                             __shfl_sync(0xffffffffu, __double2loint(c1s), 31));
-      const double need = (double)p.top_p * total;
+      const double need = (double)p.top_p * (p.nucleus_full ? row_mass_relative(p, row, lane, l0) : total);
       const unsigned m0 = __ballot_sync(0xffffffffu, lane < k_eff && c0 >= need);
       const unsigned m1 = __ballot_sync(0xffffffffu, lane + 32 < k_eff && c1s >= need);
       if (m0) last = __ffs(m0) - 1;
       else if (m1) last = 32 + __ffs(m1) - 1;
+      else if (p.nucleus_full && k_eff < p.V) status_bits |= 16u;  // the nucleus holds more ids than were resolved
     }
     cutoff = warp_dot64(p.h + (size_t)row * (size_t)p.d, p.W + (size_t)sm_id[warp][last] * (size_t)p.d, p.d, lane);
     if (tok_ok) {

@@ -87,7 +87,6 @@ def test_bad_arguments_are_refused_on_the_host():
 
     assert filtered(50, 0.95, 0) == INVALID and filtered(50, 0.95, 9) == INVALID   # 1 <= s <= 8
     assert filtered(65, 1.0, 1) == INVALID                                         # top_k <= 64
-    assert filtered(0, 0.9, 1) == INVALID                                          # a nucleus needs a top_k in front
     assert filtered(50, 0.0, 1) == INVALID and filtered(50, 1.5, 1) == INVALID
     assert filtered(50, 0.95, 4, temperature=0.0) == INVALID
     assert filtered(50, 0.95, 4, o=out(temperatures=0x10000)) == INVALID

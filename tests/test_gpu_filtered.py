@@ -179,3 +179,68 @@ def test_ipt_estimator_under_the_filter_matches_the_oracle(T, d, V, scale, tempe
     removed = ok & (k % 5 == 3) & (pt == 0.0)
     assert removed.sum() > 3 and np.allclose(got[removed], math.log(EPS), atol=1e-5)
     assert np.all(out.row_status.cpu().numpy() & 4 == 0)
+
+
+def _nucleus_sizes(h, W, temperature, top_p):
+    """Per row: how many ids the nucleus over the whole vocabulary keeps, and by how much (in mass) the prefix
+    one shorter / the kept prefix misses / passes top_p (the distance of the decision from a tie)."""
+    L = oracle.logits(h, W)
+    sizes, slack = [], []
+    for l in L:
+        z = np.sort(l)[::-1] / temperature
+        c = np.cumsum(np.exp(z - z[0]))
+        c /= c[-1]
+        n = int(np.searchsorted(c, top_p, side="left")) + 1
+        sizes.append(n)
+        near = [abs(c[n - 1] - top_p)] + ([abs(c[n - 2] - top_p)] if n >= 2 else [])
+        if len(c) >= 64:
+            near.append(abs(c[63] - top_p))
+        slack.append(min(near))
+    return np.array(sizes), np.array(slack)
+
+
+@pytest.mark.parametrize("T,d,V,scale,temperature,sigma,top_p,s", [
+    (96, 72, 9000, 5.0, 1.0, 0.3, 0.9, 4),    # peaked rows: most nuclei hold a handful of ids, some more than 64
+    (96, 64, 3000, 3.5, 0.9, 0.1, 0.85, 2),   # every id is a candidate (V < 8192)
+    (40, 64, 40, 2.0, 1.0, 0.4, 0.8, 3),      # the whole vocabulary is resolved: never flagged
+])
+def test_nucleus_over_the_whole_vocabulary(T, d, V, scale, temperature, sigma, top_p, s):
+    """top_k = 0 with top_p < 1: the nucleus takes its mass from the whole row.  Rows whose nucleus fits the 64
+    resolved ids agree with the oracle; the others carry row_status bit 4 and the 64th largest logit as cutoff."""
+    h, W, seeds, positions = _small(T, d, V, 71, scale)
+    tokens = _claims(h, W, seeds, positions, f32(temperature), 72)
+    dev = Device(h, W, seeds, positions)
+    sizes, slack = _nucleus_sizes(h, W, f32(temperature), f32(top_p))
+    clear = slack > 1e-4                      # the kernel's mass comes from fp32 sums: leave near-ties out
+    fits = sizes <= min(64, V)
+    assert fits.sum() >= 10 and (V <= 64 or (~fits).sum() >= 3)
+    L = oracle.logits(h, W)
+    kth = np.sort(L, axis=1)[:, ::-1][:, min(64, V) - 1]
+
+    out = _run(dev, tokens, temperature, sigma, 0, top_p, s)
+    flagged = (out.row_status.cpu().numpy() & 16) != 0
+    assert np.array_equal(flagged[clear], ~fits[clear])
+    want, _, cut = filtered.score_gm_filtered(h, W, tokens, seeds, positions, f32(temperature), f32(sigma), f32(EPS),
+                                              0, f32(top_p), s)
+    got, got_cut = out.score.cpu().numpy(), out.cutoff.cpu().numpy().astype(np.float64)
+    ok = clear & fits
+    np.testing.assert_allclose(got_cut[ok], cut[ok], rtol=0, atol=1e-5)
+    np.testing.assert_allclose(got[ok], want[ok], rtol=0, atol=SCORE_TOL)
+    over = clear & ~fits
+    np.testing.assert_allclose(got_cut[over], kth[over], rtol=0, atol=1e-5)
+
+    # the IPT estimator under the same nucleus
+    o2 = difr.DifrOut.allocate(T, d, V, 0.1, EPS)
+    o2.workspace = torch.empty(difr.difr_filtered_workspace_bytes(T, d, V), dtype=torch.uint8, device="cuda")
+    o2.cutoff = torch.full((T,), float("nan"), dtype=torch.float32, device="cuda")
+    difr.difr_score_ipt_filtered(dev.h, dev.W, to_dev(tokens), dev.seeds, dev.positions, f32(temperature), 0, top_p, o2)
+    torch.cuda.synchronize()
+    assert int(o2.device_status.item()) == 0
+    want2, pt, a, _, cut2 = filtered.score_ipt_filtered(h, W, tokens, seeds, positions, f32(temperature), f32(0.1),
+                                                        f32(EPS), 0, f32(top_p))
+    flagged2 = (o2.row_status.cpu().numpy() & 16) != 0
+    assert np.array_equal(flagged2[clear], ~fits[clear])
+    np.testing.assert_allclose(o2.cutoff.cpu().numpy()[ok], cut2[ok], rtol=0, atol=1e-5)
+    np.testing.assert_allclose(o2.score.cpu().numpy()[ok], want2[ok], rtol=0, atol=SCORE_TOL)
+    np.testing.assert_allclose(o2.p_claimed.cpu().numpy()[ok], pt[ok], rtol=2e-4, atol=1e-9)
+    np.testing.assert_allclose(o2.cdf_lo.cpu().numpy()[ok], a[ok], rtol=2e-4, atol=2e-6)
