@@ -6,14 +6,14 @@
  * it by eye.  It shares no code with the CUDA path and must only be used by
  * the tests, the smoke check and the CPU-baseline leg of the benchmark.
  *
- *   logits          : l[r,v] = sum_k h[r,k] * W[v,k]           (prefill's last op,
- *                     Alg. "Sampled token verification via prefill", line 2)
+ *   logits          : l[r,v] = sum_k h[r,k] * W[v,k]           (the last op of the prefill in
+ *                     Alg. "Sampled token verification via prefill")
  *   randomness      : RO(seed || i) := Philox-4x32-10 (Salmon et al., SC'11),
  *                     key = (seed lo, seed hi), counter = (id>>2, i, tag, 0)
  *   Gumbel noise    : G = -ln(-ln u), u in (0,1)              (Sec. "Gumbel-Max Trick")
  *   Gumbel-max      : argmax_v l_v + Temp * G_v               (Alg. "Gumbel-Max Sampler",
- *                     in the log-probability form of the text; Alg. Token-DiFR line
- *                     "top-s indices as ranked by l_i + T * G_i")
+ *                     in the log-probability form of the text; Alg. Token-DiFR ranks
+ *                     its active subset by the same l_i + T * G_i)
  *   Token-DiFR      : A = l_t* - l_c + Temp (G_t* - G_c), one competitor (s = 1),
  *                     Gaussian noise of std sigma on every logit, no top-k/top-p
  *                     filter: pi = E_x[ Phi((x + A)/sigma) ] = Phi(A / (sigma sqrt 2))

@@ -5,8 +5,8 @@ subset of s competitors -- TEST INFRASTRUCTURE, plain numpy / scipy.
 
 with S the top-s ids by y = l + Temp*G (the claimed token left out),
 A_i = y_t* - y_i, B_i = cutoff - l_i, and `cutoff` the smallest logit that
-survives the sampling filter (the reading of the algorithm's garbled cutoff
-line): keep the top_k largest logits, then, among those, the shortest prefix in
+survives the sampling filter (the reading of the algorithm's garbled definition
+of its cutoff): keep the top_k largest logits, then, among those, the shortest prefix in
 descending order whose renormalised temperature-softmax mass reaches top_p.
 The expectation is evaluated by adaptive quadrature (a library routine) split at
 the kinks of the integrand; the algorithm's own Monte-Carlo loop is in
