@@ -105,8 +105,14 @@ def test_margin_and_argmax_against_a_numpy_replay():
     g = np.random.default_rng(5)
     tokens = g.integers(0, V, size=T).astype(np.int32)
     temperature = 0.9
+    # every other row claims the verifier's own sample, so that both kinds of competitor occur:
+    # the sample for a wrong claim, the runner-up for a right one
+    honest, _ = oracle.sample_gm(h, W, seeds, positions, temperature)
+    tokens[::2] = honest[::2]
     r = oracle.score_gm(h, W, tokens, seeds, positions, temperature, 0.3, EPS)
     logits = _f64(h) @ _f64(W).T
+    assert np.all(r.margin[::2] > 0) and np.array_equal(r.margin[::2], r.top2_margin[::2])
+    assert np.sum(r.margin[1::2] < 0) >= T // 2 - 2
     for i in range(T):
         G = oracle.gumbel_noise_row(int(seeds[i]), int(positions[i]), V)
         y = logits[i] + temperature * G
@@ -117,7 +123,7 @@ def test_margin_and_argmax_against_a_numpy_replay():
         others = np.delete(y, tokens[i])
         assert r.margin[i] == pytest.approx(y[tokens[i]] - others.max(), abs=1e-12)
         assert r.y_claimed[i] == pytest.approx(y[tokens[i]], abs=1e-12)
-        assert r.rank[i] == int(np.sum(logits[i] > logits[i, tokens[i]]))
+        assert r.rank[i] == list(np.argsort(-logits[i], kind="stable")).index(tokens[i])  # no ties in this data
         assert r.score[i] == pytest.approx(
             math.log(ndtr(r.margin[i] / (0.3 * math.sqrt(2))) + EPS), abs=1e-12)
         assert r.lse[i] == pytest.approx(logsumexp(logits[i] / temperature), rel=1e-14)
