@@ -21,6 +21,8 @@
  *
  * Conventions
  *   - Plain C linkage, no exceptions, no global state visible to the caller.
+ *     Host threads may call concurrently (each with its own workspace; see
+ *     difr_score_gm_static for the one exception).
  *   - Every pointer is a DEVICE pointer owned by the caller unless it says
  *     "host"; the caller keeps all buffers alive until `stream` has passed the
  *     call.  The library allocates no device memory and never synchronises

@@ -7,6 +7,8 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <atomic>
+
 #include "../../include/difr.h"
 #include "difr_kernels.h"
 #include "difr_plan.h"
@@ -51,14 +53,14 @@ struct DeviceInfo {
 
 bool device_info(DeviceInfo* info) {
   constexpr int kMaxDevices = 64;
-  static int cached_pairs[kMaxDevices] = {0};  // 0: not asked yet
+  static std::atomic<int> cached_pairs[kMaxDevices];  // 0: not asked yet (threads that race here store the same value)
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return false;
   if (cudaDeviceGetAttribute(&info->major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return false;
   info->pairs = 0;
   if (info->major != 10) return true;
-  if (dev >= 0 && dev < kMaxDevices && cached_pairs[dev] > 0) {
-    info->pairs = cached_pairs[dev];
+  if (dev >= 0 && dev < kMaxDevices && cached_pairs[dev].load(std::memory_order_relaxed) > 0) {
+    info->pairs = cached_pairs[dev].load(std::memory_order_relaxed);
     return true;
   }
   int sms = 0;
@@ -66,7 +68,7 @@ bool device_info(DeviceInfo* info) {
   int pairs = k1_max_resident_pairs();
   if (pairs <= 0) return false;
   if (pairs > sms / 2) pairs = sms / 2;
-  if (dev >= 0 && dev < kMaxDevices) cached_pairs[dev] = pairs;
+  if (dev >= 0 && dev < kMaxDevices) cached_pairs[dev].store(pairs, std::memory_order_relaxed);
   info->pairs = pairs;
   return true;
 }
@@ -292,14 +294,14 @@ static void gauss_legendre(int n, double* x, double* w) {
 
 static difr_status ensure_quadrature_tables() {
   constexpr int kMaxDevices = 64;
-  static bool done[kMaxDevices] = {false};
+  static std::atomic<bool> done[kMaxDevices];  // threads that race here copy the same table
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return DIFR_ERR_CUDA;
-  if (dev >= 0 && dev < kMaxDevices && done[dev]) return DIFR_OK;
+  if (dev >= 0 && dev < kMaxDevices && done[dev].load(std::memory_order_acquire)) return DIFR_OK;
   double x[16], w[16];
   gauss_legendre(16, x, w);
   if (set_gauss_legendre(x, w) != cudaSuccess) return DIFR_ERR_CUDA;
-  if (dev >= 0 && dev < kMaxDevices) done[dev] = true;
+  if (dev >= 0 && dev < kMaxDevices) done[dev].store(true, std::memory_order_release);
   return DIFR_OK;
 }
 

@@ -265,3 +265,29 @@ def test_scores_do_not_depend_on_how_the_vocabulary_is_split(monkeypatch):
         np.testing.assert_allclose(gm["lse"], gm0["lse"], rtol=2e-6)
         np.testing.assert_allclose(ipt["cdf_lo"], ipt0["cdf_lo"], rtol=2e-5, atol=1e-7)
         np.testing.assert_allclose(ipt["score"], ipt0["score"], rtol=0, atol=2e-4)
+
+
+def test_two_calls_in_flight_on_two_streams_keep_to_their_own_workspaces():
+    """Two scoring calls enqueued back to back on different streams, each with its own workspace (its own partial
+    records and work counter), give bit for bit what each gives alone."""
+    a = _small(700, 96, 5000, 41)
+    b = _small(300, 64, 9001, 42)
+    tok_a = _claims(*a, f32(1.0), 43)
+    tok_b = _claims(*b, f32(0.8), 44)
+    dev_a, dev_b = Device(*a), Device(*b)
+    alone_a = dev_a.score("gm", tok_a, 1.0, 0.3)
+    alone_b = dev_b.score("ipt", tok_b, 0.8, 0.1)
+    out_a = difr.DifrOut.allocate(dev_a.T, dev_a.d, dev_a.V, 0.3, EPS)
+    out_b = difr.DifrOut.allocate(dev_b.T, dev_b.d, dev_b.V, 0.1, EPS)
+    ta, tb = to_dev(tok_a), to_dev(tok_b)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for _ in range(3):
+        difr.difr_score_gm(dev_a.h, dev_a.W, ta, dev_a.seeds, dev_a.positions, f32(1.0), out_a, stream=s1)
+        difr.difr_score_ipt(dev_b.h, dev_b.W, tb, dev_b.seeds, dev_b.positions, f32(0.8), out_b, stream=s2)
+    torch.cuda.synchronize()
+    assert int(out_a.device_status.item()) == 0 and int(out_b.device_status.item()) == 0
+    for k in ("score", "margin", "argmax", "runner_up", "lse"):
+        assert np.array_equal(getattr(out_a, k).cpu().numpy(), alone_a[k], equal_nan=True), k
+    for k in ("score", "p_claimed", "cdf_lo", "u", "lse"):
+        assert np.array_equal(getattr(out_b, k).cpu().numpy(), alone_b[k], equal_nan=True), k
