@@ -256,11 +256,12 @@ difr_status difr_admissible(const void* h, const void* W, const uint64_t* seeds,
 // ------------------------------------------------- full Token-DiFR estimator
 constexpr int kCandCap = 256;      // candidates kept per row when the vocabulary has at least 32 tiles
 constexpr int kFilterMinStrips = 32;
+constexpr int kFilterMaxStrips = 128;  // the bounds kernel reads at most 128 strips' records per row
 
 // Layout behind the ordinary workspace: per-row candidate counters, then the candidate lists.
 static bool filtered_layout(int64_t T, int64_t d, int64_t V, int pairs, Plan* pl, int* cap, size_t* count_off,
                             size_t* list_off, size_t* total) {
-  if (!make_plan(T, d, V, pairs, pl, kFilterMinStrips)) return false;
+  if (!make_plan(T, d, V, pairs, pl, kFilterMinStrips, kFilterMaxStrips)) return false;
   // with fewer than 32 vocabulary tiles the strips' maxima cannot bound the top_k-th logit: keep every id
   *cap = (pl->n_tiles < kFilterMinStrips) ? (int)V : kCandCap;
   *count_off = (pl->workspace_bytes + 255) & ~(size_t)255;

@@ -66,8 +66,10 @@ inline double makespan_tiles(int m_tiles, int n_tiles, int S, int gm, int num_pa
 // W tile has to survive in L2 for that long: the strip length `len` and Gm are sized so
 // that the h tiles of a group plus the W tiles in flight stay within a part of L2.
 // `num_pairs` is the number of CTA pairs resident at once (one persistent pair per two SMs).
-// `min_strips` > 0 asks for at least that many strips (fewer only if there are fewer vocabulary tiles).
-inline bool make_plan(int64_t T, int64_t d, int64_t V, int num_pairs, Plan* out, int min_strips = 0) {
+// `min_strips` > 0 asks for at least that many strips (fewer only if there are fewer vocabulary tiles),
+// `max_strips` > 0 for at most that many (the strips grow longer instead).
+inline bool make_plan(int64_t T, int64_t d, int64_t V, int num_pairs, Plan* out, int min_strips = 0,
+                      int max_strips = 0) {
   if (T <= 0 || d <= 0 || V < 2 || (d % 8) != 0) return false;
   if (T > (int64_t)1 << 30 || V >= (int64_t)1 << 31 || d > (int64_t)1 << 20) return false;
   Plan p;
@@ -103,6 +105,7 @@ inline bool make_plan(int64_t T, int64_t d, int64_t V, int num_pairs, Plan* out,
     }
   }
   if (best_S < min_strips) best_S = min_strips;
+  if (max_strips > 0 && best_S > max_strips) best_S = max_strips;
   p.S = env_int("DIFR_DEBUG_STRIPS", best_S);
   if (p.S < 1) p.S = 1;
   if (p.S > p.n_tiles) p.S = p.n_tiles;

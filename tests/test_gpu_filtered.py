@@ -74,6 +74,7 @@ def test_one_competitor_and_no_filter_is_the_plain_estimator():
     (64, 72, 9000, 3.0, 1.0, 0.5, 20, 0.9, 8),      # candidate lists bounded from the first pass (V >= 8192)
     (64, 72, 9000, 1.0, 1.0, 1.0, 0, 1.0, 8),       # no filter, many competitors, flat logits
     (40, 64, 40, 2.0, 1.0, 0.4, 64, 0.8, 3),        # top_k beyond the vocabulary: the nucleus acts on all of it
+    (48, 64, 300000, 3.0, 1.0, 0.3, 50, 0.95, 4),   # more vocabulary tiles than 128 strips of eight: longer strips
 ])
 def test_full_estimator_matches_the_oracle(T, d, V, scale, temperature, sigma, top_k, top_p, s):
     h, W, seeds, positions = _small(T, d, V, 61, scale)
