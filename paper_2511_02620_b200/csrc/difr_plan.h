@@ -112,6 +112,7 @@ inline bool make_plan(int64_t T, int64_t d, int64_t V, int num_pairs, Plan* out,
   gm = env_int("DIFR_DEBUG_GROUP", gm);
   if (gm < 1) gm = 1;
   p.Gm = gm < p.m_tiles ? gm : p.m_tiles;
+  if ((long long)p.m_tiles * p.S > 0x7fffffffLL) return false;  // unit ids are 32-bit
   p.n_units = p.m_tiles * p.S;
   p.T_pad = p.m_tiles * kPairM;
   p.n_slots = p.S;

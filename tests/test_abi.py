@@ -38,6 +38,7 @@ def test_host_only_entry_points():
     assert difr.difr_workspace_bytes(4096, 3076, 128256) == 0  # d not a multiple of 8
     assert difr.difr_workspace_bytes(4096, 3072, 1) == 0
     assert difr.difr_workspace_bytes(0, 3072, 128256) == 0
+    assert difr.difr_workspace_bytes(1 << 30, 64, (1 << 31) - 1) == 0  # more work units than 32-bit ids
     small = difr.difr_workspace_bytes(100, 64, 300)  # 100 rows pad to 256; 300 ids are two tiles: at most two strips
     assert small in (256 + 16 * 256 + 32 * 256 * s for s in (1, 2))
 
