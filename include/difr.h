@@ -56,7 +56,7 @@ typedef struct CUstream_st* difr_stream_t; /* a cudaStream_t */
 typedef enum {
   DIFR_OK = 0,
   DIFR_ERR_INVALID_ARG = -1, /* null required pointer, non-positive size, bad scalar  */
-  DIFR_ERR_SHAPE = -2,       /* d not a multiple of 8, V < 2, sizes beyond 2^31 rows  */
+  DIFR_ERR_SHAPE = -2,       /* d not a multiple of 8, V < 2, T > 2^30, d > 2^20 ...  */
   DIFR_ERR_ALIGN = -3,       /* h, W or workspace not 16-byte aligned                 */
   DIFR_ERR_WORKSPACE = -4,   /* workspace missing or smaller than difr_workspace_bytes */
   DIFR_ERR_CUDA = -5,        /* a CUDA runtime/driver call failed                     */
@@ -143,7 +143,7 @@ size_t difr_workspace_bytes(int64_t T, int64_t d, int64_t V);
  *   tokens     int32 [T] claimed ids (any value; out of range => maximally suspicious)
  *   seeds      uint64 [T], positions uint32 [T]: RO(seed || i) per row
  *   temperature  >= 0 (0: greedy replay, y = l)
- *   T >= 0, d > 0 with d % 8 == 0, 2 <= V < 2^31
+ *   0 <= T <= 2^30, 0 < d <= 2^20 with d % 8 == 0, 2 <= V <= 2^31 - 1024
  * Errors: see difr_status.  T == 0 returns DIFR_OK without launching.
  */
 difr_status difr_score_gm(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,

@@ -71,7 +71,8 @@ inline double makespan_tiles(int m_tiles, int n_tiles, int S, int gm, int num_pa
 inline bool make_plan(int64_t T, int64_t d, int64_t V, int num_pairs, Plan* out, int min_strips = 0,
                       int max_strips = 0) {
   if (T <= 0 || d <= 0 || V < 2 || (d % 8) != 0) return false;
-  if (T > (int64_t)1 << 30 || V >= (int64_t)1 << 31 || d > (int64_t)1 << 20) return false;
+  // (tile origins n * 256 and row origins m * 256 are 32-bit in the kernels: leave room for the last tile's padding)
+  if (T > (int64_t)1 << 30 || V > ((int64_t)1 << 31) - 1024 || d > (int64_t)1 << 20) return false;
   Plan p;
   p.m_tiles = (int)((T + kPairM - 1) / kPairM);
   p.n_tiles = (int)((V + kBN - 1) / kBN);
