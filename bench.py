@@ -377,6 +377,23 @@ def run_ours(args):
 
     elapsed_ms, e2e_ms, fused_avg_ms = reduce_max([elapsed_ms, e2e_ms, fused_avg_ms], device="cuda")
 
+    # ---- the other estimator on the same resident inputs (context; the headline is Token-DiFR)
+    ipt_ms = None
+    if world == 1 and temperature > 0:
+        n_ipt = max(1, min(args.steps, 10))
+        for _ in range(2):
+            difr.difr_score_ipt(h_dev, W_dev, tokens_dev, seeds_dev, pos_dev, temperature, out)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(n_ipt):
+            difr.difr_score_ipt(h_dev, W_dev, tokens_dev, seeds_dev, pos_dev, temperature, out)
+            difr.difr_detect(out.score, tau, None, None, 0, seq_dev, flags, stats)
+        b.record()
+        torch.cuda.synchronize()
+        ipt_ms = a.elapsed_time(b) / n_ipt
+        assert int(out.device_status.item()) == 0, "device-side wait timed out"
+
     if rank == 0:
         peaks = load_peaks()
         flop = 2.0 * T * d * V
@@ -403,6 +420,10 @@ def run_ours(args):
             "detect": {"threshold": tau, "n_flagged": n_flagged, "n_tampered": int(tampered.sum()),
                        "n_match": int(stats_np[:, 1].sum())},
         }
+        if ipt_ms is not None:
+            line["token_ipt_difr"] = {"value": T / (ipt_ms * 1e-3), "unit": UNIT, "ms_per_step": ipt_ms,
+                                      "tflops": flop / (ipt_ms * 1e-3) / 1e12,
+                                      "note": "difr_score_ipt + difr_detect, resident inputs, sigma in CDF units"}
         if args.variants:
             line["variants_ms"] = time_variants(difr, h_dev, W_dev, tokens_dev, seeds_dev, pos_dev, temperature, sigma,
                                                 T, d, V)
