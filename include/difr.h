@@ -92,7 +92,7 @@ typedef struct {
   float* u;           /* IPT: the uniform mu of this row                           */
   uint32_t* row_status; /* bit0: claimed id outside [0, V); bit1: non-finite logits;
                            bit2: candidate list overflow (difr_score_gm_filtered);
-                           bit3: unusable per-row temperature; bit4: the nucleus holds more
+                           bit3: unusable per-row temperature or filter values; bit4: the nucleus holds more
                            ids than the filtered calls resolve (64)                        */
   void* workspace;      /* >= difr_workspace_bytes(T, d, V) bytes, 16-byte aligned;
                            contents are scratch, overwritten by every call         */
@@ -118,7 +118,7 @@ typedef struct {
                         row (requests with their own sampling parameters in one batch); when given, the
                         `temperature` argument is ignored.  A row whose value is negative, not finite, or
                         zero where the IPT score is asked for gets a NaN score and row_status bit 3.
-                        Must be NULL for difr_score_gm_filtered.                                */
+                        The filtered calls take it too (there a row needs a temperature > 0).       */
 } difr_out;
 
 /* Scratch bytes a scoring call needs for T rows, hidden size d, vocabulary V.
@@ -228,6 +228,9 @@ difr_status difr_score_both(const void* h, const void* W, const int32_t* tokens,
  *                  less than that gets row_status bit 4 and the 64th largest logit as cutoff
  *   filter->s      1..8
  *   temperature > 0
+ *   Requests with their own sampling parameters in one batch: filter->top_k_rows, filter->top_p_rows
+ *   and out->temperatures give one value per row; a row whose values are outside the ranges above
+ *   gets a NaN score and row_status bit 3 (the scalars are checked on the host, DIFR_ERR_INVALID_ARG).
  *   out->workspace needs difr_filtered_workspace_bytes(T, d, V) bytes
  *
  * Everything difr_score_gm writes is written as there (margin, argmax, runner_up,
@@ -246,6 +249,9 @@ typedef struct {
   int32_t top_k;
   float top_p;
   int32_t s;
+  /* -- members added in version 210; zero them when unused -- */
+  const int32_t* top_k_rows; /* device [T], optional: one top_k per row (top_k is then ignored)            */
+  const float* top_p_rows;   /* device [T], optional: one top_p per row (top_p is then ignored)            */
 } difr_filter;
 size_t difr_filtered_workspace_bytes(int64_t T, int64_t d, int64_t V);
 difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,
@@ -264,7 +270,8 @@ difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* 
  *
  *   filter->top_k 1..64 (or >= V when V <= 64), or 0 with top_p < 1: a nucleus over the whole
  *   vocabulary as in difr_score_gm_filtered (row_status bit 4 when it holds more than 64 ids);
- *   filter->top_p in (0, 1]; filter->s is ignored
+ *   filter->top_p in (0, 1]; filter->s is ignored; per-row values as in difr_score_gm_filtered (a
+ *   row whose own policy filters nothing keeps the unfiltered score)
  *   temperature > 0; out->workspace needs difr_filtered_workspace_bytes(T, d, V)
  * Writes score, p_claimed, cdf_lo, u, row_status, out->cutoff (optional) and
  * lse (of the unfiltered logits).  Two passes over the logits, the second

@@ -46,7 +46,8 @@ class _COut(ctypes.Structure):
 
 
 class _CFilter(ctypes.Structure):
-    _fields_ = [("top_k", ctypes.c_int32), ("top_p", ctypes.c_float), ("s", ctypes.c_int32)]
+    _fields_ = [("top_k", ctypes.c_int32), ("top_p", ctypes.c_float), ("s", ctypes.c_int32),
+                ("top_k_rows", ctypes.c_void_p), ("top_p_rows", ctypes.c_void_p)]
 
 
 _lib = None
@@ -229,7 +230,8 @@ def difr_score_ipt_filtered(h, W, tokens, seeds, positions, temperature, top_k, 
 def difr_score_gm_filtered(h, W, tokens, seeds, positions, temperature, top_k, top_p, s, out: DifrOut, stream=None,
                            _fn="difr_score_gm_filtered"):
     """Alg. Token-DiFR in full: top-k / top-p cutoff, B_i terms, s competitors; `out.workspace` must hold
-    difr_filtered_workspace_bytes(T, d, V) bytes.  See include/difr.h."""
+    difr_filtered_workspace_bytes(T, d, V) bytes.  `top_k` (int32) and `top_p` (float32) may be device tensors
+    of T values, one per row, and `out.temperatures` one temperature per row.  See include/difr.h."""
     import torch
 
     T, d = h.shape
@@ -240,7 +242,14 @@ def difr_score_gm_filtered(h, W, tokens, seeds, positions, temperature, top_k, t
     _check(seeds, torch.int64, (T,), "seeds")
     _check(positions, torch.int32, (T,), "positions")
     c = out._c()
-    f = _CFilter(int(top_k), float(top_p), int(s))
+    k_rows = top_k if isinstance(top_k, torch.Tensor) else None
+    p_rows = top_p if isinstance(top_p, torch.Tensor) else None
+    if k_rows is not None:
+        _check(k_rows, torch.int32, (T,), "top_k")
+    if p_rows is not None:
+        _check(p_rows, torch.float32, (T,), "top_p")
+    f = _CFilter(0 if k_rows is not None else int(top_k), 1.0 if p_rows is not None else float(top_p), int(s),
+                 _ptr(k_rows), _ptr(p_rows))
     rc = getattr(lib(), _fn)(_ptr(h), _ptr(W), _ptr(tokens), _ptr(seeds), _ptr(positions),
                              float(temperature), T, d, V, ctypes.byref(f), ctypes.byref(c), _stream(stream))
     if rc != DIFR_OK:

@@ -323,17 +323,15 @@ difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* 
   if (T < 0 || d <= 0 || V <= 0) return DIFR_ERR_INVALID_ARG;
   if (!(out->sigma > 0.f) || !(out->eps >= 0.f) || !isfinite(out->sigma) || !isfinite(out->eps))
     return DIFR_ERR_INVALID_ARG;
-  if (!(temperature > 0.f) || !isfinite(temperature) || out->temperatures != nullptr) return DIFR_ERR_INVALID_ARG;
-  int top_k = filter->top_k;
+  // scalars are checked here when they apply to every row; values that come one per row are checked on the
+  // device (row_status bit 3).  How top_k and top_p combine is decided per row by the kernels.
+  if (out->temperatures == nullptr && (!(temperature > 0.f) || !isfinite(temperature))) return DIFR_ERR_INVALID_ARG;
+  if (out->temperatures != nullptr) temperature = 1.f;  // unused
+  const int top_k = filter->top_k;
   const float top_p = filter->top_p;
-  if (top_k < 0 || !(top_p > 0.f) || !(top_p <= 1.f) || filter->s < 1 || filter->s > 8) return DIFR_ERR_INVALID_ARG;
-  if (top_k >= V && top_p >= 1.f) top_k = 0;  // keeps the whole vocabulary: no filter
-  if (top_k > 64 && top_k < V) return DIFR_ERR_INVALID_ARG;
-  // a nucleus with no top-k in front of it (or one that keeps everything) is taken over the whole
-  // vocabulary's mass and resolved among the 64 largest logits
-  const int nucleus_full = (top_p < 1.f && (top_k < 1 || top_k >= V)) ? 1 : 0;
-  if (nucleus_full) top_k = 64;
-  if (top_k > V) top_k = (int)V;
+  if (filter->s < 1 || filter->s > 8) return DIFR_ERR_INVALID_ARG;
+  if (filter->top_k_rows == nullptr && (top_k < 0 || (top_k > 64 && top_k < V))) return DIFR_ERR_INVALID_ARG;
+  if (filter->top_p_rows == nullptr && (!(top_p > 0.f) || !(top_p <= 1.f))) return DIFR_ERR_INVALID_ARG;
   if ((d % 8) != 0 || V < 2) return DIFR_ERR_SHAPE;
   if (T == 0) return DIFR_OK;
   DeviceInfo info;
@@ -358,6 +356,7 @@ difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* 
   K1Params k1 = k1_params(pl, T, d, V, temperature, ws);
   k1.tokens = tokens; k1.seeds = seeds; k1.positions = positions;
   k1.device_status = out->device_status;
+  k1.temperatures = out->temperatures;
   if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
   if (launch_k1(6, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;
 
@@ -370,6 +369,7 @@ difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* 
   k2.temperature = temperature; k2.sigma = out->sigma; k2.eps = out->eps; k2.c1 = k1.c1;
   k2.score = out->score; k2.margin = out->margin; k2.argmax = out->argmax; k2.runner_up = out->runner_up;
   k2.lse = out->lse; k2.row_status = out->row_status; k2.y_max = out->y_max; k2.y_second = out->y_second;
+  k2.temperatures = out->temperatures;
   if (launch_k2(k2, s) != cudaSuccess) return DIFR_ERR_CUDA;
 
   // ---- bounds, collecting pass, finalize
@@ -378,7 +378,8 @@ difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* 
   fp.h = k2.h; fp.W = k2.W; fp.tokens = tokens; fp.seeds = seeds; fp.positions = positions;
   fp.partials = k1.partials; fp.n_slots = pl.n_slots; fp.T_pad = pl.T_pad; fp.T = (int)T; fp.d = (int)d; fp.V = (int)V;
   fp.temperature = temperature; fp.sigma = out->sigma; fp.eps = out->eps; fp.c1 = k1.c1;
-  fp.top_k = top_k; fp.top_p = top_p; fp.s = filter->s; fp.nucleus_full = nucleus_full;
+  fp.top_k = top_k; fp.top_p = top_p; fp.s = filter->s; fp.ipt = 0;
+  fp.top_k_rows = filter->top_k_rows; fp.top_p_rows = filter->top_p_rows; fp.temperatures = out->temperatures;
   fp.bounds = reinterpret_cast<float*>(ws + pl.bounds_offset);
   fp.cand_list = reinterpret_cast<const Candidate*>(ws + list_off);
   fp.cand_count = reinterpret_cast<const int*>(ws + count_off);
@@ -404,17 +405,16 @@ difr_status difr_score_ipt_filtered(const void* h, const void* W, const int32_t*
   if (T < 0 || d <= 0 || V <= 0) return DIFR_ERR_INVALID_ARG;
   if (!(out->sigma > 0.f) || !(out->eps >= 0.f) || !isfinite(out->sigma) || !isfinite(out->eps))
     return DIFR_ERR_INVALID_ARG;
-  if (!(temperature > 0.f) || !isfinite(temperature) || out->temperatures != nullptr) return DIFR_ERR_INVALID_ARG;
-  int top_k = filter->top_k;
+  if (out->temperatures == nullptr && (!(temperature > 0.f) || !isfinite(temperature))) return DIFR_ERR_INVALID_ARG;
+  if (out->temperatures != nullptr) temperature = 1.f;  // unused
+  const int top_k = filter->top_k;
   const float top_p = filter->top_p;
-  if (top_k < 0 || !(top_p > 0.f) || !(top_p <= 1.f)) return DIFR_ERR_INVALID_ARG;
-  if (top_k > V) top_k = (int)V;
-  if ((top_k < 1 || top_k >= V) && top_p >= 1.f && V > 64) return DIFR_ERR_INVALID_ARG;  // no filter: difr_score_ipt
-  if (top_k > 64 && top_k < V) return DIFR_ERR_INVALID_ARG;
-  // a nucleus with no top-k in front of it: over the whole vocabulary's mass, resolved among the 64 largest logits
-  const int nucleus_full = (top_p < 1.f && (top_k < 1 || top_k >= V)) ? 1 : 0;
-  if (nucleus_full || top_k < 1) top_k = V < 64 ? (int)V : 64;
-  if (top_k > 64) return DIFR_ERR_INVALID_ARG;  // the kept set is held in 64 slots
+  if (filter->top_k_rows == nullptr && (top_k < 0 || (top_k > 64 && top_k < V))) return DIFR_ERR_INVALID_ARG;
+  if (filter->top_p_rows == nullptr && (!(top_p > 0.f) || !(top_p <= 1.f))) return DIFR_ERR_INVALID_ARG;
+  // one policy for every row and it filters nothing: that is difr_score_ipt
+  if (filter->top_k_rows == nullptr && filter->top_p_rows == nullptr && (top_k < 1 || top_k >= V) && top_p >= 1.f &&
+      V > 64)
+    return DIFR_ERR_INVALID_ARG;
   if ((d % 8) != 0 || V < 2) return DIFR_ERR_SHAPE;
   if (T == 0) return DIFR_OK;
   DeviceInfo info;
@@ -437,6 +437,7 @@ difr_status difr_score_ipt_filtered(const void* h, const void* W, const int32_t*
   K1Params k1 = k1_params(pl, T, d, V, temperature, ws);
   k1.tokens = tokens; k1.seeds = seeds; k1.positions = positions;
   k1.device_status = out->device_status;
+  k1.temperatures = out->temperatures;
   if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
   if (launch_k1(8, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;
 
@@ -449,6 +450,7 @@ difr_status difr_score_ipt_filtered(const void* h, const void* W, const int32_t*
   k2.temperature = temperature; k2.sigma = out->sigma; k2.eps = out->eps; k2.c1 = k1.c1;
   k2.score = out->score; k2.lse = out->lse; k2.p_claimed = out->p_claimed; k2.cdf_lo = out->cdf_lo; k2.u = out->u;
   k2.row_status = out->row_status;
+  k2.temperatures = out->temperatures;
   if (launch_k2(k2, s) != cudaSuccess) return DIFR_ERR_CUDA;
 
   // ---- bound on the top_k-th logit, collecting pass by logit, finalize over the kept ids
@@ -457,7 +459,8 @@ difr_status difr_score_ipt_filtered(const void* h, const void* W, const int32_t*
   fp.h = k2.h; fp.W = k2.W; fp.tokens = tokens; fp.seeds = seeds; fp.positions = positions;
   fp.partials = k1.partials; fp.n_slots = pl.n_slots; fp.T_pad = pl.T_pad; fp.T = (int)T; fp.d = (int)d; fp.V = (int)V;
   fp.temperature = temperature; fp.sigma = out->sigma; fp.eps = out->eps; fp.c1 = k1.c1;
-  fp.top_k = top_k; fp.top_p = top_p; fp.s = 0; fp.nucleus_full = nucleus_full;
+  fp.top_k = top_k; fp.top_p = top_p; fp.s = 0; fp.ipt = 1;
+  fp.top_k_rows = filter->top_k_rows; fp.top_p_rows = filter->top_p_rows; fp.temperatures = out->temperatures;
   fp.bounds = reinterpret_cast<float*>(ws + pl.bounds_offset);
   fp.cand_list = reinterpret_cast<const Candidate*>(ws + list_off);
   fp.cand_count = reinterpret_cast<const int*>(ws + count_off);
@@ -609,6 +612,6 @@ const char* difr_status_string(difr_status status) {
   return "unknown status";
 }
 
-int difr_version(void) { return 200; }
+int difr_version(void) { return 210; }
 
 }  // extern "C"

@@ -110,10 +110,12 @@ struct FilterParams {
   const Partial* partials;  // records of the first pass (mode GmFilter)
   int n_slots, T_pad, T, d, V;
   float temperature, sigma, eps, c1;
-  int top_k;    // 0: no top-k
-  float top_p;  // 1: no nucleus
-  int nucleus_full;  // the nucleus is taken over the whole vocabulary (its mass from the first pass), resolved
-                     // among the top_k largest logits
+  int top_k;    // as the caller gave it (0 or >= V: no top-k); one per row in top_k_rows when that is given
+  float top_p;  // 1: no nucleus; one per row in top_p_rows when that is given
+  const int32_t* top_k_rows;   // nullable
+  const float* top_p_rows;     // nullable
+  const float* temperatures;   // nullable: one temperature per row (then `temperature` and `c1` are unused)
+  int ipt;      // the IPT estimator's finalize: a row without any filter keeps the first pass's outputs
   int s;        // competitors in the active subset
   float* bounds;  // [2][T_pad]: on y', on the raw logit
   const Candidate* cand_list;

@@ -79,9 +79,37 @@ __device__ __forceinline__ float warp_nth_largest(float (&v)[8], int n, int lane
   return result;
 }
 
+// The sampling policy of one row, normalised: the call's scalars or the row's own values.
+struct RowPolicy {
+  float temperature, c1, top_p;
+  int top_k;         // ids resolved by logit rank: the top-k, or kMaxK for a nucleus over the whole vocabulary; 0: none
+  int nucleus_full;  // the nucleus takes its mass from the whole row (no top-k in front of it)
+  bool none;         // no filter at all
+  bool bad;          // unusable values: the row's score is NaN and row_status bit 3 is set
+};
+
+__device__ __forceinline__ RowPolicy row_policy(const FilterParams& p, int row) {
+  RowPolicy r;
+  r.temperature = p.temperatures != nullptr ? p.temperatures[row] : p.temperature;
+  r.c1 = p.temperatures != nullptr ? (r.temperature > 0.f ? 1.4426950408889634f / r.temperature : 0.f) : p.c1;
+  int k = p.top_k_rows != nullptr ? p.top_k_rows[row] : p.top_k;
+  r.top_p = p.top_p_rows != nullptr ? p.top_p_rows[row] : p.top_p;
+  r.bad = !(r.temperature > 0.f) || isinf(r.temperature) || k < 0 || !(r.top_p > 0.f) || !(r.top_p <= 1.f);
+  if (k > p.V) k = p.V;
+  if (k > kMaxK && k < p.V) r.bad = true;
+  const bool whole = k < 1 || k >= p.V;  // no top-k in effect
+  r.nucleus_full = (whole && r.top_p < 1.f) ? 1 : 0;
+  r.none = whole && !(r.top_p < 1.f);
+  if (r.nucleus_full) k = kMaxK < p.V ? kMaxK : p.V;
+  else if (whole) k = (p.ipt && p.V <= kMaxK) ? p.V : 0;
+  if (r.bad) { k = 0; r.nucleus_full = 0; r.none = false; }
+  r.top_k = k;
+  return r;
+}
+
 // Softmax mass of the whole row in units of 2^(c1 * l0), from the first pass's records: sum_v 2^(c1 (l_v - l0)).
 // The same value in every lane.
-__device__ __forceinline__ double row_mass_relative(const FilterParams& p, int row, int lane, double l0) {
+__device__ __forceinline__ double row_mass_relative(const FilterParams& p, int row, int lane, double l0, double c1) {
   double lmax = -CUDART_INF, lsum = 0.0;
   for (int slot = lane; slot < p.n_slots; slot += 32) {
     const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * (size_t)p.T_pad + row);
@@ -99,13 +127,14 @@ __device__ __forceinline__ double row_mass_relative(const FilterParams& p, int r
   for (int m = 16; m >= 1; m >>= 1) part += shfl_xor_f64(part, m);
   part = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(part), 0),
                           __shfl_sync(0xffffffffu, __double2loint(part), 0));
-  return part * exp2(wmax - l0 * (double)p.c1);
+  return part * exp2(wmax - l0 * c1);
 }
 
 __global__ void __launch_bounds__(kFWarps * 32) filter_bounds(const FilterParams p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = blockIdx.x * kFWarps + warp;
   if (row >= p.T) return;
+  const RowPolicy rp = row_policy(p, row);
   // up to 128 strips: four records per lane, two values of each kind per record
   float yk[8], zk[8];
 #pragma unroll
@@ -132,17 +161,18 @@ __global__ void __launch_bounds__(kFWarps * 32) filter_bounds(const FilterParams
       const float ky = warp_nth_largest(yk, p.s + 3, lane);
       if (ky > -CUDART_INF_F) by = ky - 1e-4f * fmaxf(1.f, fabsf(ky));
     }
-    if (p.top_k > 0) {
-      const float kz = warp_nth_largest(zk, p.top_k, lane);
+    if (rp.top_k > 0) {
+      const float kz = warp_nth_largest(zk, rp.top_k, lane);
       bl = -CUDART_INF_F;
       if (kz > -CUDART_INF_F) {
-        const float l = kz / p.c1;
+        const float l = kz / rp.c1;
         bl = l - 1e-5f * fmaxf(1.f, fabsf(l));
       }
     }
-  } else if (p.top_k > 0) {
+  } else if (rp.top_k > 0) {
     bl = -CUDART_INF_F;
   }
+  if (rp.bad) { by = CUDART_INF_F; bl = CUDART_INF_F; }  // nothing is collected for a row that cannot be scored
   if (lane == 0) {
     p.bounds[row] = by;
     p.bounds[(size_t)p.T_pad + row] = bl;
@@ -162,8 +192,17 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
   const int n_found = p.cand_count[row];
   const int n = n_found < p.cand_cap ? n_found : p.cand_cap;
   uint32_t status_bits = (n_found > p.cand_cap) ? 4u : 0u;
+  const RowPolicy rp = row_policy(p, row);
+  if (rp.bad) {
+    if (lane == 0) {
+      p.score[row] = CUDART_NAN_F;
+      if (p.cutoff) p.cutoff[row] = CUDART_NAN_F;
+      if (p.row_status) p.row_status[row] |= 8u;
+    }
+    return;
+  }
 
-  const int k_eff = (p.top_k > 0) ? (p.top_k < n ? p.top_k : n) : 0;
+  const int k_eff = (rp.top_k > 0) ? (rp.top_k < n ? rp.top_k : n) : 0;
   int n_others = 0;  // entries that are not the claimed token
   for (int i = lane; i < n; i += 32) n_others += (list[i].id != tok) ? 1 : 0;
 #pragma unroll
@@ -195,10 +234,10 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
   __syncwarp();
   if (k_eff > 0) {
     cut_rank = k_eff - 1;  // the top_k-th largest logit
-    if (p.top_p < 1.f) {
+    if (rp.top_p < 1.f) {
       // nucleus inside the top k: shortest prefix (descending) whose renormalised softmax mass reaches top_p
       double e0 = 0.0, e1 = 0.0;
-      const double c1 = (double)p.c1, l0 = (double)sm_l[warp][0];
+      const double c1 = (double)rp.c1, l0 = (double)sm_l[warp][0];
       if (lane < k_eff) e0 = exp2(((double)sm_l[warp][lane] - l0) * c1);
       if (lane + 32 < k_eff) e1 = exp2(((double)sm_l[warp][lane + 32] - l0) * c1);
       double c0 = e0, c1s = e1;  // inclusive scans of both halves
@@ -217,13 +256,13 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
       const double total = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(c1s), 31),
                                             __shfl_sync(0xffffffffu, __double2loint(c1s), 31));
       // (a nucleus over the whole vocabulary: the mass it must reach is a share of the whole row's)
-      const double need = (double)p.top_p * (p.nucleus_full ? row_mass_relative(p, row, lane, l0) : total);
+      const double need = (double)rp.top_p * (rp.nucleus_full ? row_mass_relative(p, row, lane, l0, c1) : total);
       const unsigned m0 = __ballot_sync(0xffffffffu, lane < k_eff && c0 >= need);
       const unsigned m1 = __ballot_sync(0xffffffffu, lane + 32 < k_eff && c1s >= need);
       int last = k_eff - 1;
       if (m0) last = __ffs(m0) - 1;
       else if (m1) last = 32 + __ffs(m1) - 1;
-      else if (p.nucleus_full && k_eff < p.V) status_bits |= 16u;  // the nucleus holds more ids than were resolved
+      else if (rp.nucleus_full && k_eff < p.V) status_bits |= 16u;  // the nucleus holds more ids than were resolved
       cut_rank = last;
     }
     // the cutoff is that id's logit: re-evaluated in fp64 like every other logit the score depends on
@@ -235,7 +274,7 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
     const uint64_t seed = p.seeds[row];
     const uint32_t pos = p.positions[row];
     const uint16_t* hrow = p.h + (size_t)row * (size_t)p.d;
-    const double temp = (double)p.temperature, sigma = (double)p.sigma;
+    const double temp = (double)rp.temperature, sigma = (double)p.sigma;
     const double l_t = warp_dot64(hrow, p.W + (size_t)tok * (size_t)p.d, p.d, lane);
     const double y_t = l_t + temp * gumbel_f64(seed, pos, (uint32_t)tok);
     // exact logits and noisy logits of the s + 2 candidates; then the s best of them
@@ -326,7 +365,20 @@ __global__ void __launch_bounds__(kFWarps * 32) ipt_filtered_finalize(const Filt
   const int n_found = p.cand_count[row];
   const int n = n_found < p.cand_cap ? n_found : p.cand_cap;
   uint32_t status_bits = (n_found > p.cand_cap) ? 4u : 0u;
-  const int k_eff = p.top_k < n ? p.top_k : n;
+  const RowPolicy rp = row_policy(p, row);
+  if (rp.bad || (rp.none && rp.top_k == 0)) {
+    // unusable values: NaN; no filter at all (and a vocabulary too large to resolve here): the first pass's
+    // finalize has already written the unfiltered score
+    if (lane == 0) {
+      if (rp.bad) {
+        p.score[row] = CUDART_NAN_F;
+        if (p.row_status) p.row_status[row] |= 8u;
+      }
+      if (p.cutoff) p.cutoff[row] = rp.bad ? CUDART_NAN_F : -CUDART_INF_F;
+    }
+    return;
+  }
+  const int k_eff = rp.top_k < n ? rp.top_k : n;
 
   for (int j = 0; j < n; ++j) {
     const Candidate cj = list[j];
@@ -348,12 +400,12 @@ __global__ void __launch_bounds__(kFWarps * 32) ipt_filtered_finalize(const Filt
   const double mu = ((double)x[0] + 0.5) * (1.0 / 4294967296.0);
   double score = log((double)p.eps), pt = CUDART_NAN, a = CUDART_NAN, cutoff = -CUDART_INF;
   if (k_eff > 0) {
-    const double c1 = (double)p.c1, l0 = (double)sm_l[warp][0];
+    const double c1 = (double)rp.c1, l0 = (double)sm_l[warp][0];
     double e0 = 0.0, e1 = 0.0;  // unnormalised masses of ranks lane and lane + 32
     if (lane < k_eff) e0 = exp2(((double)sm_l[warp][lane] - l0) * c1);
     if (lane + 32 < k_eff) e1 = exp2(((double)sm_l[warp][lane + 32] - l0) * c1);
     int last = k_eff - 1;
-    if (p.top_p < 1.f) {
+    if (rp.top_p < 1.f) {
       double c0 = e0, c1s = e1;
 #pragma unroll
       for (int m = 1; m < 32; m <<= 1) {
@@ -367,12 +419,12 @@ __global__ void __launch_bounds__(kFWarps * 32) ipt_filtered_finalize(const Filt
                               __shfl_sync(0xffffffffu, __double2loint(c0), 31));
       const double total = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(c1s), 31),
                                             __shfl_sync(0xffffffffu, __double2loint(c1s), 31));
-      const double need = (double)p.top_p * (p.nucleus_full ? row_mass_relative(p, row, lane, l0) : total);
+      const double need = (double)rp.top_p * (rp.nucleus_full ? row_mass_relative(p, row, lane, l0, c1) : total);
       const unsigned m0 = __ballot_sync(0xffffffffu, lane < k_eff && c0 >= need);
       const unsigned m1 = __ballot_sync(0xffffffffu, lane + 32 < k_eff && c1s >= need);
       if (m0) last = __ffs(m0) - 1;
       else if (m1) last = 32 + __ffs(m1) - 1;
-      else if (p.nucleus_full && k_eff < p.V) status_bits |= 16u;  // the nucleus holds more ids than were resolved
+      else if (rp.nucleus_full && k_eff < p.V) status_bits |= 16u;  // the nucleus holds more ids than were resolved
     }
     cutoff = warp_dot64(p.h + (size_t)row * (size_t)p.d, p.W + (size_t)sm_id[warp][last] * (size_t)p.d, p.d, lane);
     if (tok_ok) {

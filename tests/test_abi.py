@@ -90,7 +90,9 @@ def test_bad_arguments_are_refused_on_the_host():
     assert filtered(65, 1.0, 1) == INVALID                                         # top_k <= 64
     assert filtered(50, 0.0, 1) == INVALID and filtered(50, 1.5, 1) == INVALID
     assert filtered(50, 0.95, 4, temperature=0.0) == INVALID
-    assert filtered(50, 0.95, 4, o=out(temperatures=0x10000)) == INVALID
+    assert filtered(-1, 0.95, 4) == INVALID
+    f_rows = difr._CFilter(50, 0.95, 9, 0x10000, 0x10000)  # per-row values do not excuse a bad s
+    assert L.difr_score_gm_filtered(p, p, p, p, p, 1.0, 128, 64, 1000, ctypes.byref(f_rows), ctypes.byref(out()), None) == INVALID
 
     f0 = difr._CFilter(0, 1.0, 1)
     o = out()

@@ -245,3 +245,52 @@ def test_nucleus_over_the_whole_vocabulary(T, d, V, scale, temperature, sigma, t
     np.testing.assert_allclose(o2.score.cpu().numpy()[ok], want2[ok], rtol=0, atol=SCORE_TOL)
     np.testing.assert_allclose(o2.p_claimed.cpu().numpy()[ok], pt[ok], rtol=2e-4, atol=1e-9)
     np.testing.assert_allclose(o2.cdf_lo.cpu().numpy()[ok], a[ok], rtol=2e-4, atol=2e-6)
+
+
+def test_one_sampling_policy_per_row():
+    """Requests with their own temperature, top_k and top_p in one batch: every row equals, bit for bit, the row
+    of a call that applies its policy to the whole batch; rows with unusable values are NaN and carry bit 3."""
+    T, d, V, s, sigma = 96, 72, 9000, 3, 0.3
+    h, W, seeds, positions = _small(T, d, V, 81, 4.0)
+    tokens = _claims(h, W, seeds, positions, f32(1.0), 82)
+    dev = Device(h, W, seeds, positions)
+    policies = [(1.0, 50, 0.95), (0.7, 8, 1.0), (1.3, 0, 0.9), (1.0, 0, 1.0), (0.0, 50, 0.95), (1.0, 70, 0.9),
+                (1.0, 20, 1.5)]
+    valid = [0, 1, 2, 3]
+    group = np.arange(T) % len(policies)
+    temps = torch.tensor([policies[g][0] for g in group], dtype=torch.float32, device="cuda")
+    ks = torch.tensor([policies[g][1] for g in group], dtype=torch.int32, device="cuda")
+    ps = torch.tensor([policies[g][2] for g in group], dtype=torch.float32, device="cuda")
+    tok_dev = to_dev(tokens)
+
+    def fresh():
+        out = difr.DifrOut.allocate(T, d, V, sigma, EPS)
+        out.workspace = torch.empty(difr.difr_filtered_workspace_bytes(T, d, V), dtype=torch.uint8, device="cuda")
+        out.cutoff = torch.full((T,), float("nan"), dtype=torch.float32, device="cuda")
+        return out
+
+    for fn, extra in ((difr.difr_score_gm_filtered, (s,)), (difr.difr_score_ipt_filtered, ())):
+        mixed = fresh()
+        mixed.temperatures = temps
+        fn(dev.h, dev.W, tok_dev, dev.seeds, dev.positions, 1.0, ks, ps, *extra, mixed)
+        torch.cuda.synchronize()
+        assert int(mixed.device_status.item()) == 0
+        got, cut, st = mixed.score.cpu().numpy(), mixed.cutoff.cpu().numpy(), mixed.row_status.cpu().numpy()
+        for g in valid:
+            temp, k, p = policies[g]
+            rows = group == g
+            if fn is difr.difr_score_ipt_filtered and k == 0 and p == 1.0:
+                # a row whose policy filters nothing keeps the unfiltered score
+                ref = dev.score("ipt", tokens, temp, sigma, EPS)["score"]
+                assert np.array_equal(got[rows], ref[rows]) and np.all(np.isneginf(cut[rows]))
+                continue
+            one = fresh()
+            fn(dev.h, dev.W, tok_dev, dev.seeds, dev.positions, f32(temp), k, p, *extra, one)
+            torch.cuda.synchronize()
+            assert np.array_equal(got[rows], one.score.cpu().numpy()[rows], equal_nan=True), (fn.__name__, g)
+            assert np.array_equal(cut[rows], one.cutoff.cpu().numpy()[rows], equal_nan=True), (fn.__name__, g)
+            assert np.all(np.isfinite(got[rows])) and np.all(st[rows] & 8 == 0)
+        bad = group >= len(valid)
+        assert np.all(np.isnan(got[bad])) and np.all(st[bad] & 8 != 0)
+        # the policies differ where they should: the same claims score differently under different filters
+        assert np.unique(np.round(cut[~bad & np.isfinite(cut)], 3)).size > 10
