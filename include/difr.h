@@ -90,7 +90,8 @@ typedef struct {
   float* p_claimed;   /* IPT: softmax probability of the claimed token            */
   float* cdf_lo;      /* IPT: a = sum_{v < t*} p_v                                 */
   float* u;           /* IPT: the uniform mu of this row                           */
-  uint32_t* row_status; /* bit0: claimed id outside [0, V); bit1: non-finite logits;
+  uint32_t* row_status; /* bit0: claimed id outside [0, V); bit1: non-finite logits (the
+                           scores of such a row are NaN, which difr_detect flags);
                            bit2: candidate list overflow (difr_score_gm_filtered);
                            bit3: unusable per-row temperature or filter values; bit4: the nucleus holds more
                            ids than the filtered calls resolve (64)                        */

@@ -193,11 +193,13 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
   const int n = n_found < p.cand_cap ? n_found : p.cand_cap;
   uint32_t status_bits = (n_found > p.cand_cap) ? 4u : 0u;
   const RowPolicy rp = row_policy(p, row);
-  if (rp.bad) {
+  // (the first pass's finalize leaves NaN for a row with a non-finite logit: such a row stays unscored)
+  const bool unscored = isnan(p.score[row]);
+  if (rp.bad || unscored) {
     if (lane == 0) {
       p.score[row] = CUDART_NAN_F;
       if (p.cutoff) p.cutoff[row] = CUDART_NAN_F;
-      if (p.row_status) p.row_status[row] |= 8u;
+      if (p.row_status && rp.bad) p.row_status[row] |= 8u;
     }
     return;
   }
@@ -366,7 +368,7 @@ __global__ void __launch_bounds__(kFWarps * 32) ipt_filtered_finalize(const Filt
   const int n = n_found < p.cand_cap ? n_found : p.cand_cap;
   uint32_t status_bits = (n_found > p.cand_cap) ? 4u : 0u;
   const RowPolicy rp = row_policy(p, row);
-  if (rp.bad || (rp.none && rp.top_k == 0)) {
+  if (rp.bad || isnan(p.score[row]) || (rp.none && rp.top_k == 0)) {
     // unusable values: NaN; no filter at all (and a vocabulary too large to resolve here): the first pass's
     // finalize has already written the unfiltered score
     if (lane == 0) {
@@ -374,7 +376,7 @@ __global__ void __launch_bounds__(kFWarps * 32) ipt_filtered_finalize(const Filt
         p.score[row] = CUDART_NAN_F;
         if (p.row_status) p.row_status[row] |= 8u;
       }
-      if (p.cutoff) p.cutoff[row] = rp.bad ? CUDART_NAN_F : -CUDART_INF_F;
+      if (p.cutoff) p.cutoff[row] = (rp.bad || !rp.none) ? CUDART_NAN_F : -CUDART_INF_F;
     }
     return;
   }

@@ -291,3 +291,36 @@ def test_two_calls_in_flight_on_two_streams_keep_to_their_own_workspaces():
         assert np.array_equal(getattr(out_a, k).cpu().numpy(), alone_a[k], equal_nan=True), k
     for k in ("score", "p_claimed", "cdf_lo", "u", "lse"):
         assert np.array_equal(getattr(out_b, k).cpu().numpy(), alone_b[k], equal_nan=True), k
+
+
+def test_rows_with_non_finite_logits_are_never_scored_as_safe():
+    """A NaN or an infinity in a row of h makes every logit of that row non-finite, one in a row of W makes one
+    logit of every row non-finite: the oracle marks exactly those rows (row_status bit 1), and so must the library,
+    whose scores there are NaN (flagged by the detection step) whatever the claim."""
+    T, d, V = 200, 64, 3000
+    h, W, seeds, positions = _small(T, d, V, 51)
+    tokens = _claims(h, W, seeds, positions, f32(1.0), 52)
+    h = h.copy()
+    h[3, 5] = 0x7FC0    # NaN
+    h[40, 0] = 0x7F80   # +inf
+    h[41, 63] = 0xFF80  # -inf
+    for W_case in ("clean", "nan_in_W"):
+        Wc = W.copy()
+        if W_case == "nan_in_W":
+            Wc[2999, 7] = 0x7FC0
+        dev = Device(h, Wc, seeds, positions)
+        ref = oracle.score_gm(h, Wc, tokens, seeds, positions, f32(1.0), f32(0.3), f32(EPS))
+        marked = (ref.row_status & 2) != 0
+        assert marked.sum() == (3 if W_case == "clean" else T)
+        for kind in ("gm", "ipt"):
+            got = dev.score(kind, tokens, 1.0, 0.3, EPS)
+            assert np.array_equal((got["row_status"] & 2) != 0, marked), (W_case, kind)
+            assert np.all(np.isnan(got["score"][marked])), (W_case, kind)
+            assert np.all(np.isfinite(got["score"][~marked])), (W_case, kind)
+        if W_case == "clean":
+            ok = ~marked
+            np.testing.assert_allclose(dev.score("gm", tokens, 1.0, 0.3, EPS)["score"][ok], ref.score[ok], rtol=0, atol=SCORE_TOL)
+        flags, _ = difr.difr_detect(to_dev(dev.score("gm", tokens, 1.0, 0.3, EPS)["score"]), -20.0,
+                                    flags=torch.zeros(T, dtype=torch.uint8, device="cuda"))
+        torch.cuda.synchronize()
+        assert np.all(flags.cpu().numpy()[marked] == 1)
