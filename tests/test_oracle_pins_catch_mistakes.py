@@ -34,6 +34,9 @@ MISTAKES = [
      "test_oracle_scores.py", "draws_from_the_temperature_softmax"),
     ("competitor is always the argmax", C, "int64_t c = (t == i1) ? i2 : i1; /* strongest competitor */",
      "int64_t c = i1;", "test_oracle_scores.py", "numpy_replay"),
+    ("ties go to the highest id", C, "if (i1 < 0 || y[v] > y[i1]) {\n            i2 = i1;\n            i1 = v;\n          } else if (i2 < 0 || y[v] > y[i2]) {\n            i2 = v;\n          }\n        }\n        int64_t t = tokens[r];",
+     "if (i1 < 0 || y[v] >= y[i1]) {\n            i2 = i1;\n            i1 = v;\n          } else if (i2 < 0 || y[v] >= y[i2]) {\n            i2 = v;\n          }\n        }\n        int64_t t = tokens[r];",
+     "test_oracle_scores.py", "exact_ties"),
     ("margin with the wrong sign", C, "A = y[t] - y[c];\n          if (A == 0.0", "A = y[c] - y[t];\n          if (A == 0.0",
      "test_oracle_scores.py", "nonnegative_margin"),
     ("closed form without the square root of two", C, "return std_normal_cdf(A / (sigma * sqrt(2.0)));",

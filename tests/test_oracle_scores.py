@@ -379,3 +379,29 @@ def test_detection_and_pooling_against_numpy():
     assert list(f2) == [0, 1]
     f3, st3 = oracle.detect(scores, tau, margins, None)
     assert st3["n_flagged"][0] == want_flags.sum()
+
+
+def test_exact_ties_go_to_the_lowest_id():
+    """Two identical rows of W give two identical logits; under greedy decoding (no noise) the lower id is the
+    sample, the higher id the runner-up, and claiming the higher id is a mismatch by the tie-break alone:
+    margin -0.0, not +0.0."""
+    T, d, V = 6, 16, 40
+    h, W = _small(T, d, V, 23)
+    seeds, positions = _meta(T)
+    logits = _f64(h) @ _f64(W).T
+    top = logits.argmax(axis=1)
+    W = W.copy()
+    lo_id, hi_id = 7, 31
+    # row by row: ids 7 and 31 both get the W row of that row's largest logit
+    for r in range(T):
+        Wr = W.copy()
+        Wr[lo_id] = W[top[r]]
+        Wr[hi_id] = W[top[r]]
+        if top[r] not in (lo_id, hi_id):
+            Wr[top[r]] = 0  # the original holder steps back
+        for claim, want_match, want_sign in ((lo_id, 1, False), (hi_id, 0, True)):
+            res = oracle.score_gm(h[r : r + 1], Wr, np.array([claim], dtype=np.int32), seeds[r : r + 1],
+                                  positions[r : r + 1], 0.0, 0.5, EPS)
+            assert res.argmax[0] == lo_id and res.runner_up[0] == hi_id
+            assert res.margin[0] == 0.0 and bool(np.signbit(res.margin[0])) == want_sign
+            assert res.match[0] == want_match and res.top2_margin[0] == 0.0
