@@ -316,20 +316,25 @@ def run_ours(args):
     fused_avg_ms = float(np.mean(fused_ms))
     assert int(out.device_status.item()) == 0, "device-side wait timed out"
     n_flagged = int(flags.sum().item())
+    flags_ref = flags.cpu().clone()
     stats_np = stats.cpu().numpy()
 
     # ---- end to end: per-step inputs start in pinned host memory, results end there
     out.event_fused_start = out.event_fused_stop = 0
-    score_host = torch.empty(T, dtype=torch.float32).pin_memory()
-    flags_host = torch.empty(T, dtype=torch.uint8).pin_memory()
-    stats_host = torch.empty((n_seq, 4), dtype=torch.int32).pin_memory()
-    # Two input buffers: a copy stream uploads step i + 1 while the kernels of step i run (what a serving
-    # loop does); every step's upload, kernels and read-back lie inside the timed region.
-    copy_stream, run_stream = torch.cuda.Stream(), torch.cuda.current_stream()
+    # Two input buffers and two sets of outputs: a copy stream uploads step i + 1 while the kernels of step i
+    # run, and a third stream reads the results of step i back while the kernels of step i + 1 run (what a
+    # serving loop does); every step's upload, kernels and read-back lie inside the timed region.
+    copy_stream, back_stream, run_stream = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.current_stream()
     bufs = [(torch.empty_like(h_dev), torch.empty_like(tokens_dev), torch.empty_like(seeds_dev),
              torch.empty_like(pos_dev)) for _ in range(2)]
+    outs = [out, difr.DifrOut.allocate(T, d, V, sigma, 1e-12)]
+    dev_res = [(flags, stats), (torch.empty_like(flags), torch.empty_like(stats))]
+    host_res = [(torch.empty(T, dtype=torch.float32).pin_memory(), torch.empty(T, dtype=torch.uint8).pin_memory(),
+                 torch.empty((n_seq, 4), dtype=torch.int32).pin_memory()) for _ in range(2)]
     uploaded = [torch.cuda.Event() for _ in range(2)]
     consumed = [torch.cuda.Event() for _ in range(2)]
+    scored = [torch.cuda.Event() for _ in range(2)]
+    read_back = [torch.cuda.Event() for _ in range(2)]
 
     def upload(i):
         h_in, tok_in, seed_in, pos_in = bufs[i % 2]
@@ -343,13 +348,20 @@ def run_ours(args):
 
     def run(i):
         h_in, tok_in, seed_in, pos_in = bufs[i % 2]
+        o, (fl, st) = outs[i % 2], dev_res[i % 2]
+        score_host, flags_host, stats_host = host_res[i % 2]
         run_stream.wait_event(uploaded[i % 2])
-        difr.difr_score_gm(h_in, W_dev, tok_in, seed_in, pos_in, temperature, out)
-        difr.difr_detect(out.score, tau, out.margin, None, 0, seq_dev, flags, stats)
+        run_stream.wait_event(read_back[i % 2])  # the results these outputs held two steps ago have been read
+        difr.difr_score_gm(h_in, W_dev, tok_in, seed_in, pos_in, temperature, o)
+        difr.difr_detect(o.score, tau, o.margin, None, 0, seq_dev, fl, st)
         consumed[i % 2].record(run_stream)
-        score_host.copy_(out.score, non_blocking=True)
-        flags_host.copy_(flags, non_blocking=True)
-        stats_host.copy_(stats, non_blocking=True)
+        scored[i % 2].record(run_stream)
+        with torch.cuda.stream(back_stream):
+            back_stream.wait_event(scored[i % 2])
+            score_host.copy_(o.score, non_blocking=True)
+            flags_host.copy_(fl, non_blocking=True)
+            stats_host.copy_(st, non_blocking=True)
+            read_back[i % 2].record(back_stream)
 
     def e2e_loop(n):
         upload(0)
@@ -357,13 +369,14 @@ def run_ours(args):
             if i + 1 < n:
                 upload(i + 1)
             run(i)
+        run_stream.wait_stream(back_stream)  # the last read-backs end inside the timed region
 
-    for ev in consumed:
+    for ev in consumed + read_back:
         ev.record(run_stream)
     e2e_loop(min(args.warmup, 3))
     barrier()
     e_begin, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    for ev in consumed:
+    for ev in consumed + read_back:
         ev.record(run_stream)
     e_begin.record(run_stream)
     copy_stream.wait_event(e_begin)  # the first upload starts inside the timed region
@@ -371,9 +384,13 @@ def run_ours(args):
     e_end.record(run_stream)
     barrier()
     e2e_ms = e_begin.elapsed_time(e_end)
+    assert int(outs[1].device_status.item()) == 0, "device-side wait timed out"
+    last = (args.steps - 1) % 2
+    score_host, flags_host, stats_host = host_res[last]
     h2d = h_host.numel() * 2 + tokens_host.numel() * 4 + seeds_host.numel() * 8 + pos_host.numel() * 4
     d2h = score_host.numel() * 4 + flags_host.numel() + stats_host.numel() * 4
-    assert torch.equal(flags_host, flags.cpu())
+    assert torch.equal(flags_host, dev_res[last][0].cpu())
+    assert torch.equal(flags_host, flags_ref)
 
     elapsed_ms, e2e_ms, fused_avg_ms = reduce_max([elapsed_ms, e2e_ms, fused_avg_ms], device="cuda")
 
@@ -409,7 +426,8 @@ def run_ours(args):
             "e2e": {"value": whole_job_rate(world, T, args.steps, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps,
                     "note": "per-step inputs (h, tokens, seeds, positions) from pinned host memory, uploaded on a copy "
-                            "stream one step ahead of the kernels; scores, flags and statistics read back; W resident"},
+                            "stream one step ahead of the kernels; scores, flags and statistics read back on a "
+                            "third stream; W resident"},
             "gpu_launches": 3 * args.steps,
             "roofline": {"kernel": "k1_fused_score", "bound": "tensor", "achieved": achieved,
                          "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
