@@ -100,7 +100,7 @@ __device__ __forceinline__ Unit decode_unit(const K1Params& p, int u) {
 
 // ---------------------------------------------------------- running statistics
 struct RowStats {
-  float m1, m2;  // top-2 keys of y' (low 4 mantissa bits carry the column within its 16-id group)
+  float m1, m2;  // top-2 keys of y' (low 4 mantissa bits cleared)
   int i1, i2;    // their vocabulary ids
   float lmax;    // running max of z = l * c1
   float lsum;    // sum of 2^(z - lmax)
@@ -119,7 +119,12 @@ __device__ __forceinline__ void stats_init(RowStats& s) {
   s.gm2 = -CUDART_INF_F;
 }
 
-// (k1, j1), (k2, j2): the best two of another column group of the same row, k1 >= k2.
+// Keys are y' with the low four mantissa bits cleared, so values that differ by less than 2^-19 relative count
+// as equal, and equal keys rank by vocabulary id (lowest first): of any number of exactly tied ids the two lowest
+// survive to the finalize kernel, which orders them exactly.  (Inside one 16-id group the min/max network ranks
+// tied keys by their column bits instead; three tied ids within one group are not told apart.)
+//
+// (k1, j1), (k2, j2): the best two of the next 16 ids of the same thread, k1 >= k2, all ids above those seen.
 __device__ __forceinline__ void top2_merge(RowStats& s, float k1, int j1, float k2, int j2) {
   if (k1 > s.m1) {
     const bool q = k2 > s.m1;
@@ -130,6 +135,19 @@ __device__ __forceinline__ void top2_merge(RowStats& s, float k1, int j1, float 
   } else if (k1 > s.m2) {
     s.m2 = k1;
     s.i2 = j1;
+  }
+}
+
+// One candidate of another column group (its ids may lie on either side of this group's): ties by id.
+__device__ __forceinline__ void top2_insert_any(RowStats& s, float k, int j) {
+  if (k > s.m1 || (k == s.m1 && (unsigned)j < (unsigned)s.i1)) {
+    s.m2 = s.m1;
+    s.i2 = s.i1;
+    s.m1 = k;
+    s.i1 = j;
+  } else if (k > s.m2 || (k == s.m2 && (unsigned)j < (unsigned)s.i2)) {
+    s.m2 = k;
+    s.i2 = j;
   }
 }
 
@@ -304,9 +322,12 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
         }
       }
     }
-    // merge the group's top-2 into the running top-2 (earlier ids win ties)
-    if (M::gm)
-      top2_merge(s, c1k, base + (int)(__float_as_uint(c1k) & 15u), c2k, base + (int)(__float_as_uint(c2k) & 15u));
+    // merge the group's top-2 into the running top-2 (column bits cleared: earlier ids win ties)
+    if (M::gm) {
+      const uint32_t b1 = __float_as_uint(c1k), b2 = __float_as_uint(c2k);
+      top2_merge(s, __uint_as_float(b1 & ~15u), base + (int)(b1 & 15u), __uint_as_float(b2 & ~15u),
+                 base + (int)(b2 & 15u));
+    }
   }
 }
 
@@ -332,7 +353,8 @@ __device__ __forceinline__ void record_merge(RowStats& st, const float4& a, cons
     st.cnt[2] += __float_as_int(a.z);
     st.cnt[3] += __float_as_int(a.w);
   } else {
-    top2_merge(st, a.x, __float_as_int(a.y), a.z, __float_as_int(a.w));
+    top2_insert_any(st, a.x, __float_as_int(a.y));
+    top2_insert_any(st, a.z, __float_as_int(a.w));
     if (Mode<MODE>::groupmax) st.gm2 = fmax3(st.gm2, b.w, fminf(st.lmax, b.x));  // (b.x, b.w): its two largest
     if (b.x > -CUDART_INF_F) {  // that group saw columns
       const float m = fmaxf(st.lmax, b.x);

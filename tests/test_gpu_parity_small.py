@@ -326,23 +326,25 @@ def test_rows_with_non_finite_logits_are_never_scored_as_safe():
         assert np.all(flags.cpu().numpy()[marked] == 1)
 
 
-def test_exact_ties_go_to_the_lowest_id():
-    """Greedy replay with two identical rows of W that hold the largest logit of every row: the lower id is the
-    sample, the higher id the runner-up, and a claim of the higher id is a mismatch (margin -0.0), as in the oracle."""
-    T, d, V = 64, 64, 1500
+@pytest.mark.parametrize("tied", [(37, 1301), (1301, 37, 700), (8999, 5000, 37, 700, 1301, 4096, 4111)])
+def test_exact_ties_go_to_the_lowest_id(tied):
+    """Greedy replay with identical rows of W that hold the largest logit of every row: the lowest id is the
+    sample, the next lowest the runner-up, and a claim of any other tied id is a mismatch by the tie-break alone
+    (margin -0.0), as in the oracle.  The tied ids lie in different 16-id groups, tiles and strips."""
+    T, d, V = 64, 64, 9000
     h, W, seeds, positions = _small(T, d, V, 61)
-    # one direction that dominates every row's logits: h gets a large common component, two rows of W point along it
+    # one direction that dominates every row's logits: h gets a large common component, the tied rows point along it
     h = wl.f32_to_bf16_bits(wl.bf16_bits_to_f32(h) + 4.0 * np.sign(np.arange(d) % 2 - 0.5).astype(np.float32))
     W = W.copy()
     along = wl.f32_to_bf16_bits((np.sign(np.arange(d) % 2 - 0.5)).astype(np.float32))
-    lo_id, hi_id = 37, 1301
-    W[lo_id] = along
-    W[hi_id] = along
-    tokens = np.where(np.arange(T) % 2 == 0, lo_id, hi_id).astype(np.int32)
+    for v in tied:
+        W[v] = along
+    order = sorted(tied)
+    tokens = np.array([tied[r % len(tied)] for r in range(T)], dtype=np.int32)
     ref = oracle.score_gm(h, W, tokens, seeds, positions, 0.0, f32(0.2), f32(EPS))
-    assert np.all(ref.argmax == lo_id) and np.all(ref.runner_up == hi_id) and np.all(ref.top2_margin == 0.0)
+    assert np.all(ref.argmax == order[0]) and np.all(ref.runner_up == order[1]) and np.all(ref.top2_margin == 0.0)
     got = Device(h, W, seeds, positions).score("gm", tokens, 0.0, 0.2, EPS)
     assert np.array_equal(got["argmax"], ref.argmax) and np.array_equal(got["runner_up"], ref.runner_up)
     assert np.all(got["margin"] == 0.0) and np.array_equal(np.signbit(got["margin"]), np.signbit(ref.margin))
-    assert np.array_equal(np.signbit(got["margin"]), tokens == hi_id)
+    assert np.array_equal(np.signbit(got["margin"]), tokens != order[0])
     np.testing.assert_allclose(got["score"], ref.score, rtol=0, atol=1e-6)

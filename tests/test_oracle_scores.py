@@ -391,7 +391,7 @@ def test_exact_ties_go_to_the_lowest_id():
     logits = _f64(h) @ _f64(W).T
     top = logits.argmax(axis=1)
     W = W.copy()
-    lo_id, hi_id = 7, 31
+    lo_id, hi_id, third = 7, 31, 19
     # row by row: ids 7 and 31 both get the W row of that row's largest logit
     for r in range(T):
         Wr = W.copy()
@@ -405,3 +405,9 @@ def test_exact_ties_go_to_the_lowest_id():
             assert res.argmax[0] == lo_id and res.runner_up[0] == hi_id
             assert res.margin[0] == 0.0 and bool(np.signbit(res.margin[0])) == want_sign
             assert res.match[0] == want_match and res.top2_margin[0] == 0.0
+        # a third identical row in between: it becomes the runner-up, and claiming it still loses to id 7
+        Wr[third] = Wr[lo_id]
+        res = oracle.score_gm(h[r : r + 1], Wr, np.array([third], dtype=np.int32), seeds[r : r + 1],
+                              positions[r : r + 1], 0.0, 0.5, EPS)
+        assert res.argmax[0] == lo_id and res.runner_up[0] == third and res.top23_margin[0] == 0.0
+        assert res.margin[0] == 0.0 and np.signbit(res.margin[0]) and res.match[0] == 0
