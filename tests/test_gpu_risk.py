@@ -127,7 +127,8 @@ def _noisy_logits(h, W, seeds, positions, temperature):
     return y
 
 
-@pytest.mark.parametrize("T,d,V,temperature,sigma", [(150, 64, 1200, 1.0, 1.0), (140, 72, 520, 0.7, 0.3)])
+@pytest.mark.parametrize("T,d,V,temperature,sigma", [(150, 64, 1200, 1.0, 1.0), (140, 72, 520, 0.7, 0.3),
+                                                     (130, 64, 700, 0.0, 0.5)])  # the last: greedy decoding, no noise
 def test_admissible_set_sizes_and_information_bound(T, d, V, temperature, sigma):
     h, W, seeds, positions = _small(T, d, V, 41)
     dev = Device(h, W, seeds, positions)
@@ -138,10 +139,13 @@ def test_admissible_set_sizes_and_information_bound(T, d, V, temperature, sigma)
     difr.difr_admissible(dev.h, dev.W, dev.seeds, dev.positions, f32(temperature), scored, taus, counts)
     one = torch.full((1, T), -1, dtype=torch.int32, device="cuda")
     difr.difr_admissible(dev.h, dev.W, dev.seeds, dev.positions, f32(temperature), scored, taus[1:2], one)
+    none = torch.full((1, T), -1, dtype=torch.int32, device="cuda")
+    difr.difr_admissible(dev.h, dev.W, dev.seeds, dev.positions, f32(temperature), scored, [f32(0.5)], none)
     torch.cuda.synchronize()
     assert int(scored.device_status.item()) == 0
     got = counts.cpu().numpy()
     assert np.array_equal(one.cpu().numpy()[0], got[1])  # one bound or four: the same count
+    assert np.all(none.cpu().numpy() == 0)               # no score reaches a threshold above ln(1 + eps)
 
     # the oracle's sets, and the sets reachable when every margin moves by the kernel's rounding error
     y = _noisy_logits(h, W, seeds, positions, f32(temperature))
