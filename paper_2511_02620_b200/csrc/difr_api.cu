@@ -316,9 +316,13 @@ size_t difr_filtered_workspace_bytes(int64_t T, int64_t d, int64_t V) {
   return total;
 }
 
-difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,
-                                   const uint32_t* positions, float temperature, int64_t T, int64_t d, int64_t V,
-                                   const difr_filter* filter, difr_out* out, difr_stream_t stream) {
+// The two filtered estimators share everything but the fused kernel's modes, what the first finalize writes and
+// the last kernel: scoring pass (+ the strips' group maxima), ordinary finalize, bounds, collecting pass, finalize
+// over the candidate lists.  ipt: 0 Token-DiFR in full, 1 Token-IPT-DiFR on the filtered distribution.
+static difr_status filtered_common(int ipt, const void* h, const void* W, const int32_t* tokens,
+                                   const uint64_t* seeds, const uint32_t* positions, float temperature, int64_t T,
+                                   int64_t d, int64_t V, const difr_filter* filter, difr_out* out,
+                                   difr_stream_t stream) {
   if (!h || !W || !tokens || !seeds || !positions || !out || !out->score || !filter) return DIFR_ERR_INVALID_ARG;
   if (T < 0 || d <= 0 || V <= 0) return DIFR_ERR_INVALID_ARG;
   if (!(out->sigma > 0.f) || !(out->eps >= 0.f) || !isfinite(out->sigma) || !isfinite(out->eps))
@@ -329,9 +333,14 @@ difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* 
   if (out->temperatures != nullptr) temperature = 1.f;  // unused
   const int top_k = filter->top_k;
   const float top_p = filter->top_p;
-  if (filter->s < 1 || filter->s > 8) return DIFR_ERR_INVALID_ARG;
+  const int s_comp = ipt ? 0 : filter->s;  // the IPT estimator has no competitors
+  if (!ipt && (filter->s < 1 || filter->s > 8)) return DIFR_ERR_INVALID_ARG;
   if (filter->top_k_rows == nullptr && (top_k < 0 || (top_k > 64 && top_k < V))) return DIFR_ERR_INVALID_ARG;
   if (filter->top_p_rows == nullptr && (!(top_p > 0.f) || !(top_p <= 1.f))) return DIFR_ERR_INVALID_ARG;
+  // IPT with one policy for every row that filters nothing: that is difr_score_ipt
+  if (ipt && filter->top_k_rows == nullptr && filter->top_p_rows == nullptr && (top_k < 1 || top_k >= V) &&
+      top_p >= 1.f && V > 64)
+    return DIFR_ERR_INVALID_ARG;
   if ((d % 8) != 0 || V < 2) return DIFR_ERR_SHAPE;
   if (T == 0) return DIFR_OK;
   DeviceInfo info;
@@ -344,8 +353,10 @@ difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* 
   if (!aligned16(h) || !aligned16(W)) return DIFR_ERR_ALIGN;
   if (!out->workspace || out->workspace_bytes < total) return DIFR_ERR_WORKSPACE;
   if (!aligned16(out->workspace)) return DIFR_ERR_ALIGN;
-  const difr_status qs = ensure_quadrature_tables();
-  if (qs != DIFR_OK) return qs;
+  if (!ipt) {
+    const difr_status qs = ensure_quadrature_tables();
+    if (qs != DIFR_OK) return qs;
+  }
   CUtensorMap tmap_h, tmap_w;
   if (!make_tmap(&tmap_h, h, T, d, kBM) || !make_tmap(&tmap_w, W, V, d, kBN / 2)) return DIFR_ERR_CUDA;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
@@ -358,125 +369,65 @@ difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* 
   k1.device_status = out->device_status;
   k1.temperatures = out->temperatures;
   if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
-  if (launch_k1(6, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;
+  if (launch_k1(ipt ? 8 : 6, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;
 
+  // ---- the ordinary finalize: the unfiltered outputs (and, for a row without a filter, the IPT score)
   K2Params k2;
   memset(&k2, 0, sizeof k2);
   k2.h = reinterpret_cast<const uint16_t*>(h); k2.W = reinterpret_cast<const uint16_t*>(W);
   k2.tokens = tokens; k2.seeds = seeds; k2.positions = positions;
   k2.partials = k1.partials; k2.n_slots = pl.n_slots; k2.T_pad = pl.T_pad;
-  k2.T = (int)T; k2.d = (int)d; k2.V = (int)V; k2.ipt = 0;
+  k2.T = (int)T; k2.d = (int)d; k2.V = (int)V; k2.ipt = ipt;
   k2.temperature = temperature; k2.sigma = out->sigma; k2.eps = out->eps; k2.c1 = k1.c1;
-  k2.score = out->score; k2.margin = out->margin; k2.argmax = out->argmax; k2.runner_up = out->runner_up;
-  k2.lse = out->lse; k2.row_status = out->row_status; k2.y_max = out->y_max; k2.y_second = out->y_second;
+  k2.score = out->score; k2.lse = out->lse; k2.row_status = out->row_status;
   k2.temperatures = out->temperatures;
+  if (ipt) {
+    k2.p_claimed = out->p_claimed; k2.cdf_lo = out->cdf_lo; k2.u = out->u;
+  } else {
+    k2.margin = out->margin; k2.argmax = out->argmax; k2.runner_up = out->runner_up;
+    k2.y_max = out->y_max; k2.y_second = out->y_second;
+  }
   if (launch_k2(k2, s) != cudaSuccess) return DIFR_ERR_CUDA;
 
-  // ---- bounds, collecting pass, finalize
+  // ---- bounds (on y' for the competitors, on the logit for the filter), collecting pass, finalize over the lists
   FilterParams fp;
   memset(&fp, 0, sizeof fp);
   fp.h = k2.h; fp.W = k2.W; fp.tokens = tokens; fp.seeds = seeds; fp.positions = positions;
   fp.partials = k1.partials; fp.n_slots = pl.n_slots; fp.T_pad = pl.T_pad; fp.T = (int)T; fp.d = (int)d; fp.V = (int)V;
   fp.temperature = temperature; fp.sigma = out->sigma; fp.eps = out->eps; fp.c1 = k1.c1;
-  fp.top_k = top_k; fp.top_p = top_p; fp.s = filter->s; fp.ipt = 0;
+  fp.top_k = top_k; fp.top_p = top_p; fp.s = s_comp; fp.ipt = ipt;
   fp.top_k_rows = filter->top_k_rows; fp.top_p_rows = filter->top_p_rows; fp.temperatures = out->temperatures;
   fp.bounds = reinterpret_cast<float*>(ws + pl.bounds_offset);
   fp.cand_list = reinterpret_cast<const Candidate*>(ws + list_off);
   fp.cand_count = reinterpret_cast<const int*>(ws + count_off);
   fp.cand_cap = cap;
   fp.score = out->score; fp.cutoff = out->cutoff; fp.row_status = out->row_status;
+  if (ipt) {
+    fp.p_claimed = out->p_claimed; fp.cdf_lo = out->cdf_lo; fp.u = out->u;
+  }
   if (launch_filter_bounds(fp, s) != cudaSuccess) return DIFR_ERR_CUDA;
-
   if (cudaMemsetAsync(ws + count_off, 0, (size_t)pl.T_pad * sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
   if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
   k1.bounds = fp.bounds;
   k1.cand_list = ws + list_off;
   k1.cand_count = reinterpret_cast<int*>(ws + count_off);
   k1.cand_cap = cap;
-  if (launch_k1(7, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;
-  if (launch_filtered_finalize(fp, s) != cudaSuccess) return DIFR_ERR_CUDA;
+  if (launch_k1(ipt ? 9 : 7, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;
+  if ((ipt ? launch_ipt_filtered_finalize(fp, s) : launch_filtered_finalize(fp, s)) != cudaSuccess)
+    return DIFR_ERR_CUDA;
   return DIFR_OK;
+}
+
+difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,
+                                   const uint32_t* positions, float temperature, int64_t T, int64_t d, int64_t V,
+                                   const difr_filter* filter, difr_out* out, difr_stream_t stream) {
+  return filtered_common(0, h, W, tokens, seeds, positions, temperature, T, d, V, filter, out, stream);
 }
 
 difr_status difr_score_ipt_filtered(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,
                                     const uint32_t* positions, float temperature, int64_t T, int64_t d, int64_t V,
                                     const difr_filter* filter, difr_out* out, difr_stream_t stream) {
-  if (!h || !W || !tokens || !seeds || !positions || !out || !out->score || !filter) return DIFR_ERR_INVALID_ARG;
-  if (T < 0 || d <= 0 || V <= 0) return DIFR_ERR_INVALID_ARG;
-  if (!(out->sigma > 0.f) || !(out->eps >= 0.f) || !isfinite(out->sigma) || !isfinite(out->eps))
-    return DIFR_ERR_INVALID_ARG;
-  if (out->temperatures == nullptr && (!(temperature > 0.f) || !isfinite(temperature))) return DIFR_ERR_INVALID_ARG;
-  if (out->temperatures != nullptr) temperature = 1.f;  // unused
-  const int top_k = filter->top_k;
-  const float top_p = filter->top_p;
-  if (filter->top_k_rows == nullptr && (top_k < 0 || (top_k > 64 && top_k < V))) return DIFR_ERR_INVALID_ARG;
-  if (filter->top_p_rows == nullptr && (!(top_p > 0.f) || !(top_p <= 1.f))) return DIFR_ERR_INVALID_ARG;
-  // one policy for every row and it filters nothing: that is difr_score_ipt
-  if (filter->top_k_rows == nullptr && filter->top_p_rows == nullptr && (top_k < 1 || top_k >= V) && top_p >= 1.f &&
-      V > 64)
-    return DIFR_ERR_INVALID_ARG;
-  if ((d % 8) != 0 || V < 2) return DIFR_ERR_SHAPE;
-  if (T == 0) return DIFR_OK;
-  DeviceInfo info;
-  if (!device_info(&info)) return DIFR_ERR_CUDA;
-  if (info.major != 10) return DIFR_ERR_ARCH;
-  Plan pl;
-  int cap;
-  size_t count_off, list_off, total;
-  if (!filtered_layout(T, d, V, info.pairs, &pl, &cap, &count_off, &list_off, &total)) return DIFR_ERR_SHAPE;
-  if (!aligned16(h) || !aligned16(W)) return DIFR_ERR_ALIGN;
-  if (!out->workspace || out->workspace_bytes < total) return DIFR_ERR_WORKSPACE;
-  if (!aligned16(out->workspace)) return DIFR_ERR_ALIGN;
-  CUtensorMap tmap_h, tmap_w;
-  if (!make_tmap(&tmap_h, h, T, d, kBM) || !make_tmap(&tmap_w, W, V, d, kBN / 2)) return DIFR_ERR_CUDA;
-  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-  unsigned char* ws = static_cast<unsigned char*>(out->workspace);
-  const int grid = k1_grid(pl, info.pairs);
-
-  // ---- first pass: softmax statistics (the unfiltered outputs) and the strips' group maxima
-  K1Params k1 = k1_params(pl, T, d, V, temperature, ws);
-  k1.tokens = tokens; k1.seeds = seeds; k1.positions = positions;
-  k1.device_status = out->device_status;
-  k1.temperatures = out->temperatures;
-  if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
-  if (launch_k1(8, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;
-
-  K2Params k2;
-  memset(&k2, 0, sizeof k2);
-  k2.h = reinterpret_cast<const uint16_t*>(h); k2.W = reinterpret_cast<const uint16_t*>(W);
-  k2.tokens = tokens; k2.seeds = seeds; k2.positions = positions;
-  k2.partials = k1.partials; k2.n_slots = pl.n_slots; k2.T_pad = pl.T_pad;
-  k2.T = (int)T; k2.d = (int)d; k2.V = (int)V; k2.ipt = 1;
-  k2.temperature = temperature; k2.sigma = out->sigma; k2.eps = out->eps; k2.c1 = k1.c1;
-  k2.score = out->score; k2.lse = out->lse; k2.p_claimed = out->p_claimed; k2.cdf_lo = out->cdf_lo; k2.u = out->u;
-  k2.row_status = out->row_status;
-  k2.temperatures = out->temperatures;
-  if (launch_k2(k2, s) != cudaSuccess) return DIFR_ERR_CUDA;
-
-  // ---- bound on the top_k-th logit, collecting pass by logit, finalize over the kept ids
-  FilterParams fp;
-  memset(&fp, 0, sizeof fp);
-  fp.h = k2.h; fp.W = k2.W; fp.tokens = tokens; fp.seeds = seeds; fp.positions = positions;
-  fp.partials = k1.partials; fp.n_slots = pl.n_slots; fp.T_pad = pl.T_pad; fp.T = (int)T; fp.d = (int)d; fp.V = (int)V;
-  fp.temperature = temperature; fp.sigma = out->sigma; fp.eps = out->eps; fp.c1 = k1.c1;
-  fp.top_k = top_k; fp.top_p = top_p; fp.s = 0; fp.ipt = 1;
-  fp.top_k_rows = filter->top_k_rows; fp.top_p_rows = filter->top_p_rows; fp.temperatures = out->temperatures;
-  fp.bounds = reinterpret_cast<float*>(ws + pl.bounds_offset);
-  fp.cand_list = reinterpret_cast<const Candidate*>(ws + list_off);
-  fp.cand_count = reinterpret_cast<const int*>(ws + count_off);
-  fp.cand_cap = cap;
-  fp.score = out->score; fp.cutoff = out->cutoff; fp.row_status = out->row_status;
-  fp.p_claimed = out->p_claimed; fp.cdf_lo = out->cdf_lo; fp.u = out->u;
-  if (launch_filter_bounds(fp, s) != cudaSuccess) return DIFR_ERR_CUDA;
-  if (cudaMemsetAsync(ws + count_off, 0, (size_t)pl.T_pad * sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
-  if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
-  k1.bounds = fp.bounds;
-  k1.cand_list = ws + list_off;
-  k1.cand_count = reinterpret_cast<int*>(ws + count_off);
-  k1.cand_cap = cap;
-  if (launch_k1(9, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;
-  if (launch_ipt_filtered_finalize(fp, s) != cudaSuccess) return DIFR_ERR_CUDA;
-  return DIFR_OK;
+  return filtered_common(1, h, W, tokens, seeds, positions, temperature, T, d, V, filter, out, stream);
 }
 
 difr_status difr_exfiltratable_bits(const uint8_t* classes, const int32_t* counts, int32_t rank_cutoff, int64_t V,
