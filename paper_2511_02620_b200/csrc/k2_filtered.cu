@@ -130,6 +130,41 @@ __device__ __forceinline__ double row_mass_relative(const FilterParams& p, int r
   return part * exp2(wmax - l0 * c1);
 }
 
+// The row's k_eff largest logits stand sorted (descending) in sl[].  Returns the rank of the last id the row's
+// nucleus keeps (k_eff - 1 when top_p = 1): the shortest prefix whose softmax mass reaches top_p of the top-k's
+// renormalised mass, or of the whole row's when no top-k stands in front.  e0 / e1: unnormalised masses
+// 2^(c1 (l - l0)) of ranks lane and lane + 32.  Whole warp.
+__device__ __forceinline__ int nucleus_last_rank(const FilterParams& p, const RowPolicy& rp, int row, int lane,
+                                                 const float* sl, int k_eff, double& e0, double& e1,
+                                                 uint32_t& status_bits) {
+  const double c1 = (double)rp.c1, l0 = (double)sl[0];
+  e0 = (lane < k_eff) ? exp2(((double)sl[lane] - l0) * c1) : 0.0;
+  e1 = (lane + 32 < k_eff) ? exp2(((double)sl[lane + 32] - l0) * c1) : 0.0;
+  int last = k_eff - 1;
+  if (rp.top_p < 1.f) {
+    double c0 = e0, c1s = e1;  // inclusive scans of both halves
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+      const double u0 = __hiloint2double(__shfl_up_sync(0xffffffffu, __double2hiint(c0), m),
+                                         __shfl_up_sync(0xffffffffu, __double2loint(c0), m));
+      const double u1 = __hiloint2double(__shfl_up_sync(0xffffffffu, __double2hiint(c1s), m),
+                                         __shfl_up_sync(0xffffffffu, __double2loint(c1s), m));
+      if (lane >= m) { c0 += u0; c1s += u1; }
+    }
+    c1s += __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(c0), 31),
+                            __shfl_sync(0xffffffffu, __double2loint(c0), 31));
+    const double total = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(c1s), 31),
+                                          __shfl_sync(0xffffffffu, __double2loint(c1s), 31));
+    const double need = (double)rp.top_p * (rp.nucleus_full ? row_mass_relative(p, row, lane, l0, c1) : total);
+    const unsigned m0 = __ballot_sync(0xffffffffu, lane < k_eff && c0 >= need);
+    const unsigned m1 = __ballot_sync(0xffffffffu, lane + 32 < k_eff && c1s >= need);
+    if (m0) last = __ffs(m0) - 1;
+    else if (m1) last = 32 + __ffs(m1) - 1;
+    else if (rp.nucleus_full && k_eff < p.V) status_bits |= 16u;  // the nucleus holds more ids than were resolved
+  }
+  return last;
+}
+
 __global__ void __launch_bounds__(kFWarps * 32) filter_bounds(const FilterParams p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = blockIdx.x * kFWarps + warp;
@@ -235,38 +270,8 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
   }
   __syncwarp();
   if (k_eff > 0) {
-    cut_rank = k_eff - 1;  // the top_k-th largest logit
-    if (rp.top_p < 1.f) {
-      // nucleus inside the top k: shortest prefix (descending) whose renormalised softmax mass reaches top_p
-      double e0 = 0.0, e1 = 0.0;
-      const double c1 = (double)rp.c1, l0 = (double)sm_l[warp][0];
-      if (lane < k_eff) e0 = exp2(((double)sm_l[warp][lane] - l0) * c1);
-      if (lane + 32 < k_eff) e1 = exp2(((double)sm_l[warp][lane + 32] - l0) * c1);
-      double c0 = e0, c1s = e1;  // inclusive scans of both halves
-#pragma unroll
-      for (int m = 1; m < 32; m <<= 1) {
-        int lo0 = __shfl_up_sync(0xffffffffu, __double2loint(c0), m), hi0 = __shfl_up_sync(0xffffffffu, __double2hiint(c0), m);
-        int lo1 = __shfl_up_sync(0xffffffffu, __double2loint(c1s), m), hi1 = __shfl_up_sync(0xffffffffu, __double2hiint(c1s), m);
-        if (lane >= m) {
-          c0 += __hiloint2double(hi0, lo0);
-          c1s += __hiloint2double(hi1, lo1);
-        }
-      }
-      const double half = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(c0), 31),
-                                           __shfl_sync(0xffffffffu, __double2loint(c0), 31));
-      c1s += half;
-      const double total = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(c1s), 31),
-                                            __shfl_sync(0xffffffffu, __double2loint(c1s), 31));
-      // (a nucleus over the whole vocabulary: the mass it must reach is a share of the whole row's)
-      const double need = (double)rp.top_p * (rp.nucleus_full ? row_mass_relative(p, row, lane, l0, c1) : total);
-      const unsigned m0 = __ballot_sync(0xffffffffu, lane < k_eff && c0 >= need);
-      const unsigned m1 = __ballot_sync(0xffffffffu, lane + 32 < k_eff && c1s >= need);
-      int last = k_eff - 1;
-      if (m0) last = __ffs(m0) - 1;
-      else if (m1) last = 32 + __ffs(m1) - 1;
-      else if (rp.nucleus_full && k_eff < p.V) status_bits |= 16u;  // the nucleus holds more ids than were resolved
-      cut_rank = last;
-    }
+    double e0, e1;
+    cut_rank = nucleus_last_rank(p, rp, row, lane, sm_l[warp], k_eff, e0, e1, status_bits);
     // the cutoff is that id's logit: re-evaluated in fp64 like every other logit the score depends on
     cutoff = warp_dot64(p.h + (size_t)row * (size_t)p.d, p.W + (size_t)sm_id[warp][cut_rank] * (size_t)p.d, p.d, lane);
   }
@@ -402,32 +407,8 @@ __global__ void __launch_bounds__(kFWarps * 32) ipt_filtered_finalize(const Filt
   const double mu = ((double)x[0] + 0.5) * (1.0 / 4294967296.0);
   double score = log((double)p.eps), pt = CUDART_NAN, a = CUDART_NAN, cutoff = -CUDART_INF;
   if (k_eff > 0) {
-    const double c1 = (double)rp.c1, l0 = (double)sm_l[warp][0];
-    double e0 = 0.0, e1 = 0.0;  // unnormalised masses of ranks lane and lane + 32
-    if (lane < k_eff) e0 = exp2(((double)sm_l[warp][lane] - l0) * c1);
-    if (lane + 32 < k_eff) e1 = exp2(((double)sm_l[warp][lane + 32] - l0) * c1);
-    int last = k_eff - 1;
-    if (rp.top_p < 1.f) {
-      double c0 = e0, c1s = e1;
-#pragma unroll
-      for (int m = 1; m < 32; m <<= 1) {
-        const double u0 = __hiloint2double(__shfl_up_sync(0xffffffffu, __double2hiint(c0), m),
-                                           __shfl_up_sync(0xffffffffu, __double2loint(c0), m));
-        const double u1 = __hiloint2double(__shfl_up_sync(0xffffffffu, __double2hiint(c1s), m),
-                                           __shfl_up_sync(0xffffffffu, __double2loint(c1s), m));
-        if (lane >= m) { c0 += u0; c1s += u1; }
-      }
-      c1s += __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(c0), 31),
-                              __shfl_sync(0xffffffffu, __double2loint(c0), 31));
-      const double total = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(c1s), 31),
-                                            __shfl_sync(0xffffffffu, __double2loint(c1s), 31));
-      const double need = (double)rp.top_p * (rp.nucleus_full ? row_mass_relative(p, row, lane, l0, c1) : total);
-      const unsigned m0 = __ballot_sync(0xffffffffu, lane < k_eff && c0 >= need);
-      const unsigned m1 = __ballot_sync(0xffffffffu, lane + 32 < k_eff && c1s >= need);
-      if (m0) last = __ffs(m0) - 1;
-      else if (m1) last = 32 + __ffs(m1) - 1;
-      else if (rp.nucleus_full && k_eff < p.V) status_bits |= 16u;  // the nucleus holds more ids than were resolved
-    }
+    double e0, e1;  // unnormalised masses of ranks lane and lane + 32
+    const int last = nucleus_last_rank(p, rp, row, lane, sm_l[warp], k_eff, e0, e1, status_bits);
     cutoff = warp_dot64(p.h + (size_t)row * (size_t)p.d, p.W + (size_t)sm_id[warp][last] * (size_t)p.d, p.d, lane);
     if (tok_ok) {
       // mass of the kept ids, of those below the claimed id, and whether the claimed id is kept
