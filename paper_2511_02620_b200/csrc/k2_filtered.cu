@@ -22,40 +22,6 @@ constexpr int kGlOrder = 16;
 __constant__ double c_gl_x[kGlOrder];
 __constant__ double c_gl_w[kGlOrder];
 
-__device__ __forceinline__ double shfl_xor_f64(double v, int mask) {
-  int lo = __double2loint(v), hi = __double2hiint(v);
-  lo = __shfl_xor_sync(0xffffffffu, lo, mask);
-  hi = __shfl_xor_sync(0xffffffffu, hi, mask);
-  return __hiloint2double(hi, lo);
-}
-
-__device__ __forceinline__ double bf16_f64(uint32_t bits16) { return (double)__uint_as_float(bits16 << 16); }
-
-__device__ __forceinline__ double warp_dot64(const uint16_t* a, const uint16_t* b, int d, int lane) {
-  double acc = 0.0;
-  for (int k = lane * 8; k < d; k += 32 * 8) {
-    const uint4 va = *reinterpret_cast<const uint4*>(a + k);
-    const uint4 vb = *reinterpret_cast<const uint4*>(b + k);
-    const uint32_t wa[4] = {va.x, va.y, va.z, va.w};
-    const uint32_t wb[4] = {vb.x, vb.y, vb.z, vb.w};
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      acc = fma(bf16_f64(wa[q] & 0xFFFFu), bf16_f64(wb[q] & 0xFFFFu), acc);
-      acc = fma(bf16_f64(wa[q] >> 16), bf16_f64(wb[q] >> 16), acc);
-    }
-  }
-#pragma unroll
-  for (int m = 16; m >= 1; m >>= 1) acc += shfl_xor_f64(acc, m);
-  return acc;
-}
-
-__device__ __forceinline__ double gumbel_f64(uint64_t seed, uint32_t position, uint32_t id) {
-  uint32_t x[4];
-  philox4x32_10(id >> 2, position, 0u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), x);
-  const double u = ((double)(x[id & 3u] >> 9) + 0.5) * (1.0 / 8388608.0);
-  return -log(-log(u));
-}
-
 // n-th largest (n >= 1) of the values the warp holds, eight per lane; -inf when there are fewer than n.
 __device__ __forceinline__ float warp_nth_largest(float (&v)[8], int n, int lane) {
   float result = -CUDART_INF_F;
@@ -121,10 +87,10 @@ __device__ __forceinline__ double row_mass_relative(const FilterParams& p, int r
   }
   double wmax = lmax;
 #pragma unroll
-  for (int m = 16; m >= 1; m >>= 1) wmax = fmax(wmax, shfl_xor_f64(wmax, m));
+  for (int m = 16; m >= 1; m >>= 1) wmax = fmax(wmax, shfl_xor_double(wmax, m));
   double part = (lmax == -CUDART_INF) ? 0.0 : lsum * exp2(lmax - wmax);
 #pragma unroll
-  for (int m = 16; m >= 1; m >>= 1) part += shfl_xor_f64(part, m);
+  for (int m = 16; m >= 1; m >>= 1) part += shfl_xor_double(part, m);
   part = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(part), 0),
                           __shfl_sync(0xffffffffu, __double2loint(part), 0));
   return part * exp2(wmax - l0 * c1);
@@ -273,7 +239,7 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
     double e0, e1;
     cut_rank = nucleus_last_rank(p, rp, row, lane, sm_l[warp], k_eff, e0, e1, status_bits);
     // the cutoff is that id's logit: re-evaluated in fp64 like every other logit the score depends on
-    cutoff = warp_dot64(p.h + (size_t)row * (size_t)p.d, p.W + (size_t)sm_id[warp][cut_rank] * (size_t)p.d, p.d, lane);
+    cutoff = warp_dot(p.h + (size_t)row * (size_t)p.d, p.W + (size_t)sm_id[warp][cut_rank] * (size_t)p.d, p.d, lane);
   }
 
   double score = log((double)p.eps);
@@ -282,8 +248,8 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
     const uint32_t pos = p.positions[row];
     const uint16_t* hrow = p.h + (size_t)row * (size_t)p.d;
     const double temp = (double)rp.temperature, sigma = (double)p.sigma;
-    const double l_t = warp_dot64(hrow, p.W + (size_t)tok * (size_t)p.d, p.d, lane);
-    const double y_t = l_t + temp * gumbel_f64(seed, pos, (uint32_t)tok);
+    const double l_t = warp_dot(hrow, p.W + (size_t)tok * (size_t)p.d, p.d, lane);
+    const double y_t = l_t + temp * gumbel_exact(seed, pos, (uint32_t)tok);
     // exact logits and noisy logits of the s + 2 candidates; then the s best of them
     double cl[kMaxCand], cy[kMaxCand];
     int cid[kMaxCand];
@@ -293,8 +259,8 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
       if (c < n_cand) {
         const int id = sm_cand[warp][c];
         cid[c] = id;
-        cl[c] = warp_dot64(hrow, p.W + (size_t)id * (size_t)p.d, p.d, lane);
-        cy[c] = cl[c] + temp * gumbel_f64(seed, pos, (uint32_t)id);
+        cl[c] = warp_dot(hrow, p.W + (size_t)id * (size_t)p.d, p.d, lane);
+        cy[c] = cl[c] + temp * gumbel_exact(seed, pos, (uint32_t)id);
       }
     }
     // selection sort, descending y, ties to the lower id (kMaxCand is tiny; every lane does the same)
@@ -344,7 +310,7 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
       }
       acc *= 0.5 * w * inv_sigma * 0.39894228040143267794;  // 1 / (sigma sqrt(2 pi))
 #pragma unroll
-      for (int m = 16; m >= 1; m >>= 1) acc += shfl_xor_f64(acc, m);
+      for (int m = 16; m >= 1; m >>= 1) acc += shfl_xor_double(acc, m);
       pi_hat = fmin(fmax(acc, 0.0), 1.0);
     }
     score = log(pi_hat + (double)p.eps);
@@ -409,7 +375,7 @@ __global__ void __launch_bounds__(kFWarps * 32) ipt_filtered_finalize(const Filt
   if (k_eff > 0) {
     double e0, e1;  // unnormalised masses of ranks lane and lane + 32
     const int last = nucleus_last_rank(p, rp, row, lane, sm_l[warp], k_eff, e0, e1, status_bits);
-    cutoff = warp_dot64(p.h + (size_t)row * (size_t)p.d, p.W + (size_t)sm_id[warp][last] * (size_t)p.d, p.d, lane);
+    cutoff = warp_dot(p.h + (size_t)row * (size_t)p.d, p.W + (size_t)sm_id[warp][last] * (size_t)p.d, p.d, lane);
     if (tok_ok) {
       // mass of the kept ids, of those below the claimed id, and whether the claimed id is kept
       const bool k0 = lane <= last, k1 = lane + 32 <= last;
@@ -419,9 +385,9 @@ __global__ void __launch_bounds__(kFWarps * 32) ipt_filtered_finalize(const Filt
       double mine = ((k0 && id0 == tok) ? e0 : 0.0) + ((k1 && id1 == tok) ? e1 : 0.0);
 #pragma unroll
       for (int m = 16; m >= 1; m >>= 1) {
-        z += shfl_xor_f64(z, m);
-        below += shfl_xor_f64(below, m);
-        mine += shfl_xor_f64(mine, m);
+        z += shfl_xor_double(z, m);
+        below += shfl_xor_double(below, m);
+        mine += shfl_xor_double(mine, m);
       }
       a = below / z;
       pt = mine / z;  // zero when the filter removed the claimed id

@@ -49,75 +49,6 @@ __device__ __forceinline__ void lse_merge(Merged& a, double bmax, double bsum, d
   a.lmax = m;
 }
 
-__device__ __forceinline__ double shfl_xor_double(double v, int mask) {
-  int lo = __double2loint(v), hi = __double2hiint(v);
-  lo = __shfl_xor_sync(0xffffffffu, lo, mask);
-  hi = __shfl_xor_sync(0xffffffffu, hi, mask);
-  return __hiloint2double(hi, lo);
-}
-
-__device__ __forceinline__ double bf16_to_double(uint32_t bits16) {
-  return (double)__uint_as_float(bits16 << 16);
-}
-
-// fp64 dot product of two bf16 rows of length d (d % 8 == 0, rows 16-byte aligned), whole warp.
-__device__ __forceinline__ double warp_dot(const uint16_t* a, const uint16_t* b, int d, int lane) {
-  double acc = 0.0;
-  for (int k = lane * 8; k < d; k += 32 * 8) {
-    const uint4 va = *reinterpret_cast<const uint4*>(a + k);
-    const uint4 vb = *reinterpret_cast<const uint4*>(b + k);
-    const uint32_t wa[4] = {va.x, va.y, va.z, va.w};
-    const uint32_t wb[4] = {vb.x, vb.y, vb.z, vb.w};
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      acc = fma(bf16_to_double(wa[q] & 0xFFFFu), bf16_to_double(wb[q] & 0xFFFFu), acc);
-      acc = fma(bf16_to_double(wa[q] >> 16), bf16_to_double(wb[q] >> 16), acc);
-    }
-  }
-#pragma unroll
-  for (int m = 16; m >= 1; m >>= 1) acc += shfl_xor_double(acc, m);
-  return acc;
-}
-
-// Three such dot products against the same row a, their loads in flight together; a null row gives 0.
-// Each sum is taken in warp_dot's order, so the values are the same as three separate calls.
-__device__ __forceinline__ void warp_dot3(const uint16_t* a, const uint16_t* b0, const uint16_t* b1,
-                                          const uint16_t* b2, int d, int lane, double out[3]) {
-  const uint16_t* b[3] = {b0, b1, b2};
-  double acc[3] = {0.0, 0.0, 0.0};
-  for (int k = lane * 8; k < d; k += 32 * 8) {
-    const uint4 va = *reinterpret_cast<const uint4*>(a + k);
-    uint4 vb[3];
-#pragma unroll
-    for (int j = 0; j < 3; ++j)
-      vb[j] = b[j] != nullptr ? *reinterpret_cast<const uint4*>(b[j] + k) : make_uint4(0u, 0u, 0u, 0u);
-    const uint32_t wa[4] = {va.x, va.y, va.z, va.w};
-#pragma unroll
-    for (int j = 0; j < 3; ++j) {
-      const uint32_t wb[4] = {vb[j].x, vb[j].y, vb[j].z, vb[j].w};
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        acc[j] = fma(bf16_to_double(wa[q] & 0xFFFFu), bf16_to_double(wb[q] & 0xFFFFu), acc[j]);
-        acc[j] = fma(bf16_to_double(wa[q] >> 16), bf16_to_double(wb[q] >> 16), acc[j]);
-      }
-    }
-  }
-#pragma unroll
-  for (int m = 16; m >= 1; m >>= 1) {
-#pragma unroll
-    for (int j = 0; j < 3; ++j) acc[j] += shfl_xor_double(acc[j], m);
-  }
-#pragma unroll
-  for (int j = 0; j < 3; ++j) out[j] = acc[j];
-}
-
-__device__ __forceinline__ double gumbel_exact(uint64_t seed, uint32_t position, uint32_t id) {
-  uint32_t x[4];
-  philox4x32_10(id >> 2, position, 0u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), x);
-  const double u = ((double)(x[id & 3u] >> 9) + 0.5) * (1.0 / 8388608.0);
-  return -log(-log(u));
-}
-
 // Phi(zb) - Phi(za), za <= zb, evaluated in the tail that avoids cancellation.
 __device__ __forceinline__ double normal_interval(double za, double zb) {
   const double r = 0.70710678118654752440;
