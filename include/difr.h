@@ -235,7 +235,7 @@ difr_status difr_score_both(const void* h, const void* W, const int32_t* tokens,
  *   out->workspace needs difr_filtered_workspace_bytes(T, d, V) bytes
  *
  * Everything difr_score_gm writes is written as there (margin, argmax, runner_up,
- * lse, y_max, y_second; `rank` is not available in this call); `score` holds
+ * lse, y_max, y_second, and `rank`, counted during the second pass); `score` holds
  * the full estimator and out->cutoff, if given, the cutoff per row (-inf: no
  * filter).  Two passes over the logits: the scoring pass, then a pass that
  * collects, per row, the ids that can be among the s + 2 best or among the top_k

@@ -408,6 +408,16 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
   if (launch_filter_bounds(fp, s) != cudaSuccess) return DIFR_ERR_CUDA;
   if (cudaMemsetAsync(ws + count_off, 0, (size_t)pl.T_pad * sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
   if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
+  if (!ipt && out->rank != nullptr) {
+    // the raw-logit rank of the claimed token rides on the collecting pass: claimed logits into the third
+    // plane of the bounds, the counts added up in out->rank
+    if (launch_claimed_logits(k2.h, k2.W, tokens, (int)T, (int)d, (int)V, fp.bounds + 2 * (size_t)pl.T_pad, s) !=
+        cudaSuccess)
+      return DIFR_ERR_CUDA;
+    if (cudaMemsetAsync(out->rank, 0, (size_t)T * sizeof(int32_t), s) != cudaSuccess) return DIFR_ERR_CUDA;
+    k1.rank_out = out->rank;
+    fp.rank = out->rank;
+  }
   k1.bounds = fp.bounds;
   k1.cand_list = ws + list_off;
   k1.cand_count = reinterpret_cast<int*>(ws + count_off);

@@ -22,6 +22,7 @@ struct K1Params {
   Partial* partials;  // [n_slots][T_pad]
   float* logits_out;  // dump mode only
   int32_t* device_status;
+  int* rank_out;      // Collect mode, nullable: [T] zeroed counters that receive the claimed tokens' raw-logit ranks
   int* unit_counter;  // zeroed before the launch: units are handed out in order on demand; null: round robin
   int T, d, V;
   int T_pad, m_tiles, n_tiles, k_steps;
@@ -117,12 +118,13 @@ struct FilterParams {
   const float* temperatures;   // nullable: one temperature per row (then `temperature` and `c1` are unused)
   int ipt;      // the IPT estimator's finalize: a row without any filter keeps the first pass's outputs
   int s;        // competitors in the active subset
-  float* bounds;  // [2][T_pad]: on y', on the raw logit
+  float* bounds;  // [3][T_pad]: on y', on the raw logit; claimed logits (when the rank is wanted)
   const Candidate* cand_list;
   const int* cand_count;
   int cand_cap;
   float* score;
   float* cutoff;  // nullable
+  int32_t* rank;  // nullable: counted by the collecting pass; the finalize sets V for an out-of-range claim
   uint32_t* row_status;
   float* p_claimed;  // IPT finalize only, nullable
   float* cdf_lo;

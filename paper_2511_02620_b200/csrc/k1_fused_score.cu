@@ -70,12 +70,13 @@ template <int MODE>
 struct Mode {
   static constexpr bool gm = MODE == kModeGm || MODE == kModeGmRank || MODE == kModeGmFilter;
   static constexpr bool softmax = gm || MODE == kModeIpt || MODE == kModeIptFilter;
-  static constexpr bool rank = MODE == kModeGmRank;
+  static constexpr bool rank = MODE == kModeGmRank || MODE == kModeCollect;  // Collect: only when asked for
+  static constexpr int rank_slot = MODE == kModeGmRank ? 0 : 2;  // which bound holds the claimed logit
   static constexpr bool groupmax = MODE == kModeGmFilter || MODE == kModeIptFilter;
   static constexpr bool collect = MODE == kModeCollect || MODE == kModeCollectLogit;
   static constexpr int ng = MODE == kModeCount1 ? 1 : (MODE == kModeCount4 ? 4 : 0);  // bounds per row
   static constexpr bool noise = gm || ng > 0 || MODE == kModeCollect;
-  static constexpr int ncnt = rank ? 1 : (collect ? 2 : (ng > 0 ? ng : 1));
+  static constexpr int ncnt = collect ? 3 : (rank ? 1 : (ng > 0 ? ng : 1));  // bounds loaded per row
   static constexpr bool bounds = rank || collect || ng > 0;
   static constexpr bool record = !collect && MODE != kModeDump;
 };
@@ -105,8 +106,9 @@ struct RowStats {
   float lmax;    // running max of z = l * c1
   float lsum;    // sum of 2^(z - lmax)
   float lpre;    // the same restricted to ids below the claimed one
-  int cnt[4];    // GmRank: cnt[0] = ids whose logit exceeds the claimed one; Count: ids at or above bound g
-  float bound[4];  // GmRank: bound[0] = claimed logit; Count: the row's bounds on y'; Collect: bounds on y', on l
+  int cnt[4];    // GmRank: cnt[0] (Collect: cnt[2]) = ids whose logit exceeds the claimed one; Count: ids at or above bound g
+  float bound[4];  // GmRank: bound[0] = claimed logit; Count: the row's bounds on y'; Collect: bounds on y', on l,
+                   // and the claimed logit (+inf when no rank is wanted)
   float gm2;     // GmFilter: the second largest 16-id group maximum of z (lmax is the largest)
 };
 
@@ -239,7 +241,7 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
 
   // ---- raw-logit rank of the claimed token: ids whose logit is larger (the claimed id itself left out)
   if (M::rank) {
-    const float lt = s.bound[0];
+    const float lt = s.bound[M::rank_slot];
     int c = 0;
 #pragma unroll
     for (int j = 0; j < kSub; ++j) c += (l[j] > lt) ? 1 : 0;
@@ -248,7 +250,7 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
       for (int j = 0; j < kSub; ++j)
         if (j == tl && l[j] > lt) --c;
     }
-    s.cnt[0] += c;
+    s.cnt[M::rank_slot] += c;
   }
 
   // ---- candidates by raw logit only (the IPT estimator under a filter needs no noise)
@@ -655,6 +657,8 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
         if (lane == 0) mbar_arrive_cluster_nofence(map_to_cta(acc_empty_bar(acc), 0));
         if (++acc == kAccStages) { acc = 0; acc_phase ^= 1u; }
       }
+      if (MODE == kModeCollect && ok && valid && p.rank_out != nullptr && st.cnt[2] != 0)
+        atomicAdd(p.rank_out + row, st.cnt[2]);  // this thread's share of the claimed token's raw-logit rank
       if (Mode<MODE>::record && ok) {
         // the four column groups of a row meet in shared memory; group 0 merges and writes the record
         if (colg != 0) {

@@ -193,6 +193,7 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
   const int n_found = p.cand_count[row];
   const int n = n_found < p.cand_cap ? n_found : p.cand_cap;
   uint32_t status_bits = (n_found > p.cand_cap) ? 4u : 0u;
+  if (p.rank != nullptr && !tok_ok && lane == 0) p.rank[row] = p.V;  // as in the plain call
   const RowPolicy rp = row_policy(p, row);
   // (the first pass's finalize leaves NaN for a row with a non-finite logit: such a row stays unscored)
   const bool unscored = isnan(p.score[row]);

@@ -45,6 +45,7 @@ def _run(dev, tokens, temperature, sigma, top_k, top_p, s):
     out = difr.DifrOut.allocate(dev.T, dev.d, dev.V, sigma, EPS)
     out.workspace = torch.empty(difr.difr_filtered_workspace_bytes(dev.T, dev.d, dev.V), dtype=torch.uint8, device="cuda")
     out.cutoff = torch.full((dev.T,), float("nan"), dtype=torch.float32, device="cuda")
+    out.rank = torch.full((dev.T,), -5, dtype=torch.int32, device="cuda")
     out.score.fill_(float("nan"))
     difr.difr_score_gm_filtered(dev.h, dev.W, to_dev(np.asarray(tokens, dtype=np.int32)), dev.seeds, dev.positions,
                                 f32(temperature), top_k, top_p, s, out)
@@ -92,6 +93,14 @@ def test_full_estimator_matches_the_oracle(T, d, V, scale, temperature, sigma, t
     assert same_cut.mean() >= 0.97
     np.testing.assert_allclose(got[same_cut], want[same_cut], rtol=0, atol=SCORE_TOL)
     assert got[5] == pytest.approx(math.log(EPS), abs=1e-5)
+    # the raw-logit rank rides on the second pass: the very counts of the plain call's rank mode
+    plain_out = difr.DifrOut.allocate(T, d, V, sigma, EPS)
+    plain_out.rank = torch.full((T,), -5, dtype=torch.int32, device="cuda")
+    difr.difr_score_gm(dev.h, dev.W, to_dev(tokens), dev.seeds, dev.positions, f32(temperature), plain_out)
+    torch.cuda.synchronize()
+    assert torch.equal(out.rank, plain_out.rank) and int(out.rank[5]) == V
+    ref_rank = oracle.score_gm(h, W, tokens, seeds, positions, f32(temperature), f32(sigma), f32(EPS)).rank
+    assert np.mean(out.rank.cpu().numpy() == ref_rank) >= 0.97
     # the estimate is not degenerate: the filter and the extra competitors move it
     if top_k or s > 1:
         plain = dev.score("gm", tokens, temperature, sigma, EPS)["score"]
