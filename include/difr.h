@@ -94,7 +94,7 @@ typedef struct {
                            scores of such a row are NaN, which difr_detect flags);
                            bit2: candidate list overflow (difr_score_gm_filtered);
                            bit3: unusable per-row temperature or filter values; bit4: the nucleus holds more
-                           ids than the filtered calls resolve (64)                        */
+                           ids than the filtered calls resolve (128)                       */
   void* workspace;      /* >= difr_workspace_bytes(T, d, V) bytes, 16-byte aligned;
                            contents are scratch, overwritten by every call         */
   size_t workspace_bytes;
@@ -222,11 +222,11 @@ difr_status difr_score_both(const void* h, const void* W, const int32_t* tokens,
  * mass reaches top_p.  The expectation is evaluated by Gauss-Legendre quadrature
  * (512 nodes over the range that carries the mass), not by sampling.
  *
- *   filter->top_k  0: no top-k; otherwise 1..64 (a top_k >= V filters nothing)
+ *   filter->top_k  0: no top-k; otherwise 1..128 (a top_k >= V filters nothing)
  *   filter->top_p  in (0, 1]; 1: no nucleus.  With no top-k in front of it the nucleus is the
  *                  shortest prefix that holds top_p of the whole row's softmax mass, and it is
- *                  resolved among the 64 largest logits: a row whose 64 largest logits hold
- *                  less than that gets row_status bit 4 and the 64th largest logit as cutoff
+ *                  resolved among the 128 largest logits: a row whose 128 largest logits hold
+ *                  less than that gets row_status bit 4 and the 128th largest logit as cutoff
  *   filter->s      1..8
  *   temperature > 0
  *   Requests with their own sampling parameters in one batch: filter->top_k_rows, filter->top_p_rows
@@ -239,7 +239,8 @@ difr_status difr_score_both(const void* h, const void* W, const int32_t* tokens,
  * the full estimator and out->cutoff, if given, the cutoff per row (-inf: no
  * filter).  Two passes over the logits: the scoring pass, then a pass that
  * collects, per row, the ids that can be among the s + 2 best or among the top_k
- * logits (about 3 KB of list per row; row_status bit 2 marks a row whose list
+ * logits (6 KB of list per row, or 12 V bytes per row for vocabularies below 16384 ids,
+ * where every id is listed; row_status bit 2 marks a row whose list
  * overflowed, which takes hundreds of logits within rounding of the top_k-th).
  * With s = 1 and no filter the result equals difr_score_gm's up to quadrature
  * error (< 1e-6 in the score).  The first call on a device copies the
@@ -269,8 +270,8 @@ difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* 
  * CDF in vocabulary-id order; a claimed id the filter removed has p = 0 and
  * scores ln(eps).
  *
- *   filter->top_k 1..64 (or >= V when V <= 64), or 0 with top_p < 1: a nucleus over the whole
- *   vocabulary as in difr_score_gm_filtered (row_status bit 4 when it holds more than 64 ids);
+ *   filter->top_k 1..128 (or >= V when V <= 128), or 0 with top_p < 1: a nucleus over the whole
+ *   vocabulary as in difr_score_gm_filtered (row_status bit 4 when it holds more than 128 ids);
  *   filter->top_p in (0, 1]; filter->s is ignored; per-row values as in difr_score_gm_filtered (a
  *   row whose own policy filters nothing keeps the unfiltered score)
  *   temperature > 0; out->workspace needs difr_filtered_workspace_bytes(T, d, V)

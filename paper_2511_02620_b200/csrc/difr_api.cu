@@ -254,15 +254,19 @@ difr_status difr_admissible(const void* h, const void* W, const uint64_t* seeds,
 }
 
 // ------------------------------------------------- full Token-DiFR estimator
-constexpr int kCandCap = 256;      // candidates kept per row when the vocabulary has at least 32 tiles
-constexpr int kFilterMinStrips = 32;
+constexpr int kCandCap = 512;      // candidates kept per row when the vocabulary has at least 64 tiles
+// Each strip contributes its two largest 16-id group maxima, and the k-th largest of those values bounds the row's
+// k-th largest logit from below.  The bound is tight enough to keep the lists short when there are about twice as
+// many values as k, i.e. as many strips as k: between 32 and 128 strips, by the largest top_k the call can meet.
+constexpr int kFilterFloorStrips = 32;
+constexpr int kFilterMinStrips = 64;   // vocabularies with fewer tiles than this list every id instead
 constexpr int kFilterMaxStrips = 128;  // the bounds kernel reads at most 128 strips' records per row
 
 // Layout behind the ordinary workspace: per-row candidate counters, then the candidate lists.
-static bool filtered_layout(int64_t T, int64_t d, int64_t V, int pairs, Plan* pl, int* cap, size_t* count_off,
-                            size_t* list_off, size_t* total) {
-  if (!make_plan(T, d, V, pairs, pl, kFilterMinStrips, kFilterMaxStrips)) return false;
-  // with fewer than 32 vocabulary tiles the strips' maxima cannot bound the top_k-th logit: keep every id
+static bool filtered_layout(int64_t T, int64_t d, int64_t V, int pairs, int min_strips, Plan* pl, int* cap,
+                            size_t* count_off, size_t* list_off, size_t* total) {
+  if (!make_plan(T, d, V, pairs, pl, min_strips, kFilterMaxStrips)) return false;
+  // with fewer than 64 vocabulary tiles the strips' maxima cannot bound the 128-th largest logit: keep every id
   *cap = (pl->n_tiles < kFilterMinStrips) ? (int)V : kCandCap;
   *count_off = (pl->workspace_bytes + 255) & ~(size_t)255;
   *list_off = *count_off + (((size_t)pl->T_pad * sizeof(int) + 255) & ~(size_t)255);
@@ -312,7 +316,8 @@ size_t difr_filtered_workspace_bytes(int64_t T, int64_t d, int64_t V) {
   Plan pl;
   int cap;
   size_t count_off, list_off, total;
-  if (!filtered_layout(T, d, V, info.pairs, &pl, &cap, &count_off, &list_off, &total)) return 0;
+  // sized for the most strips a call can ask for
+  if (!filtered_layout(T, d, V, info.pairs, kFilterMaxStrips, &pl, &cap, &count_off, &list_off, &total)) return 0;
   return total;
 }
 
@@ -335,11 +340,11 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
   const float top_p = filter->top_p;
   const int s_comp = ipt ? 0 : filter->s;  // the IPT estimator has no competitors
   if (!ipt && (filter->s < 1 || filter->s > 8)) return DIFR_ERR_INVALID_ARG;
-  if (filter->top_k_rows == nullptr && (top_k < 0 || (top_k > 64 && top_k < V))) return DIFR_ERR_INVALID_ARG;
+  if (filter->top_k_rows == nullptr && (top_k < 0 || (top_k > 128 && top_k < V))) return DIFR_ERR_INVALID_ARG;
   if (filter->top_p_rows == nullptr && (!(top_p > 0.f) || !(top_p <= 1.f))) return DIFR_ERR_INVALID_ARG;
   // IPT with one policy for every row that filters nothing: that is difr_score_ipt
   if (ipt && filter->top_k_rows == nullptr && filter->top_p_rows == nullptr && (top_k < 1 || top_k >= V) &&
-      top_p >= 1.f && V > 64)
+      top_p >= 1.f && V > 128)
     return DIFR_ERR_INVALID_ARG;
   if ((d % 8) != 0 || V < 2) return DIFR_ERR_SHAPE;
   if (T == 0) return DIFR_OK;
@@ -349,7 +354,17 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
   Plan pl;
   int cap;
   size_t count_off, list_off, total;
-  if (!filtered_layout(T, d, V, info.pairs, &pl, &cap, &count_off, &list_off, &total)) return DIFR_ERR_SHAPE;
+  // the largest number of ids any row resolves by logit rank (a nucleus without a top-k resolves 128)
+  int k_max = 128;
+  if (filter->top_k_rows == nullptr) {
+    const bool whole = top_k < 1 || top_k >= V;
+    if (!whole) k_max = top_k;
+    else if (filter->top_p_rows == nullptr && top_p >= 1.f) k_max = 0;
+  }
+  const int min_strips =
+      k_max < kFilterFloorStrips ? kFilterFloorStrips : (k_max > kFilterMaxStrips ? kFilterMaxStrips : k_max);
+  if (!filtered_layout(T, d, V, info.pairs, min_strips, &pl, &cap, &count_off, &list_off, &total))
+    return DIFR_ERR_SHAPE;
   if (!aligned16(h) || !aligned16(W)) return DIFR_ERR_ALIGN;
   if (!out->workspace || out->workspace_bytes < total) return DIFR_ERR_WORKSPACE;
   if (!aligned16(out->workspace)) return DIFR_ERR_ALIGN;

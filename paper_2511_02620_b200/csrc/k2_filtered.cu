@@ -15,7 +15,8 @@
 namespace difr {
 
 constexpr int kFWarps = 4;
-constexpr int kMaxK = 64;        // top_k limit (the nucleus is resolved inside the top k)
+constexpr int kMaxK = 128;       // top_k limit (the nucleus is resolved inside the top k)
+constexpr int kChunks = kMaxK / 32;  // sorted ranks held per lane
 constexpr int kMaxCand = 10;     // s + 2 with s <= 8
 constexpr int kGlOrder = 16;
 
@@ -98,35 +99,45 @@ __device__ __forceinline__ double row_mass_relative(const FilterParams& p, int r
 
 // The row's k_eff largest logits stand sorted (descending) in sl[].  Returns the rank of the last id the row's
 // nucleus keeps (k_eff - 1 when top_p = 1): the shortest prefix whose softmax mass reaches top_p of the top-k's
-// renormalised mass, or of the whole row's when no top-k stands in front.  e0 / e1: unnormalised masses
-// 2^(c1 (l - l0)) of ranks lane and lane + 32.  Whole warp.
+// renormalised mass, or of the whole row's when no top-k stands in front.  e[c]: unnormalised mass
+// 2^(c1 (l - l0)) of rank 32 c + lane.  Whole warp.
 __device__ __forceinline__ int nucleus_last_rank(const FilterParams& p, const RowPolicy& rp, int row, int lane,
-                                                 const float* sl, int k_eff, double& e0, double& e1,
+                                                 const float* sl, int k_eff, double (&e)[kChunks],
                                                  uint32_t& status_bits) {
   const double c1 = (double)rp.c1, l0 = (double)sl[0];
-  e0 = (lane < k_eff) ? exp2(((double)sl[lane] - l0) * c1) : 0.0;
-  e1 = (lane + 32 < k_eff) ? exp2(((double)sl[lane + 32] - l0) * c1) : 0.0;
+#pragma unroll
+  for (int c = 0; c < kChunks; ++c)
+    e[c] = (32 * c + lane < k_eff) ? exp2(((double)sl[32 * c + lane] - l0) * c1) : 0.0;
   int last = k_eff - 1;
   if (rp.top_p < 1.f) {
-    double c0 = e0, c1s = e1;  // inclusive scans of both halves
+    // inclusive scan over the ranks: inside each chunk of 32 by shuffles, then the chunks' totals carried over
+    double cum[kChunks];
+    double carry = 0.0;
 #pragma unroll
-    for (int m = 1; m < 32; m <<= 1) {
-      const double u0 = __hiloint2double(__shfl_up_sync(0xffffffffu, __double2hiint(c0), m),
-                                         __shfl_up_sync(0xffffffffu, __double2loint(c0), m));
-      const double u1 = __hiloint2double(__shfl_up_sync(0xffffffffu, __double2hiint(c1s), m),
-                                         __shfl_up_sync(0xffffffffu, __double2loint(c1s), m));
-      if (lane >= m) { c0 += u0; c1s += u1; }
+    for (int c = 0; c < kChunks; ++c) {
+      double v = e[c];
+#pragma unroll
+      for (int m = 1; m < 32; m <<= 1) {
+        const double up = __hiloint2double(__shfl_up_sync(0xffffffffu, __double2hiint(v), m),
+                                           __shfl_up_sync(0xffffffffu, __double2loint(v), m));
+        if (lane >= m) v += up;
+      }
+      cum[c] = v + carry;
+      carry = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(cum[c]), 31),
+                               __shfl_sync(0xffffffffu, __double2loint(cum[c]), 31));
     }
-    c1s += __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(c0), 31),
-                            __shfl_sync(0xffffffffu, __double2loint(c0), 31));
-    const double total = __hiloint2double(__shfl_sync(0xffffffffu, __double2hiint(c1s), 31),
-                                          __shfl_sync(0xffffffffu, __double2loint(c1s), 31));
+    const double total = carry;
     const double need = (double)rp.top_p * (rp.nucleus_full ? row_mass_relative(p, row, lane, l0, c1) : total);
-    const unsigned m0 = __ballot_sync(0xffffffffu, lane < k_eff && c0 >= need);
-    const unsigned m1 = __ballot_sync(0xffffffffu, lane + 32 < k_eff && c1s >= need);
-    if (m0) last = __ffs(m0) - 1;
-    else if (m1) last = 32 + __ffs(m1) - 1;
-    else if (rp.nucleus_full && k_eff < p.V) status_bits |= 16u;  // the nucleus holds more ids than were resolved
+    bool found = false;
+#pragma unroll
+    for (int c = 0; c < kChunks; ++c) {
+      const unsigned m = __ballot_sync(0xffffffffu, 32 * c + lane < k_eff && cum[c] >= need);
+      if (!found && m) {
+        last = 32 * c + __ffs(m) - 1;
+        found = true;
+      }
+    }
+    if (!found && rp.nucleus_full && k_eff < p.V) status_bits |= 16u;  // the nucleus holds more ids than were resolved
   }
   return last;
 }
@@ -237,8 +248,8 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
   }
   __syncwarp();
   if (k_eff > 0) {
-    double e0, e1;
-    cut_rank = nucleus_last_rank(p, rp, row, lane, sm_l[warp], k_eff, e0, e1, status_bits);
+    double e[kChunks];
+    cut_rank = nucleus_last_rank(p, rp, row, lane, sm_l[warp], k_eff, e, status_bits);
     // the cutoff is that id's logit: re-evaluated in fp64 like every other logit the score depends on
     cutoff = warp_dot(p.h + (size_t)row * (size_t)p.d, p.W + (size_t)sm_id[warp][cut_rank] * (size_t)p.d, p.d, lane);
   }
@@ -374,16 +385,22 @@ __global__ void __launch_bounds__(kFWarps * 32) ipt_filtered_finalize(const Filt
   const double mu = ((double)x[0] + 0.5) * (1.0 / 4294967296.0);
   double score = log((double)p.eps), pt = CUDART_NAN, a = CUDART_NAN, cutoff = -CUDART_INF;
   if (k_eff > 0) {
-    double e0, e1;  // unnormalised masses of ranks lane and lane + 32
-    const int last = nucleus_last_rank(p, rp, row, lane, sm_l[warp], k_eff, e0, e1, status_bits);
+    double e[kChunks];  // unnormalised masses of ranks 32 c + lane
+    const int last = nucleus_last_rank(p, rp, row, lane, sm_l[warp], k_eff, e, status_bits);
     cutoff = warp_dot(p.h + (size_t)row * (size_t)p.d, p.W + (size_t)sm_id[warp][last] * (size_t)p.d, p.d, lane);
     if (tok_ok) {
       // mass of the kept ids, of those below the claimed id, and whether the claimed id is kept
-      const bool k0 = lane <= last, k1 = lane + 32 <= last;
-      const int id0 = k0 ? sm_id[warp][lane] : -1, id1 = k1 ? sm_id[warp][lane + 32] : -1;
-      double z = (k0 ? e0 : 0.0) + (k1 ? e1 : 0.0);
-      double below = ((k0 && id0 < tok) ? e0 : 0.0) + ((k1 && id1 < tok) ? e1 : 0.0);
-      double mine = ((k0 && id0 == tok) ? e0 : 0.0) + ((k1 && id1 == tok) ? e1 : 0.0);
+      double z = 0.0, below = 0.0, mine = 0.0;
+#pragma unroll
+      for (int c = 0; c < kChunks; ++c) {
+        const int rank = 32 * c + lane;
+        if (rank <= last) {
+          const int id = sm_id[warp][rank];
+          z += e[c];
+          if (id < tok) below += e[c];
+          if (id == tok) mine += e[c];
+        }
+      }
 #pragma unroll
       for (int m = 16; m >= 1; m >>= 1) {
         z += shfl_xor_double(z, m);

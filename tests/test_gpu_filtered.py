@@ -70,10 +70,12 @@ def test_one_competitor_and_no_filter_is_the_plain_estimator():
 
 
 @pytest.mark.parametrize("T,d,V,scale,temperature,sigma,top_k,top_p,s", [
-    (96, 64, 3000, 2.0, 1.0, 0.3, 50, 0.95, 4),     # the paper's sampling setting; every id is a candidate (V < 8192)
+    (96, 64, 3000, 2.0, 1.0, 0.3, 50, 0.95, 4),     # the paper's sampling setting; every id is a candidate (V < 16384)
     (96, 64, 3000, 2.0, 0.7, 0.05, 8, 1.0, 2),      # top-k only, narrow noise
-    (64, 72, 9000, 3.0, 1.0, 0.5, 20, 0.9, 8),      # candidate lists bounded from the first pass (V >= 8192)
-    (64, 72, 9000, 1.0, 1.0, 1.0, 0, 1.0, 8),       # no filter, many competitors, flat logits
+    (64, 72, 20000, 3.0, 1.0, 0.5, 20, 0.9, 8),     # candidate lists bounded from the first pass (V >= 16384)
+    (64, 72, 20000, 1.0, 1.0, 1.0, 0, 1.0, 8),      # no filter, many competitors, flat logits
+    (64, 72, 20000, 3.0, 1.0, 0.3, 100, 0.98, 3),   # a top-k and a nucleus beyond 64 ids
+    (48, 64, 9000, 2.0, 1.0, 0.3, 128, 1.0, 2),     # the largest top-k
     (40, 64, 40, 2.0, 1.0, 0.4, 64, 0.8, 3),        # top_k beyond the vocabulary: the nucleus acts on all of it
     (48, 64, 300000, 3.0, 1.0, 0.3, 50, 0.95, 4),   # more vocabulary tiles than 128 strips of eight: longer strips
 ])
@@ -151,8 +153,9 @@ def test_results_do_not_depend_on_the_order_work_is_handed_out():
 
 @pytest.mark.parametrize("T,d,V,scale,temperature,sigma,top_k,top_p", [
     (96, 64, 3000, 2.0, 1.0, 0.1, 50, 0.95),
-    (80, 72, 9000, 3.0, 0.7, 0.05, 20, 0.9),
-    (64, 64, 9000, 1.0, 1.0, 1.0, 64, 1.0),
+    (80, 72, 20000, 3.0, 0.7, 0.05, 20, 0.9),
+    (64, 64, 20000, 1.0, 1.0, 1.0, 64, 1.0),
+    (64, 64, 50000, 1.0, 1.0, 0.3, 128, 0.9),   # flat logits and the largest top-k: the longest lists
     (40, 64, 40, 2.0, 1.3, 0.2, 64, 0.8),
 ])
 def test_ipt_estimator_under_the_filter_matches_the_oracle(T, d, V, scale, temperature, sigma, top_k, top_p):
@@ -203,29 +206,29 @@ def _nucleus_sizes(h, W, temperature, top_p):
         n = int(np.searchsorted(c, top_p, side="left")) + 1
         sizes.append(n)
         near = [abs(c[n - 1] - top_p)] + ([abs(c[n - 2] - top_p)] if n >= 2 else [])
-        if len(c) >= 64:
-            near.append(abs(c[63] - top_p))
+        if len(c) >= 128:
+            near.append(abs(c[127] - top_p))
         slack.append(min(near))
     return np.array(sizes), np.array(slack)
 
 
 @pytest.mark.parametrize("T,d,V,scale,temperature,sigma,top_p,s", [
-    (96, 72, 9000, 5.0, 1.0, 0.3, 0.9, 4),    # peaked rows: most nuclei hold a handful of ids, some more than 64
-    (96, 64, 3000, 3.5, 0.9, 0.1, 0.85, 2),   # every id is a candidate (V < 8192)
+    (96, 72, 20000, 4.0, 1.0, 0.3, 0.9, 4),   # peaked rows: most nuclei hold a handful of ids, some more than 128
+    (96, 64, 3000, 3.0, 0.9, 0.1, 0.85, 2),   # every id is a candidate (V < 16384)
     (40, 64, 40, 2.0, 1.0, 0.4, 0.8, 3),      # the whole vocabulary is resolved: never flagged
 ])
 def test_nucleus_over_the_whole_vocabulary(T, d, V, scale, temperature, sigma, top_p, s):
-    """top_k = 0 with top_p < 1: the nucleus takes its mass from the whole row.  Rows whose nucleus fits the 64
-    resolved ids agree with the oracle; the others carry row_status bit 4 and the 64th largest logit as cutoff."""
+    """top_k = 0 with top_p < 1: the nucleus takes its mass from the whole row.  Rows whose nucleus fits the 128
+    resolved ids agree with the oracle; the others carry row_status bit 4 and the 128th largest logit as cutoff."""
     h, W, seeds, positions = _small(T, d, V, 71, scale)
     tokens = _claims(h, W, seeds, positions, f32(temperature), 72)
     dev = Device(h, W, seeds, positions)
     sizes, slack = _nucleus_sizes(h, W, f32(temperature), f32(top_p))
     clear = slack > 1e-4                      # the kernel's mass comes from fp32 sums: leave near-ties out
-    fits = sizes <= min(64, V)
-    assert fits.sum() >= 10 and (V <= 64 or (~fits).sum() >= 3)
+    fits = sizes <= min(128, V)
+    assert fits.sum() >= 10 and (V <= 128 or (~fits).sum() >= 3)
     L = oracle.logits(h, W)
-    kth = np.sort(L, axis=1)[:, ::-1][:, min(64, V) - 1]
+    kth = np.sort(L, axis=1)[:, ::-1][:, min(128, V) - 1]
 
     out = _run(dev, tokens, temperature, sigma, 0, top_p, s)
     flagged = (out.row_status.cpu().numpy() & 16) != 0
@@ -263,7 +266,7 @@ def test_one_sampling_policy_per_row():
     h, W, seeds, positions = _small(T, d, V, 81, 4.0)
     tokens = _claims(h, W, seeds, positions, f32(1.0), 82)
     dev = Device(h, W, seeds, positions)
-    policies = [(1.0, 50, 0.95), (0.7, 8, 1.0), (1.3, 0, 0.9), (1.0, 0, 1.0), (0.0, 50, 0.95), (1.0, 70, 0.9),
+    policies = [(1.0, 50, 0.95), (0.7, 8, 1.0), (1.3, 0, 0.9), (1.0, 0, 1.0), (0.0, 50, 0.95), (1.0, 130, 0.9),
                 (1.0, 20, 1.5)]
     valid = [0, 1, 2, 3]
     group = np.arange(T) % len(policies)
