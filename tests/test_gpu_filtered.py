@@ -127,6 +127,12 @@ def test_full_estimator_at_full_size_on_sampled_rows():
     np.testing.assert_allclose(got[rows], want, rtol=0, atol=SCORE_TOL)
     assert np.all(out.row_status.cpu().numpy() == 0)
     assert np.all(np.isfinite(got)) and np.all(got <= 1e-6)
+    # the rank counted by the second pass: the oracle's on the sampled rows, up to logits within rounding of the claim
+    ref_rank = oracle.score_gm(hs, inp.W, tokens[rows], inp.seeds[rows], inp.positions[rows], f32(temperature),
+                               f32(sigma), f32(EPS)).rank
+    got_rank = out.rank.cpu().numpy()
+    assert np.mean(got_rank[rows] == ref_rank) >= 0.9 and np.max(np.abs(got_rank[rows] - ref_rank)) <= 3
+    assert got_rank.min() >= 0 and got_rank.max() < w.V
 
 
 def test_results_do_not_depend_on_the_order_work_is_handed_out():
