@@ -138,3 +138,31 @@ def test_header_is_plain_c():
         inc = os.path.join(ROOT, "include")
         subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-I", inc, path])
         subprocess.check_call(["g++", "-std=c++17", "-Wall", "-Werror", "-fsyntax-only", "-x", "c++", "-I", inc, path])
+
+
+def test_binding_structs_have_the_headers_layout():
+    """The ctypes mirrors of difr_out, difr_filter and difr_seq_stats must place every member where the C compiler
+    places it: a C program prints sizeof and offsetof for each, the binding must agree."""
+    import ctypes
+    import subprocess
+    import tempfile
+
+    structs = {"difr_out": difr._COut, "difr_filter": difr._CFilter}
+    lines = []
+    for cname, cls in structs.items():
+        lines.append(f'printf("{cname} %zu\\n", sizeof({cname}));')
+        for field, _ in cls._fields_:
+            lines.append(f'printf("{cname}.{field} %zu\\n", offsetof({cname}, {field}));')
+    src = ('#include <stddef.h>\n#include <stdio.h>\n#include "difr.h"\nint main(void) {\n' + "\n".join(lines)
+           + '\nprintf("difr_seq_stats %zu\\n", sizeof(difr_seq_stats));\nreturn 0;\n}\n')
+    with tempfile.TemporaryDirectory() as tmp:
+        c_path, exe = os.path.join(tmp, "layout.c"), os.path.join(tmp, "layout")
+        open(c_path, "w").write(src)
+        subprocess.check_call(["gcc", "-std=c99", "-I", os.path.join(ROOT, "include"), "-o", exe, c_path])
+        out = subprocess.check_output([exe], text=True)
+    got = dict(line.split() for line in out.splitlines())
+    for cname, cls in structs.items():
+        assert int(got[cname]) == ctypes.sizeof(cls), cname
+        for field, _ in cls._fields_:
+            assert int(got[f"{cname}.{field}"]) == getattr(cls, field).offset, (cname, field)
+    assert int(got["difr_seq_stats"]) == 16
