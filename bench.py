@@ -198,6 +198,8 @@ def config_dict(w, args):
     in_bytes = 2 * (w.T * w.d + w.V * w.d)
     return {"workload": w.name, "T": w.T, "d": w.d, "V": w.V, "seq_len": w.seq_len, "estimator": "token_difr_gumbel_max",
             "temperature": args.temperature, "sigma": args.sigma, "eps": 1e-12, "tamper_frac": w.tamper_frac,
+            "generator_seeds": {name: wl.stream_seed(w, k) for k, name in
+                                enumerate(("h", "W", "tamper", "seeds", "perturbation"), start=1)},
             "l2": ("inputs larger than L2 (h + W = %.0f MB)" % (in_bytes / 1e6)) if in_bytes > 2 * L2_BYTES
             else "L2 flushed between steps (256 MB write), per-step events"}
 
