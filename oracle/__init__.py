@@ -73,6 +73,10 @@ def lib() -> ctypes.CDLL:
         L.oracle_gm_pi.argtypes = [ctypes.c_double, ctypes.c_double]
         L.oracle_gm_score.restype = ctypes.c_double
         L.oracle_gm_score.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_double]
+        L.oracle_ipt_mass.restype = ctypes.c_double
+        L.oracle_ipt_mass.argtypes = [ctypes.c_double] * 4
+        L.oracle_ipt_score.restype = ctypes.c_double
+        L.oracle_ipt_score.argtypes = [ctypes.c_double] * 5
         L.oracle_philox4x32_10.restype = None
         L.oracle_philox4x32_10.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         L.oracle_logits.restype = ctypes.c_int
@@ -83,6 +87,9 @@ def lib() -> ctypes.CDLL:
         L.oracle_score_gm.argtypes = common + [ctypes.c_void_p, ctypes.POINTER(_GmOut)]
         L.oracle_score_ipt.restype = ctypes.c_int
         L.oracle_score_ipt.argtypes = common + [ctypes.POINTER(_IptOut)]
+        L.oracle_score_both.restype = ctypes.c_int
+        L.oracle_score_both.argtypes = [ctypes.c_void_p] * 6 + [ctypes.c_double] * 4 + [ctypes.c_int64] * 3 + [
+            ctypes.POINTER(_GmOut), ctypes.POINTER(_IptOut)]
         L.oracle_detect.restype = ctypes.c_int
         L.oracle_detect.argtypes = [ctypes.c_void_p, ctypes.c_double, ctypes.c_void_p, ctypes.c_void_p,
                                     ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]
@@ -160,6 +167,14 @@ def gm_pi(A: float, sigma: float) -> float:
 
 def gm_score(A: float, sigma: float, eps: float) -> float:
     return float(lib().oracle_gm_score(A, sigma, eps))
+
+
+def ipt_mass(a: float, b: float, mu: float, sigma: float) -> float:
+    return float(lib().oracle_ipt_mass(a, b, mu, sigma))
+
+
+def ipt_score(a: float, b: float, mu: float, sigma: float, eps: float) -> float:
+    return float(lib().oracle_ipt_score(a, b, mu, sigma, eps))
 
 
 def normal_interval_mass(za: float, zb: float) -> float:
@@ -259,6 +274,31 @@ def score_ipt(h_bits, W_bits, tokens, seeds, positions, temperature, sigma, eps=
     if rc != 0:
         raise RuntimeError(f"oracle_score_ipt failed: {rc}")
     return res
+
+
+def score_both(h_bits, W_bits, tokens_gm, tokens_ipt, seeds, positions, temperature, sigma_gm, sigma_ipt,
+               eps=1e-12):
+    """`score_gm` on tokens_gm and `score_ipt` on tokens_ipt from one evaluation of each row's logits."""
+    T, d = h_bits.shape
+    V = W_bits.shape[0]
+    h_bits = _bf16_bits(h_bits, (T, d))
+    W_bits = _bf16_bits(W_bits, (V, d))
+    tokens_gm, seeds, positions = _row_inputs(tokens_gm, seeds, positions, T)
+    tokens_ipt = np.ascontiguousarray(tokens_ipt, dtype=np.int32)
+    if tokens_ipt.shape != (T,):
+        raise ValueError("tokens_ipt must have shape (T,)")
+    f8 = lambda: np.zeros(T, dtype=np.float64)
+    i4 = lambda: np.zeros(T, dtype=np.int32)
+    gm = GmResult(f8(), f8(), i4(), i4(), f8(), f8(), f8(), f8(), i4(), i4(), np.zeros(T, dtype=np.uint32), f8())
+    ipt = IptResult(f8(), f8(), f8(), f8(), f8(), f8(), i4(), np.zeros(T, dtype=np.uint32))
+    gm_out = _GmOut(*[_p(getattr(gm, name)) for name, _ in _GmOut._fields_])
+    ipt_out = _IptOut(*[_p(getattr(ipt, name)) for name, _ in _IptOut._fields_])
+    rc = lib().oracle_score_both(_p(h_bits), _p(W_bits), _p(tokens_gm), _p(tokens_ipt), _p(seeds), _p(positions),
+                                 float(temperature), float(sigma_gm), float(sigma_ipt), float(eps), T, d, V,
+                                 ctypes.byref(gm_out), ctypes.byref(ipt_out))
+    if rc != 0:
+        raise RuntimeError(f"oracle_score_both failed: {rc}")
+    return gm, ipt
 
 
 def sample_ipt(h_bits, W_bits, seeds, positions, temperature) -> np.ndarray:

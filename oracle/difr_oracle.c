@@ -193,8 +193,67 @@ typedef struct {
   double* top23_margin; /* [T] y_(2) - y_(3); +inf when V < 3                     */
 } oracle_gm_out;
 
-/* noise_id (nullable): vocabulary id v draws the noise of id noise_id[v]; used
- * only by the permutation-invariance check. */
+/* One row of Token-DiFR from its logits.  y[V] is scratch.  noise_id (nullable):
+ * vocabulary id v draws the noise of id noise_id[v]; used only by the
+ * permutation-invariance check. */
+static void gm_row(const double* logit, double* y, int64_t V, int64_t t, uint64_t seed, uint32_t position,
+                   double temperature, double sigma, double eps, const int32_t* noise_id, int64_t r,
+                   oracle_gm_out* out) {
+  uint32_t status = 0;
+  for (int64_t v = 0; v < V; ++v) {
+    uint32_t id = noise_id ? (uint32_t)noise_id[v] : (uint32_t)v;
+    double G = oracle_gumbel_noise(seed, position, id);
+    y[v] = logit[v] + temperature * G;
+    if (!isfinite(logit[v])) status |= 2u;
+  }
+  /* largest and second largest, ties to the lowest id */
+  int64_t i1 = -1, i2 = -1;
+  for (int64_t v = 0; v < V; ++v) {
+    if (i1 < 0 || y[v] > y[i1]) {
+      i2 = i1;
+      i1 = v;
+    } else if (i2 < 0 || y[v] > y[i2]) {
+      i2 = v;
+    }
+  }
+  int in_range = (t >= 0 && t < V);
+  if (!in_range) status |= 1u;
+  double A, score;
+  if (in_range) {
+    int64_t c = (t == i1) ? i2 : i1; /* strongest competitor */
+    A = y[t] - y[c];
+    if (A == 0.0 && t > c) A = -0.0;
+    score = oracle_gm_score(A, sigma, eps);
+  } else {
+    A = -INFINITY;
+    score = log(eps);
+  }
+  if (out->score) out->score[r] = score;
+  if (out->margin) out->margin[r] = A;
+  if (out->argmax) out->argmax[r] = (int32_t)i1;
+  if (out->runner_up) out->runner_up[r] = (int32_t)i2;
+  if (out->top2_margin) out->top2_margin[r] = y[i1] - y[i2];
+  if (out->top23_margin) {
+    double third = -INFINITY;
+    for (int64_t v = 0; v < V; ++v)
+      if (v != i1 && v != i2 && y[v] > third) third = y[v];
+    out->top23_margin[r] = y[i2] - third;
+  }
+  if (out->lse) out->lse[r] = temperature > 0.0 ? log_sum_exp_scaled(logit, V, 1.0 / temperature) : NAN;
+  if (out->y_claimed) out->y_claimed[r] = in_range ? y[t] : NAN;
+  if (out->logit_claimed) out->logit_claimed[r] = in_range ? logit[t] : NAN;
+  if (out->rank) {
+    int32_t rank = (int32_t)V;
+    if (in_range) {
+      rank = 0;
+      for (int64_t v = 0; v < V; ++v) rank += (logit[v] > logit[t]);
+    }
+    out->rank[r] = rank;
+  }
+  if (out->match) out->match[r] = in_range && (t == i1);
+  if (out->row_status) out->row_status[r] = status;
+}
+
 int oracle_score_gm(const uint16_t* h, const uint16_t* W, const int32_t* tokens, const uint64_t* seeds,
                     const uint32_t* positions, double temperature, double sigma, double eps, int64_t T,
                     int64_t d, int64_t V, const int32_t* noise_id, oracle_gm_out* out) {
@@ -215,60 +274,7 @@ int oracle_score_gm(const uint16_t* h, const uint16_t* W, const int32_t* tokens,
 #pragma omp for schedule(dynamic, 1)
       for (int64_t r = 0; r < T; ++r) {
         row_logits(h + r * d, W, d, V, hd, logit);
-        uint32_t status = 0;
-        for (int64_t v = 0; v < V; ++v) {
-          uint32_t id = noise_id ? (uint32_t)noise_id[v] : (uint32_t)v;
-          double G = oracle_gumbel_noise(seeds[r], positions[r], id);
-          y[v] = logit[v] + temperature * G;
-          if (!isfinite(logit[v])) status |= 2u;
-        }
-        /* largest and second largest, ties to the lowest id */
-        int64_t i1 = -1, i2 = -1;
-        for (int64_t v = 0; v < V; ++v) {
-          if (i1 < 0 || y[v] > y[i1]) {
-            i2 = i1;
-            i1 = v;
-          } else if (i2 < 0 || y[v] > y[i2]) {
-            i2 = v;
-          }
-        }
-        int64_t t = tokens[r];
-        int in_range = (t >= 0 && t < V);
-        if (!in_range) status |= 1u;
-        double A, score;
-        if (in_range) {
-          int64_t c = (t == i1) ? i2 : i1; /* strongest competitor */
-          A = y[t] - y[c];
-          if (A == 0.0 && t > c) A = -0.0;
-          score = oracle_gm_score(A, sigma, eps);
-        } else {
-          A = -INFINITY;
-          score = log(eps);
-        }
-        if (out->score) out->score[r] = score;
-        if (out->margin) out->margin[r] = A;
-        if (out->argmax) out->argmax[r] = (int32_t)i1;
-        if (out->runner_up) out->runner_up[r] = (int32_t)i2;
-        if (out->top2_margin) out->top2_margin[r] = y[i1] - y[i2];
-        if (out->top23_margin) {
-          double third = -INFINITY;
-          for (int64_t v = 0; v < V; ++v)
-            if (v != i1 && v != i2 && y[v] > third) third = y[v];
-          out->top23_margin[r] = y[i2] - third;
-        }
-        if (out->lse) out->lse[r] = temperature > 0.0 ? log_sum_exp_scaled(logit, V, 1.0 / temperature) : NAN;
-        if (out->y_claimed) out->y_claimed[r] = in_range ? y[t] : NAN;
-        if (out->logit_claimed) out->logit_claimed[r] = in_range ? logit[t] : NAN;
-        if (out->rank) {
-          int32_t rank = (int32_t)V;
-          if (in_range) {
-            rank = 0;
-            for (int64_t v = 0; v < V; ++v) rank += (logit[v] > logit[t]);
-          }
-          out->rank[r] = rank;
-        }
-        if (out->match) out->match[r] = in_range && (t == i1);
-        if (out->row_status) out->row_status[r] = status;
+        gm_row(logit, y, V, tokens[r], seeds[r], positions[r], temperature, sigma, eps, noise_id, r, out);
       }
     }
     free(hd);
@@ -290,6 +296,58 @@ typedef struct {
   uint32_t* row_status;
 } oracle_ipt_out;
 
+/* Alg. Token-IPT-DiFR's last steps: the Gaussian of width sigma centred on mu,
+ * integrated over the claimed token's CDF interval [a, b], and its log-score. */
+double oracle_ipt_mass(double a, double b, double mu, double sigma) {
+  return normal_interval_mass((a - mu) / sigma, (b - mu) / sigma);
+}
+double oracle_ipt_score(double a, double b, double mu, double sigma, double eps) {
+  return log(oracle_ipt_mass(a, b, mu, sigma) + eps);
+}
+
+/* One row of Token-IPT-DiFR from its logits.  p[V] is scratch. */
+static void ipt_row(const double* logit, double* p, int64_t V, int64_t t, uint64_t seed, uint32_t position,
+                    double temperature, double sigma, double eps, int64_t r, oracle_ipt_out* out) {
+  uint32_t status = 0;
+  for (int64_t v = 0; v < V; ++v)
+    if (!isfinite(logit[v])) status |= 2u;
+  const double inv_temp = 1.0 / temperature;
+  double lse = log_sum_exp_scaled(logit, V, inv_temp);
+  for (int64_t v = 0; v < V; ++v) p[v] = exp(logit[v] * inv_temp - lse);
+  double mu = oracle_ipt_uniform(seed, position);
+  /* the IPT sampler: first id whose cumulative mass exceeds mu */
+  int64_t sampled = V - 1;
+  {
+    double C = 0.0;
+    for (int64_t v = 0; v < V; ++v) {
+      C += p[v];
+      if (C > mu) {
+        sampled = v;
+        break;
+      }
+    }
+  }
+  int in_range = (t >= 0 && t < V);
+  if (!in_range) status |= 1u;
+  double a = NAN, pt = NAN, mass = 0.0, score = log(eps);
+  if (in_range) {
+    a = 0.0;
+    for (int64_t v = 0; v < t; ++v) a += p[v];
+    pt = p[t];
+    double b = a + pt;
+    mass = oracle_ipt_mass(a, b, mu, sigma);
+    score = oracle_ipt_score(a, b, mu, sigma, eps);
+  }
+  if (out->score) out->score[r] = score;
+  if (out->p_claimed) out->p_claimed[r] = pt;
+  if (out->cdf_lo) out->cdf_lo[r] = a;
+  if (out->u) out->u[r] = mu;
+  if (out->lse) out->lse[r] = lse;
+  if (out->mass) out->mass[r] = mass;
+  if (out->sampled) out->sampled[r] = (int32_t)sampled;
+  if (out->row_status) out->row_status[r] = status;
+}
+
 int oracle_score_ipt(const uint16_t* h, const uint16_t* W, const int32_t* tokens, const uint64_t* seeds,
                      const uint32_t* positions, double temperature, double sigma, double eps, int64_t T,
                      int64_t d, int64_t V, oracle_ipt_out* out) {
@@ -310,50 +368,50 @@ int oracle_score_ipt(const uint16_t* h, const uint16_t* W, const int32_t* tokens
 #pragma omp for schedule(dynamic, 1)
       for (int64_t r = 0; r < T; ++r) {
         row_logits(h + r * d, W, d, V, hd, logit);
-        uint32_t status = 0;
-        for (int64_t v = 0; v < V; ++v)
-          if (!isfinite(logit[v])) status |= 2u;
-        const double inv_temp = 1.0 / temperature;
-        double lse = log_sum_exp_scaled(logit, V, inv_temp);
-        for (int64_t v = 0; v < V; ++v) p[v] = exp(logit[v] * inv_temp - lse);
-        double mu = oracle_ipt_uniform(seeds[r], positions[r]);
-        /* the IPT sampler: first id whose cumulative mass exceeds mu */
-        int64_t sampled = V - 1;
-        {
-          double C = 0.0;
-          for (int64_t v = 0; v < V; ++v) {
-            C += p[v];
-            if (C > mu) {
-              sampled = v;
-              break;
-            }
-          }
-        }
-        int64_t t = tokens[r];
-        int in_range = (t >= 0 && t < V);
-        if (!in_range) status |= 1u;
-        double a = NAN, pt = NAN, mass = 0.0, score = log(eps);
-        if (in_range) {
-          a = 0.0;
-          for (int64_t v = 0; v < t; ++v) a += p[v];
-          pt = p[t];
-          double b = a + pt;
-          mass = normal_interval_mass((a - mu) / sigma, (b - mu) / sigma);
-          score = log(mass + eps);
-        }
-        if (out->score) out->score[r] = score;
-        if (out->p_claimed) out->p_claimed[r] = pt;
-        if (out->cdf_lo) out->cdf_lo[r] = a;
-        if (out->u) out->u[r] = mu;
-        if (out->lse) out->lse[r] = lse;
-        if (out->mass) out->mass[r] = mass;
-        if (out->sampled) out->sampled[r] = (int32_t)sampled;
-        if (out->row_status) out->row_status[r] = status;
+        ipt_row(logit, p, V, tokens[r], seeds[r], positions[r], temperature, sigma, eps, r, out);
       }
     }
     free(hd);
     free(logit);
     free(p);
+  }
+  return err ? ORACLE_ERR_MEM : ORACLE_OK;
+}
+
+/* Both estimators from one evaluation of each row's logits: exactly what
+ * oracle_score_gm (claims tokens_gm, width sigma_gm) and oracle_score_ipt (claims
+ * tokens_ipt, width sigma_ipt) would write, row by row.  It exists so that
+ * stored expected values for the large workloads cost one contraction per row
+ * instead of two. */
+int oracle_score_both(const uint16_t* h, const uint16_t* W, const int32_t* tokens_gm, const int32_t* tokens_ipt,
+                      const uint64_t* seeds, const uint32_t* positions, double temperature, double sigma_gm,
+                      double sigma_ipt, double eps, int64_t T, int64_t d, int64_t V, oracle_gm_out* gm,
+                      oracle_ipt_out* ipt) {
+  if (!h || !W || !tokens_gm || !tokens_ipt || !seeds || !positions || !gm || !ipt || T < 0 || d <= 0 || V < 2)
+    return ORACLE_ERR_ARG;
+  if (!(sigma_gm > 0.0) || !(sigma_ipt > 0.0) || !(eps >= 0.0) || !(temperature > 0.0)) return ORACLE_ERR_ARG;
+  int err = 0;
+#pragma omp parallel
+  {
+    double* hd = (double*)malloc((size_t)d * sizeof(double));
+    double* logit = (double*)malloc((size_t)V * sizeof(double));
+    double* scratch = (double*)malloc((size_t)V * sizeof(double));
+    if (!hd || !logit || !scratch) {
+#pragma omp atomic write
+      err = 1;
+    }
+#pragma omp barrier
+    if (!err) {
+#pragma omp for schedule(dynamic, 1)
+      for (int64_t r = 0; r < T; ++r) {
+        row_logits(h + r * d, W, d, V, hd, logit);
+        gm_row(logit, scratch, V, tokens_gm[r], seeds[r], positions[r], temperature, sigma_gm, eps, NULL, r, gm);
+        ipt_row(logit, scratch, V, tokens_ipt[r], seeds[r], positions[r], temperature, sigma_ipt, eps, r, ipt);
+      }
+    }
+    free(hd);
+    free(logit);
+    free(scratch);
   }
   return err ? ORACLE_ERR_MEM : ORACLE_OK;
 }

@@ -34,10 +34,10 @@ MISTAKES = [
      "test_oracle_scores.py", "draws_from_the_temperature_softmax"),
     ("competitor is always the argmax", C, "int64_t c = (t == i1) ? i2 : i1; /* strongest competitor */",
      "int64_t c = i1;", "test_oracle_scores.py", "numpy_replay"),
-    ("ties go to the highest id", C, "if (i1 < 0 || y[v] > y[i1]) {\n            i2 = i1;\n            i1 = v;\n          } else if (i2 < 0 || y[v] > y[i2]) {\n            i2 = v;\n          }\n        }\n        int64_t t = tokens[r];",
-     "if (i1 < 0 || y[v] >= y[i1]) {\n            i2 = i1;\n            i1 = v;\n          } else if (i2 < 0 || y[v] >= y[i2]) {\n            i2 = v;\n          }\n        }\n        int64_t t = tokens[r];",
+    ("ties go to the highest id", C, "if (i1 < 0 || y[v] > y[i1]) {\n      i2 = i1;\n      i1 = v;\n    } else if (i2 < 0 || y[v] > y[i2]) {\n      i2 = v;\n    }\n  }\n  int in_range",
+     "if (i1 < 0 || y[v] >= y[i1]) {\n      i2 = i1;\n      i1 = v;\n    } else if (i2 < 0 || y[v] >= y[i2]) {\n      i2 = v;\n    }\n  }\n  int in_range",
      "test_oracle_scores.py", "exact_ties"),
-    ("margin with the wrong sign", C, "A = y[t] - y[c];\n          if (A == 0.0", "A = y[c] - y[t];\n          if (A == 0.0",
+    ("margin with the wrong sign", C, "A = y[t] - y[c];\n    if (A == 0.0", "A = y[c] - y[t];\n    if (A == 0.0",
      "test_oracle_scores.py", "nonnegative_margin"),
     ("closed form without the square root of two", C, "return std_normal_cdf(A / (sigma * sqrt(2.0)));",
      "return std_normal_cdf(A / sigma);", "test_oracle_scores.py", "sampling_loop_of_the_algorithm"),
@@ -86,7 +86,8 @@ def _mirror(tmp, file=None, old=None, new=None):
     for name in os.listdir(os.path.join(ROOT, "tests")):
         if name == "conftest.py" or name.startswith("test_oracle_"):
             shutil.copy(os.path.join(ROOT, "tests", name), os.path.join(tmp, "tests", name))
-    shutil.copytree(os.path.join(ROOT, "tests", "golden"), os.path.join(tmp, "tests", "golden"))
+    shutil.copytree(os.path.join(ROOT, "tests", "golden"), os.path.join(tmp, "tests", "golden"),
+                    ignore=shutil.ignore_patterns("full_*.npz"))  # stored full-size values: GPU tests only
     if file is not None:
         path = os.path.join(tmp, "oracle", file)
         text = open(path).read()
