@@ -331,9 +331,13 @@ difr_status difr_exfiltratable_bits(const uint8_t* classes, const int32_t* count
  *   scores      float [T]
  *   threshold   tau; a score equal to tau is safe, NaN is flagged
  *   margins     float [T], nullable: rows without a sign bit count as matches
- *   ranks, rank_cutoff   nullable / ignored when NULL: with raw-logit ranks (difr_out.rank) a
- *               flagged row whose rank exceeds the cutoff gets flag 2 (Alg. "Per-Token Risk
- *               Classification via GLS and Rank": 0 safe, 1 suspicious, 2 dangerous)
+ *   ranks, rank_cutoff   nullable / ignored when NULL: with raw-logit ranks (difr_out.rank, counted
+ *               from 0) a flagged row whose claimed token is not among the R = rank_cutoff largest
+ *               logits (rank >= R) gets flag 2 (Alg. "Per-Token Risk Classification via GLS and
+ *               Rank": 0 safe, 1 suspicious, 2 dangerous).  With R = 1 only the top-ranked token
+ *               can be suspicious; a suspicious token is one of R ids, hence log2 R bits
+ *               (appendix "Logit-Rank Ablations").  The algorithm prints the test as rank > R,
+ *               which is this rule for a rank counted from 1.
  *   seq_offsets int32 [n_seq + 1] ascending row offsets, nullable => one sequence [0, T)
  *   flags       uint8 [T], nullable: 0 safe, 1 flagged (suspicious), 2 dangerous
  *   seq_stats   difr_seq_stats [n_seq] (or [1]), nullable

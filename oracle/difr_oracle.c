@@ -453,15 +453,21 @@ int oracle_detect(const double* scores, double threshold, const double* margins,
 
 /* ------------------------------------------------------- risk classes */
 /* Alg. "Per-Token Risk Classification via GLS and Rank": 0 safe if score >= tau;
- * otherwise 2 (dangerous) if the raw-logit rank exceeds R, else 1 (suspicious).
- * A NaN score is not >= tau.  ranks nullable => classes 0/1 only. */
+ * otherwise suspicious (1) if the claimed token is among the R largest raw logits,
+ * else dangerous (2).  `ranks` are 0-based (0 = largest logit, the convention of
+ * the paper's rank histograms), so "among the R largest" is rank < R: with cutoff 1
+ * only the top-ranked token can be suspicious and with cutoff 4 the top four, which
+ * is what makes log2 R the information a suspicious token can carry (appendix
+ * "Logit-Rank Ablations").  The algorithm's printed test "rank > R" is the same rule
+ * for a rank counted from 1.  A NaN score is not >= tau.  ranks nullable => classes
+ * 0/1 only. */
 int oracle_classify(const double* scores, double threshold, const int32_t* ranks, int32_t rank_cutoff, int64_t T,
                     uint8_t* classes) {
   if (!scores || !classes || T < 0) return ORACLE_ERR_ARG;
   for (int64_t r = 0; r < T; ++r) {
     if (scores[r] >= threshold) {
       classes[r] = 0;
-    } else if (ranks && ranks[r] > rank_cutoff) {
+    } else if (ranks && ranks[r] >= rank_cutoff) {
       classes[r] = 2;
     } else {
       classes[r] = 1;

@@ -18,7 +18,7 @@ struct SeqAcc {
 __device__ __forceinline__ void row_update(const K3Params& p, int64_t r, float s, SeqAcc& a) {
   const bool flagged = (s < p.threshold) || isnan(s);
   uint8_t f = flagged ? 1 : 0;
-  if (flagged && p.ranks != nullptr && p.ranks[r] > p.rank_cutoff) f = 2;
+  if (flagged && p.ranks != nullptr && p.ranks[r] >= p.rank_cutoff) f = 2;
   if (p.flags) p.flags[r] = f;
   a.n_flag += flagged;
   if (p.margins) {

@@ -56,8 +56,8 @@ MISTAKES = [
      "test_oracle_scores.py", "brute_force_cdf or follow_the_softmax"),
     ("raw-logit rank counts the claim itself", C, "rank += (logit[v] > logit[t]);", "rank += (logit[v] >= logit[t]);",
      "test_oracle_scores.py", "numpy_replay"),
-    ("dangerous from rank R on", C, "ranks[r] > rank_cutoff", "ranks[r] >= rank_cutoff",
-     "test_oracle_risk.py", "three_classes"),
+    ("suspicious class one id too large", C, "ranks[r] >= rank_cutoff", "ranks[r] > rank_cutoff",
+     "test_oracle_risk.py", "three_classes or rank_cutoff_counts"),
     ("suspicious bits in nats", C, "b = log2((double)rank_cutoff);", "b = log((double)rank_cutoff);",
      "test_oracle_risk.py", "exfiltratable"),
     ("admissible set: the sample is its own competitor", C, "int64_t c = (i == i1) ? i2 : i1;", "int64_t c = i1;",

@@ -26,15 +26,39 @@ def _small(T, d, V, seed):
 
 
 def test_three_classes_follow_the_algorithm_case_by_case():
-    # (score, rank) pairs around tau = -2, R = 3, one of each branch plus the boundaries
+    # (score, rank) pairs around tau = -2, R = 3 (ranks count from 0: the suspicious ids are ranks 0, 1, 2),
+    # one of each branch plus the boundaries
     scores = np.array([-1.0, -2.0, -2.0000001, -5.0, -5.0, -5.0, np.nan, np.nan])
-    ranks = np.array([100, 100, 0, 3, 4, 0, 0, 9], dtype=np.int32)
+    ranks = np.array([100, 100, 0, 2, 3, 0, 0, 9], dtype=np.int32)
     got = oracle.classify(scores, -2.0, ranks, 3)
-    #   safe   safe (equal)  susp.  susp. (rank == R)  danger  susp.  NaN is not >= tau: susp. / danger
+    #   safe   safe (equal)  susp.  susp. (last of the top R)  danger  susp.  NaN is not >= tau: susp. / danger
     assert got.tolist() == [0, 0, 1, 1, 2, 1, 1, 2]
     # without ranks only the threshold acts, exactly like the detection flags
     flags, _ = oracle.detect(scores, -2.0)
     assert np.array_equal(oracle.classify(scores, -2.0), flags)
+
+
+def test_rank_cutoff_counts_ids_the_way_the_ablations_describe():
+    """Appendix "Logit-Rank Ablations": with cutoff 1 only the top-ranked token may be suspicious; with cutoff 4
+    the top four, which is why such a token carries log2(4) = 2 bits.  Worked through on a row of known
+    logits: the flagged claim is moved down the ranking and the suspicious ids are counted."""
+    d, V = 8, 12
+    # h = e_0 and W[v, 0] = -v: logits 0, -1, -2, ... so id v has exactly v larger logits (rank v)
+    h = _bits(np.eye(1, d))
+    W = np.zeros((V, d), dtype=np.float32)
+    W[:, 0] = -np.arange(V)
+    W = _bits(W)
+    seeds, positions = np.array([7], dtype=np.uint64), np.array([1], dtype=np.uint32)
+    ranks = np.array([oracle.score_gm(h, W, np.array([v], dtype=np.int32), seeds, positions, 1.0, 1.0, EPS).rank[0]
+                      for v in range(V)], dtype=np.int32)
+    assert ranks.tolist() == list(range(V))
+    flagged = np.full(V, -30.0)  # every claim fails the threshold
+    for R in (1, 4, 8):
+        classes = oracle.classify(flagged, -2.0, ranks, R)
+        assert (classes == 1).sum() == R  # a suspicious token is one of exactly R ids => log2 R bits
+        assert classes.tolist() == [1] * R + [2] * (V - R)
+    # cutoff 1: the claim holding the second-largest logit is already dangerous
+    assert oracle.classify(flagged[:2], -2.0, ranks[:2], 1).tolist() == [1, 2]
 
 
 @pytest.mark.parametrize("sigma,temperature", [(1.0, 1.0), (0.3, 0.7), (0.05, 1.0)])
