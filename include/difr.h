@@ -17,7 +17,8 @@
  *                pooling), difr_admissible (sizes of the admissible sets), difr_exfiltratable_bits
  *   randomness   difr_expand_seeds (seeds that also depend on the context)
  *   sizes        difr_workspace_bytes, difr_filtered_workspace_bytes
- *   aids         difr_logits, difr_philox, difr_selftest_wait, difr_status_string, difr_version
+ *   aids         difr_logits, difr_philox, difr_selftest_wait, difr_debug_plan_override,
+ *                difr_status_string, difr_version
  *
  * Conventions
  *   - Plain C linkage, no exceptions, no global state visible to the caller.
@@ -243,9 +244,7 @@ difr_status difr_score_both(const void* h, const void* W, const int32_t* tokens,
  * where every id is listed; row_status bit 2 marks a row whose list
  * overflowed, which takes hundreds of logits within rounding of the top_k-th).
  * With s = 1 and no filter the result equals difr_score_gm's up to quadrature
- * error (< 1e-6 in the score).  The first call on a device copies the
- * quadrature nodes (256 bytes) into the library's constant memory with a
- * synchronous cudaMemcpyToSymbol.
+ * error (< 1e-6 in the score).
  */
 typedef struct {
   int32_t top_k;
@@ -396,6 +395,15 @@ difr_status difr_philox(const uint32_t* ctr, const uint32_t* key, int64_t n, uin
  * either way and the context stays usable.
  */
 difr_status difr_selftest_wait(int32_t* status2, int64_t limit_cycles, difr_stream_t stream);
+
+/*
+ * Validation aid: overrides the work planner's choices for every later call of the process (0 = the planner's
+ * own value): the number of vocabulary strips, the number of 256-row tiles per raster group, and the megabytes
+ * of h per raster group the planner aims at.  Results do not depend on these values (tests sweep them to show
+ * it); speed and the workspace size do, so query difr_workspace_bytes again after changing them, and do not
+ * change them while a call is being issued on another thread.  Not meant for production use.
+ */
+difr_status difr_debug_plan_override(int32_t strips, int32_t group, int32_t l2_mb);
 
 const char* difr_status_string(difr_status status); /* host pointer to a static string */
 int difr_version(void);

@@ -21,7 +21,7 @@ STATUS_NAMES = {0: "DIFR_OK", -1: "DIFR_ERR_INVALID_ARG", -2: "DIFR_ERR_SHAPE", 
 EXPORTS = ("difr_workspace_bytes", "difr_filtered_workspace_bytes", "difr_score_gm", "difr_score_ipt",
            "difr_score_both", "difr_score_gm_filtered", "difr_score_ipt_filtered", "difr_score_gm_static",
            "difr_admissible", "difr_exfiltratable_bits", "difr_detect", "difr_expand_seeds", "difr_logits", "difr_philox",
-           "difr_selftest_wait", "difr_status_string", "difr_version")
+           "difr_selftest_wait", "difr_debug_plan_override", "difr_status_string", "difr_version")
 STATIC_SCRATCH_BYTES = 16 << 20  # DIFR_STATIC_SCRATCH_BYTES
 
 
@@ -97,6 +97,8 @@ def lib() -> ctypes.CDLL:
         L.difr_philox.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]
         L.difr_selftest_wait.restype = ctypes.c_int
         L.difr_selftest_wait.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p]
+        L.difr_debug_plan_override.restype = ctypes.c_int
+        L.difr_debug_plan_override.argtypes = [ctypes.c_int32] * 3
         L.difr_status_string.restype = ctypes.c_char_p
         L.difr_status_string.argtypes = [ctypes.c_int]
         L.difr_version.restype = ctypes.c_int
@@ -338,6 +340,13 @@ def difr_selftest_wait(status2, limit_cycles, stream=None):
     if rc != DIFR_OK:
         raise DifrError(rc, "difr_selftest_wait")
     return status2
+
+
+def difr_debug_plan_override(strips: int = 0, group: int = 0, l2_mb: int = 0) -> None:
+    """Validation aid: fixes the planner's strip count / raster group / L2 share for later calls (0: its own)."""
+    rc = lib().difr_debug_plan_override(int(strips), int(group), int(l2_mb))
+    if rc != DIFR_OK:
+        raise DifrError(rc, "difr_debug_plan_override")
 
 
 def difr_philox(ctr, key, out, stream=None):

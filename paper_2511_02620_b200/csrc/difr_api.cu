@@ -8,6 +8,8 @@
 #include <string.h>
 
 #include <atomic>
+#include <mutex>
+#include <vector>
 
 #include "../../include/difr.h"
 #include "difr_kernels.h"
@@ -34,7 +36,7 @@ EncodeTiledFn encode_tiled_fn() {
 }
 
 // bf16 [rows, cols] row-major, box = 64 columns (128 bytes, 128-byte swizzle) x box_rows rows.
-bool make_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows) {
+bool encode_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (fn == nullptr) return false;
   const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
@@ -46,6 +48,40 @@ bool make_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, i
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// A tensor map is a host object that depends on the base address and the shape only (never on the contents), and
+// callers pass the same W, and often the same h buffers, call after call: the encoded maps are remembered in a
+// short most-recently-used list under a mutex.
+bool make_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows) {
+  struct Entry {
+    const void* base;
+    int64_t rows, cols;
+    int box_rows;
+    CUtensorMap map;
+  };
+  constexpr size_t kEntries = 16;
+  static std::mutex mu;
+  static std::vector<Entry> cache;  // most recently used first
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    for (size_t i = 0; i < cache.size(); ++i) {
+      if (cache[i].base == base && cache[i].rows == rows && cache[i].cols == cols && cache[i].box_rows == box_rows) {
+        *map = cache[i].map;
+        if (i != 0) {
+          const Entry hit = cache[i];
+          cache.erase(cache.begin() + (long)i);
+          cache.insert(cache.begin(), hit);
+        }
+        return true;
+      }
+    }
+  }
+  if (!encode_tmap(map, base, rows, cols, box_rows)) return false;
+  std::lock_guard<std::mutex> lock(mu);
+  if (cache.size() >= kEntries) cache.pop_back();
+  cache.insert(cache.begin(), Entry{base, rows, cols, box_rows, *map});
+  return true;
+}
+
 struct DeviceInfo {
   int major;
   int pairs;  // CTA pairs of the fused kernel that are resident at once (0 on other architectures)
@@ -53,23 +89,30 @@ struct DeviceInfo {
 
 bool device_info(DeviceInfo* info) {
   constexpr int kMaxDevices = 64;
-  static std::atomic<int> cached_pairs[kMaxDevices];  // 0: not asked yet (threads that race here store the same value)
+  // 0: not asked yet; otherwise (major << 16) | pairs + 1 (threads that race here store the same value)
+  static std::atomic<int> cached[kMaxDevices];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  const bool slot = dev >= 0 && dev < kMaxDevices;
+  if (slot) {
+    const int c = cached[dev].load(std::memory_order_relaxed);
+    if (c != 0) {
+      info->major = c >> 16;
+      info->pairs = (c & 0xffff) - 1;
+      return true;
+    }
+  }
   if (cudaDeviceGetAttribute(&info->major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return false;
   info->pairs = 0;
-  if (info->major != 10) return true;
-  if (dev >= 0 && dev < kMaxDevices && cached_pairs[dev].load(std::memory_order_relaxed) > 0) {
-    info->pairs = cached_pairs[dev].load(std::memory_order_relaxed);
-    return true;
+  if (info->major == 10) {
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+    int pairs = k1_max_resident_pairs();
+    if (pairs <= 0) return false;
+    if (pairs > sms / 2) pairs = sms / 2;
+    info->pairs = pairs;
   }
-  int sms = 0;
-  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
-  int pairs = k1_max_resident_pairs();
-  if (pairs <= 0) return false;
-  if (pairs > sms / 2) pairs = sms / 2;
-  if (dev >= 0 && dev < kMaxDevices) cached_pairs[dev].store(pairs, std::memory_order_relaxed);
-  info->pairs = pairs;
+  if (slot) cached[dev].store((info->major << 16) | (info->pairs + 1), std::memory_order_relaxed);
   return true;
 }
 
@@ -274,42 +317,6 @@ static bool filtered_layout(int64_t T, int64_t d, int64_t V, int pairs, int min_
   return true;
 }
 
-// Nodes and weights of the n-point Gauss-Legendre rule on [-1, 1]: Newton's iteration on the Legendre
-// polynomial from the Chebyshev-like starting points, weights 2 / ((1 - x^2) P_n'(x)^2).
-static void gauss_legendre(int n, double* x, double* w) {
-  const double pi = 3.14159265358979323846;
-  for (int i = 0; i < n; ++i) {
-    double z = cos(pi * (i + 0.75) / (n + 0.5)), dp = 1.0;
-    for (int it = 0; it < 100; ++it) {
-      double p0 = 1.0, p1 = z;
-      for (int k = 2; k <= n; ++k) {
-        const double pk = ((2.0 * k - 1.0) * z * p1 - (k - 1.0) * p0) / k;
-        p0 = p1;
-        p1 = pk;
-      }
-      dp = n * (z * p1 - p0) / (z * z - 1.0);
-      const double dz = p1 / dp;
-      z -= dz;
-      if (fabs(dz) < 1e-16) break;
-    }
-    x[i] = z;
-    w[i] = 2.0 / ((1.0 - z * z) * dp * dp);
-  }
-}
-
-static difr_status ensure_quadrature_tables() {
-  constexpr int kMaxDevices = 64;
-  static std::atomic<bool> done[kMaxDevices];  // threads that race here copy the same table
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return DIFR_ERR_CUDA;
-  if (dev >= 0 && dev < kMaxDevices && done[dev].load(std::memory_order_acquire)) return DIFR_OK;
-  double x[16], w[16];
-  gauss_legendre(16, x, w);
-  if (set_gauss_legendre(x, w) != cudaSuccess) return DIFR_ERR_CUDA;
-  if (dev >= 0 && dev < kMaxDevices) done[dev].store(true, std::memory_order_release);
-  return DIFR_OK;
-}
-
 size_t difr_filtered_workspace_bytes(int64_t T, int64_t d, int64_t V) {
   DeviceInfo info;
   if (!device_info(&info)) info.pairs = 0;
@@ -368,10 +375,6 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
   if (!aligned16(h) || !aligned16(W)) return DIFR_ERR_ALIGN;
   if (!out->workspace || out->workspace_bytes < total) return DIFR_ERR_WORKSPACE;
   if (!aligned16(out->workspace)) return DIFR_ERR_ALIGN;
-  if (!ipt) {
-    const difr_status qs = ensure_quadrature_tables();
-    if (qs != DIFR_OK) return qs;
-  }
   CUtensorMap tmap_h, tmap_w;
   if (!make_tmap(&tmap_h, h, T, d, kBM) || !make_tmap(&tmap_w, W, V, d, kBN / 2)) return DIFR_ERR_CUDA;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
@@ -534,16 +537,19 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 // to be asked for, once per device, while that device is current.
 static difr_status static_scratch_address(void** ptr) {
   constexpr int kMaxDevices = 64;
-  static void* cached[kMaxDevices] = {nullptr};
+  static std::atomic<void*> cached[kMaxDevices];  // host threads may call concurrently
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return DIFR_ERR_CUDA;
-  if (dev >= 0 && dev < kMaxDevices && cached[dev] != nullptr) {
-    *ptr = cached[dev];
-    return DIFR_OK;
+  if (dev >= 0 && dev < kMaxDevices) {
+    void* known = cached[dev].load(std::memory_order_relaxed);
+    if (known != nullptr) {
+      *ptr = known;
+      return DIFR_OK;
+    }
   }
   void* p = nullptr;
   if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return DIFR_ERR_CUDA;
-  if (dev >= 0 && dev < kMaxDevices) cached[dev] = p;  // same value whichever thread gets here first
+  if (dev >= 0 && dev < kMaxDevices) cached[dev].store(p, std::memory_order_relaxed);  // same value whoever is first
   *ptr = p;
   return DIFR_OK;
 }
@@ -567,6 +573,14 @@ difr_status difr_score_gm_static(const void* h, const void* W, const int32_t* to
   return score_common(0, h, W, tokens, seeds, positions, temperature, T, d, V, &local, stream);
 }
 
+difr_status difr_debug_plan_override(int32_t strips, int32_t group, int32_t l2_mb) {
+  if (strips < 0 || group < 0 || l2_mb < 0) return DIFR_ERR_INVALID_ARG;
+  plan_override_word(0).store(strips, std::memory_order_relaxed);
+  plan_override_word(1).store(group, std::memory_order_relaxed);
+  plan_override_word(2).store(l2_mb, std::memory_order_relaxed);
+  return DIFR_OK;
+}
+
 difr_status difr_selftest_wait(int32_t* status2, int64_t limit_cycles, difr_stream_t stream) {
   if (!status2 || limit_cycles < 1 || limit_cycles > 1000000000LL) return DIFR_ERR_INVALID_ARG;
   if (launch_wait_selftest(status2, (long long)limit_cycles, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
@@ -588,6 +602,6 @@ const char* difr_status_string(difr_status status) {
   return "unknown status";
 }
 
-int difr_version(void) { return 210; }
+int difr_version(void) { return 220; }
 
 }  // extern "C"

@@ -130,7 +130,6 @@ struct FilterParams {
   float* cdf_lo;
   float* u;
 };
-cudaError_t set_gauss_legendre(const double* x, const double* w);  // 16 nodes / weights on [-1, 1]
 cudaError_t launch_filter_bounds(const FilterParams& p, cudaStream_t stream);
 cudaError_t launch_filtered_finalize(const FilterParams& p, cudaStream_t stream);
 cudaError_t launch_ipt_filtered_finalize(const FilterParams& p, cudaStream_t stream);

@@ -4,9 +4,10 @@
 #pragma once
 #include <stddef.h>
 #include <stdint.h>
-#include <stdlib.h>
 
+#include <atomic>
 #include <functional>
+#include <mutex>
 #include <queue>
 #include <vector>
 
@@ -31,9 +32,23 @@ struct Plan {
   size_t workspace_bytes;
 };
 
-inline int env_int(const char* name, int fallback) {
-  const char* v = getenv(name);
-  return (v && *v) ? atoi(v) : fallback;
+// Overrides of the planner's choices, for validation sweeps only (difr_debug_plan_override): 0 = the planner's own
+// value.  Process-wide; part of the plan cache's key.
+struct PlanOverride {
+  int strips;    // number of vocabulary strips S
+  int group;     // row tiles per raster group Gm
+  int l2_mb;     // megabytes of h per raster group that the planner aims at (default 40)
+};
+inline std::atomic<int>& plan_override_word(int i) {
+  static std::atomic<int> words[3];
+  return words[i];
+}
+inline PlanOverride plan_override() {
+  PlanOverride o;
+  o.strips = plan_override_word(0).load(std::memory_order_relaxed);
+  o.group = plan_override_word(1).load(std::memory_order_relaxed);
+  o.l2_mb = plan_override_word(2).load(std::memory_order_relaxed);
+  return o;
 }
 
 // Tile times until the last pair is done when the units (in raster order, each as long as its strip, plus
@@ -68,8 +83,8 @@ inline double makespan_tiles(int m_tiles, int n_tiles, int S, int gm, int num_pa
 // `num_pairs` is the number of CTA pairs resident at once (one persistent pair per two SMs).
 // `min_strips` > 0 asks for at least that many strips (fewer only if there are fewer vocabulary tiles),
 // `max_strips` > 0 for at most that many (the strips grow longer instead).
-inline bool make_plan(int64_t T, int64_t d, int64_t V, int num_pairs, Plan* out, int min_strips = 0,
-                      int max_strips = 0) {
+inline bool compute_plan(int64_t T, int64_t d, int64_t V, int num_pairs, Plan* out, int min_strips, int max_strips,
+                         const PlanOverride& ov) {
   if (T <= 0 || d <= 0 || V < 2 || (d % 8) != 0) return false;
   // (tile origins n * 256 and row origins m * 256 are 32-bit in the kernels: leave room for the last tile's padding)
   if (T > (int64_t)1 << 30 || V > ((int64_t)1 << 31) - 1024 || d > (int64_t)1 << 20) return false;
@@ -81,7 +96,7 @@ inline bool make_plan(int64_t T, int64_t d, int64_t V, int num_pairs, Plan* out,
   // Measured on B200 (126 MB of L2): DRAM traffic is lowest with about 40 MB of h per raster group
   // and strips of about eight tiles; larger groups push W out of L2 before its strip is done with it.
   const double tile_bytes = 2.0 * kPairM * (double)d;  // one 256-row tile of h or of W
-  const double group_bytes = (double)env_int("DIFR_DEBUG_L2_MB", 40) * 1048576.0;
+  const double group_bytes = (double)(ov.l2_mb > 0 ? ov.l2_mb : 40) * 1048576.0;
   int gm = (int)(group_bytes / tile_bytes);
   if (gm < 4) gm = 4;
   int len_target = 8;
@@ -107,10 +122,10 @@ inline bool make_plan(int64_t T, int64_t d, int64_t V, int num_pairs, Plan* out,
   }
   if (best_S < min_strips) best_S = min_strips;
   if (max_strips > 0 && best_S > max_strips) best_S = max_strips;
-  p.S = env_int("DIFR_DEBUG_STRIPS", best_S);
+  p.S = ov.strips > 0 ? ov.strips : best_S;
   if (p.S < 1) p.S = 1;
   if (p.S > p.n_tiles) p.S = p.n_tiles;
-  gm = env_int("DIFR_DEBUG_GROUP", gm);
+  if (ov.group > 0) gm = ov.group;
   if (gm < 1) gm = 1;
   p.Gm = gm < p.m_tiles ? gm : p.m_tiles;
   if ((long long)p.m_tiles * p.S > 0x7fffffffLL) return false;  // unit ids are 32-bit
@@ -120,6 +135,49 @@ inline bool make_plan(int64_t T, int64_t d, int64_t V, int num_pairs, Plan* out,
   p.partial_bytes = (size_t)p.n_slots * (size_t)p.T_pad * 32;
   p.bounds_offset = p.partial_bytes + 256;
   p.workspace_bytes = p.bounds_offset + (size_t)4 * (size_t)p.T_pad * sizeof(float);
+  *out = p;
+  return true;
+}
+
+// The plan of a problem, remembered: small problems pick their strip count by simulating the on-demand schedule
+// for a few dozen candidates, which costs about a millisecond of host time, and callers score the same shapes
+// over and over.  A short most-recently-used list under a mutex (a hit costs a lock and a few compares).
+inline bool make_plan(int64_t T, int64_t d, int64_t V, int num_pairs, Plan* out, int min_strips = 0,
+                      int max_strips = 0) {
+  struct Entry {
+    int64_t T, d, V;
+    int pairs, min_strips, max_strips;
+    PlanOverride ov;
+    Plan plan;
+  };
+  constexpr size_t kEntries = 32;
+  static std::mutex mu;
+  static std::vector<Entry> cache;  // most recently used first
+  const PlanOverride ov = plan_override();
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    for (size_t i = 0; i < cache.size(); ++i) {
+      const Entry& e = cache[i];
+      if (e.T == T && e.d == d && e.V == V && e.pairs == num_pairs && e.min_strips == min_strips &&
+          e.max_strips == max_strips && e.ov.strips == ov.strips && e.ov.group == ov.group &&
+          e.ov.l2_mb == ov.l2_mb) {
+        *out = e.plan;
+        if (i != 0) {
+          const Entry hit = e;
+          cache.erase(cache.begin() + (long)i);
+          cache.insert(cache.begin(), hit);
+        }
+        return true;
+      }
+    }
+  }
+  Plan p;
+  if (!compute_plan(T, d, V, num_pairs, &p, min_strips, max_strips, ov)) return false;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (cache.size() >= kEntries) cache.pop_back();
+    cache.insert(cache.begin(), Entry{T, d, V, num_pairs, min_strips, max_strips, ov, p});
+  }
   *out = p;
   return true;
 }

@@ -20,8 +20,18 @@ constexpr int kChunks = kMaxK / 32;  // sorted ranks held per lane
 constexpr int kMaxCand = 10;     // s + 2 with s <= 8
 constexpr int kGlOrder = 16;
 
-__constant__ double c_gl_x[kGlOrder];
-__constant__ double c_gl_w[kGlOrder];
+// Nodes and weights of the 16-point Gauss-Legendre rule on [-1, 1] (roots of the Legendre polynomial P_16,
+// weights 2 / ((1 - x^2) P_16'(x)^2)), to double precision.
+__constant__ double c_gl_x[kGlOrder] = {
+    -0.98940093499164994, -0.9445750230732326,  -0.86563120238783176, -0.755404408355003,
+    -0.61787624440264377, -0.45801677765722737, -0.28160355077925892, -0.095012509837637441,
+    0.095012509837637441, 0.28160355077925892,  0.45801677765722737,  0.61787624440264377,
+    0.755404408355003,    0.86563120238783176,  0.9445750230732326,   0.98940093499164994};
+__constant__ double c_gl_w[kGlOrder] = {
+    0.027152459411754176, 0.062253523938647456, 0.095158511682492605, 0.12462897125553407,
+    0.14959598881657671,  0.16915651939500265,  0.18260341504492364,  0.18945061045506864,
+    0.18945061045506864,  0.18260341504492364,  0.16915651939500265,  0.14959598881657671,
+    0.12462897125553407,  0.095158511682492605, 0.062253523938647456, 0.027152459411754176};
 
 // n-th largest (n >= 1) of the values the warp holds, eight per lane; -inf when there are fewer than n.
 __device__ __forceinline__ float warp_nth_largest(float (&v)[8], int n, int lane) {
@@ -431,12 +441,6 @@ __global__ void __launch_bounds__(kFWarps * 32) ipt_filtered_finalize(const Filt
 cudaError_t launch_ipt_filtered_finalize(const FilterParams& p, cudaStream_t stream) {
   ipt_filtered_finalize<<<(p.T + kFWarps - 1) / kFWarps, kFWarps * 32, 0, stream>>>(p);
   return cudaGetLastError();
-}
-
-cudaError_t set_gauss_legendre(const double* x, const double* w) {
-  cudaError_t e = cudaMemcpyToSymbol(c_gl_x, x, sizeof(double) * kGlOrder);
-  if (e != cudaSuccess) return e;
-  return cudaMemcpyToSymbol(c_gl_w, w, sizeof(double) * kGlOrder);
 }
 
 cudaError_t launch_filter_bounds(const FilterParams& p, cudaStream_t stream) {

@@ -1,8 +1,9 @@
 // K2: split-V finalize.  One warp per row merges the row's partial records with
 // warp shuffles, re-evaluates in fp64 the few logits the score depends on (the
-// claimed token and the two Gumbel-max candidates: three gathered rows of W
-// against the row of h), re-ranks them, and turns the margin (Token-DiFR) or the
-// CDF interval (Token-IPT-DiFR) into the log-score.
+// claimed token and every Gumbel-max candidate whose key lies within the fused
+// kernel's ranking noise of the second largest: gathered rows of W against the
+// row of h), ranks them exactly, and turns the margin (Token-DiFR) or the CDF
+// interval (Token-IPT-DiFR) into the log-score.
 #include <cuda_runtime.h>
 #include <math_constants.h>
 
@@ -118,57 +119,72 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
   if (temp_bad) status |= 8u;
   const double lse = (temp_f > 0.f) ? (acc.lmax + log2(acc.lsum)) * ln2 : CUDART_NAN;
 
-  // the exact logits of the claimed token and (Token-DiFR) of the two candidates, in one pass over h's row
-  const int c1 = (p.ipt != 1 && acc.i1 >= 0 && acc.i1 < p.V) ? acc.i1 : -1;
-  const int c2 = (p.ipt != 1 && acc.i2 >= 0 && acc.i2 < p.V) ? acc.i2 : -1;
-  double l_exact[3];
-  warp_dot3(hrow, tok_ok ? p.W + (size_t)tok * (size_t)p.d : nullptr,
-            c1 >= 0 ? p.W + (size_t)c1 * (size_t)p.d : nullptr,
-            c2 >= 0 ? p.W + (size_t)c2 * (size_t)p.d : nullptr, p.d, lane, l_exact);
-  const double l_tok = l_exact[0];
+  // the exact logit of the claimed token
+  double l_tok = 0.0;
+  if (tok_ok) l_tok = warp_dot(hrow, p.W + (size_t)tok * (size_t)p.d, p.d, lane);
 
   if (p.ipt != 1) {
-    // ---- Token-DiFR: exact y = l + Temp * G for the claimed token and the two candidates
-    double y1 = -CUDART_INF, y2 = -CUDART_INF, yt = -CUDART_INF;
-    if (c1 >= 0) y1 = l_exact[1] + temp * gumbel_exact(seed, pos, c1);
-    if (c2 >= 0) y2 = l_exact[2] + temp * gumbel_exact(seed, pos, c2);
-    if (tok_ok) yt = l_tok + temp * gumbel_exact(seed, pos, (uint32_t)tok);
-    if (lane == 0) {
-      // order the two candidates exactly (ties: lowest id)
-      int a = c1, b = c2;
-      double ya = y1, yb = y2;
-      if (b >= 0 && (a < 0 || yb > ya || (yb == ya && b < a))) {
-        int ti = a; a = b; b = ti;
-        double tv = ya; ya = yb; yb = tv;
+    // ---- Token-DiFR: exact y = l + Temp * G of the claimed token and of every candidate that can be among the
+    // two largest.  The fused kernel ranks by fp32 keys whose error (tensor-core accumulation, lg2.approx in the
+    // noise, the index bits in the low mantissa) is bounded by `noise`; an id whose exact y is among the two
+    // largest has a key within 2 * noise of the second largest key, so every candidate of the strips' records
+    // inside that window is re-evaluated in fp64 and the two largest are taken exactly (ties: lowest id).
+    const float noise = 3e-4f * temp_f + 1e-4f + 3.9e-6f * fabsf(acc.m2);
+    const float window = acc.m2 - 2.f * noise;  // -inf when there is no second candidate: everything qualifies
+    double yb1 = -CUDART_INF, yb2 = -CUDART_INF;
+    int ib1 = -1, ib2 = -1;
+    auto place = [&](double y, int id) {
+      if (ib1 < 0 || y > yb1 || (y == yb1 && id < ib1)) {
+        yb2 = yb1; ib2 = ib1;
+        yb1 = y; ib1 = id;
+      } else if (ib2 < 0 || y > yb2 || (y == yb2 && id < ib2)) {
+        yb2 = y; ib2 = id;
       }
-      int best = a, second = b;
-      double ybest = ya, ysecond = yb;
+    };
+    double yt = -CUDART_INF;
+    if (tok_ok) {
+      yt = l_tok + temp * gumbel_exact(seed, pos, (uint32_t)tok);
+      place(yt, tok);
+    }
+    for (int base = 0; base < p.n_slots; base += 32) {
+      const int slot = base + lane;
+      float4 a = make_float4(-CUDART_INF_F, __int_as_float(-1), -CUDART_INF_F, __int_as_float(-1));
+      if (slot < p.n_slots) a = *reinterpret_cast<const float4*>(p.partials + (size_t)slot * (size_t)p.T_pad + row);
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const float key = e ? a.z : a.x;
+        const int id = __float_as_int(e ? a.w : a.y);
+        unsigned todo = __ballot_sync(0xffffffffu, id >= 0 && id < p.V && id != tok && !(key < window));
+        while (todo) {
+          const int src = __ffs(todo) - 1;
+          todo &= todo - 1;
+          const int cid = __shfl_sync(0xffffffffu, id, src);
+          const double l = warp_dot(hrow, p.W + (size_t)cid * (size_t)p.d, p.d, lane);
+          place(l + temp * gumbel_exact(seed, pos, (uint32_t)cid), cid);
+        }
+      }
+    }
+    if (lane == 0) {
       double A = -CUDART_INF;
       if (tok_ok) {
-        // strongest competitor: the best candidate that is not the claimed token
-        const int c = (a != tok) ? a : b;
-        const double yc = (a != tok) ? ya : yb;
+        // strongest competitor: the best id that is not the claimed token
+        const int c = (ib1 != tok) ? ib1 : ib2;
+        const double yc = (ib1 != tok) ? yb1 : yb2;
         A = (c >= 0) ? yt - yc : CUDART_INF;
         if (A == 0.0 && tok > c) A = -0.0;
-        const bool tok_first = (c < 0) || (yt > yc) || (yt == yc && tok < c);
-        if (tok != a && tok != b) {
-          // the claimed token was not among the candidates: place it
-          if (tok_first) { second = a; ysecond = ya; best = tok; ybest = yt; }
-          else if (b < 0 || yt > yb || (yt == yb && tok < b)) { second = tok; ysecond = yt; }
-        }
       }
       const double pi = 0.5 * erfc(-A / (2.0 * sigma));  // Phi(A / (sigma sqrt 2))
       double score = tok_ok ? log(pi + eps) : log(eps);
       if (temp_bad || !lse_finite) score = CUDART_NAN;  // a row with a non-finite logit is never scored as safe
       p.score[row] = (float)score;
       if (p.margin) p.margin[row] = (float)A;
-      if (p.argmax) p.argmax[row] = best;
-      if (p.runner_up) p.runner_up[row] = second;
+      if (p.argmax) p.argmax[row] = ib1;
+      if (p.runner_up) p.runner_up[row] = ib2;
       if (p.lse) p.lse[row] = (float)lse;
       if (p.row_status) p.row_status[row] = status;
       if (p.rank) p.rank[row] = tok_ok ? acc.larger : p.V;
-      if (p.y_max) p.y_max[row] = (float)ybest;
-      if (p.y_second) p.y_second[row] = (float)ysecond;
+      if (p.y_max) p.y_max[row] = (float)yb1;
+      if (p.y_second) p.y_second[row] = (float)yb2;
     }
   }
   if (p.ipt != 0) {

@@ -166,3 +166,59 @@ def test_binding_structs_have_the_headers_layout():
         for field, _ in cls._fields_:
             assert int(got[f"{cname}.{field}"]) == getattr(cls, field).offset, (cname, field)
     assert int(got["difr_seq_stats"]) == 16
+
+
+def test_planning_is_remembered():
+    """The work plan of a shape is computed once (small problems simulate their schedule for a few dozen strip
+    counts, about a millisecond each time) and then looked up: a thousand repeated size queries take a few
+    milliseconds in all, and an explicit override of the planner takes effect at once and is undone at once."""
+    import time
+
+    shape = (16384, 4096, 128256)
+    first = difr.difr_workspace_bytes(*shape)
+    t0 = time.perf_counter()
+    for _ in range(1000):
+        assert difr.difr_workspace_bytes(*shape) == first
+    assert time.perf_counter() - t0 < 0.02  # 20 us per call, most of it the ctypes call itself
+    # llama3b-sized problems take the slow planning path (few rounds of work units)
+    t0 = time.perf_counter()
+    for _ in range(200):
+        difr.difr_workspace_bytes(4096, 3072, 128256)
+    assert time.perf_counter() - t0 < 0.02
+    try:
+        difr.difr_debug_plan_override(7, 0, 0)
+        T_pad = 16384
+        assert difr.difr_workspace_bytes(*shape) == 7 * 32 * T_pad + 256 + 16 * T_pad
+    finally:
+        difr.difr_debug_plan_override()
+    assert difr.difr_workspace_bytes(*shape) == first
+    with pytest.raises(difr.DifrError):
+        difr.difr_debug_plan_override(-1)
+
+
+def test_a_well_formed_call_without_a_device_reports_a_cuda_error():
+    """The host-side failure path: every argument is acceptable, but the CUDA runtime cannot give a device
+    (none is visible here), so the call returns DIFR_ERR_CUDA before anything is launched.  Runs in a child
+    process with the devices hidden, so it means the same on a machine that has GPUs."""
+    import subprocess
+    import sys
+
+    code = r'''
+import ctypes, sys
+sys.path.insert(0, %r)
+import paper_2511_02620_b200 as difr
+L = difr.lib()
+p = ctypes.c_void_p(0x10000)
+o = difr._COut()
+o.sigma, o.eps, o.score, o.workspace, o.workspace_bytes = 0.3, 1e-12, 0x10000, 0x10000, 1 << 40
+rc = [L.difr_score_gm(p, p, p, p, p, 1.0, 128, 64, 1000, ctypes.byref(o), None),
+      L.difr_score_ipt(p, p, p, p, p, 1.0, 128, 64, 1000, ctypes.byref(o), None),
+      L.difr_score_gm_static(p, p, p, p, p, 1.0, 128, 64, 1000, ctypes.byref(o), None),
+      L.difr_logits(p, p, 128, 64, 1000, p, None, None)]
+print(rc, difr.difr_status_string(rc[0]))
+sys.exit(0 if rc == [-5, -5, -5, -5] else 1)
+''' % ROOT
+    env = dict(os.environ, CUDA_VISIBLE_DEVICES="")
+    r = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stdout + r.stderr
+    assert "CUDA call failed" in r.stdout

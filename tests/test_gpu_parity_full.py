@@ -1,8 +1,8 @@
-"""Parity at the full sizes of the five workloads, in the launch configuration
-the benchmark times: the GPU scores every row, the oracle re-scores a seeded
-sample of rows one by one (its honest claims come from its own sampler on the
-server-side hidden states), and properties that hold at any size are checked on
-all rows."""
+"""The widened calls (raw-logit rank, both estimators in one pass, admissible sets) at
+full size, in the launch configuration the benchmark times: the oracle re-scores a
+seeded sample of rows one by one, and properties that hold at any size are checked
+on all rows.  (The two estimators themselves are compared row by row with stored
+oracle values in test_gpu_golden_full.py.)"""
 import numpy as np
 import pytest
 import torch
@@ -20,15 +20,6 @@ LSE_RTOL = 1e-3
 ARGMAX_MARGIN = 1e-3
 EPS = 1e-12
 N_SAMPLE = 48
-
-CASES = [
-    ("llama3b", 0, 0.7, 0.05),
-    ("llama3b", 0, 1.0, 1.0),
-    ("llama8b", 0, 1.0, 0.05),
-    ("moe30b", 0, 0.7, 0.05),
-    ("longstream", 4096, 1.0, 0.05),
-    ("longstream", 131072, 1.0, 1.0),
-]
 
 _cache = {}
 
@@ -60,78 +51,6 @@ def _sampled_claims(w, inp, rows, temperature, kind):
     rnd = g.integers(0, w.V, size=len(rows))
     claims[k % 6 == 4] = rnd[k % 6 == 4]
     return claims.astype(np.int32)
-
-
-def _threshold_in_a_gap(scores, quantile=0.3, min_gap=2e-2):
-    s = np.sort(scores)
-    gaps = np.diff(s)
-    ok = np.nonzero(gaps >= min_gap)[0]
-    assert len(ok), "no gap wide enough for an unambiguous threshold"
-    i = ok[np.argmin(np.abs(ok - quantile * len(s)))]
-    return float(np.float32(0.5 * (s[i] + s[i + 1])))
-
-
-@pytest.mark.parametrize("name,T,temperature,sigma", CASES)
-def test_full_size_gm(name, T, temperature, sigma):
-    w, inp, dev = _inputs(name, T)
-    rows = wl.sample_rows(w, N_SAMPLE)
-    g = np.random.default_rng(wl.stream_seed(w, 7))
-    tokens = g.integers(0, w.V, size=w.T).astype(np.int32)
-    tokens[rows] = _sampled_claims(w, inp, rows, f32(temperature), "gm")
-    got = dev.score("gm", tokens, temperature, sigma, EPS)
-    ref = oracle.score_gm(np.ascontiguousarray(inp.h[rows]), inp.W, tokens[rows], inp.seeds[rows],
-                          inp.positions[rows], f32(temperature), f32(sigma), f32(EPS))
-    np.testing.assert_allclose(got["score"][rows], ref.score, rtol=0, atol=SCORE_TOL)
-    np.testing.assert_allclose(got["margin"][rows], ref.margin, rtol=0, atol=1e-4)
-    clear = ref.top2_margin >= ARGMAX_MARGIN
-    assert np.array_equal(got["argmax"][rows][clear], ref.argmax[clear])
-    clear2 = clear & (ref.top23_margin >= ARGMAX_MARGIN)
-    assert np.array_equal(got["runner_up"][rows][clear2], ref.runner_up[clear2])
-    np.testing.assert_allclose(got["lse"][rows], ref.lse, rtol=LSE_RTOL)
-    # every row: well-formed outputs and the exact-match bookkeeping
-    assert np.all(got["row_status"] == 0)
-    assert np.all(np.isfinite(got["score"])) and np.all(got["score"] <= 1e-6)
-    assert np.all((got["argmax"] >= 0) & (got["argmax"] < w.V) & (got["runner_up"] >= 0) & (got["runner_up"] < w.V))
-    assert np.all(got["argmax"] != got["runner_up"])
-    assert np.array_equal(got["argmax"] == tokens, ~np.signbit(got["margin"]))
-    # most honest claims of the sample match even though the server saw perturbed hidden states
-    honest_rows = np.arange(len(rows)) % 6 != 1
-    honest_rows &= np.arange(len(rows)) % 6 != 4
-    assert ref.match[honest_rows].mean() > 0.8
-    # detection decisions on the sample, threshold placed in a gap of the oracle's scores
-    tau = _threshold_in_a_gap(ref.score)
-    ref_flags, _ = oracle.detect(ref.score, tau, ref.margin, None)
-    flags = torch.empty(w.T, dtype=torch.uint8, device="cuda")
-    stats = torch.zeros((len(inp.seq_offsets) - 1, 4), dtype=torch.int32, device="cuda")
-    difr.difr_detect(to_dev(got["score"]), tau, to_dev(got["margin"]), None, 0, to_dev(inp.seq_offsets), flags, stats)
-    torch.cuda.synchronize()
-    f = flags.cpu().numpy()
-    assert np.array_equal(f[rows], ref_flags)
-    st = stats.cpu().numpy().view(SEQ_STATS_DTYPE).reshape(-1)
-    assert st["n_flagged"].sum() == f.sum()
-    assert st["n_match"].sum() == (got["argmax"] == tokens).sum()
-    per_seq = got["score"].reshape(-1, w.seq_len)
-    np.testing.assert_allclose(st["sum"], per_seq.astype(np.float64).sum(axis=1), rtol=1e-4)
-    assert np.array_equal(st["min"], per_seq.min(axis=1))
-
-
-@pytest.mark.parametrize("name,T,temperature,sigma", [("llama3b", 0, 1.0, 1.0), ("moe30b", 0, 0.7, 0.05)])
-def test_full_size_ipt(name, T, temperature, sigma):
-    w, inp, dev = _inputs(name, T)
-    rows = wl.sample_rows(w, N_SAMPLE, salt=1)
-    g = np.random.default_rng(wl.stream_seed(w, 8))
-    tokens = g.integers(0, w.V, size=w.T).astype(np.int32)
-    tokens[rows] = _sampled_claims(w, inp, rows, f32(temperature), "ipt")
-    got = dev.score("ipt", tokens, temperature, sigma, EPS)
-    ref = oracle.score_ipt(np.ascontiguousarray(inp.h[rows]), inp.W, tokens[rows], inp.seeds[rows],
-                           inp.positions[rows], f32(temperature), f32(sigma), f32(EPS))
-    np.testing.assert_allclose(got["score"][rows], ref.score, rtol=0, atol=SCORE_TOL)
-    np.testing.assert_allclose(got["lse"][rows], ref.lse, rtol=LSE_RTOL)
-    np.testing.assert_allclose(got["cdf_lo"][rows], ref.cdf_lo, rtol=0, atol=2e-6)
-    np.testing.assert_allclose(got["p_claimed"][rows], ref.p_claimed, rtol=1e-3, atol=1e-12)
-    assert np.all(got["row_status"] == 0)
-    assert np.all((got["cdf_lo"] >= -1e-6) & (got["cdf_lo"] <= 1 + 1e-6))
-    assert np.all((got["u"] > 0) & (got["u"] < 1))
 
 
 @pytest.mark.parametrize("name,T,temperature,sigma", [("llama3b", 0, 1.0, 1.0), ("moe30b", 0, 0.7, 0.3)])
