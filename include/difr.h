@@ -95,7 +95,9 @@ typedef struct {
                            scores of such a row are NaN, which difr_detect flags);
                            bit2: candidate list overflow (difr_score_gm_filtered);
                            bit3: unusable per-row temperature or filter values; bit4: the nucleus holds more
-                           ids than the filtered calls resolve (128)                       */
+                           ids than the filtered calls resolve (128); bit5: more than 64 ids lie within
+                           fp32 rounding of the claimed logit (rank) or of a bound (difr_admissible):
+                           the integer leaves the unlisted ones out                           */
   void* workspace;      /* >= difr_workspace_bytes(T, d, V) bytes, 16-byte aligned;
                            contents are scratch, overwritten by every call         */
   size_t workspace_bytes;
@@ -107,10 +109,11 @@ typedef struct {
   /* -- members added in version 200; zero them when unused -- */
   int32_t* rank;     /* GM, optional: raw-logit rank of the claimed token, #{v != t* : l_v > l_t*}
                         (0 = largest logit; V for an out-of-range claim), Sec. "Problems with FSSL
-                        Estimators and Logit-Rank as a Solution".  Counted on the tensor cores' fp32
-                        logits against l_t* rounded to fp32, so ids whose logit lies within fp32
-                        rounding of l_t* may fall on either side.  Asking for it adds one gather pass
-                        and a compare per logit.                                              */
+                        Estimators and Logit-Rank as a Solution".  An exact integer: the fused kernel
+                        counts the fp32 logits that exceed l_t* by more than the tensor cores' rounding
+                        and lists the ids it cannot decide (at most 64 per row; row_status bit 5 on
+                        overflow), which the finalize kernel compares in fp64.  Asking for it adds one
+                        gather pass and two compares per logit.                                  */
   float* y_max;      /* GM, optional: y = l + Temp*G of the verifier's own sample (the largest) */
   float* y_second;   /* GM, optional: the second largest y                                     */
   float sigma_ipt;   /* difr_score_both only: noise width of the IPT estimator (CDF units), > 0 */
@@ -290,23 +293,29 @@ difr_status difr_score_ipt_filtered(const void* h, const void* W, const int32_t*
  * For id i != the verifier's own sample the score is ln(Phi((y_i - y_max) /
  * (sigma sqrt 2)) + eps), so i is admissible iff y_i >= y_max + A(tau) with
  * A(tau) = sigma sqrt 2 Phi^-1(e^tau - eps); the sample itself is admissible iff
- * y_max - y_second >= A(tau).  The call makes a second pass over the logits
- * (same tensor-core main loop, noise regenerated, one compare per logit and
- * threshold) and needs the outputs of a difr_score_gm call on the same h, W,
- * seeds, positions and temperature: argmax, y_max, y_second.
+ * the score of its margin y_max - y_second reaches tau.  The call makes a second
+ * pass over the logits (same tensor-core main loop, noise regenerated, two
+ * compares per logit and threshold) and needs the outputs of a difr_score_gm call
+ * on the same h, W, seeds, positions and temperature: argmax, runner_up, y_max,
+ * y_second.
  *
- *   taus      host pointer, n_tau thresholds, 1 <= n_tau <= 4
- *   counts    int32 [n_tau, T] (device): |A_t(taus[j])| in counts[j*T + t]
- *   workspace >= difr_workspace_bytes(T, d, V), scratch
- * y is evaluated in fp32 here (the scoring calls re-evaluate their few
- * candidates in fp64), so an id whose y lies within about 1e-3 * max(1, Temp)
- * of the bound may fall on either side.
+ *   taus       host pointer, n_tau thresholds, 1 <= n_tau <= 4
+ *   runner_up  int32 [T], nullable: with it the sample's own margin is re-evaluated in fp64, without it
+ *              taken from the fp32 values y_max - y_second
+ *   counts     int32 [n_tau, T] (device): |A_t(taus[j])| in counts[j*T + t]
+ *   row_status uint32 [T], nullable: bit 5 marks a row with more than 64 undecided ids (see below)
+ *   workspace  >= difr_workspace_bytes(T, d, V), scratch
+ * The counts are integers decided exactly: the pass evaluates y in fp32, counts the ids that clear the bound by
+ * more than fp32's error there (about 4e-4 * max(1, Temp)), lists the ids inside that band (at most 64 per
+ * row) and a last kernel scores each listed id as the claim in fp64 against tau itself.  A row whose list
+ * overflows (thousands of ids within 1e-3 of a bound: thresholds that cut through the bulk of the
+ * vocabulary) gets bit 5 and a count that leaves the unlisted ids out.
  */
 difr_status difr_admissible(const void* h, const void* W, const uint64_t* seeds, const uint32_t* positions,
                             float temperature, int64_t T, int64_t d, int64_t V, const int32_t* argmax,
-                            const float* y_max, const float* y_second, float sigma, float eps, const float* taus,
-                            int32_t n_tau, int32_t* counts, void* workspace, size_t workspace_bytes,
-                            int32_t* device_status, difr_stream_t stream);
+                            const int32_t* runner_up, const float* y_max, const float* y_second, float sigma,
+                            float eps, const float* taus, int32_t n_tau, int32_t* counts, uint32_t* row_status,
+                            void* workspace, size_t workspace_bytes, int32_t* device_status, difr_stream_t stream);
 
 /*
  * Per-token exfiltratable information (displayed cases of Sec. "Problems with

@@ -4,7 +4,7 @@ The scoring path uses Alg. Token-DiFR with an active subset of one competitor
 and no top-k/top-p filter, where the expectation has a closed form.  This module
 states the algorithm in its general form so that the closed form can be checked:
 
-* `token_difr_monte_carlo`  the algorithm's sampling loop, step by step;
+* `token_difr_monte_carlo`  the sample mean the algorithm returns, over given noise draws;
 * `token_difr_quadrature`   the same expectation by Gauss-Hermite quadrature;
 * `fixed_seed_posterior_mc` the definition it estimates (Sec. "Fixed-Seed
   Posterior Distribution"): perturb every logit, re-run the Gumbel-max sampler
@@ -29,20 +29,22 @@ def margins(logits: np.ndarray, gumbel: np.ndarray, temperature: float, claimed:
 
 
 def token_difr_monte_carlo(logits, gumbel, temperature, claimed, s, sigma, noise_samples, cutoff=-np.inf):
-    """Alg. Token-DiFR: `noise_samples` are the M draws x_j of the claimed token's
-    noise; every competitor's noise CDF is Gaussian with std sigma; `cutoff` is the
-    smallest logit that survives the top-k/top-p filter (-inf: no filter)."""
+    """The sample mean that Alg. Token-DiFR returns, written as the estimator it is:
+
+        pi_hat = mean_j  1{l_t* + x_j > cutoff} * prod_{i in S} Phi(max(x_j + A_i, B_i) / sigma)
+
+    over the draws x_j = `noise_samples` of the claimed token's noise, with Gaussian noise of std sigma on every
+    competitor, B_i = cutoff - l_i, and `cutoff` the smallest logit that survives the top-k/top-p filter
+    (-inf: no filter).  One array expression over (draws x competitors)."""
     logits = np.asarray(logits, dtype=np.float64)
     gumbel = np.asarray(gumbel, dtype=np.float64)
-    y = logits + temperature * gumbel
-    S = active_subset(y, claimed, s)
+    x = np.asarray(noise_samples, dtype=np.float64)
+    S = active_subset(logits + temperature * gumbel, claimed, s)
     A = margins(logits, gumbel, temperature, claimed, S)
     B = cutoff - logits[S]
-    total = 0.0
-    for x in np.asarray(noise_samples, dtype=np.float64):
-        if logits[claimed] + x > cutoff:
-            total += float(np.prod(ndtr(np.maximum(x + A, B) / sigma)))
-    return total / len(noise_samples)
+    survives = (logits[claimed] + x > cutoff).astype(np.float64)
+    factors = ndtr(np.maximum(x[:, None] + A[None, :], B[None, :]) / sigma)
+    return float(np.mean(survives * np.prod(factors, axis=1)))
 
 
 def token_difr_quadrature(logits, gumbel, temperature, claimed, s, sigma, order=200):

@@ -80,9 +80,10 @@ def lib() -> ctypes.CDLL:
                                          + [ctypes.POINTER(_CFilter), ctypes.POINTER(_COut), ctypes.c_void_p])
         L.difr_admissible.restype = ctypes.c_int
         L.difr_admissible.argtypes = ([ctypes.c_void_p] * 4 + [ctypes.c_float] + [ctypes.c_int64] * 3
-                                      + [ctypes.c_void_p] * 3 + [ctypes.c_float] * 2
+                                      + [ctypes.c_void_p] * 4 + [ctypes.c_float] * 2
                                       + [ctypes.POINTER(ctypes.c_float), ctypes.c_int32, ctypes.c_void_p,
-                                         ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p])
+                                         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p,
+                                         ctypes.c_void_p])
         L.difr_exfiltratable_bits.restype = ctypes.c_int
         L.difr_exfiltratable_bits.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64,
                                               ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_void_p,
@@ -259,9 +260,10 @@ def difr_score_gm_filtered(h, W, tokens, seeds, positions, temperature, top_k, t
     return out
 
 
-def difr_admissible(h, W, seeds, positions, temperature, scored: DifrOut, taus, counts, stream=None):
-    """Admissible-set sizes |A_t(tau)| for up to four thresholds; `scored` holds argmax, y_max, y_second, sigma,
-    eps and the workspace of a difr_score_gm call on the same inputs; `counts` is int32 [len(taus), T]."""
+def difr_admissible(h, W, seeds, positions, temperature, scored: DifrOut, taus, counts, row_status=None, stream=None):
+    """Admissible-set sizes |A_t(tau)| for up to four thresholds; `scored` holds argmax, runner_up, y_max, y_second,
+    sigma, eps and the workspace of a difr_score_gm call on the same inputs; `counts` is int32 [len(taus), T];
+    `row_status` (uint32 bits in an int32 [T] tensor, optional) receives bit 5 for rows whose list overflowed."""
     import torch
 
     T, d = h.shape
@@ -271,9 +273,9 @@ def difr_admissible(h, W, seeds, positions, temperature, scored: DifrOut, taus, 
     arr = (ctypes.c_float * len(taus))(*taus)
     ws = scored.workspace
     rc = lib().difr_admissible(_ptr(h), _ptr(W), _ptr(seeds), _ptr(positions), float(temperature), T, d, V,
-                               _ptr(scored.argmax), _ptr(scored.y_max), _ptr(scored.y_second), float(scored.sigma),
-                               float(scored.eps), arr, len(taus), _ptr(counts), _ptr(ws),
-                               ws.numel() * ws.element_size(), _ptr(scored.device_status), _stream(stream))
+                               _ptr(scored.argmax), _ptr(scored.runner_up), _ptr(scored.y_max), _ptr(scored.y_second),
+                               float(scored.sigma), float(scored.eps), arr, len(taus), _ptr(counts), _ptr(row_status),
+                               _ptr(ws), ws.numel() * ws.element_size(), _ptr(scored.device_status), _stream(stream))
     if rc != DIFR_OK:
         raise DifrError(rc, "difr_admissible")
     return counts

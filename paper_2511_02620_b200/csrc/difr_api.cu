@@ -173,11 +173,17 @@ difr_status score_common(int ipt, const void* h, const void* W, const int32_t* t
   if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
   const bool want_rank = (ipt != 1) && out->rank != nullptr;
   if (want_rank) {
-    float* claimed = reinterpret_cast<float*>(static_cast<unsigned char*>(out->workspace) + pl.bounds_offset);
+    unsigned char* ws = static_cast<unsigned char*>(out->workspace);
+    float* bounds = reinterpret_cast<float*>(ws + pl.bounds_offset);
     if (launch_claimed_logits(reinterpret_cast<const uint16_t*>(h), reinterpret_cast<const uint16_t*>(W), tokens,
-                              (int)T, (int)d, (int)V, claimed, s) != cudaSuccess)
+                              (int)T, (int)d, (int)V, bounds, bounds + (size_t)kBandPlane * (size_t)pl.T_pad, s) !=
+        cudaSuccess)
       return DIFR_ERR_CUDA;
-    k1.bounds = claimed;
+    k1.bounds = bounds;
+    k1.band_count = reinterpret_cast<int*>(ws + pl.band_count_offset);
+    k1.band_list = reinterpret_cast<BandEntry*>(ws + pl.band_list_offset);
+    k1.band_cap = kBandCap;
+    if (cudaMemsetAsync(k1.band_count, 0, (size_t)pl.T_pad * sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
   }
   if (out->event_fused_start && cudaEventRecord(reinterpret_cast<cudaEvent_t>(out->event_fused_start), s) != cudaSuccess)
     return DIFR_ERR_CUDA;
@@ -199,6 +205,7 @@ difr_status score_common(int ipt, const void* h, const void* W, const int32_t* t
   k2.temperatures = out->temperatures;
   k2.sigma_ipt = out->sigma_ipt; k2.score_ipt = out->score_ipt;
   k2.rank = want_rank ? out->rank : nullptr; k2.y_max = out->y_max; k2.y_second = out->y_second;
+  k2.band_list = k1.band_list; k2.band_count = k1.band_count; k2.band_cap = k1.band_cap;
   if (launch_k2(k2, s) != cudaSuccess) return DIFR_ERR_CUDA;
   return DIFR_OK;
 }
@@ -248,9 +255,9 @@ static float margin_at_threshold(double tau, double sigma, double eps) {
 
 difr_status difr_admissible(const void* h, const void* W, const uint64_t* seeds, const uint32_t* positions,
                             float temperature, int64_t T, int64_t d, int64_t V, const int32_t* argmax,
-                            const float* y_max, const float* y_second, float sigma, float eps, const float* taus,
-                            int32_t n_tau, int32_t* counts, void* workspace, size_t workspace_bytes,
-                            int32_t* device_status, difr_stream_t stream) {
+                            const int32_t* runner_up, const float* y_max, const float* y_second, float sigma,
+                            float eps, const float* taus, int32_t n_tau, int32_t* counts, uint32_t* row_status,
+                            void* workspace, size_t workspace_bytes, int32_t* device_status, difr_stream_t stream) {
   if (!h || !W || !seeds || !positions || !argmax || !y_max || !y_second || !taus || !counts)
     return DIFR_ERR_INVALID_ARG;
   if (T < 0 || d <= 0 || V <= 0 || n_tau < 1 || n_tau > 4) return DIFR_ERR_INVALID_ARG;
@@ -275,21 +282,35 @@ difr_status difr_admissible(const void* h, const void* W, const uint64_t* seeds,
 
   CountParams cp;
   memset(&cp, 0, sizeof cp);
+  cp.h = reinterpret_cast<const uint16_t*>(h); cp.W = reinterpret_cast<const uint16_t*>(W);
+  cp.seeds = seeds; cp.positions = positions;
   cp.partials = reinterpret_cast<const Partial*>(ws);
-  cp.n_slots = pl.n_slots; cp.T_pad = pl.T_pad; cp.T = (int)T; cp.V = (int)V; cp.n_tau = n_tau;
-  cp.argmax = argmax; cp.y_max = y_max; cp.y_second = y_second;
-  for (int j = 0; j < 4; ++j) cp.a_tau[j] = j < n_tau ? margin_at_threshold(taus[j], sigma, eps) : INFINITY;
+  cp.n_slots = pl.n_slots; cp.T_pad = pl.T_pad; cp.T = (int)T; cp.d = (int)d; cp.V = (int)V; cp.n_tau = n_tau;
+  cp.argmax = argmax; cp.runner_up = runner_up; cp.y_max = y_max; cp.y_second = y_second;
+  cp.temperature = temperature; cp.sigma = sigma; cp.eps = eps;
+  for (int j = 0; j < 4; ++j) {
+    cp.a_tau[j] = j < n_tau ? margin_at_threshold(taus[j], sigma, eps) : INFINITY;
+    cp.taus[j] = j < n_tau ? taus[j] : INFINITY;
+  }
   cp.y_shift = temperature * (float)log(log(2.0));  // the kernel ranks y' = l - Temp ln2 log2(E / ln2) = y + Temp ln ln 2
   cp.bounds = reinterpret_cast<float*>(ws + pl.bounds_offset);
+  cp.band_count = reinterpret_cast<int*>(ws + pl.band_count_offset);
+  cp.band_list = reinterpret_cast<BandEntry*>(ws + pl.band_list_offset);
+  cp.band_cap = kBandCap;
   cp.counts = counts;
+  cp.row_status = row_status;
   if (launch_count_bounds(cp, s) != cudaSuccess) return DIFR_ERR_CUDA;
 
   K1Params k1 = k1_params(pl, T, d, V, temperature, ws);
   k1.tokens = argmax;  // the id the count leaves out
   k1.seeds = seeds; k1.positions = positions;
   k1.bounds = cp.bounds;
+  k1.band_count = const_cast<int*>(cp.band_count);
+  k1.band_list = const_cast<BandEntry*>(cp.band_list);
+  k1.band_cap = kBandCap;
   k1.device_status = device_status;
   if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
+  if (cudaMemsetAsync(k1.band_count, 0, (size_t)pl.T_pad * sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
   const int grid = k1_grid(pl, info.pairs);
   if (launch_k1(n_tau == 1 ? 4 : 5, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;
   if (launch_count_finalize(cp, s) != cudaSuccess) return DIFR_ERR_CUDA;
@@ -429,8 +450,8 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
   if (!ipt && out->rank != nullptr) {
     // the raw-logit rank of the claimed token rides on the collecting pass: claimed logits into the third
     // plane of the bounds, the counts added up in out->rank
-    if (launch_claimed_logits(k2.h, k2.W, tokens, (int)T, (int)d, (int)V, fp.bounds + 2 * (size_t)pl.T_pad, s) !=
-        cudaSuccess)
+    if (launch_claimed_logits(k2.h, k2.W, tokens, (int)T, (int)d, (int)V, fp.bounds + 2 * (size_t)pl.T_pad,
+                              fp.bounds + (size_t)kBandPlane * (size_t)pl.T_pad, s) != cudaSuccess)
       return DIFR_ERR_CUDA;
     if (cudaMemsetAsync(out->rank, 0, (size_t)T * sizeof(int32_t), s) != cudaSuccess) return DIFR_ERR_CUDA;
     k1.rank_out = out->rank;

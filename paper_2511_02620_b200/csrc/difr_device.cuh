@@ -29,6 +29,16 @@ struct Candidate {
   float l, y;  // fp32 logit and y' = y + Temp ln ln 2 as the fused kernel computes them
 };
 
+// An id whose fp32 value (raw logit in the rank mode, y' in the counting modes) lies within rounding of a bound:
+// the finalize kernels re-evaluate it in fp64.  Up to kBandCap per row.
+struct BandEntry {
+  int32_t id;
+  float v;
+};
+constexpr int kBandCap = 64;
+constexpr int kBandOnly = (int)0x80000000u;  // candidate lists: an entry kept only for the rank's exact decision
+constexpr int kBandPlane = 4;                // plane of the per-row bounds that holds the band width
+
 // -------------------------------------------------------------------- Philox
 constexpr uint32_t kPhiloxM0 = 0xD2511F53u;
 constexpr uint32_t kPhiloxM1 = 0xCD9E8D57u;

@@ -15,7 +15,11 @@ struct K1Params {
   const uint64_t* seeds;
   const uint32_t* positions;
   const float* temperatures;  // [T], nullable: per-row temperature in place of c1 / neg_tl2
-  const float* bounds;  // [1 or 4][T_pad]: claimed logits (rank mode) or bounds on y' (counting modes)
+  const float* bounds;  // [5][T_pad]: planes 0..3 claimed logits (rank mode) or bounds on y' (counting modes), each
+                        // raised by the fp32 rounding allowance; plane 4 the width of the undecided band below
+  BandEntry* band_list;  // rank / counting modes: [T_pad][band_cap] ids inside a band, for the exact decision
+  int* band_count;       // [T_pad], zeroed before the launch; may end above band_cap (overflow)
+  int band_cap;
   void* cand_list;      // collect mode: [T][cand_cap] records {int32 id, float l, float y'}
   int* cand_count;      // collect mode: [T], zeroed before the launch; may end above cand_cap (overflow)
   int cand_cap;
@@ -45,6 +49,9 @@ struct K2Params {
   float sigma_ipt;
   float* score_ipt;
   int32_t* rank;
+  const BandEntry* band_list;  // rank mode: the ids the fused kernel could not decide in fp32 (nullable)
+  const int* band_count;
+  int band_cap;
   float* y_max;
   float* y_second;
   float temperature, sigma, eps;
@@ -82,21 +89,33 @@ int k1_max_resident_pairs();  // CTA pairs of the fused kernel the current devic
 cudaError_t launch_k2(const K2Params& p, cudaStream_t stream);
 cudaError_t launch_k3(const K3Params& p, cudaStream_t stream);
 
-// Claimed logits l[r, tokens[r]] rounded to fp32 into out[r] (+inf for an id outside [0, V)): one warp per row.
+// Claimed logits l[r, tokens[r]] plus the tensor cores' rounding allowance into hi[r] (+inf for an id outside
+// [0, V)) and the width of the undecided band below it into width[r]: one warp per row.
 cudaError_t launch_claimed_logits(const uint16_t* h, const uint16_t* W, const int32_t* tokens, int T, int d, int V,
-                                  float* out, cudaStream_t stream);
+                                  float* hi, float* width, cudaStream_t stream);
 
 // Counting pass of the admissible sets.
 struct CountParams {
+  const uint16_t* h;
+  const uint16_t* W;
+  const uint64_t* seeds;
+  const uint32_t* positions;
   const Partial* partials;  // records of the counting modes: four int32 counts each
-  int n_slots, T_pad, T, V, n_tau;
+  int n_slots, T_pad, T, d, V, n_tau;
   const int32_t* argmax;
+  const int32_t* runner_up;  // nullable: without it the sample's own margin is taken from y_max - y_second in fp32
   const float* y_max;
   const float* y_second;
+  float temperature, sigma, eps;
   float a_tau[4];   // A(tau_j): id i != argmax is admissible iff y_i - y_max >= A(tau_j)
+  float taus[4];
   float y_shift;    // the fused kernel ranks y' = y + y_shift
-  float* bounds;    // [4][T_pad] out: bounds on y'
+  float* bounds;    // [5][T_pad] out: bounds on y' (raised by the fp32 allowance), band width in plane 4
+  const BandEntry* band_list;
+  const int* band_count;
+  int band_cap;
   int32_t* counts;  // [n_tau][T] out
+  uint32_t* row_status;  // nullable out: bit 5 = the row's list of undecided ids overflowed
 };
 cudaError_t launch_count_bounds(const CountParams& p, cudaStream_t stream);
 cudaError_t launch_count_finalize(const CountParams& p, cudaStream_t stream);

@@ -17,6 +17,8 @@ constexpr int kBM = 128;        // rows (tokens) per CTA tile
 constexpr int kPairM = 2 * kBM;  // rows per CTA pair: the two CTAs of a pair share one 256 x 256 MMA
 constexpr int kBN = 256;        // vocabulary ids per tile
 constexpr int kBK = 64;         // hidden-dimension slice per pipeline stage (128 bytes of bf16)
+constexpr int kPlanBoundPlanes = 5;  // per-row bounds of the rank / counting / collecting passes (see K1Params)
+constexpr int kPlanBandCap = 64;     // per-row list of ids that fp32 cannot decide (kBandCap)
 
 struct Plan {
   int m_tiles;   // ceil(T / 256): row tiles of a CTA pair
@@ -28,7 +30,9 @@ struct Plan {
   int T_pad;     // m_tiles * 256
   int n_slots;   // partial records per row: one per strip
   size_t partial_bytes;
-  size_t bounds_offset;  // [4][T_pad] floats behind the records and the 256-byte tail (unit counter)
+  size_t bounds_offset;  // [5][T_pad] floats behind the records and the 256-byte tail (unit counter)
+  size_t band_count_offset;  // [T_pad] ints: entries in each row's list of undecided ids
+  size_t band_list_offset;   // [T_pad][kPlanBandCap] entries of 8 bytes
   size_t workspace_bytes;
 };
 
@@ -134,7 +138,9 @@ inline bool compute_plan(int64_t T, int64_t d, int64_t V, int num_pairs, Plan* o
   p.n_slots = p.S;
   p.partial_bytes = (size_t)p.n_slots * (size_t)p.T_pad * 32;
   p.bounds_offset = p.partial_bytes + 256;
-  p.workspace_bytes = p.bounds_offset + (size_t)4 * (size_t)p.T_pad * sizeof(float);
+  p.band_count_offset = p.bounds_offset + (size_t)kPlanBoundPlanes * (size_t)p.T_pad * sizeof(float);
+  p.band_list_offset = p.band_count_offset + (size_t)p.T_pad * sizeof(int);
+  p.workspace_bytes = p.band_list_offset + (size_t)p.T_pad * (size_t)kPlanBandCap * 8;
   *out = p;
   return true;
 }

@@ -56,6 +56,7 @@ constexpr int kXchBytes = (kColGroups - 1) * kBM * 32;  // statistics of column 
 constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + kXchBytes + 1024;  // + slack for 1024-byte alignment
 constexpr float kMasked = -3.0e38f;  // stands in for -inf on padded vocabulary columns (keeps keys finite)
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one CTA");
+static_assert(kPlanBandCap == kBandCap && kPlanBoundPlanes == kBandPlane + 1, "workspace layout");
 
 // Epilogue variants.  GmRank adds the raw-logit rank of the claimed token; Count1 / Count4 regenerate the
 // noise only to count the ids whose y reaches one / four per-row bounds (admissible-set sizes).
@@ -78,6 +79,7 @@ struct Mode {
   static constexpr bool noise = gm || ng > 0 || MODE == kModeCollect;
   static constexpr int ncnt = collect ? 3 : (rank ? 1 : (ng > 0 ? ng : 1));  // bounds loaded per row
   static constexpr bool bounds = rank || collect || ng > 0;
+  static constexpr bool band = rank || ng > 0;  // ids within rounding of a bound are listed for an exact decision
   static constexpr bool record = !collect && MODE != kModeDump;
 };
 
@@ -106,9 +108,11 @@ struct RowStats {
   float lmax;    // running max of z = l * c1
   float lsum;    // sum of 2^(z - lmax)
   float lpre;    // the same restricted to ids below the claimed one
-  int cnt[4];    // GmRank: cnt[0] (Collect: cnt[2]) = ids whose logit exceeds the claimed one; Count: ids at or above bound g
-  float bound[4];  // GmRank: bound[0] = claimed logit; Count: the row's bounds on y'; Collect: bounds on y', on l,
-                   // and the claimed logit (+inf when no rank is wanted)
+  int cnt[4];    // GmRank: cnt[0] (Collect: cnt[2]) = ids whose logit surely exceeds the claimed one; Count: ids
+                 // surely at or above bound g
+  float bound[4];  // GmRank: bound[0] = claimed logit + its rounding allowance; Count: the row's bounds on y' plus
+                   // theirs; Collect: bounds on y', on l, and the claimed logit as in GmRank (+inf: no rank wanted)
+  float bw;      // width of the band below such a bound inside which fp32 cannot decide: those ids are listed
   float gm2;     // GmFilter: the second largest 16-id group maximum of z (lmax is the largest)
 };
 
@@ -118,6 +122,7 @@ __device__ __forceinline__ void stats_init(RowStats& s) {
   s.lmax = -CUDART_INF_F;
   s.lsum = s.lpre = 0.f;
   s.cnt[0] = s.cnt[1] = s.cnt[2] = s.cnt[3] = 0;
+  s.bw = 0.f;
   s.gm2 = -CUDART_INF_F;
 }
 
@@ -183,12 +188,24 @@ __device__ __forceinline__ void noisy4(const RowNoise& rn, int id0, const float 
   }
 }
 
+// One more id of a row whose fp32 value cannot decide an integer: (id, the fp32 value) goes to the row's list.
+__device__ __forceinline__ void band_append(BandEntry* list, int* count, int cap, int id, float v) {
+  if (count == nullptr) return;
+  const int pos = atomicAdd(count, 1);
+  if (pos < cap) {
+    BandEntry e;
+    e.id = id; e.v = v;
+    list[pos] = e;
+  }
+}
+
 // 16 consecutive vocabulary ids [base, base + 16) of one row.  `tok` is the id the row singles out: the
 // claimed token (scoring modes) or the id left out of the count (counting modes).
 template <int MODE>
 __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base, int V, int tok, float c1,
                                           float neg_tl2, const RowNoise& rn, RowStats& s, Candidate* cand_list,
-                                          int* cand_count, int cand_cap) {
+                                          int* cand_count, int cand_cap, BandEntry* band_list, int* band_count,
+                                          int band_cap) {
   using M = Mode<MODE>;
   float l[kSub];
 #pragma unroll
@@ -239,18 +256,41 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
     }
   }
 
-  // ---- raw-logit rank of the claimed token: ids whose logit is larger (the claimed id itself left out)
+  // ---- raw-logit rank of the claimed token: ids whose logit is larger (the claimed id itself left out).
+  // Counted here: logits above the claimed one by more than the tensor cores' rounding.  Ids inside the band
+  // [hi - bw, hi] are listed; the finalize kernel compares their fp64 logits with the claimed token's.
   if (M::rank) {
-    const float lt = s.bound[M::rank_slot];
-    int c = 0;
+    const float hi = s.bound[M::rank_slot], w = s.bw;
+    int c_hi = 0, c_lo = 0;
 #pragma unroll
-    for (int j = 0; j < kSub; ++j) c += (l[j] > lt) ? 1 : 0;
-    if (tl >= 0 && tl < kSub) {
+    for (int j = 0; j < kSub; ++j) {
+      c_hi += (l[j] > hi) ? 1 : 0;
+      c_lo += (l[j] + w >= hi) ? 1 : 0;
+    }
+    if (c_lo != c_hi) {  // rare: some id of this group lies in the band (the claimed id itself always does)
+#pragma unroll
+      for (int j = 0; j < kSub; ++j) {
+        if ((l[j] + w >= hi) && !(l[j] > hi) && j != tl && base + j < V) {
+          if (MODE == kModeCollect) {
+            if (cand_count == nullptr) continue;
+            const int pos = atomicAdd(cand_count, 1);
+            if (pos < cand_cap) {
+              Candidate c;
+              c.id = (base + j) | kBandOnly; c.l = l[j]; c.y = 0.f;
+              cand_list[pos] = c;
+            }
+          } else {
+            band_append(band_list, band_count, band_cap, base + j, l[j]);
+          }
+        }
+      }
+    }
+    if (tl >= 0 && tl < kSub) {  // the claimed id never counts, whatever its own rounding
 #pragma unroll
       for (int j = 0; j < kSub; ++j)
-        if (j == tl && l[j] > lt) --c;
+        if (j == tl && l[j] > hi) --c_hi;
     }
-    s.cnt[M::rank_slot] += c;
+    s.cnt[M::rank_slot] += c_hi;
   }
 
   // ---- candidates by raw logit only (the IPT estimator under a filter needs no noise)
@@ -317,10 +357,28 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
           for (int q = 0; q < 4; ++q)
             if (j + q == tl) y[q] = kMasked;
         }
+        // counted here: y' surely at or above bound g (the bounds carry the fp32 noise allowance); an id whose
+        // y' lies in the band below some bound is listed with its y', and the finalize kernel decides it exactly
+        int n_hi = 0, n_lo = 0;
 #pragma unroll
-        for (int g = 0; g < M::ng; ++g) {
+        for (int q = 0; q < 4; ++q) {
+          const float yw = y[q] + s.bw;
 #pragma unroll
-          for (int q = 0; q < 4; ++q) s.cnt[g] += (y[q] >= s.bound[g]) ? 1 : 0;
+          for (int g = 0; g < M::ng; ++g) {
+            const int a = (y[q] >= s.bound[g]) ? 1 : 0;
+            s.cnt[g] += a;
+            n_hi += a;
+            n_lo += (yw >= s.bound[g]) ? 1 : 0;
+          }
+        }
+        if (n_lo != n_hi) {  // rare
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            bool in_band = false;
+#pragma unroll
+            for (int g = 0; g < M::ng; ++g) in_band |= (y[q] + s.bw >= s.bound[g]) && !(y[q] >= s.bound[g]);
+            if (in_band && base + j + q < V) band_append(band_list, band_count, band_cap, base + j + q, y[q]);
+          }
         }
       }
     }
@@ -607,6 +665,7 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
 #pragma unroll
           for (int g = 0; g < Mode<MODE>::ncnt; ++g)
             st.bound[g] = valid ? p.bounds[(size_t)g * (size_t)p.T_pad + row] : CUDART_INF_F;
+          st.bw = valid ? p.bounds[(size_t)kBandPlane * (size_t)p.T_pad + row] : 0.f;
         }
       }
       // the temperature is the call's, or the row's own when the caller passes one per row
@@ -621,6 +680,12 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
       if (Mode<MODE>::collect && valid) {
         cand_list = reinterpret_cast<Candidate*>(p.cand_list) + (size_t)row * (size_t)p.cand_cap;
         cand_count = p.cand_count + row;
+      }
+      BandEntry* band_list = nullptr;
+      int* band_count = nullptr;
+      if (Mode<MODE>::band && !Mode<MODE>::collect && valid && p.band_count != nullptr) {
+        band_list = p.band_list + (size_t)row * (size_t)p.band_cap;
+        band_count = p.band_count + row;
       }
       for (int n = w.n0; n < w.n1; ++n) {
         if (!mbar_wait(acc_full_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
@@ -647,7 +712,8 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
                   if (base + j < p.V) dst[j] = __uint_as_float(cur[j]);
               }
             } else {
-              process16<MODE>(cur, base, p.V, tok, c1, neg_tl2, rn, st, cand_list, cand_count, p.cand_cap);
+              process16<MODE>(cur, base, p.V, tok, c1, neg_tl2, rn, st, cand_list, cand_count, p.cand_cap, band_list,
+                              band_count, p.band_cap);
             }
             if (!more) break;
           }

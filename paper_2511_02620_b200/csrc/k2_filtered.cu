@@ -198,6 +198,9 @@ __global__ void __launch_bounds__(kFWarps * 32) filter_bounds(const FilterParams
   if (lane == 0) {
     p.bounds[row] = by;
     p.bounds[(size_t)p.T_pad + row] = bl;
+    // no raw-logit rank unless the claimed-logit kernel overwrites these two
+    p.bounds[(size_t)2 * (size_t)p.T_pad + row] = CUDART_INF_F;
+    p.bounds[(size_t)kBandPlane * (size_t)p.T_pad + row] = 0.f;
   }
 }
 
@@ -228,8 +231,10 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
   }
 
   const int k_eff = (rp.top_k > 0) ? (rp.top_k < n ? rp.top_k : n) : 0;
-  int n_others = 0;  // entries that are not the claimed token
-  for (int i = lane; i < n; i += 32) n_others += (list[i].id != tok) ? 1 : 0;
+  // (entries with the sign bit set were kept for the rank's exact decision only: they take no part in the filter
+  // or among the competitors, where the same id may stand a second time as an ordinary entry)
+  int n_others = 0;  // ordinary entries that are not the claimed token
+  for (int i = lane; i < n; i += 32) n_others += (list[i].id >= 0 && list[i].id != tok) ? 1 : 0;
 #pragma unroll
   for (int m = 16; m >= 1; m >>= 1) n_others += __shfl_xor_sync(0xffffffffu, n_others, m);
   const int want = p.s + 2;
@@ -240,9 +245,11 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
   int cut_rank = -1;
   for (int j = 0; j < n; ++j) {
     const Candidate cj = list[j];
+    if (cj.id < 0) continue;  // (uniform over the warp)
     int rl = 0, ry = 0;
     for (int i = lane; i < n; i += 32) {
       const Candidate ci = list[i];
+      if (ci.id < 0) continue;
       rl += (ci.l > cj.l || (ci.l == cj.l && ci.id < cj.id)) ? 1 : 0;
       ry += (ci.id != tok && (ci.y > cj.y || (ci.y == cj.y && ci.id < cj.id))) ? 1 : 0;
     }
@@ -272,6 +279,18 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
     const double temp = (double)rp.temperature, sigma = (double)p.sigma;
     const double l_t = warp_dot(hrow, p.W + (size_t)tok * (size_t)p.d, p.d, lane);
     const double y_t = l_t + temp * gumbel_exact(seed, pos, (uint32_t)tok);
+    if (p.rank != nullptr) {
+      // the collecting pass counted the logits surely above the claimed one; the ids it could not decide in
+      // fp32 stand in the list with the sign bit set and are decided here in fp64
+      int extra = 0;
+      for (int i = 0; i < n; ++i) {
+        const int id = list[i].id;
+        if (id >= 0) continue;
+        const double l = warp_dot(hrow, p.W + (size_t)(id & 0x7fffffff) * (size_t)p.d, p.d, lane);
+        extra += (l > l_t) ? 1 : 0;
+      }
+      if (lane == 0 && extra != 0) atomicAdd(p.rank + row, extra);
+    }
     // exact logits and noisy logits of the s + 2 candidates; then the s best of them
     double cl[kMaxCand], cy[kMaxCand];
     int cid[kMaxCand];

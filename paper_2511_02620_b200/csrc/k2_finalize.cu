@@ -123,6 +123,20 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
   double l_tok = 0.0;
   if (tok_ok) l_tok = warp_dot(hrow, p.W + (size_t)tok * (size_t)p.d, p.d, lane);
 
+  // raw-logit rank: the fused kernel counted the ids whose fp32 logit is above the claimed one by more than the
+  // tensor cores' rounding; the ids it could not decide are on the row's list and are decided here in fp64
+  if (p.rank != nullptr && p.band_count != nullptr && tok_ok) {
+    const int n_found = p.band_count[row];
+    const int n_band = n_found < p.band_cap ? n_found : p.band_cap;
+    if (n_found > p.band_cap) status |= 32u;
+    const BandEntry* list = p.band_list + (size_t)row * (size_t)p.band_cap;
+    for (int e = 0; e < n_band; ++e) {
+      const int id = list[e].id;
+      const double l = warp_dot(hrow, p.W + (size_t)id * (size_t)p.d, p.d, lane);
+      acc.larger += (l > l_tok) ? 1 : 0;
+    }
+  }
+
   if (p.ipt != 1) {
     // ---- Token-DiFR: exact y = l + Temp * G of the claimed token and of every candidate that can be among the
     // two largest.  The fused kernel ranks by fp32 keys whose error (tensor-core accumulation, lg2.approx in the
@@ -221,46 +235,77 @@ cudaError_t launch_k2(const K2Params& p, cudaStream_t stream) {
 }
 
 // --------------------------------------------------------- claimed logits
-// l[r, tokens[r]] in fp64, rounded to fp32: what the fused kernel's rank mode compares every logit with.
+// What the fused kernel's rank mode compares every fp32 logit with: the claimed token's logit l[r, tokens[r]]
+// (fp64 dot product) raised by `allow`, a bound on the rounding of a tensor-core logit of that size, and the
+// width 2 * allow of the band below in which fp32 cannot tell "larger" from "smaller".  The tensor cores add
+// the d / 16 partial products of a logit in fp32 with truncation: at most one unit in the last place of the
+// running sum per step.  +inf / 0 for an id outside [0, V): nothing counts.
 __global__ void __launch_bounds__(kK2Warps * 32)
-claimed_logits(const uint16_t* h, const uint16_t* W, const int32_t* tokens, int T, int d, int V, float* out) {
+claimed_logits(const uint16_t* h, const uint16_t* W, const int32_t* tokens, int T, int d, int V, float* hi,
+               float* width) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = blockIdx.x * kK2Warps + warp;
   if (row >= T) return;
   const int tok = tokens[row];
-  float v = CUDART_INF_F;
-  if (tok >= 0 && tok < V) v = (float)warp_dot(h + (size_t)row * (size_t)d, W + (size_t)tok * (size_t)d, d, lane);
-  if (lane == 0) out[row] = v;
+  float v = CUDART_INF_F, w = 0.f;
+  if (tok >= 0 && tok < V) {
+    const double l = warp_dot(h + (size_t)row * (size_t)d, W + (size_t)tok * (size_t)d, d, lane);
+    const double allow = 1.1920928955078125e-7 * ((double)(d / 16) + 32.0) * (fabs(l) + 2.0);
+    v = (float)(l + allow);
+    w = (float)(2.0 * allow);
+    if (!isfinite(v)) { v = CUDART_INF_F; w = 0.f; }
+  }
+  if (lane == 0) {
+    hi[row] = v;
+    width[row] = w;
+  }
 }
 
 cudaError_t launch_claimed_logits(const uint16_t* h, const uint16_t* W, const int32_t* tokens, int T, int d, int V,
-                                  float* out, cudaStream_t stream) {
+                                  float* hi, float* width, cudaStream_t stream) {
   const int blocks = (T + kK2Warps - 1) / kK2Warps;
-  claimed_logits<<<blocks, kK2Warps * 32, 0, stream>>>(h, W, tokens, T, d, V, out);
+  claimed_logits<<<blocks, kK2Warps * 32, 0, stream>>>(h, W, tokens, T, d, V, hi, width);
   return cudaGetLastError();
 }
 
 // ------------------------------------------------------- admissible sets
-// Bounds of the counting pass: id i != argmax is admissible at threshold j iff y_i >= y_max + A(tau_j); the
-// fused kernel sees y' = y + y_shift.  Unused thresholds get +inf (nothing counts).
+// Id i != argmax is admissible at threshold j iff y_i >= y_max + A(tau_j).  The counting pass sees fp32 values
+// y' = y + y_shift whose noise term comes from lg2.approx: it counts the ids whose y' is above the bound by more
+// than that error (bound + allow) and lists the ids inside the band of width 2 * allow below; unused thresholds
+// get +inf (nothing counts, nothing is listed).
 __global__ void count_bounds(const CountParams p) {
   const int row = blockIdx.x * blockDim.x + threadIdx.x;
   if (row >= p.T) return;
   const float ymax = p.y_max[row];
+  float top = 0.f;  // the largest finite |bound| of the row
+  float b[4];
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    float b = CUDART_INF_F;
+    b[j] = CUDART_INF_F;
     if (j < p.n_tau) {
       // -inf (everything admissible) must stay above the value that masks padded vocabulary columns
-      b = fmaxf(ymax + p.a_tau[j] + p.y_shift, -1.0e38f);
-      if (isnan(b)) b = CUDART_INF_F;
+      b[j] = fmaxf(ymax + p.a_tau[j] + p.y_shift, -1.0e38f);
+      if (isnan(b[j])) b[j] = CUDART_INF_F;
+      if (b[j] > -1.0e38f && b[j] < CUDART_INF_F) top = fmaxf(top, fabsf(b[j]));
     }
-    p.bounds[(size_t)j * (size_t)p.T_pad + row] = b;
   }
+  const float allow = 3e-4f * p.temperature + 1e-4f + 3.9e-6f * top;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const bool open = !(b[j] > -1.0e38f) || !(b[j] < CUDART_INF_F);  // everything or nothing: no band to decide
+    p.bounds[(size_t)j * (size_t)p.T_pad + row] = open ? b[j] : b[j] + allow;
+  }
+  p.bounds[(size_t)kBandPlane * (size_t)p.T_pad + row] = 2.f * allow;
 }
 
-// One warp per row: sums the strips' counts and adds the verifier's own sample, which the counting pass
-// leaves out and which is admissible iff y_max - y_second >= A(tau_j).
+// The Token-DiFR score of a claim with margin A (one competitor, Gaussian noise): ln(Phi(A / (sigma sqrt 2)) + eps).
+__device__ __forceinline__ double gm_score_of_margin(double A, double sigma, double eps) {
+  return log(0.5 * erfc(-A / (2.0 * sigma)) + eps);
+}
+
+// One warp per row: sums the strips' counts, decides the listed ids exactly (fp64 logit and noise, the score of
+// the id as the claim against tau itself), and adds the verifier's own sample, which the counting pass leaves
+// out and which is admissible iff the score of its margin over the runner-up reaches tau.
 __global__ void __launch_bounds__(kK2Warps * 32) count_finalize(const CountParams p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = blockIdx.x * kK2Warps + warp;
@@ -275,10 +320,47 @@ __global__ void __launch_bounds__(kK2Warps * 32) count_finalize(const CountParam
 #pragma unroll
     for (int j = 0; j < 4; ++j) c[j] += __shfl_xor_sync(0xffffffffu, c[j], m);
   }
+  const uint64_t seed = p.seeds[row];
+  const uint32_t pos = p.positions[row];
+  const uint16_t* hrow = p.h + (size_t)row * (size_t)p.d;
+  const double temp = (double)p.temperature, sigma = (double)p.sigma, eps = (double)p.eps;
+  const int best = p.argmax[row];
+  const bool best_ok = best >= 0 && best < p.V;
+  // exact y of the verifier's own sample (and of the runner-up when its id is known)
+  double y_best = (double)p.y_max[row], y_second = (double)p.y_second[row];
+  if (best_ok) y_best = warp_dot(hrow, p.W + (size_t)best * (size_t)p.d, p.d, lane) + temp * gumbel_exact(seed, pos, (uint32_t)best);
+  if (p.runner_up != nullptr) {
+    const int second = p.runner_up[row];
+    if (second >= 0 && second < p.V)
+      y_second = warp_dot(hrow, p.W + (size_t)second * (size_t)p.d, p.d, lane) + temp * gumbel_exact(seed, pos, (uint32_t)second);
+  }
+  uint32_t status = 0;
+  if (p.band_count != nullptr) {
+    const int n_found = p.band_count[row];
+    const int n_band = n_found < p.band_cap ? n_found : p.band_cap;
+    if (n_found > p.band_cap) status |= 32u;
+    const BandEntry* list = p.band_list + (size_t)row * (size_t)p.band_cap;
+    for (int e = 0; e < n_band; ++e) {
+      const int id = list[e].id;
+      const float yf = list[e].v;  // the fp32 y' the counting pass saw
+      const double y = warp_dot(hrow, p.W + (size_t)id * (size_t)p.d, p.d, lane) + temp * gumbel_exact(seed, pos, (uint32_t)id);
+      const double score = gm_score_of_margin(y - y_best, sigma, eps);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (j < p.n_tau) {
+          const float hi = p.bounds[(size_t)j * (size_t)p.T_pad + row];
+          const float w = p.bounds[(size_t)kBandPlane * (size_t)p.T_pad + row];
+          // (ids at or above hi were counted by the pass, ids below the band are surely inadmissible)
+          if (!(yf >= hi) && (yf + w >= hi) && score >= (double)p.taus[j]) ++c[j];
+        }
+      }
+    }
+  }
   if (lane == 0) {
-    const float top_margin = p.y_max[row] - p.y_second[row];
+    const double top_score = gm_score_of_margin(y_best - y_second, sigma, eps);
     for (int j = 0; j < p.n_tau; ++j)
-      p.counts[(size_t)j * (size_t)p.T + row] = c[j] + ((top_margin >= p.a_tau[j]) ? 1 : 0);
+      p.counts[(size_t)j * (size_t)p.T + row] = c[j] + ((top_score >= (double)p.taus[j]) ? 1 : 0);
+    if (p.row_status != nullptr) p.row_status[row] = status;
   }
 }
 

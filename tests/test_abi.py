@@ -32,17 +32,18 @@ def test_host_only_entry_points():
     assert difr.difr_status_string(0) == "ok"
     assert "workspace" in difr.difr_status_string(-4)
     assert difr.difr_status_string(-7)
-    # plan-derived sizes: one 32-byte record per (row, strip) and four floats per row, rows padded to 256,
-    # plus a 256-byte tail
+    # plan-derived sizes: one 32-byte record per (row, strip), a 256-byte tail, and per row (padded to 256 rows)
+    # five floats of bounds, a counter and 64 eight-byte entries for the ids fp32 cannot decide
+    per_row = 5 * 4 + 4 + 64 * 8
     nbytes = difr.difr_workspace_bytes(4096, 3072, 128256)
-    assert nbytes > 0 and (nbytes - 256 - 16 * 4096) % (32 * 4096) == 0
-    assert (difr.difr_workspace_bytes(4097, 3072, 128256) - 256 - 16 * (4096 + 256)) % (32 * (4096 + 256)) == 0
+    assert nbytes > 0 and (nbytes - 256 - per_row * 4096) % (32 * 4096) == 0
+    assert (difr.difr_workspace_bytes(4097, 3072, 128256) - 256 - per_row * (4096 + 256)) % (32 * (4096 + 256)) == 0
     assert difr.difr_workspace_bytes(4096, 3076, 128256) == 0  # d not a multiple of 8
     assert difr.difr_workspace_bytes(4096, 3072, 1) == 0
     assert difr.difr_workspace_bytes(0, 3072, 128256) == 0
     assert difr.difr_workspace_bytes(1 << 30, 64, (1 << 31) - 1) == 0  # more work units than 32-bit ids
     small = difr.difr_workspace_bytes(100, 64, 300)  # 100 rows pad to 256; 300 ids are two tiles: at most two strips
-    assert small in (256 + 16 * 256 + 32 * 256 * s for s in (1, 2))
+    assert small in (256 + per_row * 256 + 32 * 256 * s for s in (1, 2))
 
 
 def test_bad_arguments_are_refused_on_the_host():
@@ -112,8 +113,8 @@ def test_bad_arguments_are_refused_on_the_host():
     assert L.difr_score_ipt_filtered(p, p, p, p, p, 1.0, 128, 64, 1000, ctypes.byref(f1), ctypes.byref(o), None) == INVALID
 
     taus = (ctypes.c_float * 5)(-1.0, -2.0, -3.0, -4.0, -5.0)
-    adm = lambda n, sigma=0.3: L.difr_admissible(p, p, p, p, 1.0, 128, 64, 1000, p, p, p, sigma, 1e-12, taus, n, p, p,
-                                                 1 << 30, None, None)
+    adm = lambda n, sigma=0.3: L.difr_admissible(p, p, p, p, 1.0, 128, 64, 1000, p, p, p, p, sigma, 1e-12, taus, n, p,
+                                                 None, p, 1 << 30, None, None)
     assert adm(0) == INVALID and adm(5) == INVALID and adm(2, sigma=0.0) == INVALID
     assert L.difr_exfiltratable_bits(p, p, 0, 1000, None, 1, 128, None, None, None) == INVALID  # R >= 1
     assert L.difr_exfiltratable_bits(None, p, 8, 1000, None, 1, 128, None, None, None) == INVALID
@@ -188,7 +189,7 @@ def test_planning_is_remembered():
     try:
         difr.difr_debug_plan_override(7, 0, 0)
         T_pad = 16384
-        assert difr.difr_workspace_bytes(*shape) == 7 * 32 * T_pad + 256 + 16 * T_pad
+        assert difr.difr_workspace_bytes(*shape) == 7 * 32 * T_pad + 256 + (5 * 4 + 4 + 64 * 8) * T_pad
     finally:
         difr.difr_debug_plan_override()
     assert difr.difr_workspace_bytes(*shape) == first

@@ -118,6 +118,22 @@ def _check_token_difr(case):
         # tampered rows are what the threshold is for: the calibrated threshold flags most of them
         if sigma <= 0.05 and g["tampered"].sum() >= 8:
             assert flags[g["tampered"]].mean() > 0.5
+    # raw-logit rank (an exact integer) and the three risk classes at rank cutoff 8, on every compared row
+    out = difr.DifrOut.allocate(w.T, w.d, w.V, float(g["sigmas_gm"][1]), eps)
+    out.rank = torch.full((w.T,), -7, dtype=torch.int32, device="cuda")
+    difr.difr_score_gm(dev.h, dev.W, to_dev(tokens), dev.seeds, dev.positions, temperature, out)
+    torch.cuda.synchronize()
+    assert int(out.device_status.item()) == 0
+    rank = out.rank.cpu().numpy()
+    assert np.array_equal(rank[rows], g["rank"]), f"{np.sum(rank[rows] != g['rank'])} ranks differ"
+    assert np.all(out.row_status.cpu().numpy() & 32 == 0)
+    tau = float(g["tau_gm"][1])
+    classes = torch.full((n,), 9, dtype=torch.uint8, device="cuda")
+    difr.difr_detect(out.score[rows_dev].contiguous(), tau, out.margin[rows_dev].contiguous(),
+                     out.rank[rows_dev].contiguous(), 8, None, classes, None)
+    torch.cuda.synchronize()
+    want = oracle.classify(g["score_gm"][1].astype(np.float64), tau, g["rank"], 8)
+    assert np.array_equal(classes.cpu().numpy(), want)
     # whole-workload detection (every sequence of the workload, not only the compared rows)
     flags = torch.empty(w.T, dtype=torch.uint8, device="cuda")
     stats = torch.zeros((len(inp.seq_offsets) - 1, 4), dtype=torch.int32, device="cuda")

@@ -56,10 +56,7 @@ def _sampled_claims(w, inp, rows, temperature, kind):
 @pytest.mark.parametrize("name,T,temperature,sigma", [("llama3b", 0, 1.0, 1.0), ("moe30b", 0, 0.7, 0.3)])
 def test_full_size_rank_both_and_admissible_sets(name, T, temperature, sigma):
     """The widened calls at full size: ranks, both scores and admissible-set sizes on sampled rows against the
-    oracle (integers within the reach of the kernel's fp32 rounding, equal on almost every row), and
-    size-independent properties on all rows."""
-    from scipy.special import ndtr
-
+    oracle (the integers identical), and size-independent properties on all rows."""
     w, inp, dev = _inputs(name, T)
     rows = wl.sample_rows(w, 24, salt=2)
     g = np.random.default_rng(wl.stream_seed(w, 9))
@@ -83,29 +80,15 @@ def test_full_size_rank_both_and_admissible_sets(name, T, temperature, sigma):
                                f32(0.05), f32(EPS))
     np.testing.assert_allclose(out.score.cpu().numpy()[rows], ref.score, rtol=0, atol=SCORE_TOL)
     np.testing.assert_allclose(out.score_ipt.cpu().numpy()[rows], ref_ipt.score, rtol=0, atol=SCORE_TOL)
-    # ranks
-    logits = oracle.logits(hs, Ws)
-    lt = logits[np.arange(len(rows)), tokens[rows]][:, None]
-    others = np.ones_like(logits, dtype=bool)
-    others[np.arange(len(rows)), tokens[rows]] = False
-    lo = ((logits > lt + 2e-5) & others).sum(axis=1)
-    hi = ((logits > lt - 2e-5) & others).sum(axis=1)
+    # ranks: the oracle's integers
     rank = out.rank.cpu().numpy()
-    assert np.all(rank[rows] >= lo) and np.all(rank[rows] <= hi)
-    assert (rank[rows] == ref.rank).mean() >= 0.9
+    assert np.array_equal(rank[rows], ref.rank)
     assert np.all((rank >= 0) & (rank < w.V))
-    # admissible sets
-    y = logits.copy()
-    for i, r in enumerate(rows):
-        y[i] += f32(temperature) * oracle.gumbel_noise_row(int(inp.seeds[r]), int(inp.positions[r]), w.V)
-    order = np.sort(y, axis=1)
-    ymax, ysec = order[:, -1:], order[:, -2:-1]
-    A = np.where(y == ymax, ymax - ysec, y - ymax)
+    assert np.all(out.row_status.cpu().numpy() & 32 == 0)
+    # admissible sets: the oracle's integers
     got = counts.cpu().numpy()
     for j, tau in enumerate(taus):
-        size = lambda shift: (np.log(ndtr((A + shift) / (f32(sigma) * np.sqrt(2.0))) + f32(EPS)) >= tau).sum(axis=1)
         want = oracle.admissible_count(hs, Ws, inp.seeds[rows], inp.positions[rows], f32(temperature), f32(sigma),
                                        tau, f32(EPS))
-        assert np.array_equal(size(0.0), want)
-        assert np.all(got[j][rows] >= size(-1e-3)) and np.all(got[j][rows] <= size(1e-3))
+        assert np.array_equal(got[j][rows], want), (j, got[j][rows], want)
     assert np.all(got[0] <= got[1]) and np.all(got[1] >= 1) and np.all(got[1] <= w.V)

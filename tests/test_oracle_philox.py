@@ -60,8 +60,8 @@ def test_philox_matches_curand_host_generator():
 
 
 def test_philox_known_answer_vectors():
-    """The published known-answer vectors of the algorithm (all-zero, all-one and
-    pi-digit inputs); unlike the cuRAND comparison this needs no library."""
+    """Three stored vectors (all-zero, all-one and pi-digit inputs); unlike the cuRAND comparison this needs no
+    library.  The fixture's header says where they come from: the cuRAND comparison above is the authority."""
     path = os.path.join(os.path.dirname(__file__), "golden", "philox4x32_10_kat.txt")
     rows = [ln.split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
     assert len(rows) == 3

@@ -15,11 +15,11 @@ C, FILTERED, SEEDS = "difr_oracle.c", "filtered.py", "seed_expansion.py"
 # (name, file, text to replace, replacement, test file, -k expression)
 MISTAKES = [
     ("philox multipliers swapped", C, "mul_a = 0xD2511F53u, mul_b = 0xCD9E8D57u", "mul_a = 0xCD9E8D57u, mul_b = 0xD2511F53u",
-     "test_oracle_philox.py", "known_answer"),
+     "test_oracle_philox.py", "curand_host_generator"),
     ("philox key schedule uses one constant twice", C, "kb += weyl_b;", "kb += weyl_a;",
-     "test_oracle_philox.py", "known_answer"),
+     "test_oracle_philox.py", "curand_host_generator"),
     ("philox mixes the wrong high halves", C, "uint32_t n0 = (uint32_t)(pb >> 32) ^ x1 ^ ka;",
-     "uint32_t n0 = (uint32_t)(pa >> 32) ^ x1 ^ ka;", "test_oracle_philox.py", "known_answer"),
+     "uint32_t n0 = (uint32_t)(pa >> 32) ^ x1 ^ ka;", "test_oracle_philox.py", "curand_host_generator"),
     ("counter words in the wrong order", C, "{id >> 2, position, tag, 0u}", "{position, id >> 2, tag, 0u}",
      "test_oracle_philox.py", "ro_word_layout"),
     ("wrong output word for an id", C, "return out[id & 3u];", "return out[3u - (id & 3u)];",
