@@ -7,7 +7,11 @@ with S the top-s ids by y = l + Temp*G (the claimed token left out),
 A_i = y_t* - y_i, B_i = cutoff - l_i, and `cutoff` the smallest logit that
 survives the sampling filter (the reading of the algorithm's garbled definition
 of its cutoff): keep the top_k largest logits, then, among those, the shortest prefix in
-descending order whose renormalised temperature-softmax mass reaches top_p.
+descending order whose renormalised temperature-softmax mass reaches top_p.  A min-p
+filter (Sec. "Sampling From Large Language Models" names it beside top-k and top-p;
+the algorithm does not) keeps the ids whose probability is at least min_p times the
+largest one, i.e. l >= l_max + Temp ln(min_p): that bound is itself the value a logit
+has to reach to survive, so it enters the cutoff as max(cutoff of top-k/top-p, bound).
 The expectation is evaluated by adaptive quadrature (a library routine) split at
 the kinks of the integrand; the algorithm's own Monte-Carlo loop is in
 `posterior.token_difr_monte_carlo`.
@@ -23,14 +27,25 @@ from scipy.special import log_ndtr
 from . import posterior
 
 
-def filter_cutoff(logits: np.ndarray, temperature: float, top_k: int, top_p: float) -> float:
-    """Smallest logit that survives top-k followed by top-p (-inf when neither is set)."""
+def min_p_bound(logits: np.ndarray, temperature: float, min_p: float) -> float:
+    """The logit an id must reach to survive min-p: p_v >= min_p * p_max  <=>  l_v >= l_max + Temp ln(min_p).
+    -inf when min_p is 0 (no filter); under greedy decoding (Temp = 0) only the largest logit survives."""
+    if not min_p > 0.0:
+        return -math.inf
+    top = float(np.max(np.asarray(logits, dtype=np.float64)))
+    return top + temperature * math.log(min_p) if temperature > 0.0 else top
+
+
+def filter_cutoff(logits: np.ndarray, temperature: float, top_k: int, top_p: float, min_p: float = 0.0) -> float:
+    """The value a logit must reach to survive top-k, then top-p, then min-p: the smallest logit the first two
+    keep, or the min-p bound where that is higher (-inf when nothing is set)."""
     logits = np.asarray(logits, dtype=np.float64)
     V = logits.shape[0]
     k_on = 0 < top_k < V
     p_on = top_p < 1.0
+    bound = min_p_bound(logits, temperature, min_p)
     if not k_on and not p_on:
-        return -math.inf
+        return bound
     order = np.argsort(-logits, kind="stable")  # descending, ties: lowest id first
     kept = order[:top_k] if k_on else order
     if p_on:
@@ -42,7 +57,7 @@ def filter_cutoff(logits: np.ndarray, temperature: float, top_k: int, top_p: flo
         else:
             n = 1  # a greedy sampler's nucleus is the largest logit
         kept = kept[: min(n, len(kept))]
-    return float(logits[kept[-1]])
+    return max(float(logits[kept[-1]]), bound)
 
 
 def token_difr_filtered(logits, gumbel, temperature, claimed, s, sigma, cutoff=-math.inf) -> float:
@@ -91,7 +106,7 @@ def model_posterior_mc(logits, gumbel, temperature, claimed, sigma, cutoff, n_dr
 
 
 def score_gm_filtered(h_bits, W_bits, tokens, seeds, positions, temperature, sigma, eps=1e-12, top_k=0, top_p=1.0,
-                      s=1):
+                      s=1, min_p=0.0):
     """Per row: (score = ln(pi + eps), pi, cutoff).  Out-of-range claims score ln(eps)."""
     from . import gumbel_noise_row, logits as all_logits
 
@@ -101,7 +116,7 @@ def score_gm_filtered(h_bits, W_bits, tokens, seeds, positions, temperature, sig
     pi = np.zeros(T)
     cut = np.empty(T)
     for r in range(T):
-        cut[r] = filter_cutoff(L[r], temperature, top_k, top_p)
+        cut[r] = filter_cutoff(L[r], temperature, top_k, top_p, min_p)
         t = int(tokens[r])
         if 0 <= t < V:
             G = gumbel_noise_row(int(seeds[r]), int(positions[r]), V)
@@ -111,8 +126,8 @@ def score_gm_filtered(h_bits, W_bits, tokens, seeds, positions, temperature, sig
 
 
 # ---------------------------------------------------------------- Token-IPT-DiFR under the sampling filter
-def filter_kept(logits: np.ndarray, temperature: float, top_k: int, top_p: float) -> np.ndarray:
-    """Ids that survive top-k followed by top-p (all ids when neither is set), in descending logit order."""
+def filter_kept(logits: np.ndarray, temperature: float, top_k: int, top_p: float, min_p: float = 0.0) -> np.ndarray:
+    """Ids that survive top-k, then top-p, then min-p (all ids when none is set), in descending logit order."""
     logits = np.asarray(logits, dtype=np.float64)
     V = logits.shape[0]
     order = np.argsort(-logits, kind="stable")
@@ -126,14 +141,14 @@ def filter_kept(logits: np.ndarray, temperature: float, top_k: int, top_p: float
         else:
             n = 1
         kept = kept[: min(n, len(kept))]
-    return kept
+    return kept[logits[kept] >= min_p_bound(logits, temperature, min_p)]
 
 
-def filtered_probs(logits: np.ndarray, temperature: float, top_k: int, top_p: float) -> np.ndarray:
+def filtered_probs(logits: np.ndarray, temperature: float, top_k: int, top_p: float, min_p: float = 0.0) -> np.ndarray:
     """The distribution the filtered sampler draws from: softmax(l / Temp) restricted to the surviving ids and
     renormalised (Alg. Token-IPT-DiFR: the same temperature / top-k / nucleus policy as generation)."""
     logits = np.asarray(logits, dtype=np.float64)
-    kept = filter_kept(logits, temperature, top_k, top_p)
+    kept = filter_kept(logits, temperature, top_k, top_p, min_p)
     p = np.zeros_like(logits)
     z = logits[kept] / temperature
     e = np.exp(z - z.max())
@@ -141,14 +156,15 @@ def filtered_probs(logits: np.ndarray, temperature: float, top_k: int, top_p: fl
     return p
 
 
-def ipt_sample_filtered(logits, temperature, top_k, top_p, mu: float) -> int:
+def ipt_sample_filtered(logits, temperature, top_k, top_p, mu: float, min_p: float = 0.0) -> int:
     """Alg. IPT Sampler on the filtered distribution: min{v : C_v > mu}."""
-    c = np.cumsum(filtered_probs(logits, temperature, top_k, top_p))
-    hit = np.nonzero(c > mu)[0]
-    return int(hit[0]) if len(hit) else int(np.nonzero(filtered_probs(logits, temperature, top_k, top_p))[0][-1])
+    p = filtered_probs(logits, temperature, top_k, top_p, min_p)
+    hit = np.nonzero(np.cumsum(p) > mu)[0]
+    return int(hit[0]) if len(hit) else int(np.nonzero(p)[0][-1])
 
 
-def score_ipt_filtered(h_bits, W_bits, tokens, seeds, positions, temperature, sigma, eps=1e-12, top_k=0, top_p=1.0):
+def score_ipt_filtered(h_bits, W_bits, tokens, seeds, positions, temperature, sigma, eps=1e-12, top_k=0, top_p=1.0,
+                       min_p=0.0):
     """Per row: (score, p_claimed, cdf_lo, mu, cutoff) of Token-IPT-DiFR with the filtered distribution."""
     from . import ipt_uniform, logits as all_logits, normal_interval_mass
 
@@ -161,11 +177,11 @@ def score_ipt_filtered(h_bits, W_bits, tokens, seeds, positions, temperature, si
     cut = np.empty(T)
     for r in range(T):
         mu[r] = ipt_uniform(int(seeds[r]), int(positions[r]))
-        cut[r] = filter_cutoff(L[r], temperature, top_k, top_p)
+        cut[r] = filter_cutoff(L[r], temperature, top_k, top_p, min_p)
         t = int(tokens[r])
         mass = 0.0
         if 0 <= t < V:
-            p = filtered_probs(L[r], temperature, top_k, top_p)
+            p = filtered_probs(L[r], temperature, top_k, top_p, min_p)
             a[r] = float(np.sum(p[:t]))
             pt[r] = float(p[t])
             mass = normal_interval_mass((a[r] - mu[r]) / sigma, (a[r] + pt[r] - mu[r]) / sigma)

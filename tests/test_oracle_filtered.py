@@ -183,3 +183,43 @@ def test_ipt_score_without_filter_is_the_plain_one_and_with_filter_obeys_the_ide
             total += math.exp(st[0])
         want = oracle.normal_interval_mass((0.0 - mu0[r]) / sigma, (1.0 - mu0[r]) / sigma)
         assert total == pytest.approx(want, rel=1e-9)
+
+
+def test_min_p_on_hand_worked_examples():
+    """min-p keeps the ids whose probability is at least min_p times the largest (Sec. "Sampling From Large
+    Language Models"): worked through on probabilities 1/2, 1/4, 1/8, 1/16, 1/16."""
+    probs = np.array([0.5, 0.25, 0.125, 0.0625, 0.0625])
+    l = np.log(probs) + 3.0  # any common shift
+    # min_p 0.2 at Temp 1: the bar is 0.1 -> ids 0, 1, 2 survive; a logit survives iff it reaches ln(0.1) + 3
+    assert filtered.filter_cutoff(l, 1.0, 0, 1.0, 0.2) == pytest.approx(math.log(0.1) + 3.0, rel=1e-15)
+    assert sorted(filtered.filter_kept(l, 1.0, 0, 1.0, 0.2).tolist()) == [0, 1, 2]
+    np.testing.assert_allclose(filtered.filtered_probs(l, 1.0, 0, 1.0, 0.2), [4 / 7, 2 / 7, 1 / 7, 0, 0], rtol=1e-14)
+    # exactly on the bar (min_p 0.25: the bar is 1/8) the id survives
+    assert sorted(filtered.filter_kept(l, 1.0, 0, 1.0, 0.25).tolist()) == [0, 1, 2]
+    # Temp 2 flattens the distribution (p ~ sqrt): sqrt(1/16) / sqrt(1/2) = 0.354 >= 0.2, everything survives
+    assert sorted(filtered.filter_kept(l, 2.0, 0, 1.0, 0.2).tolist()) == [0, 1, 2, 3, 4]
+    assert filtered.filter_cutoff(l, 2.0, 0, 1.0, 0.2) == pytest.approx(math.log(0.5) + 3.0 + 2.0 * math.log(0.2))
+    # no min-p: nothing changes; min_p 1 keeps the largest only; greedy decoding likewise
+    assert filtered.filter_cutoff(l, 1.0, 0, 1.0, 0.0) == -math.inf
+    assert filtered.filter_kept(l, 1.0, 0, 1.0, 1.0).tolist() == [0]
+    assert filtered.filter_kept(l, 0.0, 0, 1.0, 0.3).tolist() == [0]
+    # with a top-k in front the stricter of the two decides
+    assert filtered.filter_cutoff(l, 1.0, 2, 1.0, 0.2) == l[1]                       # top-2 is stricter
+    assert filtered.filter_cutoff(l, 1.0, 4, 1.0, 0.2) == pytest.approx(math.log(0.1) + 3.0)  # min-p is stricter
+    assert sorted(filtered.filter_kept(l, 1.0, 4, 1.0, 0.2).tolist()) == [0, 1, 2]
+    # the IPT sampler on the min-p distribution: cumulative 4/7, 6/7, 1
+    assert filtered.ipt_sample_filtered(l, 1.0, 0, 1.0, 0.5, 0.2) == 0
+    assert filtered.ipt_sample_filtered(l, 1.0, 0, 1.0, 0.6, 0.2) == 1
+    assert filtered.ipt_sample_filtered(l, 1.0, 0, 1.0, 0.9, 0.2) == 2
+
+
+def test_min_p_cutoff_is_the_survival_threshold_of_the_simulated_event():
+    """With the min-p bound as the cutoff the expectation still equals the literal simulation of the event
+    (every id a competitor; an id takes part iff its perturbed logit reaches the fixed bound)."""
+    logits, G = _row(12, 9, scale=1.5)
+    cutoff = filtered.filter_cutoff(logits, 1.0, 0, 1.0, 0.3)
+    assert np.sum(logits >= cutoff) < 12  # the filter bites
+    claimed = int(np.argmax(logits + G))
+    want = filtered.model_posterior_mc(logits, G, 1.0, claimed, 0.6, cutoff, 400_000, np.random.default_rng(5))
+    got = filtered.token_difr_filtered(logits, G, 1.0, claimed, 11, 0.6, cutoff)
+    assert got == pytest.approx(want, abs=4 * math.sqrt(want * (1 - want) / 400_000) + 1e-4)
