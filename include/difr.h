@@ -232,6 +232,11 @@ difr_status difr_score_both(const void* h, const void* W, const int32_t* tokens,
  *                  resolved among the 128 largest logits: a row whose 128 largest logits hold
  *                  less than that gets row_status bit 4 and the 128th largest logit as cutoff
  *   filter->s      1..8
+ *   filter->min_p  in [0, 1]; 0: none.  min-p (Sec. "Sampling From Large Language Models") keeps the ids whose
+ *                  probability is at least min_p times the largest one, i.e. whose logit reaches
+ *                  l_max + Temp ln(min_p); that bound is the value a (perturbed) logit has to reach to
+ *                  survive, so the cutoff is the larger of it and the top-k / top-p cutoff.  l_max is
+ *                  re-evaluated in fp64.
  *   temperature > 0
  *   Requests with their own sampling parameters in one batch: filter->top_k_rows, filter->top_p_rows
  *   and out->temperatures give one value per row; a row whose values are outside the ranges above
@@ -256,6 +261,9 @@ typedef struct {
   /* -- members added in version 210; zero them when unused -- */
   const int32_t* top_k_rows; /* device [T], optional: one top_k per row (top_k is then ignored)            */
   const float* top_p_rows;   /* device [T], optional: one top_p per row (top_p is then ignored)            */
+  /* -- members added in version 220; zero them when unused -- */
+  float min_p;               /* in [0, 1]; 0: no min-p filter                                               */
+  const float* min_p_rows;   /* device [T], optional: one min_p per row (min_p is then ignored)            */
 } difr_filter;
 size_t difr_filtered_workspace_bytes(int64_t T, int64_t d, int64_t V);
 difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,
@@ -274,8 +282,9 @@ difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* 
  *
  *   filter->top_k 1..128 (or >= V when V <= 128), or 0 with top_p < 1: a nucleus over the whole
  *   vocabulary as in difr_score_gm_filtered (row_status bit 4 when it holds more than 128 ids);
- *   filter->top_p in (0, 1]; filter->s is ignored; per-row values as in difr_score_gm_filtered (a
- *   row whose own policy filters nothing keeps the unfiltered score)
+ *   filter->top_p in (0, 1]; filter->min_p in [0, 1] (the ids that reach l_max + Temp ln(min_p); resolved
+ *   among the 128 largest logits, row_status bit 4 when more survive); filter->s is ignored; per-row values
+ *   as in difr_score_gm_filtered (a row whose own policy filters nothing keeps the unfiltered score)
  *   temperature > 0; out->workspace needs difr_filtered_workspace_bytes(T, d, V)
  * Writes score, p_claimed, cdf_lo, u, row_status, out->cutoff (optional) and
  * lse (of the unfiltered logits).  Two passes over the logits, the second

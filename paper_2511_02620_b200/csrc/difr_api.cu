@@ -370,9 +370,12 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
   if (!ipt && (filter->s < 1 || filter->s > 8)) return DIFR_ERR_INVALID_ARG;
   if (filter->top_k_rows == nullptr && (top_k < 0 || (top_k > 128 && top_k < V))) return DIFR_ERR_INVALID_ARG;
   if (filter->top_p_rows == nullptr && (!(top_p > 0.f) || !(top_p <= 1.f))) return DIFR_ERR_INVALID_ARG;
+  const float min_p = filter->min_p;
+  if (filter->min_p_rows == nullptr && (!(min_p >= 0.f) || !(min_p <= 1.f))) return DIFR_ERR_INVALID_ARG;
+  const bool min_p_on = filter->min_p_rows != nullptr || min_p > 0.f;
   // IPT with one policy for every row that filters nothing: that is difr_score_ipt
-  if (ipt && filter->top_k_rows == nullptr && filter->top_p_rows == nullptr && (top_k < 1 || top_k >= V) &&
-      top_p >= 1.f && V > 128)
+  if (ipt && filter->top_k_rows == nullptr && filter->top_p_rows == nullptr && !min_p_on &&
+      (top_k < 1 || top_k >= V) && top_p >= 1.f && V > 128)
     return DIFR_ERR_INVALID_ARG;
   if ((d % 8) != 0 || V < 2) return DIFR_ERR_SHAPE;
   if (T == 0) return DIFR_OK;
@@ -387,7 +390,7 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
   if (filter->top_k_rows == nullptr) {
     const bool whole = top_k < 1 || top_k >= V;
     if (!whole) k_max = top_k;
-    else if (filter->top_p_rows == nullptr && top_p >= 1.f) k_max = 0;
+    else if (filter->top_p_rows == nullptr && top_p >= 1.f) k_max = (min_p_on && ipt) ? 128 : 0;
   }
   const int min_strips =
       k_max < kFilterFloorStrips ? kFilterFloorStrips : (k_max > kFilterMaxStrips ? kFilterMaxStrips : k_max);
@@ -436,6 +439,7 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
   fp.temperature = temperature; fp.sigma = out->sigma; fp.eps = out->eps; fp.c1 = k1.c1;
   fp.top_k = top_k; fp.top_p = top_p; fp.s = s_comp; fp.ipt = ipt;
   fp.top_k_rows = filter->top_k_rows; fp.top_p_rows = filter->top_p_rows; fp.temperatures = out->temperatures;
+  fp.min_p = min_p; fp.min_p_rows = filter->min_p_rows;
   fp.bounds = reinterpret_cast<float*>(ws + pl.bounds_offset);
   fp.cand_list = reinterpret_cast<const Candidate*>(ws + list_off);
   fp.cand_count = reinterpret_cast<const int*>(ws + count_off);

@@ -134,6 +134,8 @@ struct FilterParams {
   float top_p;  // 1: no nucleus; one per row in top_p_rows when that is given
   const int32_t* top_k_rows;   // nullable
   const float* top_p_rows;     // nullable
+  float min_p;                 // 0: no min-p; one per row in min_p_rows when that is given
+  const float* min_p_rows;     // nullable
   const float* temperatures;   // nullable: one temperature per row (then `temperature` and `c1` are unused)
   int ipt;      // the IPT estimator's finalize: a row without any filter keeps the first pass's outputs
   int s;        // competitors in the active subset

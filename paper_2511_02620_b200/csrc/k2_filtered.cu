@@ -58,9 +58,11 @@ __device__ __forceinline__ float warp_nth_largest(float (&v)[8], int n, int lane
 
 // The sampling policy of one row, normalised: the call's scalars or the row's own values.
 struct RowPolicy {
-  float temperature, c1, top_p;
-  int top_k;         // ids resolved by logit rank: the top-k, or kMaxK for a nucleus over the whole vocabulary; 0: none
+  float temperature, c1, top_p, min_p;
+  int top_k;         // ids resolved by logit rank: the top-k, or kMaxK for a nucleus over the whole vocabulary or
+                     // a min-p set; 1 when only the largest logit is needed (min-p bound); 0: none
   int nucleus_full;  // the nucleus takes its mass from the whole row (no top-k in front of it)
+  bool by_rank;      // a top-k or a nucleus is in effect: the cutoff by rank is one of the resolved logits
   bool none;         // no filter at all
   bool bad;          // unusable values: the row's score is NaN and row_status bit 3 is set
 };
@@ -71,17 +73,39 @@ __device__ __forceinline__ RowPolicy row_policy(const FilterParams& p, int row) 
   r.c1 = p.temperatures != nullptr ? (r.temperature > 0.f ? 1.4426950408889634f / r.temperature : 0.f) : p.c1;
   int k = p.top_k_rows != nullptr ? p.top_k_rows[row] : p.top_k;
   r.top_p = p.top_p_rows != nullptr ? p.top_p_rows[row] : p.top_p;
-  r.bad = !(r.temperature > 0.f) || isinf(r.temperature) || k < 0 || !(r.top_p > 0.f) || !(r.top_p <= 1.f);
+  r.min_p = p.min_p_rows != nullptr ? p.min_p_rows[row] : p.min_p;
+  r.bad = !(r.temperature > 0.f) || isinf(r.temperature) || k < 0 || !(r.top_p > 0.f) || !(r.top_p <= 1.f) ||
+          !(r.min_p >= 0.f) || !(r.min_p <= 1.f);
   if (k > p.V) k = p.V;
   if (k > kMaxK && k < p.V) r.bad = true;
   const bool whole = k < 1 || k >= p.V;  // no top-k in effect
   r.nucleus_full = (whole && r.top_p < 1.f) ? 1 : 0;
-  r.none = whole && !(r.top_p < 1.f);
+  r.by_rank = !whole || r.nucleus_full;
+  r.none = whole && !(r.top_p < 1.f) && !(r.min_p > 0.f);
   if (r.nucleus_full) k = kMaxK < p.V ? kMaxK : p.V;
-  else if (whole) k = (p.ipt && p.V <= kMaxK) ? p.V : 0;
-  if (r.bad) { k = 0; r.nucleus_full = 0; r.none = false; }
+  else if (whole) {
+    k = (p.ipt && p.V <= kMaxK) ? p.V : 0;
+    // min-p alone: the IPT estimator needs the surviving ids (resolved among the largest kMaxK), Token-DiFR
+    // only the largest logit
+    if (r.min_p > 0.f) k = p.ipt ? (kMaxK < p.V ? kMaxK : p.V) : (k > 1 ? k : 1);
+  }
+  if (r.bad) { k = 0; r.nucleus_full = 0; r.by_rank = false; r.none = false; }
   r.top_k = k;
   return r;
+}
+
+// The min-p bound l_max + Temp ln(min_p) with l_max in fp64: the sorted list's first ranks whose fp32 logit lies
+// within rounding of the largest are all re-evaluated, the largest exact value counts.  Whole warp.
+__device__ __forceinline__ double min_p_bound_exact(const FilterParams& p, const RowPolicy& rp, int row, int lane,
+                                                    const float* sl, const int* sid, int k_eff) {
+  const uint16_t* hrow = p.h + (size_t)row * (size_t)p.d;
+  double l_max = -CUDART_INF;
+  const float near = sl[0] - 1e-4f * fmaxf(1.f, fabsf(sl[0]));
+  for (int r = 0; r < k_eff && r < 8; ++r) {
+    if (r > 0 && sl[r] < near) break;
+    l_max = fmax(l_max, warp_dot(hrow, p.W + (size_t)sid[r] * (size_t)p.d, p.d, lane));
+  }
+  return l_max + (double)rp.temperature * log((double)rp.min_p);
 }
 
 // Softmax mass of the whole row in units of 2^(c1 * l0), from the first pass's records: sum_v 2^(c1 (l_v - l0)).
@@ -264,12 +288,15 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
     }
   }
   __syncwarp();
-  if (k_eff > 0) {
+  if (k_eff > 0 && rp.by_rank) {
     double e[kChunks];
     cut_rank = nucleus_last_rank(p, rp, row, lane, sm_l[warp], k_eff, e, status_bits);
     // the cutoff is that id's logit: re-evaluated in fp64 like every other logit the score depends on
     cutoff = warp_dot(p.h + (size_t)row * (size_t)p.d, p.W + (size_t)sm_id[warp][cut_rank] * (size_t)p.d, p.d, lane);
   }
+  // min-p: a logit survives iff it reaches l_max + Temp ln(min_p); the stricter of the two bounds is the cutoff
+  if (k_eff > 0 && rp.min_p > 0.f)
+    cutoff = fmax(cutoff, min_p_bound_exact(p, rp, row, lane, sm_l[warp], sm_id[warp], k_eff));
 
   double score = log((double)p.eps);
   if (tok_ok) {
@@ -415,8 +442,32 @@ __global__ void __launch_bounds__(kFWarps * 32) ipt_filtered_finalize(const Filt
   double score = log((double)p.eps), pt = CUDART_NAN, a = CUDART_NAN, cutoff = -CUDART_INF;
   if (k_eff > 0) {
     double e[kChunks];  // unnormalised masses of ranks 32 c + lane
-    const int last = nucleus_last_rank(p, rp, row, lane, sm_l[warp], k_eff, e, status_bits);
-    cutoff = warp_dot(p.h + (size_t)row * (size_t)p.d, p.W + (size_t)sm_id[warp][last] * (size_t)p.d, p.d, lane);
+    RowPolicy rank_policy = rp;
+    if (!rp.by_rank) rank_policy.top_p = 1.f;  // no filter by rank: every resolved id stays
+    int last = nucleus_last_rank(p, rank_policy, row, lane, sm_l[warp], k_eff, e, status_bits);
+    if (rp.by_rank)
+      cutoff = warp_dot(p.h + (size_t)row * (size_t)p.d, p.W + (size_t)sm_id[warp][last] * (size_t)p.d, p.d, lane);
+    if (rp.min_p > 0.f) {
+      // min-p: of the ids kept so far, those that reach the bound; logits within fp32 rounding of the bound
+      // are compared in fp64
+      const double bound = min_p_bound_exact(p, rp, row, lane, sm_l[warp], sm_id[warp], k_eff);
+      const uint16_t* hrow = p.h + (size_t)row * (size_t)p.d;
+      int keep = -1;
+      for (int r = 0; r <= last; ++r) {  // descending logits: stop at the first id below the bound
+        const double lf = (double)sm_l[warp][r];
+        const double slack = 1e-4 * fmax(1.0, fabs(bound));
+        bool in = lf >= bound + slack;
+        if (!in && lf > bound - slack)
+          in = warp_dot(hrow, p.W + (size_t)sm_id[warp][r] * (size_t)p.d, p.d, lane) >= bound;
+        else if (!in)
+          break;
+        if (in) keep = r;
+      }
+      if (keep < 0) keep = 0;  // the largest logit always survives
+      if (!rp.by_rank && keep == k_eff - 1 && k_eff < p.V) status_bits |= 16u;  // more survivors than resolved
+      last = keep;
+      cutoff = fmax(cutoff, bound);
+    }
     if (tok_ok) {
       // mass of the kept ids, of those below the claimed id, and whether the claimed id is kept
       double z = 0.0, below = 0.0, mine = 0.0;

@@ -312,3 +312,81 @@ def test_one_sampling_policy_per_row():
         assert np.all(np.isnan(got[bad])) and np.all(st[bad] & 8 != 0)
         # the policies differ where they should: the same claims score differently under different filters
         assert np.unique(np.round(cut[~bad & np.isfinite(cut)], 3)).size > 10
+
+
+@pytest.mark.parametrize("T,d,V,scale,temperature,sigma,top_k,top_p,min_p,s", [
+    (96, 72, 20000, 4.0, 1.0, 0.3, 0, 1.0, 0.05, 3),     # min-p alone (the largest logit is all the filter needs)
+    (96, 64, 3000, 3.0, 0.8, 0.05, 0, 1.0, 0.3, 2),      # every id is a candidate (V < 16384), a strict bar
+    (64, 72, 20000, 4.0, 1.0, 0.3, 50, 0.95, 0.02, 4),   # behind top-k and top-p: the stricter bound decides
+    (64, 72, 20000, 2.0, 1.2, 0.5, 100, 1.0, 0.2, 1),
+])
+def test_min_p_filter_matches_the_oracle(T, d, V, scale, temperature, sigma, top_k, top_p, min_p, s):
+    """min-p keeps the ids whose probability is at least min_p times the largest: the cutoff is the larger of the
+    top-k / top-p cutoff and l_max + Temp ln(min_p), with l_max re-evaluated in fp64."""
+    h, W, seeds, positions = _small(T, d, V, 93, scale)
+    tokens = _claims(h, W, seeds, positions, f32(temperature), 94)
+    tokens[5] = V + 1
+    dev = Device(h, W, seeds, positions)
+    out = difr.DifrOut.allocate(T, d, V, sigma, EPS)
+    out.workspace = torch.empty(difr.difr_filtered_workspace_bytes(T, d, V), dtype=torch.uint8, device="cuda")
+    out.cutoff = torch.full((T,), float("nan"), dtype=torch.float32, device="cuda")
+    out.score.fill_(float("nan"))
+    difr.difr_score_gm_filtered(dev.h, dev.W, to_dev(tokens), dev.seeds, dev.positions, f32(temperature), top_k, top_p,
+                                s, out, min_p=f32(min_p))
+    torch.cuda.synchronize()
+    assert int(out.device_status.item()) == 0
+    want, _, cut = filtered.score_gm_filtered(h, W, tokens, seeds, positions, f32(temperature), f32(sigma), f32(EPS),
+                                              top_k, f32(top_p), s, f32(min_p))
+    got, got_cut = out.score.cpu().numpy(), out.cutoff.cpu().numpy().astype(np.float64)
+    same_cut = np.isclose(got_cut, cut, rtol=0, atol=1e-5)
+    assert same_cut.mean() >= 0.97
+    np.testing.assert_allclose(got[same_cut], want[same_cut], rtol=0, atol=SCORE_TOL)
+    assert got[5] == pytest.approx(math.log(EPS), abs=1e-5)
+    # the bar really is the binding part of the filter on some rows, and the rank filter on others (when both act)
+    L = oracle.logits(h, W)
+    bar = L.max(axis=1) + f32(temperature) * math.log(f32(min_p))
+    assert np.isclose(cut, bar, atol=1e-9).sum() > 5
+    if top_k and top_p < 1.0:
+        assert (~np.isclose(cut, bar, atol=1e-9)).sum() > 5
+    # without min-p the same call gives other scores
+    plain = _run(dev, tokens, temperature, sigma, top_k, top_p, s).score.cpu().numpy()
+    assert np.abs(plain - got)[np.isfinite(plain)].max() > 0.01
+
+
+@pytest.mark.parametrize("T,d,V,scale,temperature,sigma,top_k,top_p,min_p", [
+    (96, 72, 20000, 5.0, 1.0, 0.1, 0, 1.0, 0.05),    # min-p alone: the survivors are found among the 128 largest logits
+    (80, 64, 3000, 4.0, 0.8, 0.05, 40, 0.9, 0.1),
+    (40, 64, 40, 2.0, 1.0, 0.2, 0, 1.0, 0.3),
+])
+def test_ipt_estimator_under_min_p_matches_the_oracle(T, d, V, scale, temperature, sigma, top_k, top_p, min_p):
+    h, W, seeds, positions = _small(T, d, V, 95, scale)
+    L = oracle.logits(h, W)
+    mu = np.array([oracle.ipt_uniform(int(s), int(p)) for s, p in zip(seeds, positions)])
+    tokens = np.array([filtered.ipt_sample_filtered(L[r], f32(temperature), top_k, f32(top_p), mu[r], f32(min_p))
+                       for r in range(T)], dtype=np.int32)
+    k = np.arange(T)
+    tokens[k % 5 == 1] = np.argsort(-L, axis=1)[k % 5 == 1, 1]
+    tokens[k % 5 == 3] = np.argmin(L, axis=1)[k % 5 == 3]
+    dev = Device(h, W, seeds, positions)
+    out = difr.DifrOut.allocate(T, d, V, sigma, EPS)
+    out.workspace = torch.empty(difr.difr_filtered_workspace_bytes(T, d, V), dtype=torch.uint8, device="cuda")
+    out.cutoff = torch.full((T,), float("nan"), dtype=torch.float32, device="cuda")
+    difr.difr_score_ipt_filtered(dev.h, dev.W, to_dev(tokens), dev.seeds, dev.positions, f32(temperature), top_k, top_p,
+                                 out, min_p=f32(min_p))
+    torch.cuda.synchronize()
+    assert int(out.device_status.item()) == 0
+    want, pt, a, _, cut = filtered.score_ipt_filtered(h, W, tokens, seeds, positions, f32(temperature), f32(sigma),
+                                                      f32(EPS), top_k, f32(top_p), f32(min_p))
+    n_kept = np.array([len(filtered.filter_kept(L[r], f32(temperature), top_k, f32(top_p), f32(min_p)))
+                       for r in range(T)])
+    status = out.row_status.cpu().numpy()
+    resolved = n_kept < min(128, V) if not top_k else np.ones(T, dtype=bool)
+    assert resolved.sum() >= T // 2
+    assert np.all(status[resolved] & 16 == 0)
+    got_cut = out.cutoff.cpu().numpy().astype(np.float64)
+    ok = resolved & np.isclose(got_cut, cut, rtol=0, atol=1e-5)
+    assert ok.sum() >= 0.95 * resolved.sum()
+    np.testing.assert_allclose(out.score.cpu().numpy()[ok], want[ok], rtol=0, atol=SCORE_TOL)
+    np.testing.assert_allclose(out.p_claimed.cpu().numpy()[ok], pt[ok], rtol=2e-4, atol=1e-9)
+    np.testing.assert_allclose(out.cdf_lo.cpu().numpy()[ok], a[ok], rtol=2e-4, atol=2e-6)
+    assert (n_kept[resolved] > 1).sum() > 5  # the bar keeps more than the top id on some rows
