@@ -114,6 +114,7 @@ struct RowStats {
                    // theirs; Collect: bounds on y', on l, and the claimed logit as in GmRank (+inf: no rank wanted)
   float bw;      // width of the band below such a bound inside which fp32 cannot decide: those ids are listed
   float gm2;     // GmFilter: the second largest 16-id group maximum of z (lmax is the largest)
+  uint32_t tie;  // Gumbel-max modes: nonzero once the two best keys of some 16-id group were equal
 };
 
 __device__ __forceinline__ void stats_init(RowStats& s) {
@@ -124,12 +125,14 @@ __device__ __forceinline__ void stats_init(RowStats& s) {
   s.cnt[0] = s.cnt[1] = s.cnt[2] = s.cnt[3] = 0;
   s.bw = 0.f;
   s.gm2 = -CUDART_INF_F;
+  s.tie = 0u;
 }
 
 // Keys are y' with the low four mantissa bits cleared, so values that differ by less than 2^-19 relative count
 // as equal, and equal keys rank by vocabulary id (lowest first): of any number of exactly tied ids the two lowest
 // survive to the finalize kernel, which orders them exactly.  (Inside one 16-id group the min/max network ranks
-// tied keys by their column bits instead; three tied ids within one group are not told apart.)
+// tied keys by their column bits instead; a record whose strip saw such a tie is marked, and the finalize kernel
+// then re-evaluates every id of its candidates' groups.)
 //
 // (k1, j1), (k2, j2): the best two of the next 16 ids of the same thread, k1 >= k2, all ids above those seen.
 __device__ __forceinline__ void top2_merge(RowStats& s, float k1, int j1, float k2, int j2) {
@@ -385,6 +388,9 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
     // merge the group's top-2 into the running top-2 (column bits cleared: earlier ids win ties)
     if (M::gm) {
       const uint32_t b1 = __float_as_uint(c1k), b2 = __float_as_uint(c2k);
+      // Equal keys inside one group were ranked by their column bits (the highest column first), not by id: the
+      // record says so, and the finalize kernel then looks at every id of its candidates' groups.
+      s.tie |= ((b1 ^ b2) < 16u) ? 1u : 0u;
       top2_merge(s, __uint_as_float(b1 & ~15u), base + (int)(b1 & 15u), __uint_as_float(b2 & ~15u),
                  base + (int)(b2 & 15u));
     }
@@ -402,7 +408,9 @@ __device__ __forceinline__ void record_pack(const RowStats& st, float4& a, float
     b = make_float4(0.f, 0.f, 0.f, 0.f);
   } else {
     a = make_float4(st.m1, __int_as_float(st.i1), st.m2, __int_as_float(st.i2));
-    b = make_float4(st.lmax, st.lsum, st.lpre, Mode<MODE>::groupmax ? st.gm2 : __int_as_float(st.cnt[0]));
+    // (the sum is never negative: its sign bit carries the tie mark)
+    b = make_float4(st.lmax, (Mode<MODE>::gm && st.tie) ? -st.lsum : st.lsum, st.lpre,
+                    Mode<MODE>::groupmax ? st.gm2 : __int_as_float(st.cnt[0]));
   }
 }
 template <int MODE>
@@ -415,11 +423,12 @@ __device__ __forceinline__ void record_merge(RowStats& st, const float4& a, cons
   } else {
     top2_insert_any(st, a.x, __float_as_int(a.y));
     top2_insert_any(st, a.z, __float_as_int(a.w));
+    if (Mode<MODE>::gm) st.tie |= __float_as_uint(b.y) >> 31;
     if (Mode<MODE>::groupmax) st.gm2 = fmax3(st.gm2, b.w, fminf(st.lmax, b.x));  // (b.x, b.w): its two largest
     if (b.x > -CUDART_INF_F) {  // that group saw columns
       const float m = fmaxf(st.lmax, b.x);
       const float fa = ex2_approx(st.lmax - m), fb = ex2_approx(b.x - m);
-      st.lsum = st.lsum * fa + b.y * fb;
+      st.lsum = st.lsum * fa + fabsf(b.y) * fb;
       st.lpre = st.lpre * fa + b.z * fb;
       st.lmax = m;
     }

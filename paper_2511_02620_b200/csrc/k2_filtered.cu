@@ -115,7 +115,7 @@ __device__ __forceinline__ double row_mass_relative(const FilterParams& p, int r
   for (int slot = lane; slot < p.n_slots; slot += 32) {
     const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * (size_t)p.T_pad + row);
     const float4 b = src[1];
-    const double bm = (double)b.x, bs = (double)b.y;
+    const double bm = (double)b.x, bs = (double)fabsf(b.y);  // (the sign bit is the fused kernel's tie mark)
     if (bm == -CUDART_INF) continue;
     if (bm > lmax) { lsum = lsum * exp2(lmax - bm) + bs; lmax = bm; }
     else lsum += bs * exp2(bm - lmax);

@@ -75,7 +75,7 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
     const float4 a = src[0], b = src[1];
     top2_insert(acc, a.x, __float_as_int(a.y));
     top2_insert(acc, a.z, __float_as_int(a.w));
-    lse_merge(acc, (double)b.x, (double)b.y, (double)b.z);
+    lse_merge(acc, (double)b.x, (double)fabsf(b.y), (double)b.z);  // (the sign bit of the sum is the tie mark)
     acc.larger += __float_as_int(b.w);
   }
 #pragma unroll
@@ -148,12 +148,17 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
     double yb1 = -CUDART_INF, yb2 = -CUDART_INF;
     int ib1 = -1, ib2 = -1;
     auto place = [&](double y, int id) {
+      if (id == ib1 || id == ib2) return;  // (a group that is walked whole can bring an id a second time)
       if (ib1 < 0 || y > yb1 || (y == yb1 && id < ib1)) {
         yb2 = yb1; ib2 = ib1;
         yb1 = y; ib1 = id;
       } else if (ib2 < 0 || y > yb2 || (y == yb2 && id < ib2)) {
         yb2 = y; ib2 = id;
       }
+    };
+    auto place_id = [&](int cid) {
+      const double l = warp_dot(hrow, p.W + (size_t)cid * (size_t)p.d, p.d, lane);
+      place(l + temp * gumbel_exact(seed, pos, (uint32_t)cid), cid);
     };
     double yt = -CUDART_INF;
     if (tok_ok) {
@@ -163,18 +168,31 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
     for (int base = 0; base < p.n_slots; base += 32) {
       const int slot = base + lane;
       float4 a = make_float4(-CUDART_INF_F, __int_as_float(-1), -CUDART_INF_F, __int_as_float(-1));
-      if (slot < p.n_slots) a = *reinterpret_cast<const float4*>(p.partials + (size_t)slot * (size_t)p.T_pad + row);
+      bool tie_mark = false;
+      if (slot < p.n_slots) {
+        const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * (size_t)p.T_pad + row);
+        a = src[0];
+        tie_mark = signbit(src[1].y);
+      }
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
         const float key = e ? a.z : a.x;
         const int id = __float_as_int(e ? a.w : a.y);
-        unsigned todo = __ballot_sync(0xffffffffu, id >= 0 && id < p.V && id != tok && !(key < window));
+        unsigned todo = __ballot_sync(0xffffffffu, id >= 0 && id < p.V && !(key < window));
+        const unsigned marked = __ballot_sync(0xffffffffu, tie_mark);
         while (todo) {
-          const int src = __ffs(todo) - 1;
+          const int src_lane = __ffs(todo) - 1;
           todo &= todo - 1;
-          const int cid = __shfl_sync(0xffffffffu, id, src);
-          const double l = warp_dot(hrow, p.W + (size_t)cid * (size_t)p.d, p.d, lane);
-          place(l + temp * gumbel_exact(seed, pos, (uint32_t)cid), cid);
+          const int cid = __shfl_sync(0xffffffffu, id, src_lane);
+          if ((marked >> src_lane) & 1u) {
+            // this strip ranked equal keys inside a 16-id group by column, not by id: every id of the
+            // candidate's group is a candidate
+            const int g0 = cid & ~15;
+            for (int v = g0; v < g0 + 16 && v < p.V; ++v)
+              if (v != tok) place_id(v);
+          } else if (cid != tok) {
+            place_id(cid);
+          }
         }
       }
     }

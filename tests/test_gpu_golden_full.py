@@ -115,8 +115,10 @@ def _check_token_difr(case):
         assert np.array_equal(stats["n_match"], ref_stats["n_match"])
         np.testing.assert_allclose(stats["sum"], ref_stats["sum"], rtol=1e-5, atol=0.02)
         np.testing.assert_allclose(stats["min"], ref_stats["min"], rtol=0, atol=SCORE_TOL)
-        # tampered rows are what the threshold is for: the calibrated threshold flags most of them
-        if sigma <= 0.05 and g["tampered"].sum() >= 8:
+        # tampered rows are what the threshold is for: where honest claims (almost) always replay, the calibrated
+        # threshold flags most of them.  (Where more than 1 % of the honest claims fail to replay because the
+        # server saw perturbed hidden states, their scores reach the floor and the 1 % threshold sits at it.)
+        if sigma <= 0.05 and g["tampered"].sum() >= 8 and float(g["honest_match_rate"]) > 0.995:
             assert flags[g["tampered"]].mean() > 0.5
     # raw-logit rank (an exact integer) and the three risk classes at rank cutoff 8, on every compared row
     out = difr.DifrOut.allocate(w.T, w.d, w.V, float(g["sigmas_gm"][1]), eps)

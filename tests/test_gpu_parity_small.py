@@ -326,11 +326,15 @@ def test_rows_with_non_finite_logits_are_never_scored_as_safe():
         assert np.all(flags.cpu().numpy()[marked] == 1)
 
 
-@pytest.mark.parametrize("tied", [(37, 1301), (1301, 37, 700), (8999, 5000, 37, 700, 1301, 4096, 4111)])
+@pytest.mark.parametrize("tied", [(37, 1301), (1301, 37, 700), (8999, 5000, 37, 700, 1301, 4096, 4111),
+                                  (4098, 4100, 4111), (4111, 4097, 4103, 4100, 8990),   # three and more in one 16-id group
+                                  (37, 4098, 4100, 4111), (36, 37, 39, 44, 47)])
 def test_exact_ties_go_to_the_lowest_id(tied):
     """Greedy replay with identical rows of W that hold the largest logit of every row: the lowest id is the
     sample, the next lowest the runner-up, and a claim of any other tied id is a mismatch by the tie-break alone
-    (margin -0.0), as in the oracle.  The tied ids lie in different 16-id groups, tiles and strips."""
+    (margin -0.0), as in the oracle.  The tied ids lie in different 16-id groups, tiles and strips, or several of
+    them inside one aligned group of 16 ids (where the fused kernel ranks equal keys by column and marks the
+    record, and the finalize kernel walks the group)."""
     T, d, V = 64, 64, 9000
     h, W, seeds, positions = _small(T, d, V, 61)
     # one direction that dominates every row's logits: h gets a large common component, the tied rows point along it
