@@ -389,10 +389,10 @@ def timed_steps(prob, steps, warmup, events, local_rank, barrier, flush=None):
 
 
 def strips_of(difr, w):
-    """Partial records per row, recovered from the workspace size (records, a 256-byte tail, 536 bytes per row of
+    """Partial records per row, recovered from the workspace size (records, a 256-byte tail, 540 bytes per row of
     bounds and lists for the integer outputs)."""
     T_pad = -(-w.T // 256) * 256
-    return (difr.difr_workspace_bytes(w.T, w.d, w.V) - 256 - 536 * T_pad) // (32 * T_pad)
+    return (difr.difr_workspace_bytes(w.T, w.d, w.V) - 256 - 540 * T_pad) // (32 * T_pad)
 
 
 def roofline_of(difr, w, k1_ms, k2_ms, k3_ms, peaks, n_seq):

@@ -171,6 +171,12 @@ difr_status score_common(int ipt, const void* h, const void* W, const int32_t* t
   const int grid = k1_grid(pl, info.pairs);
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
+  if (ipt != 1) {
+    // the rows' running floors (last plane of the bounds): 0x80 in every byte is a float below every key
+    k1.row_floor = reinterpret_cast<int*>(static_cast<unsigned char*>(out->workspace) + pl.bounds_offset) +
+                   (size_t)(kPlanBoundPlanes - 1) * (size_t)pl.T_pad;
+    if (cudaMemsetAsync(k1.row_floor, 0x80, (size_t)pl.T_pad * sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
+  }
   const bool want_rank = (ipt != 1) && out->rank != nullptr;
   if (want_rank) {
     unsigned char* ws = static_cast<unsigned char*>(out->workspace);

@@ -26,6 +26,8 @@ struct K1Params {
   Partial* partials;  // [n_slots][T_pad]
   float* logits_out;  // dump mode only
   int32_t* device_status;
+  int* row_floor;     // Gumbel-max scoring modes, nullable: [T_pad] per-row lower bounds of the second largest key
+                      // (order-preserving integers), every byte preset to 0x80 (a value below every key)
   int* rank_out;      // Collect mode, nullable: [T] zeroed counters that receive the claimed tokens' raw-logit ranks
   int* unit_counter;  // zeroed before the launch: units are handed out in order on demand; null: round robin
   int T, d, V;

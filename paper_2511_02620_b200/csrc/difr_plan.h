@@ -17,7 +17,8 @@ constexpr int kBM = 128;        // rows (tokens) per CTA tile
 constexpr int kPairM = 2 * kBM;  // rows per CTA pair: the two CTAs of a pair share one 256 x 256 MMA
 constexpr int kBN = 256;        // vocabulary ids per tile
 constexpr int kBK = 64;         // hidden-dimension slice per pipeline stage (128 bytes of bf16)
-constexpr int kPlanBoundPlanes = 5;  // per-row bounds of the rank / counting / collecting passes (see K1Params)
+constexpr int kPlanBoundPlanes = 6;  // per-row bounds of the rank / counting / collecting passes (see K1Params);
+                                     // the last plane holds the rows' running floors of the scoring pass
 constexpr int kPlanBandCap = 64;     // per-row list of ids that fp32 cannot decide (kBandCap)
 
 struct Plan {
@@ -30,7 +31,7 @@ struct Plan {
   int T_pad;     // m_tiles * 256
   int n_slots;   // partial records per row: one per strip
   size_t partial_bytes;
-  size_t bounds_offset;  // [5][T_pad] floats behind the records and the 256-byte tail (unit counter)
+  size_t bounds_offset;  // [6][T_pad] floats behind the records and the 256-byte tail (unit counter)
   size_t band_count_offset;  // [T_pad] ints: entries in each row's list of undecided ids
   size_t band_list_offset;   // [T_pad][kPlanBandCap] entries of 8 bytes
   size_t workspace_bytes;

@@ -56,7 +56,7 @@ constexpr int kXchBytes = (kColGroups - 1) * kBM * 32;  // statistics of column 
 constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + kXchBytes + 1024;  // + slack for 1024-byte alignment
 constexpr float kMasked = -3.0e38f;  // stands in for -inf on padded vocabulary columns (keeps keys finite)
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one CTA");
-static_assert(kPlanBandCap == kBandCap && kPlanBoundPlanes == kBandPlane + 1, "workspace layout");
+static_assert(kPlanBandCap == kBandCap && kPlanBoundPlanes == kBandPlane + 2, "workspace layout");
 
 // Epilogue variants.  GmRank adds the raw-logit rank of the claimed token; Count1 / Count4 regenerate the
 // noise only to count the ids whose y reaches one / four per-row bounds (admissible-set sizes).
@@ -80,6 +80,9 @@ struct Mode {
   static constexpr int ncnt = collect ? 3 : (rank ? 1 : (ng > 0 ? ng : 1));  // bounds loaded per row
   static constexpr bool bounds = rank || collect || ng > 0;
   static constexpr bool band = rank || ng > 0;  // ids within rounding of a bound are listed for an exact decision
+  // Gumbel-max modes whose records feed the finalize kernel only: an id whose noise word cannot lift it to the
+  // row's second best so far skips the Gumbel transform and the top-2 network
+  static constexpr bool skip = MODE == kModeGm || MODE == kModeGmRank;
   static constexpr bool record = !collect && MODE != kModeDump;
 };
 
@@ -115,6 +118,8 @@ struct RowStats {
   float bw;      // width of the band below such a bound inside which fp32 cannot decide: those ids are listed
   float gm2;     // GmFilter: the second largest 16-id group maximum of z (lmax is the largest)
   uint32_t tie;  // Gumbel-max modes: nonzero once the two best keys of some 16-id group were equal
+  float floor;   // skip modes: a lower bound of the row's second largest key (from other strips' records)
+  float thrz;    // skip modes: (max(floor, m2) - allowance) * c1, the key an id must be able to reach; -inf: none
 };
 
 __device__ __forceinline__ void stats_init(RowStats& s) {
@@ -126,6 +131,7 @@ __device__ __forceinline__ void stats_init(RowStats& s) {
   s.bw = 0.f;
   s.gm2 = -CUDART_INF_F;
   s.tie = 0u;
+  s.floor = s.thrz = -CUDART_INF_F;
 }
 
 // Keys are y' with the low four mantissa bits cleared, so values that differ by less than 2^-19 relative count
@@ -161,11 +167,9 @@ __device__ __forceinline__ void top2_insert_any(RowStats& s, float k, int j) {
   }
 }
 
-// y' = l - Temp ln2 log2(-log2 u) = l + Temp G + Temp ln(ln 2) for ids [id0, id0 + 4) of one row (id0 % 4 == 0).
-__device__ __forceinline__ void noisy4(const RowNoise& rn, int id0, const float (&l)[4], float neg_tl2,
-                                       float (&y)[4]) {
-  uint32_t x[4];
-  row_noise_block(rn, (uint32_t)id0 >> 2, x);
+// y' = l - Temp ln2 log2(-log2 u) = l + Temp G + Temp ln(ln 2) from the four noise words x of ids [id0, id0 + 4).
+__device__ __forceinline__ void noisy4_from_words(const uint32_t (&x)[4], const float (&l)[4], float neg_tl2,
+                                                  float (&y)[4]) {
   const float2 minus1 = make_float2(-0.99999994f, -0.99999994f), ntl2 = make_float2(neg_tl2, neg_tl2);
 #pragma unroll
   for (int q = 0; q < 4; q += 2) {
@@ -189,6 +193,23 @@ __device__ __forceinline__ void noisy4(const RowNoise& rn, int id0, const float 
       }
     }
   }
+}
+
+__device__ __forceinline__ void noisy4(const RowNoise& rn, int id0, const float (&l)[4], float neg_tl2,
+                                       float (&y)[4]) {
+  uint32_t x[4];
+  row_noise_block(rn, (uint32_t)id0 >> 2, x);
+  noisy4_from_words(x, l, neg_tl2, y);
+}
+
+// The key an id must be able to reach to matter to the finalize kernel, times c1: the larger of the row's floor
+// and this thread's own second best, less the allowance by which the finalize kernel looks below the second
+// best key (twice the keys' error) and a little more.
+__device__ __forceinline__ float skip_threshold_z(float floor, float m2, float c1, float neg_tl2) {
+  const float m = fmaxf(floor, m2);
+  const float temp = neg_tl2 * -1.4426950408889634f;
+  const float thr = m - (1e-3f * temp + 4e-4f + 1.6e-5f * fabsf(m));
+  return (c1 > 0.f && m > -CUDART_INF_F) ? thr * c1 : -CUDART_INF_F;  // greedy replay (c1 = 0): no noise to skip
 }
 
 // One more id of a row whose fp32 value cannot decide an integer: (id, the fp32 value) goes to the row's list.
@@ -220,6 +241,7 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
   }
   const int tl = tok - base;  // position of the singled-out id relative to this group
 
+  float zmax_group = 0.f;  // largest z = l * c1 of these 16 ids
   // ---- softmax statistics (online log-sum-exp in base 2)
   if (M::softmax) {
     float cm = fmax3(l[0], l[1], l[2]);
@@ -227,6 +249,7 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
     for (int j = 3; j + 1 < kSub; j += 2) cm = fmax3(cm, l[j], l[j + 1]);
     cm = fmaxf(cm, l[kSub - 1]);
     const float zmax = cm * c1;
+    zmax_group = zmax;
     if (M::groupmax) s.gm2 = fmaxf(s.gm2, fminf(s.lmax, zmax));
     if (zmax > s.lmax) {  // rare after the first few groups of a strip
       const float scale = ex2_approx(s.lmax - zmax);  // 0 on the first group
@@ -320,12 +343,24 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
   // ---- Gumbel-max replay: top-2 of y' = l - Temp*ln2 * log2(-log2 u), or counts of y' against the row's bounds
   if (M::noise) {
     float c1k = -CUDART_INF_F, c2k = -CUDART_INF_F;
+    // Skip modes: y' >= thr needs -ln u <= ln2 2^((l - thr) c1), and 1 - u <= -ln u, so a noise word below
+    // x_need (taken with the group's largest logit, rounded to the safe side) cannot lift its id to thr.
+    uint32_t x_need = 0u;
+    if (M::skip) x_need = ~__float2uint_rz(fmaf(ex2_approx(zmax_group - s.thrz), 2.9799e9f, 1024.f));
 #pragma unroll
     for (int j = 0; j < kSub; j += 4) {
       const float l4[4] = {l[j], l[j + 1], l[j + 2], l[j + 3]};
       float y[4];
-      noisy4(rn, base + j, l4, neg_tl2, y);
-      if (M::gm) {
+      bool live = true;
+      if (M::skip) {
+        uint32_t x[4];
+        row_noise_block(rn, (uint32_t)(base + j) >> 2, x);
+        live = max(max(x[0], x[1]), max(x[2], x[3])) >= x_need;
+        if (live) noisy4_from_words(x, l4, neg_tl2, y);  // rare once the row's second best is known
+      } else {
+        noisy4(rn, base + j, l4, neg_tl2, y);
+      }
+      if (M::gm && live) {
         float key[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) key[q] = __uint_as_float((__float_as_uint(y[q]) & ~15u) | (uint32_t)(j + q));
@@ -390,12 +425,21 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
       const uint32_t b1 = __float_as_uint(c1k), b2 = __float_as_uint(c2k);
       // Equal keys inside one group were ranked by their column bits (the highest column first), not by id: the
       // record says so, and the finalize kernel then looks at every id of its candidates' groups.
-      s.tie |= ((b1 ^ b2) < 16u) ? 1u : 0u;
+      s.tie |= ((b1 ^ b2) < 16u && c1k > -CUDART_INF_F) ? 1u : 0u;
+      const float m2_before = s.m2;
       top2_merge(s, __uint_as_float(b1 & ~15u), base + (int)(b1 & 15u), __uint_as_float(b2 & ~15u),
                  base + (int)(b2 & 15u));
+      if (M::skip && s.m2 != m2_before) s.thrz = skip_threshold_z(s.floor, s.m2, c1, neg_tl2);  // rare
     }
   }
 }
+
+// Floats as integers that order the same way (for atomicMax on a float kept in global memory).
+__device__ __forceinline__ int float_to_ordered(float f) {
+  const int b = __float_as_int(f);
+  return b >= 0 ? b : b ^ 0x7fffffff;
+}
+__device__ __forceinline__ float ordered_to_float(int o) { return __int_as_float(o >= 0 ? o : o ^ 0x7fffffff); }
 
 // The 32-byte record of a row: what leaves a column group for shared memory and a unit for the workspace.
 //   scoring modes:  {m1, i1, m2, i2, lse2_max, lse2_sum, prefix2, count of larger logits}
@@ -684,6 +728,11 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
         c1 = temp > 0.f ? 1.4426950408889634f / temp : 0.f;
         neg_tl2 = -temp * 0.6931471805599453f;
       }
+      if (Mode<MODE>::skip && valid && p.row_floor != nullptr) {
+        // what earlier units of this row (other strips) found as their second best: nothing below it matters
+        st.floor = ordered_to_float(__ldcg(p.row_floor + row));
+        st.thrz = skip_threshold_z(st.floor, st.m2, c1, neg_tl2);
+      }
       Candidate* cand_list = nullptr;
       int* cand_count = nullptr;
       if (Mode<MODE>::collect && valid) {
@@ -754,6 +803,9 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
           if (valid) {
             float4* dst = reinterpret_cast<float4*>(p.partials + (size_t)w.strip * (size_t)p.T_pad + row);
             record_pack<MODE>(st, dst[0], dst[1]);
+            // this strip's second best is a lower bound of the row's: later units of the row skip below it
+            if (Mode<MODE>::skip && p.row_floor != nullptr && st.m2 > st.floor)
+              atomicMax(p.row_floor + row, float_to_ordered(st.m2));
           }
         }
         xch_phase ^= 1u;

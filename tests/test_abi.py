@@ -33,8 +33,8 @@ def test_host_only_entry_points():
     assert "workspace" in difr.difr_status_string(-4)
     assert difr.difr_status_string(-7)
     # plan-derived sizes: one 32-byte record per (row, strip), a 256-byte tail, and per row (padded to 256 rows)
-    # five floats of bounds, a counter and 64 eight-byte entries for the ids fp32 cannot decide
-    per_row = 5 * 4 + 4 + 64 * 8
+    # six floats of bounds, a counter and 64 eight-byte entries for the ids fp32 cannot decide
+    per_row = 6 * 4 + 4 + 64 * 8
     nbytes = difr.difr_workspace_bytes(4096, 3072, 128256)
     assert nbytes > 0 and (nbytes - 256 - per_row * 4096) % (32 * 4096) == 0
     assert (difr.difr_workspace_bytes(4097, 3072, 128256) - 256 - per_row * (4096 + 256)) % (32 * (4096 + 256)) == 0
@@ -189,7 +189,7 @@ def test_planning_is_remembered():
     try:
         difr.difr_debug_plan_override(7, 0, 0)
         T_pad = 16384
-        assert difr.difr_workspace_bytes(*shape) == 7 * 32 * T_pad + 256 + (5 * 4 + 4 + 64 * 8) * T_pad
+        assert difr.difr_workspace_bytes(*shape) == 7 * 32 * T_pad + 256 + (6 * 4 + 4 + 64 * 8) * T_pad
     finally:
         difr.difr_debug_plan_override()
     assert difr.difr_workspace_bytes(*shape) == first
