@@ -217,10 +217,10 @@ def kernel_source_digest():
 
 def captured_traffic(w):
     """dram__bytes_read.sum + dram__bytes_write.sum of one fused-kernel launch on this workload, from the ncu
-    capture recorded in profiles/k1_fused_score_traffic.json; None when there is no capture for the workload or
+    capture recorded in profiles/k1_fused_score_traffic.txt; None when there is no capture for the workload or
     the kernel's sources have changed since it was taken.  A capture taken at fewer rows is scaled by the rows
     (W is streamed once per group of rows, so traffic grows in proportion)."""
-    path = os.path.join(ROOT, "profiles", "k1_fused_score_traffic.json")
+    path = os.path.join(ROOT, "profiles", "k1_fused_score_traffic.txt")
     if not os.path.exists(path):
         return None, "no capture"
     with open(path) as f:
@@ -325,6 +325,23 @@ class Problem:
         difr.difr_detect(o.score, self.tau, o.margin, None, 0, self.seq, self.flags, self.stats)
         if ev is not None:
             events.record(ev[3], stream)
+
+    def detect_us_back_to_back(self, n=200):
+        """Microseconds per difr_detect call when many are enqueued back to back (two events around all of them):
+        what the kernel costs a stream that is kept busy, without the event records between single launches."""
+        import torch
+
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        o = self.out
+        for _ in range(10):
+            self.difr.difr_detect(o.score, self.tau, o.margin, None, 0, self.seq, self.flags, self.stats)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(n):
+            self.difr.difr_detect(o.score, self.tau, o.margin, None, 0, self.seq, self.flags, self.stats)
+        b.record()
+        torch.cuda.synchronize()
+        return 1e3 * a.elapsed_time(b) / n
 
     def host_us_per_call(self, n=8):
         """Host time of one difr_score_gm call through the raw C ABI (arguments marshalled beforehand)."""
@@ -520,6 +537,7 @@ def per_config_entry(difr, w, temperature, sigma, events, local_rank, barrier, p
     steps = int(min(2000, max(3, np.ceil(1100.0 / est_ms))))
     elapsed, (k1, k2, k3), clocks = timed_steps(prob, steps, 3, events, local_rank, barrier)
     host_us = prob.host_us_per_call()
+    k3_us = prob.detect_us_back_to_back()
     roof = roofline_of(difr, w, k1, k2, k3, peaks, prob.n_seq)
     mhz = clocks.get("sm_mhz")
     entry = {
@@ -530,7 +548,8 @@ def per_config_entry(difr, w, temperature, sigma, events, local_rank, barrier, p
         "fused_ms": k1, "fused_ms_x_sm_mhz": (k1 * mhz) if mhz else None,
         "traffic": roof["traffic"], "traffic_source": roof["traffic_source"],
         "k2_finalize": {k: roof["other_kernels"]["k2_finalize"][k] for k in ("ms_per_launch", "achieved", "frac")},
-        "k3_detect": {k: roof["other_kernels"]["k3_detect"][k] for k in ("ms_per_launch", "achieved", "frac")},
+        "k3_detect": dict({k: roof["other_kernels"]["k3_detect"][k] for k in ("ms_per_launch", "achieved", "frac")},
+                          us_back_to_back=k3_us),
         "host_us_per_call": host_us, "clocks": clocks,
         "detect": {"threshold": prob.tau, "n_flagged": int(prob.flags.sum().item()),
                    "n_tampered": int(prob.tampered.sum())},
@@ -574,6 +593,13 @@ def run_ours(args):
     flags_ref = prob.flags.cpu().clone()
     stats_np = prob.stats.cpu().numpy()
     host_us = prob.host_us_per_call()
+    k3_us = prob.detect_us_back_to_back()
+    k3_us_one_sequence = None
+    if world == 1:
+        seq_keep, stats_keep = prob.seq, prob.stats
+        prob.seq, prob.stats = None, torch.empty((1, 4), dtype=torch.int32, device="cuda")
+        k3_us_one_sequence = prob.detect_us_back_to_back()  # seq_offsets == NULL: all T rows are one sequence
+        prob.seq, prob.stats = seq_keep, stats_keep
 
     # ---- end to end
     e2e_ms, h2d, d2h, e2e_flags = e2e_rate(prob, args.steps, args.warmup, barrier)
@@ -632,6 +658,8 @@ def run_ours(args):
         roof = roofline_of(difr, w, k1_ms, k2_ms, k3_ms, peaks, T // w.seq_len)
         mhz = clocks.get("sm_mhz")
         roof["ms_per_launch_x_sm_mhz"] = (k1_ms * mhz) if mhz else None
+        roof["other_kernels"]["k3_detect"]["us_back_to_back"] = k3_us
+        roof["other_kernels"]["k3_detect"]["us_back_to_back_one_sequence"] = k3_us_one_sequence
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
