@@ -425,6 +425,38 @@ __device__ __forceinline__ double warp_dot(const uint16_t* a, const uint16_t* b,
   return acc;
 }
 
+// Up to three such dot products against the same row a, their loads in flight together; a null row gives 0.
+// Each sum is taken in warp_dot's order, so the values are the same as separate calls.
+__device__ __forceinline__ void warp_dot3(const uint16_t* a, const uint16_t* b0, const uint16_t* b1,
+                                          const uint16_t* b2, int d, int lane, double out[3]) {
+  const uint16_t* b[3] = {b0, b1, b2};
+  double acc[3] = {0.0, 0.0, 0.0};
+  for (int k = lane * 8; k < d; k += 32 * 8) {
+    const uint4 va = *reinterpret_cast<const uint4*>(a + k);
+    uint4 vb[3];
+#pragma unroll
+    for (int j = 0; j < 3; ++j)
+      vb[j] = b[j] != nullptr ? *reinterpret_cast<const uint4*>(b[j] + k) : make_uint4(0u, 0u, 0u, 0u);
+    const uint32_t wa[4] = {va.x, va.y, va.z, va.w};
+#pragma unroll
+    for (int j = 0; j < 3; ++j) {
+      const uint32_t wb[4] = {vb[j].x, vb[j].y, vb[j].z, vb[j].w};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        acc[j] = fma(bf16_to_double(wa[q] & 0xFFFFu), bf16_to_double(wb[q] & 0xFFFFu), acc[j]);
+        acc[j] = fma(bf16_to_double(wa[q] >> 16), bf16_to_double(wb[q] >> 16), acc[j]);
+      }
+    }
+  }
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) {
+#pragma unroll
+    for (int j = 0; j < 3; ++j) acc[j] += shfl_xor_double(acc[j], m);
+  }
+#pragma unroll
+  for (int j = 0; j < 3; ++j) out[j] = acc[j];
+}
+
 __device__ __forceinline__ double gumbel_exact(uint64_t seed, uint32_t position, uint32_t id) {
   uint32_t x[4];
   philox4x32_10(id >> 2, position, 0u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), x);

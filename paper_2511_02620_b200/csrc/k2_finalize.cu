@@ -70,12 +70,14 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
   acc.lmax = -CUDART_INF;
   acc.lsum = acc.lpre = 0.0;
   acc.larger = 0;
+  uint32_t tie_bits = 0u;  // bit j: this lane's record of slot lane + 32 j carries the fused kernel's tie mark
   for (int slot = lane; slot < p.n_slots; slot += 32) {
     const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * (size_t)p.T_pad + row);
     const float4 a = src[0], b = src[1];
     top2_insert(acc, a.x, __float_as_int(a.y));
     top2_insert(acc, a.z, __float_as_int(a.w));
     lse_merge(acc, (double)b.x, (double)fabsf(b.y), (double)b.z);  // (the sign bit of the sum is the tie mark)
+    if (signbit(b.y) && slot < 1024) tie_bits |= 1u << (slot >> 5);
     acc.larger += __float_as_int(b.w);
   }
 #pragma unroll
@@ -119,52 +121,51 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
   if (temp_bad) status |= 8u;
   const double lse = (temp_f > 0.f) ? (acc.lmax + log2(acc.lsum)) * ln2 : CUDART_NAN;
 
-  // the exact logit of the claimed token
-  double l_tok = 0.0;
-  if (tok_ok) l_tok = warp_dot(hrow, p.W + (size_t)tok * (size_t)p.d, p.d, lane);
-
-  // raw-logit rank: the fused kernel counted the ids whose fp32 logit is above the claimed one by more than the
-  // tensor cores' rounding; the ids it could not decide are on the row's list and are decided here in fp64
-  if (p.rank != nullptr && p.band_count != nullptr && tok_ok) {
-    const int n_found = p.band_count[row];
-    const int n_band = n_found < p.band_cap ? n_found : p.band_cap;
-    if (n_found > p.band_cap) status |= 32u;
-    const BandEntry* list = p.band_list + (size_t)row * (size_t)p.band_cap;
-    for (int e = 0; e < n_band; ++e) {
-      const int id = list[e].id;
-      const double l = warp_dot(hrow, p.W + (size_t)id * (size_t)p.d, p.d, lane);
-      acc.larger += (l > l_tok) ? 1 : 0;
+  // ---- exact (fp64) values.  Token-DiFR: y = l + Temp * G of the claimed token and of every candidate that can
+  // be among the two largest.  The fused kernel ranks by fp32 keys whose error (tensor-core accumulation,
+  // lg2.approx in the noise, the index bits in the low mantissa) is bounded by `noise`; an id whose exact y is
+  // among the two largest has a key within 2 * noise of the second largest key, so every candidate of the strips'
+  // records inside that window is re-evaluated and the two largest are taken exactly (ties: lowest id).  The dot
+  // products go three at a time (the claimed token and, normally, the two candidates) with their loads in flight
+  // together.
+  double l_tok = 0.0, yt = -CUDART_INF;
+  double yb1 = -CUDART_INF, yb2 = -CUDART_INF;
+  int ib1 = -1, ib2 = -1;
+  auto place = [&](double y, int id) {
+    if (id == ib1 || id == ib2) return;  // (a group that is walked whole can bring an id a second time)
+    if (ib1 < 0 || y > yb1 || (y == yb1 && id < ib1)) {
+      yb2 = yb1; ib2 = ib1;
+      yb1 = y; ib1 = id;
+    } else if (ib2 < 0 || y > yb2 || (y == yb2 && id < ib2)) {
+      yb2 = y; ib2 = id;
     }
-  }
-
+  };
+  int pend[3] = {-1, -1, -1};
+  int n_pend = 0;
+  auto flush = [&]() {
+    if (n_pend == 0) return;
+    double l[3];
+    warp_dot3(hrow, pend[0] >= 0 ? p.W + (size_t)pend[0] * (size_t)p.d : nullptr,
+              pend[1] >= 0 ? p.W + (size_t)pend[1] * (size_t)p.d : nullptr,
+              pend[2] >= 0 ? p.W + (size_t)pend[2] * (size_t)p.d : nullptr, p.d, lane, l);
+#pragma unroll
+    for (int i = 0; i < 3; ++i) {
+      if (pend[i] < 0) continue;
+      const double y = (p.ipt != 1) ? l[i] + temp * gumbel_exact(seed, pos, (uint32_t)pend[i]) : 0.0;
+      if (pend[i] == tok) { l_tok = l[i]; yt = y; }
+      if (p.ipt != 1) place(y, pend[i]);
+      pend[i] = -1;
+    }
+    n_pend = 0;
+  };
+  auto push = [&](int id) {
+    if (n_pend == 0) pend[0] = id; else if (n_pend == 1) pend[1] = id; else pend[2] = id;
+    if (++n_pend == 3) flush();
+  };
+  if (tok_ok) push(tok);
   if (p.ipt != 1) {
-    // ---- Token-DiFR: exact y = l + Temp * G of the claimed token and of every candidate that can be among the
-    // two largest.  The fused kernel ranks by fp32 keys whose error (tensor-core accumulation, lg2.approx in the
-    // noise, the index bits in the low mantissa) is bounded by `noise`; an id whose exact y is among the two
-    // largest has a key within 2 * noise of the second largest key, so every candidate of the strips' records
-    // inside that window is re-evaluated in fp64 and the two largest are taken exactly (ties: lowest id).
     const float noise = 3e-4f * temp_f + 1e-4f + 3.9e-6f * fabsf(acc.m2);
     const float window = acc.m2 - 2.f * noise;  // -inf when there is no second candidate: everything qualifies
-    double yb1 = -CUDART_INF, yb2 = -CUDART_INF;
-    int ib1 = -1, ib2 = -1;
-    auto place = [&](double y, int id) {
-      if (id == ib1 || id == ib2) return;  // (a group that is walked whole can bring an id a second time)
-      if (ib1 < 0 || y > yb1 || (y == yb1 && id < ib1)) {
-        yb2 = yb1; ib2 = ib1;
-        yb1 = y; ib1 = id;
-      } else if (ib2 < 0 || y > yb2 || (y == yb2 && id < ib2)) {
-        yb2 = y; ib2 = id;
-      }
-    };
-    auto place_id = [&](int cid) {
-      const double l = warp_dot(hrow, p.W + (size_t)cid * (size_t)p.d, p.d, lane);
-      place(l + temp * gumbel_exact(seed, pos, (uint32_t)cid), cid);
-    };
-    double yt = -CUDART_INF;
-    if (tok_ok) {
-      yt = l_tok + temp * gumbel_exact(seed, pos, (uint32_t)tok);
-      place(yt, tok);
-    }
     for (int base = 0; base < p.n_slots; base += 32) {
       const int slot = base + lane;
       float4 a = make_float4(-CUDART_INF_F, __int_as_float(-1), -CUDART_INF_F, __int_as_float(-1));
@@ -172,7 +173,7 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
       if (slot < p.n_slots) {
         const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * (size_t)p.T_pad + row);
         a = src[0];
-        tie_mark = signbit(src[1].y);
+        tie_mark = base < 1024 ? ((tie_bits >> (base >> 5)) & 1u) != 0u : signbit(src[1].y);
       }
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
@@ -189,13 +190,35 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
             // candidate's group is a candidate
             const int g0 = cid & ~15;
             for (int v = g0; v < g0 + 16 && v < p.V; ++v)
-              if (v != tok) place_id(v);
+              if (v != tok) push(v);
           } else if (cid != tok) {
-            place_id(cid);
+            push(cid);
           }
         }
       }
     }
+  }
+  flush();
+
+  // raw-logit rank: the fused kernel counted the ids whose fp32 logit is above the claimed one by more than the
+  // tensor cores' rounding; the ids it could not decide are on the row's list and are decided here in fp64
+  if (p.rank != nullptr && p.band_count != nullptr && tok_ok) {
+    const int n_found = p.band_count[row];
+    const int n_band = n_found < p.band_cap ? n_found : p.band_cap;
+    if (n_found > p.band_cap) status |= 32u;
+    const BandEntry* list = p.band_list + (size_t)row * (size_t)p.band_cap;
+    for (int e = 0; e < n_band; e += 3) {
+      double l[3];
+      const int i0 = list[e].id, i1 = e + 1 < n_band ? list[e + 1].id : -1, i2 = e + 2 < n_band ? list[e + 2].id : -1;
+      warp_dot3(hrow, p.W + (size_t)i0 * (size_t)p.d, i1 >= 0 ? p.W + (size_t)i1 * (size_t)p.d : nullptr,
+                i2 >= 0 ? p.W + (size_t)i2 * (size_t)p.d : nullptr, p.d, lane, l);
+      acc.larger += (l[0] > l_tok) ? 1 : 0;
+      acc.larger += (i1 >= 0 && l[1] > l_tok) ? 1 : 0;
+      acc.larger += (i2 >= 0 && l[2] > l_tok) ? 1 : 0;
+    }
+  }
+
+  if (p.ipt != 1) {
     if (lane == 0) {
       double A = -CUDART_INF;
       if (tok_ok) {
