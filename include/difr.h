@@ -226,11 +226,16 @@ difr_status difr_score_both(const void* h, const void* W, const int32_t* tokens,
  * mass reaches top_p.  The expectation is evaluated by Gauss-Legendre quadrature
  * (512 nodes over the range that carries the mass), not by sampling.
  *
- *   filter->top_k  0: no top-k; otherwise 1..128 (a top_k >= V filters nothing)
+ *   filter->top_k  0: no top-k; otherwise >= 1 (a top_k >= V filters nothing)
  *   filter->top_p  in (0, 1]; 1: no nucleus.  With no top-k in front of it the nucleus is the
- *                  shortest prefix that holds top_p of the whole row's softmax mass, and it is
- *                  resolved among the 128 largest logits: a row whose 128 largest logits hold
- *                  less than that gets row_status bit 4 and the 128th largest logit as cutoff
+ *                  shortest prefix that holds top_p of the whole row's softmax mass.
+ *   Filters of any size: with one policy for the whole call (no *_rows arrays), a top_k above 128 or a
+ *   nucleus over the whole vocabulary is resolved exactly by a selection over the rows' logits, which are
+ *   written out a block of rows at a time (about 1 GiB of the workspace) by the tensor-core main loop: one
+ *   more pass over the logits plus the selection (a dozen walks over each row, from L2).  Per-row policies
+ *   (the *_rows arrays) are resolved among each row's 128 largest logits: a row's top_k must be <= 128 (or
+ *   >= V), and a row whose whole-vocabulary nucleus holds more than 128 ids gets row_status bit 4 and the
+ *   128th largest logit as cutoff.
  *   filter->s      1..8
  *   filter->min_p  in [0, 1]; 0: none.  min-p (Sec. "Sampling From Large Language Models") keeps the ids whose
  *                  probability is at least min_p times the largest one, i.e. whose logit reaches
@@ -280,10 +285,11 @@ difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* 
  * CDF in vocabulary-id order; a claimed id the filter removed has p = 0 and
  * scores ln(eps).
  *
- *   filter->top_k 1..128 (or >= V when V <= 128), or 0 with top_p < 1: a nucleus over the whole
- *   vocabulary as in difr_score_gm_filtered (row_status bit 4 when it holds more than 128 ids);
- *   filter->top_p in (0, 1]; filter->min_p in [0, 1] (the ids that reach l_max + Temp ln(min_p); resolved
- *   among the 128 largest logits, row_status bit 4 when more survive); filter->s is ignored; per-row values
+ *   filter->top_k and filter->top_p as in difr_score_gm_filtered (any size with one policy for the call:
+ *   the selection also sums the kept ids' masses; per-row policies within the 128 largest logits);
+ *   filter->top_p in (0, 1]; filter->min_p in [0, 1] (the ids that reach l_max + Temp ln(min_p); any number of them
+ *   with one policy for the call, else resolved among the 128 largest logits with row_status bit 4 when more
+ *   survive); filter->s is ignored; per-row values
  *   as in difr_score_gm_filtered (a row whose own policy filters nothing keeps the unfiltered score)
  *   temperature > 0; out->workspace needs difr_filtered_workspace_bytes(T, d, V)
  * Writes score, p_claimed, cdf_lo, u, row_status, out->cutoff (optional) and

@@ -7,7 +7,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(CSRC, "libdifr.so")
-SOURCES = ["difr_api.cu", "k0_expand_seeds.cu", "k1_fused_score.cu", "k2_finalize.cu", "k2_filtered.cu", "k3_detect.cu"]
+SOURCES = ["difr_api.cu", "k0_expand_seeds.cu", "k1_fused_score.cu", "k2_finalize.cu", "k2_filtered.cu", "k2_select.cu", "k3_detect.cu"]
 HEADERS = ["difr_device.cuh", "difr_kernels.h", "difr_plan.h", os.path.join("..", "..", "include", "difr.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC"]

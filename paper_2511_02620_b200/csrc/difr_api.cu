@@ -332,15 +332,32 @@ constexpr int kFilterFloorStrips = 32;
 constexpr int kFilterMinStrips = 64;   // vocabularies with fewer tiles than this list every id instead
 constexpr int kFilterMaxStrips = 128;  // the bounds kernel reads at most 128 strips' records per row
 
-// Layout behind the ordinary workspace: per-row candidate counters, then the candidate lists.
+// Rows whose logits are written out at a time for filters of any size: about a gibibyte of fp32 logits.
+static int select_chunk_rows(int64_t T_pad, int64_t V) {
+  int64_t rows = (((int64_t)1 << 30) / (4 * V)) & ~(int64_t)255;
+  if (rows < 256) rows = 256;
+  if (rows > T_pad) rows = T_pad;
+  return (int)rows;
+}
+
+// Layout behind the ordinary workspace: per-row candidate counters, the candidate lists, and for filters of any
+// size six per-row words of the selection's results and the block of logits it reads.
 static bool filtered_layout(int64_t T, int64_t d, int64_t V, int pairs, int min_strips, Plan* pl, int* cap,
-                            size_t* count_off, size_t* list_off, size_t* total) {
+                            size_t* count_off, size_t* list_off, size_t* total, size_t* sel_off = nullptr,
+                            size_t* logits_off = nullptr) {
   if (!make_plan(T, d, V, pairs, pl, min_strips, kFilterMaxStrips)) return false;
   // with fewer than 64 vocabulary tiles the strips' maxima cannot bound the 128-th largest logit: keep every id
   *cap = (pl->n_tiles < kFilterMinStrips) ? (int)V : kCandCap;
   *count_off = (pl->workspace_bytes + 255) & ~(size_t)255;
   *list_off = *count_off + (((size_t)pl->T_pad * sizeof(int) + 255) & ~(size_t)255);
-  *total = *list_off + (size_t)T * (size_t)*cap * sizeof(Candidate);
+  const size_t sel = (*list_off + (size_t)T * (size_t)*cap * sizeof(Candidate) + 255) & ~(size_t)255;
+  // selection results: three ints and three doubles per padded row, each array 256-byte aligned
+  const size_t ints = ((size_t)pl->T_pad * sizeof(int) + 255) & ~(size_t)255;
+  const size_t dbls = ((size_t)pl->T_pad * sizeof(double) + 255) & ~(size_t)255;
+  const size_t lg = sel + 3 * ints + 3 * dbls;
+  if (sel_off) *sel_off = sel;
+  if (logits_off) *logits_off = lg;
+  *total = lg + (size_t)select_chunk_rows(pl->T_pad, V) * (size_t)V * sizeof(float);
   return true;
 }
 
@@ -374,7 +391,7 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
   const float top_p = filter->top_p;
   const int s_comp = ipt ? 0 : filter->s;  // the IPT estimator has no competitors
   if (!ipt && (filter->s < 1 || filter->s > 8)) return DIFR_ERR_INVALID_ARG;
-  if (filter->top_k_rows == nullptr && (top_k < 0 || (top_k > 128 && top_k < V))) return DIFR_ERR_INVALID_ARG;
+  if (filter->top_k_rows == nullptr && top_k < 0) return DIFR_ERR_INVALID_ARG;
   if (filter->top_p_rows == nullptr && (!(top_p > 0.f) || !(top_p <= 1.f))) return DIFR_ERR_INVALID_ARG;
   const float min_p = filter->min_p;
   if (filter->min_p_rows == nullptr && (!(min_p >= 0.f) || !(min_p <= 1.f))) return DIFR_ERR_INVALID_ARG;
@@ -390,17 +407,27 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
   if (info.major != 10) return DIFR_ERR_ARCH;
   Plan pl;
   int cap;
-  size_t count_off, list_off, total;
+  size_t count_off, list_off, total, sel_off, logits_off;
+  // One policy for the whole call whose kept set can exceed what the candidate lists resolve (a top-k above
+  // 128, a nucleus or a min-p set over the whole vocabulary): the kept prefix is found by selection over the
+  // rows' logits, written out a block of rows at a time.  (Per-row policies stay within the lists' reach.)
+  const bool scalar_policy = !filter->top_k_rows && !filter->top_p_rows && !filter->min_p_rows;
+  const bool whole_vocab = top_k < 1 || top_k >= V;
+  const bool select_path = scalar_policy && V > 128 &&
+                           ((!whole_vocab && top_k > 128) || (whole_vocab && top_p < 1.f) ||
+                            (ipt && whole_vocab && min_p > 0.f));
   // the largest number of ids any row resolves by logit rank (a nucleus without a top-k resolves 128)
   int k_max = 128;
-  if (filter->top_k_rows == nullptr) {
-    const bool whole = top_k < 1 || top_k >= V;
-    if (!whole) k_max = top_k;
+  if (select_path) {
+    k_max = (min_p_on && !ipt) ? 1 : 0;
+  } else if (filter->top_k_rows == nullptr) {
+    if (!whole_vocab) k_max = top_k;
     else if (filter->top_p_rows == nullptr && top_p >= 1.f) k_max = (min_p_on && ipt) ? 128 : 0;
   }
   const int min_strips =
       k_max < kFilterFloorStrips ? kFilterFloorStrips : (k_max > kFilterMaxStrips ? kFilterMaxStrips : k_max);
-  if (!filtered_layout(T, d, V, info.pairs, min_strips, &pl, &cap, &count_off, &list_off, &total))
+  if (!filtered_layout(T, d, V, info.pairs, min_strips, &pl, &cap, &count_off, &list_off, &total, &sel_off,
+                       &logits_off))
     return DIFR_ERR_SHAPE;
   if (!aligned16(h) || !aligned16(W)) return DIFR_ERR_ALIGN;
   if (!out->workspace || out->workspace_bytes < total) return DIFR_ERR_WORKSPACE;
@@ -453,6 +480,48 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
   fp.score = out->score; fp.cutoff = out->cutoff; fp.row_status = out->row_status;
   if (ipt) {
     fp.p_claimed = out->p_claimed; fp.cdf_lo = out->cdf_lo; fp.u = out->u;
+  }
+  if (select_path) {
+    // ---- logits of a block of rows (the fused kernel's main loop in its dump mode), then the selection
+    const size_t ints = ((size_t)pl.T_pad * sizeof(int) + 255) & ~(size_t)255;
+    const size_t dbls = ((size_t)pl.T_pad * sizeof(double) + 255) & ~(size_t)255;
+    int* sel_cut = reinterpret_cast<int*>(ws + sel_off);
+    int* sel_top = reinterpret_cast<int*>(ws + sel_off + ints);
+    int* sel_n = reinterpret_cast<int*>(ws + sel_off + 2 * ints);
+    double* sel_z = reinterpret_cast<double*>(ws + sel_off + 3 * ints);
+    double* sel_below = reinterpret_cast<double*>(ws + sel_off + 3 * ints + dbls);
+    double* sel_mine = reinterpret_cast<double*>(ws + sel_off + 3 * ints + 2 * dbls);
+    float* logits_buf = reinterpret_cast<float*>(ws + logits_off);
+    const int chunk = select_chunk_rows(pl.T_pad, V);
+    for (int64_t r0 = 0; r0 < T; r0 += chunk) {
+      const int64_t rows = T - r0 < chunk ? T - r0 : chunk;
+      Plan pc;
+      if (!make_plan(rows, d, V, info.pairs, &pc)) return DIFR_ERR_SHAPE;
+      CUtensorMap tmap_hc;
+      const unsigned char* h_chunk = static_cast<const unsigned char*>(h) + (size_t)r0 * (size_t)d * 2;
+      if (!make_tmap(&tmap_hc, h_chunk, rows, d, kBM)) return DIFR_ERR_CUDA;
+      K1Params kd = k1_params(pc, rows, d, V, 1.f, nullptr);  // no counter: units go round robin
+      kd.logits_out = logits_buf;
+      kd.device_status = out->device_status;
+      if (launch_k1(2, tmap_hc, tmap_w, kd, k1_grid(pc, info.pairs), s) != cudaSuccess) return DIFR_ERR_CUDA;
+      SelectParams sp;
+      memset(&sp, 0, sizeof sp);
+      sp.logits = logits_buf; sp.rows = (int)rows; sp.V = (int)V; sp.row0 = (int)r0;
+      sp.tokens = tokens; sp.temperatures = out->temperatures; sp.temperature = temperature;
+      sp.top_k = top_k; sp.top_p = top_p;
+      sp.min_p = ipt ? min_p : 0.f;  // Token-DiFR takes the min-p bound itself as cutoff (exact l_max, below)
+      sp.cut_id = sel_cut; sp.top_id = sel_top; sp.kept_n = sel_n;
+      sp.kept_z = sel_z; sp.kept_below = sel_below; sp.kept_mine = sel_mine;
+      sp.row_status = out->row_status;
+      if (launch_select_cutoff(sp, s) != cudaSuccess) return DIFR_ERR_CUDA;
+    }
+    fp.sel_cut_id = sel_cut; fp.sel_top_id = sel_top; fp.sel_kept_n = sel_n;
+    fp.sel_z = sel_z; fp.sel_below = sel_below; fp.sel_mine = sel_mine;
+    if (ipt) {
+      // the selection has summed the kept set: no candidate lists are needed
+      if (launch_ipt_select_finalize(fp, s) != cudaSuccess) return DIFR_ERR_CUDA;
+      return DIFR_OK;
+    }
   }
   if (launch_filter_bounds(fp, s) != cudaSuccess) return DIFR_ERR_CUDA;
   if (cudaMemsetAsync(ws + count_off, 0, (size_t)pl.T_pad * sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;

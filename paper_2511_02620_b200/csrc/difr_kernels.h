@@ -152,10 +152,38 @@ struct FilterParams {
   float* p_claimed;  // IPT finalize only, nullable
   float* cdf_lo;
   float* u;
+  // filters of any size (one policy for the whole call): the kept prefix found by select_cutoff; null otherwise
+  const int* sel_cut_id;
+  const int* sel_top_id;
+  const int* sel_kept_n;  // negative: the min-p bound ended the prefix
+  const double* sel_z;
+  const double* sel_below;
+  const double* sel_mine;
 };
 cudaError_t launch_filter_bounds(const FilterParams& p, cudaStream_t stream);
 cudaError_t launch_filtered_finalize(const FilterParams& p, cudaStream_t stream);
 cudaError_t launch_ipt_filtered_finalize(const FilterParams& p, cudaStream_t stream);
+cudaError_t launch_ipt_select_finalize(const FilterParams& p, cudaStream_t stream);
+
+// Filters of any size: exact length and last id of the kept prefix from a block of rows' fp32 logits.
+struct SelectParams {
+  const float* logits;   // [rows][V]: the logits of rows row0 .. row0 + rows - 1
+  int rows, V, row0;
+  const int32_t* tokens;       // [T]
+  const float* temperatures;   // [T], nullable
+  float temperature;
+  int top_k;      // 0 or >= V: none
+  float top_p;    // 1: none
+  float min_p;    // 0: none
+  int* cut_id;    // [T] out: the last kept id in the order (logit descending, id ascending)
+  int* top_id;    // [T] out: the id of the largest logit (lowest id among equals)
+  int* kept_n;    // [T] out: how many ids are kept; negated when the min-p bound ended the prefix
+  double* kept_z;      // [T] out: mass of the kept ids, of those below the claimed id, of the claimed id if kept,
+  double* kept_below;  //         all in units of 2^-40 of the row's largest term
+  double* kept_mine;
+  uint32_t* row_status;  // nullable: bit 4 when more than 256 ids tie exactly at the cutoff
+};
+cudaError_t launch_select_cutoff(const SelectParams& p, cudaStream_t stream);
 
 struct BitsParams {
   const uint8_t* classes;

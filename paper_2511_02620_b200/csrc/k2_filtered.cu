@@ -77,7 +77,8 @@ __device__ __forceinline__ RowPolicy row_policy(const FilterParams& p, int row) 
   r.bad = !(r.temperature > 0.f) || isinf(r.temperature) || k < 0 || !(r.top_p > 0.f) || !(r.top_p <= 1.f) ||
           !(r.min_p >= 0.f) || !(r.min_p <= 1.f);
   if (k > p.V) k = p.V;
-  if (k > kMaxK && k < p.V) r.bad = true;
+  const bool selected = p.sel_cut_id != nullptr;  // one policy for the call, resolved by the selection kernel
+  if (k > kMaxK && k < p.V && !selected) r.bad = true;
   const bool whole = k < 1 || k >= p.V;  // no top-k in effect
   r.nucleus_full = (whole && r.top_p < 1.f) ? 1 : 0;
   r.by_rank = !whole || r.nucleus_full;
@@ -88,6 +89,11 @@ __device__ __forceinline__ RowPolicy row_policy(const FilterParams& p, int row) 
     // min-p alone: the IPT estimator needs the surviving ids (resolved among the largest kMaxK), Token-DiFR
     // only the largest logit
     if (r.min_p > 0.f) k = p.ipt ? (kMaxK < p.V ? kMaxK : p.V) : (k > 1 ? k : 1);
+  }
+  if (selected && !r.bad) {
+    // the cutoff by rank comes from the selection: only the min-p bound still needs the largest logit here
+    k = (r.min_p > 0.f && !p.ipt) ? 1 : 0;
+    r.nucleus_full = 0;
   }
   if (r.bad) { k = 0; r.nucleus_full = 0; r.by_rank = false; r.none = false; }
   r.top_k = k;
@@ -288,7 +294,12 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
     }
   }
   __syncwarp();
-  if (k_eff > 0 && rp.by_rank) {
+  if (p.sel_cut_id != nullptr && rp.by_rank) {
+    // a filter of any size: the last kept id was found by the selection over the row's logits
+    const int cid = p.sel_cut_id[row];
+    if (cid >= 0 && cid < p.V)
+      cutoff = warp_dot(p.h + (size_t)row * (size_t)p.d, p.W + (size_t)cid * (size_t)p.d, p.d, lane);
+  } else if (k_eff > 0 && rp.by_rank) {
     double e[kChunks];
     cut_rank = nucleus_last_rank(p, rp, row, lane, sm_l[warp], k_eff, e, status_bits);
     // the cutoff is that id's logit: re-evaluated in fp64 like every other logit the score depends on
@@ -506,6 +517,65 @@ __global__ void __launch_bounds__(kFWarps * 32) ipt_filtered_finalize(const Filt
     if (p.cutoff) p.cutoff[row] = (float)cutoff;
     if (p.row_status && status_bits) p.row_status[row] |= status_bits;
   }
+}
+
+// Token-IPT-DiFR on a filtered distribution of any size: the selection kernel has summed the kept ids' masses
+// (all of them, those below the claimed id, the claimed id's own); what is left is the uniform, the interval
+// and the score, and the cutoff in fp64.  One warp per row.
+__global__ void __launch_bounds__(kFWarps * 32) ipt_select_finalize(const FilterParams p) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * kFWarps + warp;
+  if (row >= p.T) return;
+  const int tok = p.tokens[row];
+  const bool tok_ok = tok >= 0 && tok < p.V;
+  const RowPolicy rp = row_policy(p, row);
+  if (rp.bad || isnan(p.score[row])) {
+    if (lane == 0) {
+      if (rp.bad) {
+        p.score[row] = CUDART_NAN_F;
+        if (p.row_status) p.row_status[row] |= 8u;
+      }
+      if (p.cutoff) p.cutoff[row] = CUDART_NAN_F;
+    }
+    return;
+  }
+  const uint16_t* hrow = p.h + (size_t)row * (size_t)p.d;
+  const int cid = p.sel_cut_id[row], top = p.sel_top_id[row];
+  const bool by_min_p = p.sel_kept_n[row] < 0;  // the min-p bound, not the rank filter, ended the kept prefix
+  double cutoff = -CUDART_INF;
+  if (by_min_p && top >= 0 && top < p.V)
+    cutoff = warp_dot(hrow, p.W + (size_t)top * (size_t)p.d, p.d, lane) + (double)rp.temperature * log((double)rp.min_p);
+  else if (cid >= 0 && cid < p.V)
+    cutoff = warp_dot(hrow, p.W + (size_t)cid * (size_t)p.d, p.d, lane);
+  if (lane == 0) {
+    const uint64_t seed = p.seeds[row];
+    uint32_t x[4];
+    philox4x32_10(0u, p.positions[row], 1u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), x);
+    const double mu = ((double)x[0] + 0.5) * (1.0 / 4294967296.0);
+    double score = log((double)p.eps), pt = CUDART_NAN, a = CUDART_NAN;
+    if (tok_ok) {
+      const double z = p.sel_z[row];
+      a = p.sel_below[row] / z;
+      pt = p.sel_mine[row] / z;  // zero when the filter removed the claimed id
+      const double sigma = (double)p.sigma;
+      const double za = (a - mu) / sigma, zb = (a + pt - mu) / sigma, r2 = 0.70710678118654752440;
+      double mass;
+      if (za >= 0.0) mass = 0.5 * (erfc(za * r2) - erfc(zb * r2));
+      else if (zb <= 0.0) mass = 0.5 * (erfc(-zb * r2) - erfc(-za * r2));
+      else mass = 1.0 - 0.5 * erfc(zb * r2) - 0.5 * erfc(-za * r2);
+      score = log(mass + (double)p.eps);
+    }
+    p.score[row] = (float)score;
+    if (p.p_claimed) p.p_claimed[row] = (float)pt;
+    if (p.cdf_lo) p.cdf_lo[row] = (float)a;
+    if (p.u) p.u[row] = (float)mu;
+    if (p.cutoff) p.cutoff[row] = (float)cutoff;
+  }
+}
+
+cudaError_t launch_ipt_select_finalize(const FilterParams& p, cudaStream_t stream) {
+  ipt_select_finalize<<<(p.T + kFWarps - 1) / kFWarps, kFWarps * 32, 0, stream>>>(p);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_ipt_filtered_finalize(const FilterParams& p, cudaStream_t stream) {

@@ -1,0 +1,303 @@
+// Sampling filters of any size (a top-k above 128 ids, a nucleus over the whole vocabulary, a min-p set): the
+// filter keeps a prefix of the row's ids in the order (logit descending, id ascending), and this kernel finds the
+// length N of that prefix and its last id exactly, by radix selection over a block of rows whose fp32 logits the
+// fused kernel's main loop has written to memory (difr_logits' mode), one CTA per row:
+//
+//   top-k   keeps positions [0, K)
+//   top-p   keeps the shortest prefix whose softmax(l / Temp) mass reaches top_p of the mass of [0, K)
+//   min-p   keeps the ids whose logit reaches l_max + Temp ln(min_p), a prefix as well
+//
+// N is the smallest of the three.  Masses are summed as 64-bit fixed-point integers (2^-40 of the largest
+// term), so sums do not depend on the order of the additions and the result is the same on every run.  The
+// row (V floats) is walked up to a dozen times; after the first walk it is in L2.
+#include <cuda_runtime.h>
+#include <math_constants.h>
+
+#include "difr_kernels.h"
+
+namespace difr {
+
+constexpr int kSelThreads = 512;
+constexpr int kSelBins = 2048;
+constexpr int kSelTieCap = 256;
+
+// keys that ascend as the logit descends
+__device__ __forceinline__ uint32_t desc_key(float l) {
+  const uint32_t b = __float_as_uint(l);
+  return ~(b ^ ((b >> 31) ? 0xFFFFFFFFu : 0x80000000u));
+}
+
+struct SelShared {
+  unsigned int cnt[kSelBins];
+  unsigned long long mass[kSelBins];
+  unsigned int warp_cnt[kSelThreads / 32];
+  unsigned long long warp_mass[kSelThreads / 32];
+  unsigned int found_bin;
+  unsigned int c_before;
+  unsigned long long m_before;
+  unsigned int bin_cnt;
+  unsigned long long bin_mass;
+  float red_f[kSelThreads / 32];
+  unsigned long long red_u[kSelThreads / 32];
+  int tie_ids[kSelTieCap];
+  unsigned int tie_n;
+};
+
+struct Selected {
+  uint32_t key;            // key of the element found
+  unsigned int c_gt;       // elements with a larger logit
+  unsigned long long m_gt; // their mass
+  unsigned int ties;       // elements with exactly this logit
+  unsigned long long m_tie;  // mass of all of them
+};
+
+__device__ __forceinline__ unsigned long long fixed_mass(float l, float lmax, float c1) {
+  // 2^(c1 (l - lmax)) in units of 2^-40, rounded to nearest; terms below 2^-41 of the largest count as zero
+  const double e = exp2((double)c1 * ((double)l - (double)lmax));
+  return (unsigned long long)(e * 1099511627776.0 + 0.5);
+}
+
+// One radix selection over the row.  by_mass == false: the element at position `pos` (0-based) of the descending
+// order.  by_mass == true: the first element at which the cumulative mass reaches `target`.  Whole CTA.
+__device__ Selected radix_select(const float* row, int V, float lmax, float c1, bool by_mass, unsigned int pos,
+                                 unsigned long long target, SelShared& sh) {
+  uint32_t prefix = 0;       // the key bits decided so far (high bits)
+  int decided = 0;           // how many
+  unsigned int c_acc = 0;
+  unsigned long long m_acc = 0;
+  const int shifts[3] = {21, 10, 0};
+  const int widths[3] = {11, 11, 10};
+  Selected out;
+  for (int round = 0; round < 3; ++round) {
+    const int shift = shifts[round], width = widths[round];
+    for (int b = threadIdx.x; b < kSelBins; b += kSelThreads) { sh.cnt[b] = 0; sh.mass[b] = 0; }
+    if (threadIdx.x == 0) sh.found_bin = 0xFFFFFFFFu;
+    __syncthreads();
+    for (int v = threadIdx.x; v < V; v += kSelThreads) {
+      const float l = row[v];
+      const uint32_t k = desc_key(l);
+      if (decided == 0 || (k >> (32 - decided)) == prefix) {
+        const uint32_t bin = (k >> shift) & ((1u << width) - 1u);
+        atomicAdd(&sh.cnt[bin], 1u);
+        atomicAdd(&sh.mass[bin], fixed_mass(l, lmax, c1));
+      }
+    }
+    __syncthreads();
+    // block scan over the bins (four consecutive bins per thread), then the first bin that holds the answer
+    const int per = kSelBins / kSelThreads;
+    unsigned int tc = 0;
+    unsigned long long tm = 0;
+    for (int i = 0; i < per; ++i) { tc += sh.cnt[threadIdx.x * per + i]; tm += sh.mass[threadIdx.x * per + i]; }
+    unsigned int sc = tc;
+    unsigned long long sm = tm;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int m = 1; m < 32; m <<= 1) {
+      const unsigned int oc = __shfl_up_sync(0xffffffffu, sc, m);
+      const unsigned long long om = __shfl_up_sync(0xffffffffu, sm, m);
+      if (lane >= m) { sc += oc; sm += om; }
+    }
+    if (lane == 31) { sh.warp_cnt[warp] = sc; sh.warp_mass[warp] = sm; }
+    __syncthreads();
+    unsigned int base_c = c_acc;
+    unsigned long long base_m = m_acc;
+    for (int w = 0; w < warp; ++w) { base_c += sh.warp_cnt[w]; base_m += sh.warp_mass[w]; }
+    base_c += sc - tc;
+    base_m += sm - tm;  // sums of everything before this thread's first bin
+    const unsigned int start_c = base_c;
+    const unsigned long long start_m = base_m;
+    for (int i = 0; i < per; ++i) {
+      const int b = threadIdx.x * per + i;
+      const unsigned int bc = sh.cnt[b];
+      const unsigned long long bm = sh.mass[b];
+      const bool here = bc != 0 && (by_mass ? (base_m + bm >= target) : (base_c + bc > pos));
+      if (here) {
+        const unsigned int old = atomicMin(&sh.found_bin, (unsigned int)b);
+        (void)old;
+      }
+      base_c += bc;
+      base_m += bm;
+    }
+    __syncthreads();
+    unsigned int fb = sh.found_bin;
+    if (fb == 0xFFFFFFFFu) {
+      // the target lies beyond the row's total (rounding of the target): the last non-empty bin
+      if (threadIdx.x == 0) {
+        unsigned int last = 0;
+        for (int b = 0; b < (1 << width); ++b) if (sh.cnt[b] != 0) last = (unsigned int)b;
+        sh.found_bin = last;
+      }
+      __syncthreads();
+      fb = sh.found_bin;
+    }
+    if (threadIdx.x == fb / per) {  // the bin's owner knows what lies before it
+      unsigned int c = start_c;
+      unsigned long long m = start_m;
+      for (unsigned int b = (unsigned int)(threadIdx.x * per); b < fb; ++b) { c += sh.cnt[b]; m += sh.mass[b]; }
+      sh.c_before = c; sh.m_before = m; sh.bin_cnt = sh.cnt[fb]; sh.bin_mass = sh.mass[fb];
+    }
+    __syncthreads();
+    c_acc = sh.c_before;
+    m_acc = sh.m_before;
+    prefix = (prefix << width) | fb;
+    decided += width;
+    out.ties = sh.bin_cnt;
+    out.m_tie = sh.bin_mass;
+    __syncthreads();
+  }
+  out.key = prefix;
+  out.c_gt = c_acc;
+  out.m_gt = m_acc;
+  return out;
+}
+
+__device__ __forceinline__ float block_max(float v, SelShared& sh) {
+  for (int m = 16; m >= 1; m >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, m));
+  if ((threadIdx.x & 31) == 0) sh.red_f[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float r = sh.red_f[0];
+  for (int w = 1; w < kSelThreads / 32; ++w) r = fmaxf(r, sh.red_f[w]);
+  __syncthreads();
+  return r;
+}
+
+__device__ __forceinline__ unsigned long long block_sum(unsigned long long v, SelShared& sh) {
+  for (int m = 16; m >= 1; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
+  if ((threadIdx.x & 31) == 0) sh.red_u[threadIdx.x >> 5] = v;
+  __syncthreads();
+  unsigned long long r = 0;
+  for (int w = 0; w < kSelThreads / 32; ++w) r += sh.red_u[w];
+  __syncthreads();
+  return r;
+}
+
+__global__ void __launch_bounds__(kSelThreads) select_cutoff(const SelectParams p) {
+  __shared__ SelShared sh;
+  const int r_local = blockIdx.x;
+  const int row = p.row0 + r_local;
+  const float* lrow = p.logits + (size_t)r_local * (size_t)p.V;
+  const int V = p.V;
+  float temp = p.temperatures != nullptr ? p.temperatures[row] : p.temperature;
+  const bool usable = temp > 0.f && !isinf(temp);
+  if (!usable) temp = 1.f;  // (the finalize kernels mark such a row; keep the arithmetic finite here)
+  const float c1 = 1.4426950408889634f / temp;
+
+  float lm = -CUDART_INF_F;
+  for (int v = threadIdx.x; v < V; v += kSelThreads) lm = fmaxf(lm, lrow[v]);
+  const float lmax = block_max(lm, sh);
+
+  // total mass, and how many ids reach the min-p bound
+  const float bound = p.min_p > 0.f ? lmax + temp * logf(p.min_p) : -CUDART_INF_F;
+  unsigned long long tm = 0, tb = 0;
+  for (int v = threadIdx.x; v < V; v += kSelThreads) {
+    const float l = lrow[v];
+    tm += fixed_mass(l, lmax, c1);
+    tb += (l >= bound) ? 1u : 0u;
+  }
+  const unsigned long long m_total = block_sum(tm, sh);
+  const unsigned int n_minp = (unsigned int)block_sum(tb, sh);
+
+  const unsigned int k_eff = (p.top_k >= 1 && p.top_k < V) ? (unsigned int)p.top_k : (unsigned int)V;
+  unsigned int n_keep = k_eff;
+  Selected last;       // the selection whose position is N - 1, when one of them is
+  bool have_last = false;
+  unsigned int last_pos = 0;
+
+  unsigned long long m_topk = m_total;
+  if (k_eff < (unsigned int)V) {
+    const Selected sk = radix_select(lrow, V, lmax, c1, false, k_eff - 1, 0ull, sh);
+    const unsigned long long e = sk.ties ? sk.m_tie / sk.ties : 0ull;
+    m_topk = sk.m_gt + (unsigned long long)(k_eff - sk.c_gt) * e;
+    last = sk; have_last = true; last_pos = k_eff - 1;
+  }
+  if (p.top_p < 1.f) {
+    // the shortest prefix whose mass reaches top_p of the mass the top-k keeps
+    const double want = (double)p.top_p * (double)m_topk;
+    unsigned long long target = (unsigned long long)want;
+    if ((double)target < want) ++target;
+    if (target < 1ull) target = 1ull;
+    const Selected sn = radix_select(lrow, V, lmax, c1, true, 0u, target, sh);
+    const unsigned long long e = sn.ties ? sn.m_tie / sn.ties : 0ull;
+    unsigned int in_tie = sn.ties;
+    if (e > 0ull && target > sn.m_gt) {
+      const unsigned long long need = target - sn.m_gt;
+      const unsigned long long q = (need + e - 1ull) / e;
+      if (q < (unsigned long long)in_tie) in_tie = (unsigned int)q;
+    }
+    if (in_tie < 1u) in_tie = 1u;
+    const unsigned int n_nucleus = sn.c_gt + in_tie;
+    if (n_nucleus < n_keep) {
+      n_keep = n_nucleus;
+      last = sn; have_last = true; last_pos = n_nucleus - 1;
+    }
+  }
+  bool by_min_p = false;
+  if (n_minp >= 1u && n_minp < n_keep) { n_keep = n_minp; have_last = false; by_min_p = true; }
+  if (n_keep < 1u) n_keep = 1u;
+  if (n_keep > (unsigned int)V) n_keep = (unsigned int)V;
+  if (!have_last || last_pos != n_keep - 1u || !(last.c_gt <= n_keep - 1u && n_keep - 1u < last.c_gt + last.ties)) {
+    last = radix_select(lrow, V, lmax, c1, false, n_keep - 1u, 0ull, sh);
+  }
+
+  // the id at position N - 1: the (N - c_gt)-th lowest id among the elements with that logit
+  const unsigned int j = n_keep - 1u - last.c_gt;
+  if (threadIdx.x == 0) sh.tie_n = 0u;
+  __syncthreads();
+  for (int v = threadIdx.x; v < V; v += kSelThreads) {
+    if (desc_key(lrow[v]) == last.key) {
+      const unsigned int at = atomicAdd(&sh.tie_n, 1u);
+      if (at < (unsigned int)kSelTieCap) sh.tie_ids[at] = v;
+    }
+  }
+  __syncthreads();
+  const unsigned int n_tie = sh.tie_n < (unsigned int)kSelTieCap ? sh.tie_n : (unsigned int)kSelTieCap;
+  int cut_id = -1;
+  if (threadIdx.x == 0) sh.found_bin = n_tie ? (unsigned int)sh.tie_ids[0] : 0u;
+  __syncthreads();
+  for (unsigned int a = threadIdx.x; a < n_tie; a += kSelThreads) {
+    unsigned int before = 0;
+    for (unsigned int b = 0; b < n_tie; ++b) before += (sh.tie_ids[b] < sh.tie_ids[a]) ? 1u : 0u;
+    if (before == (j < n_tie ? j : n_tie - 1u)) sh.found_bin = (unsigned int)sh.tie_ids[a];
+  }
+  __syncthreads();
+  cut_id = (int)sh.found_bin;
+  __syncthreads();
+
+  // sums over the kept ids (Token-IPT-DiFR on the filtered distribution)
+  const int tok = p.tokens[row];
+  unsigned long long kz = 0, kb = 0, km = 0;
+  for (int v = threadIdx.x; v < V; v += kSelThreads) {
+    const float l = lrow[v];
+    const uint32_t k = desc_key(l);
+    if (k < last.key || (k == last.key && v <= cut_id)) {
+      const unsigned long long q = fixed_mass(l, lmax, c1);
+      kz += q;
+      if (v < tok) kb += q;
+      if (v == tok) km += q;
+    }
+  }
+  const unsigned long long z = block_sum(kz, sh), below = block_sum(kb, sh), mine = block_sum(km, sh);
+  // the id of the largest logit (the lowest such id)
+  if (threadIdx.x == 0) sh.found_bin = 0x7fffffffu;
+  __syncthreads();
+  for (int v = threadIdx.x; v < V; v += kSelThreads)
+    if (lrow[v] == lmax) atomicMin(&sh.found_bin, (unsigned int)v);
+  __syncthreads();
+  const int top_id = sh.found_bin == 0x7fffffffu ? -1 : (int)sh.found_bin;
+  if (threadIdx.x == 0) {
+    p.cut_id[row] = cut_id;
+    p.top_id[row] = top_id;
+    p.kept_n[row] = by_min_p ? -(int)n_keep : (int)n_keep;
+    p.kept_z[row] = (double)z;
+    p.kept_below[row] = (double)below;
+    p.kept_mine[row] = (double)mine;
+    if (sh.tie_n > (unsigned int)kSelTieCap && p.row_status != nullptr) p.row_status[row] |= 16u;
+  }
+}
+
+cudaError_t launch_select_cutoff(const SelectParams& p, cudaStream_t stream) {
+  if (p.rows <= 0) return cudaSuccess;
+  select_cutoff<<<p.rows, kSelThreads, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace difr

@@ -99,7 +99,6 @@ def test_bad_arguments_are_refused_on_the_host():
         return L.difr_score_gm_filtered(p, p, p, p, p, temperature, 128, 64, 1000, ctypes.byref(f), ctypes.byref(o), None)
 
     assert filtered(50, 0.95, 0) == INVALID and filtered(50, 0.95, 9) == INVALID   # 1 <= s <= 8
-    assert filtered(129, 1.0, 1) == INVALID                                        # top_k <= 128
     assert filtered(50, 0.0, 1) == INVALID and filtered(50, 1.5, 1) == INVALID
     assert filtered(50, 0.95, 4, temperature=0.0) == INVALID
     assert filtered(-1, 0.95, 4) == INVALID
@@ -109,8 +108,6 @@ def test_bad_arguments_are_refused_on_the_host():
     f0 = difr._CFilter(0, 1.0, 1)
     o = out()
     assert L.difr_score_ipt_filtered(p, p, p, p, p, 1.0, 128, 64, 1000, ctypes.byref(f0), ctypes.byref(o), None) == INVALID
-    f1 = difr._CFilter(129, 1.0, 1)
-    assert L.difr_score_ipt_filtered(p, p, p, p, p, 1.0, 128, 64, 1000, ctypes.byref(f1), ctypes.byref(o), None) == INVALID
 
     taus = (ctypes.c_float * 5)(-1.0, -2.0, -3.0, -4.0, -5.0)
     adm = lambda n, sigma=0.3: L.difr_admissible(p, p, p, p, 1.0, 128, 64, 1000, p, p, p, p, sigma, 1e-12, taus, n, p,

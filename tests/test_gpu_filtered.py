@@ -224,8 +224,10 @@ def _nucleus_sizes(h, W, temperature, top_p):
     (40, 64, 40, 2.0, 1.0, 0.4, 0.8, 3),      # the whole vocabulary is resolved: never flagged
 ])
 def test_nucleus_over_the_whole_vocabulary(T, d, V, scale, temperature, sigma, top_p, s):
-    """top_k = 0 with top_p < 1: the nucleus takes its mass from the whole row.  Rows whose nucleus fits the 128
-    resolved ids agree with the oracle; the others carry row_status bit 4 and the 128th largest logit as cutoff."""
+    """top_k = 0 with top_p < 1 given per row: the nucleus takes its mass from the whole row and is resolved among
+    the row's 128 largest logits.  Rows whose nucleus fits agree with the oracle; the others carry row_status bit 4
+    and the 128th largest logit as cutoff.  (With one policy for the call the selection path resolves any size:
+    test_filters_of_any_size_match_the_oracle.)"""
     h, W, seeds, positions = _small(T, d, V, 71, scale)
     tokens = _claims(h, W, seeds, positions, f32(temperature), 72)
     dev = Device(h, W, seeds, positions)
@@ -236,7 +238,9 @@ def test_nucleus_over_the_whole_vocabulary(T, d, V, scale, temperature, sigma, t
     L = oracle.logits(h, W)
     kth = np.sort(L, axis=1)[:, ::-1][:, min(128, V) - 1]
 
-    out = _run(dev, tokens, temperature, sigma, 0, top_p, s)
+    k_rows = torch.zeros(T, dtype=torch.int32, device="cuda")
+    p_rows = torch.full((T,), top_p, dtype=torch.float32, device="cuda")
+    out = _run(dev, tokens, temperature, sigma, k_rows, p_rows, s)
     flagged = (out.row_status.cpu().numpy() & 16) != 0
     assert np.array_equal(flagged[clear], ~fits[clear])
     want, _, cut = filtered.score_gm_filtered(h, W, tokens, seeds, positions, f32(temperature), f32(sigma), f32(EPS),
@@ -252,7 +256,7 @@ def test_nucleus_over_the_whole_vocabulary(T, d, V, scale, temperature, sigma, t
     o2 = difr.DifrOut.allocate(T, d, V, 0.1, EPS)
     o2.workspace = torch.empty(difr.difr_filtered_workspace_bytes(T, d, V), dtype=torch.uint8, device="cuda")
     o2.cutoff = torch.full((T,), float("nan"), dtype=torch.float32, device="cuda")
-    difr.difr_score_ipt_filtered(dev.h, dev.W, to_dev(tokens), dev.seeds, dev.positions, f32(temperature), 0, top_p, o2)
+    difr.difr_score_ipt_filtered(dev.h, dev.W, to_dev(tokens), dev.seeds, dev.positions, f32(temperature), k_rows, p_rows, o2)
     torch.cuda.synchronize()
     assert int(o2.device_status.item()) == 0
     want2, pt, a, _, cut2 = filtered.score_ipt_filtered(h, W, tokens, seeds, positions, f32(temperature), f32(0.1),
@@ -302,8 +306,10 @@ def test_one_sampling_policy_per_row():
                 ref = dev.score("ipt", tokens, temp, sigma, EPS)["score"]
                 assert np.array_equal(got[rows], ref[rows]) and np.all(np.isneginf(cut[rows]))
                 continue
-            one = fresh()
-            fn(dev.h, dev.W, tok_dev, dev.seeds, dev.positions, f32(temp), k, p, *extra, one)
+            one = fresh()  # the same policy for every row, given per row like the mixed call's
+            k_all = torch.full((T,), k, dtype=torch.int32, device="cuda")
+            p_all = torch.full((T,), p, dtype=torch.float32, device="cuda")
+            fn(dev.h, dev.W, tok_dev, dev.seeds, dev.positions, f32(temp), k_all, p_all, *extra, one)
             torch.cuda.synchronize()
             assert np.array_equal(got[rows], one.score.cpu().numpy()[rows], equal_nan=True), (fn.__name__, g)
             assert np.array_equal(cut[rows], one.cutoff.cpu().numpy()[rows], equal_nan=True), (fn.__name__, g)
@@ -390,3 +396,126 @@ def test_ipt_estimator_under_min_p_matches_the_oracle(T, d, V, scale, temperatur
     np.testing.assert_allclose(out.p_claimed.cpu().numpy()[ok], pt[ok], rtol=2e-4, atol=1e-9)
     np.testing.assert_allclose(out.cdf_lo.cpu().numpy()[ok], a[ok], rtol=2e-4, atol=2e-6)
     assert (n_kept[resolved] > 1).sum() > 5  # the bar keeps more than the top id on some rows
+
+
+def _filtered_call(fn, dev, tokens, temperature, sigma, top_k, top_p, min_p, s=None):
+    T, d, V = dev.T, dev.d, dev.V
+    out = difr.DifrOut.allocate(T, d, V, sigma, EPS)
+    out.workspace = torch.empty(difr.difr_filtered_workspace_bytes(T, d, V), dtype=torch.uint8, device="cuda")
+    out.cutoff = torch.full((T,), float("nan"), dtype=torch.float32, device="cuda")
+    for name in ("score", "p_claimed", "cdf_lo", "u"):
+        getattr(out, name).fill_(float("nan"))
+    args = (dev.h, dev.W, to_dev(np.asarray(tokens, dtype=np.int32)), dev.seeds, dev.positions, f32(temperature),
+            top_k, top_p)
+    if s is None:
+        fn(*args, out, min_p=f32(min_p))
+    else:
+        fn(*args, s, out, min_p=f32(min_p))
+    torch.cuda.synchronize()
+    assert int(out.device_status.item()) == 0
+    return out
+
+
+def _cutoff_agrees(l_row, temperature, top_k, top_p, min_p, got_cut, want_cut, tol_mass=3e-5):
+    """The kernel's cutoff is the oracle's, or the logit at a neighbouring position of the sorted row where the
+    nucleus decision "does this prefix hold top_p of the mass" lies within tol_mass of a tie (the kernel sums
+    masses of fp32 logits).  Returns (acceptable, identical)."""
+    if abs(got_cut - want_cut) <= 1e-5 or (np.isneginf(got_cut) and np.isneginf(want_cut)):
+        return True, True
+    if not top_p < 1.0:
+        return False, False
+    V = l_row.shape[0]
+    z = np.sort(l_row)[::-1]
+    k = top_k if 0 < top_k < V else V
+    e = np.exp((z[:k] - z[0]) / temperature)
+    c = np.cumsum(e) / e.sum()
+    q = int(np.argmin(np.abs(z[:k] - got_cut)))
+    if abs(z[q] - got_cut) > 1e-5:
+        return False, False
+    n = int(np.searchsorted(c, top_p, side="left")) + 1
+    if q + 1 < n:   # the kernel stopped earlier: it saw the mass of its prefix reach top_p
+        return bool(top_p - c[q] <= tol_mass), False
+    return bool(c[q - 1] - top_p <= tol_mass), False   # it stopped later: it saw the shorter prefix fall short
+
+
+@pytest.mark.parametrize("T,d,V,scale,temperature,sigma,top_k,top_p,min_p,s", [
+    (64, 72, 20000, 1.0, 1.0, 0.3, 0, 0.95, 0.0, 3),      # flat logits: the nucleus holds most of the vocabulary
+    (64, 72, 20000, 3.0, 1.0, 0.3, 0, 0.9, 0.0, 2),       # peaked rows: nuclei from a handful to thousands of ids
+    (48, 64, 9000, 2.0, 0.8, 0.1, 1000, 1.0, 0.0, 4),     # a top-k above the lists' reach
+    (48, 64, 9000, 2.0, 1.0, 0.3, 2000, 0.9, 0.0, 2),     # both: the nucleus inside a large top-k
+    (48, 64, 9000, 2.0, 1.0, 0.3, 500, 0.97, 0.05, 2),    # ... with a min-p bound behind them
+    (40, 64, 300, 2.0, 1.0, 0.4, 200, 0.9, 0.0, 3),       # one vocabulary tile, ragged
+])
+def test_filters_of_any_size_match_the_oracle(T, d, V, scale, temperature, sigma, top_k, top_p, min_p, s):
+    """One policy for the whole call with a kept set beyond the candidate lists (top_k > 128, a nucleus over the
+    whole vocabulary): the kept prefix is found by selection over the rows' logits.  The cutoff is the oracle's
+    (or its neighbour in the sorted row where the nucleus decision is within 3e-5 of a tie in relative mass),
+    the score the oracle's on every row."""
+    h, W, seeds, positions = _small(T, d, V, 97, scale)
+    tokens = _claims(h, W, seeds, positions, f32(temperature), 98)
+    tokens[5] = V + 1
+    dev = Device(h, W, seeds, positions)
+    out = _filtered_call(difr.difr_score_gm_filtered, dev, tokens, temperature, sigma, top_k, top_p, min_p, s)
+    want, _, cut = filtered.score_gm_filtered(h, W, tokens, seeds, positions, f32(temperature), f32(sigma), f32(EPS),
+                                              top_k, f32(top_p), s, f32(min_p))
+    L = oracle.logits(h, W)
+    got, got_cut = out.score.cpu().numpy(), out.cutoff.cpu().numpy().astype(np.float64)
+    status = out.row_status.cpu().numpy()
+    assert np.all(status & (4 | 8 | 16) == 0)  # nothing unresolved, nothing overflowed
+    bar = L.max(axis=1) + f32(temperature) * math.log(f32(min_p)) if min_p > 0 else np.full(T, -np.inf)
+    agree = [_cutoff_agrees(L[r], f32(temperature), top_k, f32(top_p), f32(min_p), max(got_cut[r], -np.inf),
+                            cut[r]) if not (min_p > 0 and np.isclose(cut[r], bar[r], atol=1e-9))
+             else (bool(abs(got_cut[r] - cut[r]) <= 1e-5),) * 2 for r in range(T)]
+    ok = np.array([a[0] for a in agree])
+    same = np.array([a[1] for a in agree])
+    assert ok.all(), np.nonzero(~ok)[0]
+    assert same.mean() > 0.8
+    np.testing.assert_allclose(got, want, rtol=0, atol=SCORE_TOL)
+    assert got[5] == pytest.approx(math.log(EPS), abs=1e-5)
+    # the kept sets really are large
+    n_kept = np.array([len(filtered.filter_kept(L[r], f32(temperature), top_k, f32(top_p), f32(min_p))) for r in range(T)])
+    assert n_kept.max() > 128 or V <= 300
+
+    # Token-IPT-DiFR on the same filtered distribution
+    mu = np.array([oracle.ipt_uniform(int(sd), int(ps)) for sd, ps in zip(seeds, positions)])
+    tok2 = np.array([filtered.ipt_sample_filtered(L[r], f32(temperature), top_k, f32(top_p), mu[r], f32(min_p))
+                     for r in range(T)], dtype=np.int32)
+    k = np.arange(T)
+    tok2[k % 5 == 1] = np.argsort(-L, axis=1)[k % 5 == 1, 1]
+    tok2[k % 5 == 3] = np.argmin(L, axis=1)[k % 5 == 3]
+    o2 = _filtered_call(difr.difr_score_ipt_filtered, dev, tok2, temperature, 0.1, top_k, top_p, min_p)
+    want2, pt, a, _, cut2 = filtered.score_ipt_filtered(h, W, tok2, seeds, positions, f32(temperature), f32(0.1),
+                                                        f32(EPS), top_k, f32(top_p), f32(min_p))
+    assert np.all(o2.row_status.cpu().numpy() & (8 | 16) == 0)
+    cut_ipt = o2.cutoff.cpu().numpy().astype(np.float64)
+    same2 = np.isclose(cut_ipt, cut2, rtol=0, atol=1e-5)   # the same kept set (compared where it is)
+    assert same2.mean() > 0.8
+    np.testing.assert_allclose(o2.score.cpu().numpy()[same2], want2[same2], rtol=0, atol=SCORE_TOL)
+    np.testing.assert_allclose(o2.p_claimed.cpu().numpy()[same2], pt[same2], rtol=2e-4, atol=1e-9)
+    np.testing.assert_allclose(o2.cdf_lo.cpu().numpy()[same2], a[same2], rtol=2e-4, atol=2e-6)
+
+
+def test_min_p_set_of_any_size_for_the_ipt_estimator():
+    """min-p alone on flat logits keeps thousands of ids: with one policy for the call the IPT estimator's kept
+    set is summed by the selection, none is left unresolved."""
+    T, d, V, temperature, min_p = 64, 72, 20000, 1.0, 0.05
+    h, W, seeds, positions = _small(T, d, V, 99, 1.0)
+    L = oracle.logits(h, W)
+    mu = np.array([oracle.ipt_uniform(int(sd), int(ps)) for sd, ps in zip(seeds, positions)])
+    tokens = np.array([filtered.ipt_sample_filtered(L[r], f32(temperature), 0, 1.0, mu[r], f32(min_p)) for r in range(T)],
+                      dtype=np.int32)
+    tokens[::4] = np.argmin(L, axis=1)[::4]
+    dev = Device(h, W, seeds, positions)
+    out = _filtered_call(difr.difr_score_ipt_filtered, dev, tokens, temperature, 0.1, 0, 1.0, min_p)
+    want, pt, a, _, cut = filtered.score_ipt_filtered(h, W, tokens, seeds, positions, f32(temperature), f32(0.1), f32(EPS),
+                                                      0, 1.0, f32(min_p))
+    n_kept = np.array([len(filtered.filter_kept(L[r], f32(temperature), 0, 1.0, f32(min_p))) for r in range(T)])
+    assert n_kept.min() > 128
+    # ids whose logit lies within fp32 rounding of the bound may fall on either side: leave those rows out
+    bar = L.max(axis=1, keepdims=True) + f32(temperature) * math.log(f32(min_p))
+    clear = np.abs(L - bar).min(axis=1) > 2e-5
+    assert clear.mean() > 0.8
+    assert np.all(out.row_status.cpu().numpy() & (8 | 16) == 0)
+    np.testing.assert_allclose(out.cutoff.cpu().numpy()[clear], cut[clear], rtol=0, atol=1e-5)
+    np.testing.assert_allclose(out.score.cpu().numpy()[clear], want[clear], rtol=0, atol=SCORE_TOL)
+    np.testing.assert_allclose(out.cdf_lo.cpu().numpy()[clear], a[clear], rtol=2e-4, atol=2e-6)
