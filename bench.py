@@ -723,6 +723,10 @@ def time_variants(difr, h, W, tokens, seeds, pos, temperature, sigma, T, d, V, i
                                                                              50, 0.95, 4, out),
         "score_ipt_filtered_k50_p095": lambda: difr.difr_score_ipt_filtered(h, W, tokens, seeds, pos, temperature,
                                                                            50, 0.95, out),
+        "score_gm_filtered_whole_vocabulary_nucleus_p095_s4": lambda: difr.difr_score_gm_filtered(
+            h, W, tokens, seeds, pos, temperature, 0, 0.95, 4, out),
+        "score_ipt_filtered_k1000": lambda: difr.difr_score_ipt_filtered(h, W, tokens, seeds, pos, temperature,
+                                                                        1000, 1.0, out),
     }
     res = {}
     calls["score_gm"]()

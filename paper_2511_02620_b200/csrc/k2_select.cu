@@ -8,8 +8,10 @@
 //   min-p   keeps the ids whose logit reaches l_max + Temp ln(min_p), a prefix as well
 //
 // N is the smallest of the three.  Masses are summed as 64-bit fixed-point integers (2^-40 of the largest
-// term), so sums do not depend on the order of the additions and the result is the same on every run.  The
-// row (V floats) is walked up to a dozen times; after the first walk it is in L2.
+// term), so sums do not depend on the order of the additions and the result is the same on every run.  One
+// walk over the row builds a histogram in bins of 1/64 of (l_max - l); each selection then scans it, gathers
+// the ids of one bin and pins the exact value by radix rounds over their key bits.  The row (V floats) is
+// walked about seven times; after the first walk it is in L2.
 #include <cuda_runtime.h>
 #include <math_constants.h>
 
@@ -27,9 +29,15 @@ __device__ __forceinline__ uint32_t desc_key(float l) {
   return ~(b ^ ((b >> 31) ? 0xFFFFFFFFu : 0x80000000u));
 }
 
+constexpr int kSelListCap = 2048;
+
 struct SelShared {
-  unsigned int cnt[kSelBins];
+  unsigned int cnt0[kSelBins];         // level 0: bins of 1/64 in (l_max - l), all ids of the row
+  unsigned long long mass0[kSelBins];
+  unsigned int cnt[kSelBins];          // inner rounds: key bits of the ids of one level-0 bin
   unsigned long long mass[kSelBins];
+  int list[kSelListCap];               // the ids of that level-0 bin (when they fit)
+  unsigned int list_n;
   unsigned int warp_cnt[kSelThreads / 32];
   unsigned long long warp_mass[kSelThreads / 32];
   unsigned int found_bin;
@@ -52,29 +60,112 @@ struct Selected {
 };
 
 __device__ __forceinline__ unsigned long long fixed_mass(float l, float lmax, float c1) {
-  // 2^(c1 (l - lmax)) in units of 2^-40, rounded to nearest; terms below 2^-41 of the largest count as zero
-  const double e = exp2((double)c1 * ((double)l - (double)lmax));
-  return (unsigned long long)(e * 1099511627776.0 + 0.5);
+  // 2^(c1 (l - lmax)) in units of 2^-40; terms below 2^-41 of the largest count as zero.  fp32 arithmetic (a
+  // relative error of 1e-7 per term, against the 1e-5 the fp32 logits themselves carry): a pure function of
+  // its arguments, so the integer sums stay independent of the order of the additions.
+  const float e = exp2f(c1 * (l - lmax));  // in [0, 1]
+  return (unsigned long long)__float2ull_rn(e * 1099511627776.0f);
 }
 
-// One radix selection over the row.  by_mass == false: the element at position `pos` (0-based) of the descending
-// order.  by_mass == true: the first element at which the cumulative mass reaches `target`.  Whole CTA.
+// Level-0 bin of a logit: monotone in l (larger logits in lower bins, equal logits in one bin), 1/64 wide, the
+// last bin open-ended.
+__device__ __forceinline__ unsigned int level0_bin(float l, float lmax) {
+  const unsigned int b = __float2uint_rz((lmax - l) * 64.f);
+  return b < (unsigned int)(kSelBins - 1) ? b : (unsigned int)(kSelBins - 1);
+}
+
+// Scan of a histogram (bins in descending order of the logit) from the carried sums (c_acc, m_acc): the first
+// bin in which the position `pos` lies (by_mass == false) or the cumulative mass reaches `target`
+// (by_mass == true); a target beyond the total gives the last non-empty bin.  Leaves the bin, the sums before
+// it and the bin's own count and mass in shared memory.  Whole CTA.
+__device__ void locate(const unsigned int* cnt, const unsigned long long* mass, bool by_mass, unsigned int pos,
+                       unsigned long long target, unsigned int c_acc, unsigned long long m_acc, SelShared& sh) {
+  if (threadIdx.x == 0) sh.found_bin = 0xFFFFFFFFu;
+  const int per = kSelBins / kSelThreads;
+  unsigned int tc = 0;
+  unsigned long long tm = 0;
+  for (int i = 0; i < per; ++i) { tc += cnt[threadIdx.x * per + i]; tm += mass[threadIdx.x * per + i]; }
+  unsigned int sc = tc;
+  unsigned long long sm = tm;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int m = 1; m < 32; m <<= 1) {
+    const unsigned int oc = __shfl_up_sync(0xffffffffu, sc, m);
+    const unsigned long long om = __shfl_up_sync(0xffffffffu, sm, m);
+    if (lane >= m) { sc += oc; sm += om; }
+  }
+  if (lane == 31) { sh.warp_cnt[warp] = sc; sh.warp_mass[warp] = sm; }
+  __syncthreads();
+  unsigned int base_c = c_acc;
+  unsigned long long base_m = m_acc;
+  for (int w = 0; w < warp; ++w) { base_c += sh.warp_cnt[w]; base_m += sh.warp_mass[w]; }
+  base_c += sc - tc;
+  base_m += sm - tm;  // sums of everything before this thread's first bin
+  const unsigned int start_c = base_c;
+  const unsigned long long start_m = base_m;
+  for (int i = 0; i < per; ++i) {
+    const int b = threadIdx.x * per + i;
+    const unsigned int bc = cnt[b];
+    const unsigned long long bm = mass[b];
+    if (bc != 0 && (by_mass ? (base_m + bm >= target) : (base_c + bc > pos))) atomicMin(&sh.found_bin, (unsigned int)b);
+    base_c += bc;
+    base_m += bm;
+  }
+  __syncthreads();
+  unsigned int fb = sh.found_bin;
+  if (fb == 0xFFFFFFFFu) {
+    if (threadIdx.x == 0) {
+      unsigned int last = 0;
+      for (int b = 0; b < kSelBins; ++b) if (cnt[b] != 0) last = (unsigned int)b;
+      sh.found_bin = last;
+    }
+    __syncthreads();
+    fb = sh.found_bin;
+  }
+  if (threadIdx.x == fb / per) {  // the bin's owner knows what lies before it
+    unsigned int c = start_c;
+    unsigned long long m = start_m;
+    for (unsigned int b = (unsigned int)(threadIdx.x * per); b < fb; ++b) { c += cnt[b]; m += mass[b]; }
+    sh.c_before = c; sh.m_before = m; sh.bin_cnt = cnt[fb]; sh.bin_mass = mass[fb];
+  }
+  __syncthreads();
+}
+
+// One selection over the row, from its level-0 histogram (built by the caller).  by_mass == false: the element at
+// position `pos` (0-based) of the descending order.  by_mass == true: the first element at which the cumulative
+// mass reaches `target`.  The level-0 bin that holds the answer is found by a scan; its ids are gathered into a
+// list (one walk over the row) and three radix rounds over their key bits (11 + 11 + 10) pin the exact value.
+// Whole CTA.
 __device__ Selected radix_select(const float* row, int V, float lmax, float c1, bool by_mass, unsigned int pos,
                                  unsigned long long target, SelShared& sh) {
-  uint32_t prefix = 0;       // the key bits decided so far (high bits)
-  int decided = 0;           // how many
-  unsigned int c_acc = 0;
-  unsigned long long m_acc = 0;
+  locate(sh.cnt0, sh.mass0, by_mass, pos, target, 0u, 0ull, sh);
+  const unsigned int bin0 = sh.found_bin;
+  unsigned int c_acc = sh.c_before;
+  unsigned long long m_acc = sh.m_before;
+  if (threadIdx.x == 0) sh.list_n = 0u;
+  __syncthreads();
+  for (int v = threadIdx.x; v < V; v += kSelThreads) {
+    if (level0_bin(row[v], lmax) == bin0) {
+      const unsigned int at = atomicAdd(&sh.list_n, 1u);
+      if (at < (unsigned int)kSelListCap) sh.list[at] = v;
+    }
+  }
+  __syncthreads();
+  const unsigned int n_sub = sh.list_n;
+  const bool listed = n_sub <= (unsigned int)kSelListCap;  // else: walk the whole row in every round
+  uint32_t prefix = 0;  // the key bits decided so far (high bits)
+  int decided = 0;      // how many
   const int shifts[3] = {21, 10, 0};
   const int widths[3] = {11, 11, 10};
   Selected out;
   for (int round = 0; round < 3; ++round) {
     const int shift = shifts[round], width = widths[round];
     for (int b = threadIdx.x; b < kSelBins; b += kSelThreads) { sh.cnt[b] = 0; sh.mass[b] = 0; }
-    if (threadIdx.x == 0) sh.found_bin = 0xFFFFFFFFu;
     __syncthreads();
-    for (int v = threadIdx.x; v < V; v += kSelThreads) {
+    const int n_walk = listed ? (int)n_sub : V;
+    for (int i = threadIdx.x; i < n_walk; i += kSelThreads) {
+      const int v = listed ? sh.list[i] : i;
       const float l = row[v];
+      if (!listed && level0_bin(l, lmax) != bin0) continue;
       const uint32_t k = desc_key(l);
       if (decided == 0 || (k >> (32 - decided)) == prefix) {
         const uint32_t bin = (k >> shift) & ((1u << width) - 1u);
@@ -83,62 +174,10 @@ __device__ Selected radix_select(const float* row, int V, float lmax, float c1, 
       }
     }
     __syncthreads();
-    // block scan over the bins (four consecutive bins per thread), then the first bin that holds the answer
-    const int per = kSelBins / kSelThreads;
-    unsigned int tc = 0;
-    unsigned long long tm = 0;
-    for (int i = 0; i < per; ++i) { tc += sh.cnt[threadIdx.x * per + i]; tm += sh.mass[threadIdx.x * per + i]; }
-    unsigned int sc = tc;
-    unsigned long long sm = tm;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int m = 1; m < 32; m <<= 1) {
-      const unsigned int oc = __shfl_up_sync(0xffffffffu, sc, m);
-      const unsigned long long om = __shfl_up_sync(0xffffffffu, sm, m);
-      if (lane >= m) { sc += oc; sm += om; }
-    }
-    if (lane == 31) { sh.warp_cnt[warp] = sc; sh.warp_mass[warp] = sm; }
-    __syncthreads();
-    unsigned int base_c = c_acc;
-    unsigned long long base_m = m_acc;
-    for (int w = 0; w < warp; ++w) { base_c += sh.warp_cnt[w]; base_m += sh.warp_mass[w]; }
-    base_c += sc - tc;
-    base_m += sm - tm;  // sums of everything before this thread's first bin
-    const unsigned int start_c = base_c;
-    const unsigned long long start_m = base_m;
-    for (int i = 0; i < per; ++i) {
-      const int b = threadIdx.x * per + i;
-      const unsigned int bc = sh.cnt[b];
-      const unsigned long long bm = sh.mass[b];
-      const bool here = bc != 0 && (by_mass ? (base_m + bm >= target) : (base_c + bc > pos));
-      if (here) {
-        const unsigned int old = atomicMin(&sh.found_bin, (unsigned int)b);
-        (void)old;
-      }
-      base_c += bc;
-      base_m += bm;
-    }
-    __syncthreads();
-    unsigned int fb = sh.found_bin;
-    if (fb == 0xFFFFFFFFu) {
-      // the target lies beyond the row's total (rounding of the target): the last non-empty bin
-      if (threadIdx.x == 0) {
-        unsigned int last = 0;
-        for (int b = 0; b < (1 << width); ++b) if (sh.cnt[b] != 0) last = (unsigned int)b;
-        sh.found_bin = last;
-      }
-      __syncthreads();
-      fb = sh.found_bin;
-    }
-    if (threadIdx.x == fb / per) {  // the bin's owner knows what lies before it
-      unsigned int c = start_c;
-      unsigned long long m = start_m;
-      for (unsigned int b = (unsigned int)(threadIdx.x * per); b < fb; ++b) { c += sh.cnt[b]; m += sh.mass[b]; }
-      sh.c_before = c; sh.m_before = m; sh.bin_cnt = sh.cnt[fb]; sh.bin_mass = sh.mass[fb];
-    }
-    __syncthreads();
+    locate(sh.cnt, sh.mass, by_mass, pos, target, c_acc, m_acc, sh);
     c_acc = sh.c_before;
     m_acc = sh.m_before;
-    prefix = (prefix << width) | fb;
+    prefix = (prefix << width) | sh.found_bin;
     decided += width;
     out.ties = sh.bin_cnt;
     out.m_tie = sh.bin_mass;
@@ -171,7 +210,8 @@ __device__ __forceinline__ unsigned long long block_sum(unsigned long long v, Se
 }
 
 __global__ void __launch_bounds__(kSelThreads) select_cutoff(const SelectParams p) {
-  __shared__ SelShared sh;
+  extern __shared__ __align__(16) unsigned char sel_smem[];
+  SelShared& sh = *reinterpret_cast<SelShared*>(sel_smem);
   const int r_local = blockIdx.x;
   const int row = p.row0 + r_local;
   const float* lrow = p.logits + (size_t)r_local * (size_t)p.V;
@@ -185,12 +225,18 @@ __global__ void __launch_bounds__(kSelThreads) select_cutoff(const SelectParams 
   for (int v = threadIdx.x; v < V; v += kSelThreads) lm = fmaxf(lm, lrow[v]);
   const float lmax = block_max(lm, sh);
 
-  // total mass, and how many ids reach the min-p bound
+  // level-0 histogram (count and mass per 1/64 of l_max - l), total mass, and how many ids reach the min-p bound
   const float bound = p.min_p > 0.f ? lmax + temp * logf(p.min_p) : -CUDART_INF_F;
+  for (int b = threadIdx.x; b < kSelBins; b += kSelThreads) { sh.cnt0[b] = 0; sh.mass0[b] = 0; }
+  __syncthreads();
   unsigned long long tm = 0, tb = 0;
   for (int v = threadIdx.x; v < V; v += kSelThreads) {
     const float l = lrow[v];
-    tm += fixed_mass(l, lmax, c1);
+    const unsigned long long q = fixed_mass(l, lmax, c1);
+    const unsigned int b0 = level0_bin(l, lmax);
+    atomicAdd(&sh.cnt0[b0], 1u);
+    atomicAdd(&sh.mass0[b0], q);
+    tm += q;
     tb += (l >= bound) ? 1u : 0u;
   }
   const unsigned long long m_total = block_sum(tm, sh);
@@ -296,7 +342,10 @@ __global__ void __launch_bounds__(kSelThreads) select_cutoff(const SelectParams 
 
 cudaError_t launch_select_cutoff(const SelectParams& p, cudaStream_t stream) {
   if (p.rows <= 0) return cudaSuccess;
-  select_cutoff<<<p.rows, kSelThreads, 0, stream>>>(p);
+  const cudaError_t e =
+      cudaFuncSetAttribute(select_cutoff, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SelShared));
+  if (e != cudaSuccess) return e;
+  select_cutoff<<<p.rows, kSelThreads, sizeof(SelShared), stream>>>(p);
   return cudaGetLastError();
 }
 

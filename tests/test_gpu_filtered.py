@@ -519,3 +519,34 @@ def test_min_p_set_of_any_size_for_the_ipt_estimator():
     np.testing.assert_allclose(out.cutoff.cpu().numpy()[clear], cut[clear], rtol=0, atol=1e-5)
     np.testing.assert_allclose(out.score.cpu().numpy()[clear], want[clear], rtol=0, atol=SCORE_TOL)
     np.testing.assert_allclose(out.cdf_lo.cpu().numpy()[clear], a[clear], rtol=2e-4, atol=2e-6)
+
+
+def test_filters_of_any_size_at_full_size_on_sampled_rows():
+    """llama3b at full size with the nucleus taken over the whole vocabulary (flat synthetic logits: it holds about
+    three quarters of the ids) and with a top-k of 1000: the logits go through the selection three blocks of rows
+    at a time; sampled rows against the oracle, twice (the results are the same bits on every run)."""
+    w = wl.WORKLOADS["llama3b"]
+    inp = wl.make_inputs(w)
+    dev = Device(inp.h, inp.W, inp.seeds, inp.positions)
+    rows = wl.sample_rows(w, 10, salt=4)
+    temperature, sigma, s = 1.0, 0.3, 2
+    g = np.random.default_rng(7)
+    tokens = g.integers(0, w.V, size=w.T).astype(np.int32)
+    hs = np.ascontiguousarray(inp.h[rows])
+    tokens[rows] = _claims(hs, inp.W, inp.seeds[rows], inp.positions[rows], f32(temperature), 8)
+    L = oracle.logits(hs, inp.W)
+    for top_k, top_p in ((0, 0.95), (1000, 1.0)):
+        out = _filtered_call(difr.difr_score_gm_filtered, dev, tokens, temperature, sigma, top_k, top_p, 0.0, s)
+        again = _filtered_call(difr.difr_score_gm_filtered, dev, tokens, temperature, sigma, top_k, top_p, 0.0, s)
+        assert torch.equal(out.score.view(torch.int32), again.score.view(torch.int32))
+        assert torch.equal(out.cutoff.view(torch.int32), again.cutoff.view(torch.int32))
+        want, _, cut = filtered.score_gm_filtered(hs, inp.W, tokens[rows], inp.seeds[rows], inp.positions[rows],
+                                                  f32(temperature), f32(sigma), f32(EPS), top_k, f32(top_p), s)
+        got, got_cut = out.score.cpu().numpy(), out.cutoff.cpu().numpy().astype(np.float64)
+        for i, r in enumerate(rows):
+            ok, _ = _cutoff_agrees(L[i], f32(temperature), top_k, f32(top_p), 0.0, got_cut[r], cut[i])
+            assert ok, (top_k, top_p, int(r), got_cut[r], cut[i])
+        np.testing.assert_allclose(got[rows], want, rtol=0, atol=SCORE_TOL)
+        assert np.all(out.row_status.cpu().numpy() & (4 | 8 | 16) == 0)
+        assert np.all(np.isfinite(got)) and np.all(got <= 1e-6)
+        assert np.all(np.isfinite(got_cut))
