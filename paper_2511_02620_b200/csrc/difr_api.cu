@@ -211,6 +211,7 @@ difr_status score_common(int ipt, const void* h, const void* W, const int32_t* t
   k2.temperatures = out->temperatures;
   k2.sigma_ipt = out->sigma_ipt; k2.score_ipt = out->score_ipt;
   k2.rank = want_rank ? out->rank : nullptr; k2.y_max = out->y_max; k2.y_second = out->y_second;
+  k2.tok_logit_in_records = want_rank ? 0 : 1;  // (the rank mode counts in that word)
   k2.band_list = k1.band_list; k2.band_count = k1.band_count; k2.band_cap = k1.band_cap;
   if (launch_k2(k2, s) != cudaSuccess) return DIFR_ERR_CUDA;
   return DIFR_OK;

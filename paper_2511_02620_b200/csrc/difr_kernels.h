@@ -48,6 +48,7 @@ struct K2Params {
   int T, d, V;
   const float* temperatures;  // [T], nullable: per-row temperature in place of `temperature` / `c1`
   int ipt;  // 0: Token-DiFR (Gumbel-max), 1: Token-IPT-DiFR, 2: both (IPT score to score_ipt with sigma_ipt)
+  int tok_logit_in_records;  // the records' last words add up to the bits of the claimed token's fp32 logit
   float sigma_ipt;
   float* score_ipt;
   int32_t* rank;

@@ -273,12 +273,18 @@ __device__ __forceinline__ void process16(const uint32_t (&raw)[kSub], int base,
     // ids below the claimed one: all, none, or the first tl of this group
     if (tl >= kSub) {
       s.lpre += cs;
-    } else if (tl > 0) {
-      float ps = 0.f;
+    } else if (tl >= 0) {  // this group holds the claimed id
+      float ps = 0.f, lt = 0.f;
 #pragma unroll
-      for (int j = 0; j < kSub; ++j)
+      for (int j = 0; j < kSub; ++j) {
         if (j < tl) ps += ex2_approx(fmaf(l[j], c1, shift));
+        if (j == tl) lt = l[j];
+      }
       s.lpre += ps;
+      // the claimed token's own fp32 logit travels in the record's last word (modes that do not count there):
+      // the finalize kernel swaps its term of the sum for the fp64 one, so that p[t*] is not off by the tensor
+      // cores' rounding of the largest logit
+      if (!M::rank && !M::groupmax) s.cnt[0] = __float_as_int(lt);
     }
   }
 

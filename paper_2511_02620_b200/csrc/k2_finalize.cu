@@ -119,7 +119,7 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
   if (!lse_finite) status |= 2u;
   const bool temp_bad = !(temp_f >= 0.f) || isinf(temp_f) || (p.ipt != 0 && temp_f == 0.f);
   if (temp_bad) status |= 8u;
-  const double lse = (temp_f > 0.f) ? (acc.lmax + log2(acc.lsum)) * ln2 : CUDART_NAN;
+  double lse = (temp_f > 0.f) ? (acc.lmax + log2(acc.lsum)) * ln2 : CUDART_NAN;
 
   // ---- exact (fp64) values.  Token-DiFR: y = l + Temp * G of the claimed token and of every candidate that can
   // be among the two largest.  The fused kernel ranks by fp32 keys whose error (tensor-core accumulation,
@@ -199,6 +199,20 @@ __global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
     }
   }
   flush();
+
+  // The softmax sums come from the tensor cores' fp32 logits, the claimed token's own logit from the fp64 dot
+  // product: where the claimed token carries much of the mass, the rounding of its fp32 logit (1e-5 of a unit
+  // per ten units of magnitude) would go straight into p[t*].  The fused kernel sent that fp32 logit along;
+  // its term of the sum is replaced by the exact one.
+  if (p.tok_logit_in_records && tok_ok && acc.larger != 0 && temp_f > 0.f && isfinite(acc.lmax)) {
+    const double l_fp32 = (double)__int_as_float(acc.larger);
+    const double c1d = (double)c1_f;
+    const double swapped = acc.lsum - exp2(l_fp32 * c1d - acc.lmax) + exp2(l_tok * c1d - acc.lmax);
+    if (swapped > 0.0 && isfinite(swapped)) {
+      acc.lsum = swapped;
+      lse = (acc.lmax + log2(acc.lsum)) * ln2;
+    }
+  }
 
   // raw-logit rank: the fused kernel counted the ids whose fp32 logit is above the claimed one by more than the
   // tensor cores' rounding; the ids it could not decide are on the row's list and are decided here in fp64

@@ -304,7 +304,10 @@ def test_one_sampling_policy_per_row():
             if fn is difr.difr_score_ipt_filtered and k == 0 and p == 1.0:
                 # a row whose policy filters nothing keeps the unfiltered score
                 ref = dev.score("ipt", tokens, temp, sigma, EPS)["score"]
-                assert np.array_equal(got[rows], ref[rows]) and np.all(np.isneginf(cut[rows]))
+                # (up to the last digits: the plain call also swaps the claimed token's fp32 softmax term for
+                # the fp64 one, the filtered call's first pass keeps another statistic in that record word)
+                np.testing.assert_allclose(got[rows], ref[rows], rtol=0, atol=2e-5)
+                assert np.all(np.isneginf(cut[rows]))
                 continue
             one = fresh()  # the same policy for every row, given per row like the mixed call's
             k_all = torch.full((T,), k, dtype=torch.int32, device="cuda")

@@ -399,3 +399,36 @@ def test_small_noise_widths_of_the_papers_sweep(T, d, V, temperature, sigma):
     np.testing.assert_allclose(got["margin"], ref.margin, rtol=2e-6, atol=1e-6)
     clear = ref.top2_margin >= 1e-6
     assert np.array_equal(got["argmax"][clear], ref.argmax[clear])
+
+
+@pytest.mark.parametrize("d,kind", [(512, "peaked"), (5120, "unit"), (5120, "peaked")])
+def test_ipt_score_holds_its_tolerance_over_widths_and_logit_magnitudes(d, kind):
+    """The IPT estimator divides by sigma^2: at sigma 0.01 an error of 1e-7 in a CDF value is 1e-3 of score.  The
+    softmax sums come from the tensor cores' fp32 logits; the claimed token's own term is swapped for the fp64
+    one in the finalize kernel.  Unit-variance logits at d = 5120 and heads whose logits reach +-200 (one or two
+    ids far ahead) stay within 2e-3 for sigma from 0.2 down to 0.01."""
+    T, V = 128, 8192
+    g = np.random.default_rng(12)
+    hf = g.standard_normal((T, d)).astype(np.float32)
+    if kind == "unit":
+        Wf = (g.standard_normal((V, d)) / math.sqrt(d)).astype(np.float32)
+    else:
+        Wf = (6.0 * g.standard_normal((V, d)) / math.sqrt(d)).astype(np.float32)
+        bias_dir = g.standard_normal(d).astype(np.float32) / math.sqrt(d)
+        hf += 4.0 * math.sqrt(d) * bias_dir
+        Wf += 7.0 * bias_dir / math.sqrt(d)
+        Wf[g.integers(0, V, size=40)] *= 1.8
+    h, W = wl.f32_to_bf16_bits(hf), wl.f32_to_bf16_bits(Wf)
+    seeds = np.array([wl.splitmix64(900 + r // 32) for r in range(T)], dtype=np.uint64)
+    positions = (np.arange(T) % 32 + 1).astype(np.uint32)
+    itok = oracle.sample_ipt(h, W, seeds, positions, 1.0).astype(np.int32)
+    itok[::5] = g.integers(0, V, size=len(itok[::5]))
+    if kind == "peaked":
+        assert np.abs(oracle.logits(h[:8], W)).max() > 100
+    dev = Device(h, W, seeds, positions)
+    for sigma in (0.2, 0.05, 0.01):
+        ref = oracle.score_ipt(h, W, itok, seeds, positions, 1.0, f32(sigma), f32(EPS))
+        got = dev.score("ipt", itok, 1.0, sigma, EPS)
+        np.testing.assert_allclose(got["score"], ref.score, rtol=0, atol=SCORE_TOL, err_msg=f"sigma {sigma}")
+        np.testing.assert_allclose(got["lse"], ref.lse, rtol=LSE_RTOL)
+        np.testing.assert_allclose(got["p_claimed"], ref.p_claimed, rtol=2e-4, atol=1e-12)
