@@ -238,6 +238,7 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
   __shared__ float sm_l[kFWarps][kMaxK];
   __shared__ int sm_id[kFWarps][kMaxK];
   __shared__ int sm_cand[kFWarps][kMaxCand];
+  __shared__ float sm_cand_y[kFWarps][kMaxCand];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = blockIdx.x * kFWarps + warp;
   if (row >= p.T) return;
@@ -267,8 +268,12 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
   for (int i = lane; i < n; i += 32) n_others += (list[i].id >= 0 && list[i].id != tok) ? 1 : 0;
 #pragma unroll
   for (int m = 16; m >= 1; m >>= 1) n_others += __shfl_xor_sync(0xffffffffu, n_others, m);
+  // The s competitors are the exact best s; the list ranks by the fused kernel's fp32 y'.  Taken for exact
+  // re-evaluation: the first s + 2 by that ranking, and beyond them every entry within the keys' error of the
+  // s-th (up to kMaxCand in all), so that near-ties at the edge of the active subset are decided in fp64.
   const int want = p.s + 2;
-  const int n_cand = n_others < want ? n_others : want;
+  const int n_top = n_others < kMaxCand ? n_others : kMaxCand;  // entries whose rank by y' is kept
+  int n_cand = n_others < want ? n_others : want;
 
   // ---- order statistics of the list: rank by raw logit (the filter) and by y' (the competitors)
   double cutoff = -CUDART_INF;
@@ -290,10 +295,15 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
     }
     if (lane == 0) {
       if (rl < k_eff) { sm_l[warp][rl] = cj.l; sm_id[warp][rl] = cj.id; }
-      if (cj.id != tok && ry < n_cand) sm_cand[warp][ry] = cj.id;
+      if (cj.id != tok && ry < n_top) { sm_cand[warp][ry] = cj.id; sm_cand_y[warp][ry] = cj.y; }
     }
   }
   __syncwarp();
+  if (n_top > n_cand && p.s <= n_top) {
+    const float ys = sm_cand_y[warp][p.s - 1];
+    const float edge = ys - 2.f * (3e-4f * rp.temperature + 1e-4f + 3.9e-6f * fabsf(ys));
+    while (n_cand < n_top && sm_cand_y[warp][n_cand] >= edge) ++n_cand;
+  }
   if (p.sel_cut_id != nullptr && rp.by_rank) {
     // a filter of any size: the last kept id was found by the selection over the row's logits
     const int cid = p.sel_cut_id[row];
