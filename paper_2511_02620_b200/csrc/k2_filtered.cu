@@ -234,6 +234,36 @@ __global__ void __launch_bounds__(kFWarps * 32) filter_bounds(const FilterParams
   }
 }
 
+// The k-th largest (k >= 1) logit, or y' among the entries that are not the claimed token, of a candidate list
+// (band-only entries left out); -inf when there are fewer than k.  Bisection on keys that order like the floats:
+// the largest key that at least k entries reach.  Whole warp; every lane gets the value.
+__device__ __forceinline__ float warp_kth_largest(const Candidate* list, int n, int k, bool by_y, int tok, int lane) {
+  auto key_of = [](float f) {
+    const uint32_t b = __float_as_uint(f);
+    return b ^ ((b >> 31) ? 0xFFFFFFFFu : 0x80000000u);
+  };
+  uint32_t lo = 0u, hi = 0xFFFFFFFFu;  // invariant: count(key >= lo) >= k (or lo == 0)
+  int total = 0;
+  for (int i = lane; i < n; i += 32) total += (list[i].id >= 0 && (!by_y || list[i].id != tok)) ? 1 : 0;
+#pragma unroll
+  for (int m = 16; m >= 1; m >>= 1) total += __shfl_xor_sync(0xffffffffu, total, m);
+  if (total < k) return -CUDART_INF_F;
+  while (lo < hi) {
+    const uint32_t mid = lo + (hi - lo) / 2u + 1u;  // upper middle: the loop ends with lo == hi
+    int c = 0;
+    for (int i = lane; i < n; i += 32) {
+      const Candidate ci = list[i];
+      if (ci.id < 0 || (by_y && ci.id == tok)) continue;
+      c += key_of(by_y ? ci.y : ci.l) >= mid ? 1 : 0;
+    }
+#pragma unroll
+    for (int m = 16; m >= 1; m >>= 1) c += __shfl_xor_sync(0xffffffffu, c, m);
+    if (c >= k) lo = mid; else hi = mid - 1u;
+  }
+  const uint32_t b = lo ^ ((lo >> 31) ? 0x80000000u : 0xFFFFFFFFu);
+  return __uint_as_float(b);
+}
+
 __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterParams p) {
   __shared__ float sm_l[kFWarps][kMaxK];
   __shared__ int sm_id[kFWarps][kMaxK];
@@ -275,12 +305,21 @@ __global__ void __launch_bounds__(kFWarps * 32) filtered_finalize(const FilterPa
   const int n_top = n_others < kMaxCand ? n_others : kMaxCand;  // entries whose rank by y' is kept
   int n_cand = n_others < want ? n_others : want;
 
-  // ---- order statistics of the list: rank by raw logit (the filter) and by y' (the competitors)
+  // ---- order statistics of the list: rank by raw logit (the filter) and by y' (the competitors).
+  // A long list (vocabularies below 64 tiles list every id) is first cut down: the k_eff-th largest logit and the
+  // n_top-th largest y' are found by bisection on order-preserving keys (32 counting sweeps), and only entries
+  // that reach one of them are ranked against the list.
+  float need_l = -CUDART_INF_F, need_y = -CUDART_INF_F;
+  if (n > 256) {
+    need_l = k_eff > 0 ? warp_kth_largest(list, n, k_eff, false, tok, lane) : CUDART_INF_F;
+    need_y = n_top > 0 ? warp_kth_largest(list, n, n_top, true, tok, lane) : CUDART_INF_F;
+  }
   double cutoff = -CUDART_INF;
   int cut_rank = -1;
   for (int j = 0; j < n; ++j) {
     const Candidate cj = list[j];
     if (cj.id < 0) continue;  // (uniform over the warp)
+    if (n > 256 && !(cj.l >= need_l) && !(cj.y >= need_y)) continue;
     int rl = 0, ry = 0;
     for (int i = lane; i < n; i += 32) {
       const Candidate ci = list[i];
@@ -442,8 +481,11 @@ __global__ void __launch_bounds__(kFWarps * 32) ipt_filtered_finalize(const Filt
   }
   const int k_eff = rp.top_k < n ? rp.top_k : n;
 
+  // (a long list is cut down to the entries that reach its k_eff-th largest logit before they are ranked)
+  const float need_l = (n > 256 && k_eff > 0) ? warp_kth_largest(list, n, k_eff, false, -1, lane) : -CUDART_INF_F;
   for (int j = 0; j < n; ++j) {
     const Candidate cj = list[j];
+    if (n > 256 && !(cj.l >= need_l)) continue;
     int rl = 0;
     for (int i = lane; i < n; i += 32) {
       const Candidate ci = list[i];
