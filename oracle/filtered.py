@@ -73,13 +73,16 @@ def token_difr_filtered(logits, gumbel, temperature, claimed, s, sigma, cutoff=-
         t = np.maximum(x + A, B) / sigma
         return math.exp(-0.5 * (x / sigma) ** 2 + float(np.sum(log_ndtr(t)))) / (sigma * math.sqrt(2.0 * math.pi))
 
-    lo = max(cutoff - logits[claimed], -14.0 * sigma)
-    hi = max(14.0 * sigma, float(np.max(-A, initial=0.0)) + 14.0 * sigma)
+    # The expectation runs over the whole real line; below cutoff - l_claimed the claimed token is filtered out
+    # and the integrand is zero.  Outside +-38 sigma (and 38 sigma past the largest -A) the weight of
+    # x ~ N(0, sigma^2) is below 1e-313, the smallest magnitudes fp64 still represents.
+    lo = max(cutoff - logits[claimed], -38.0 * sigma)
+    hi = max(38.0 * sigma, float(np.max(-A, initial=0.0)) + 38.0 * sigma)
     if lo >= hi:
         return 0.0
     kinks = [float(b - a) for a, b in zip(A, B) if np.isfinite(b) and lo < b - a < hi]
     # break the range where the integrand peaks as well: the peak is narrow (about sigma) in a wide range
-    grid = np.linspace(lo, hi, 2001)
+    grid = np.linspace(lo, hi, 6001)
     peak = float(grid[int(np.argmax([integrand(x) for x in grid]))])
     pts = sorted(set(kinks + [p for p in (peak - sigma, peak, peak + sigma) if lo < p < hi]))
     val, _ = quad(integrand, lo, hi, points=pts or None, epsabs=1e-18, epsrel=1e-11, limit=400)
