@@ -209,9 +209,15 @@ def kernel_source_digest():
     import hashlib
 
     hsh = hashlib.sha256()
-    for name in ("k1_fused_score.cu", "difr_device.cuh", "difr_plan.h", "difr_kernels.h"):
-        with open(os.path.join(ROOT, "paper_2511_02620_b200", "csrc", name), "rb") as f:
+    csrc = os.path.join(ROOT, "paper_2511_02620_b200", "csrc")
+    for name in ("k1_fused_score.cu", "difr_device.cuh", "difr_plan.h"):
+        with open(os.path.join(csrc, name), "rb") as f:
             hsh.update(f.read())
+    # of the shared header only the fused kernel's own parameter block
+    with open(os.path.join(csrc, "difr_kernels.h"), "rb") as f:
+        text = f.read()
+    start = text.index(b"struct K1Params")
+    hsh.update(text[start:text.index(b"};", start)])
     return hsh.hexdigest()[:16]
 
 
