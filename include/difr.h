@@ -238,9 +238,11 @@ difr_status difr_score_both(const void* h, const void* W, const int32_t* tokens,
  *   nucleus over the whole vocabulary is resolved exactly by a selection over the rows' logits, which are
  *   written out a block of rows at a time (about 1 GiB of the workspace) by the tensor-core main loop: one
  *   more pass over the logits plus the selection (a dozen walks over each row, from L2).  Per-row policies
- *   (the *_rows arrays) are resolved among each row's 128 largest logits: a row's top_k must be <= 128 (or
- *   >= V), and a row whose whole-vocabulary nucleus holds more than 128 ids gets row_status bit 4 and the
- *   128th largest logit as cutoff.
+ *   (the *_rows arrays) are by default resolved among each row's 128 largest logits: a row's top_k must be
+ *   <= 128 (or >= V), and a row whose whole-vocabulary nucleus holds more than 128 ids gets row_status
+ *   bit 4 and the 128th largest logit as cutoff.  The host cannot see the rows' values, so the caller says
+ *   when they may go beyond that: filter->any_size != 0 sends every row of a per-row call through the
+ *   selection (same cost as above, same results where both paths apply).
  *   filter->s      1..8
  *   filter->min_p  in [0, 1]; 0: none.  min-p (Sec. "Sampling From Large Language Models") keeps the ids whose
  *                  probability is at least min_p times the largest one, i.e. whose logit reaches
@@ -274,6 +276,9 @@ typedef struct {
   /* -- members added in version 220; zero them when unused -- */
   float min_p;               /* in [0, 1]; 0: no min-p filter                                               */
   const float* min_p_rows;   /* device [T], optional: one min_p per row (min_p is then ignored)            */
+  /* -- member added in version 221; zero it when unused -- */
+  int32_t any_size;          /* with *_rows arrays: non-zero resolves every row by the selection over its   */
+                             /* logits (no limit of 128 ids); ignored when there is one policy for the call */
 } difr_filter;
 size_t difr_filtered_workspace_bytes(int64_t T, int64_t d, int64_t V);
 difr_status difr_score_gm_filtered(const void* h, const void* W, const int32_t* tokens, const uint64_t* seeds,

@@ -48,7 +48,7 @@ class _COut(ctypes.Structure):
 class _CFilter(ctypes.Structure):
     _fields_ = [("top_k", ctypes.c_int32), ("top_p", ctypes.c_float), ("s", ctypes.c_int32),
                 ("top_k_rows", ctypes.c_void_p), ("top_p_rows", ctypes.c_void_p),
-                ("min_p", ctypes.c_float), ("min_p_rows", ctypes.c_void_p)]
+                ("min_p", ctypes.c_float), ("min_p_rows", ctypes.c_void_p), ("any_size", ctypes.c_int32)]
 
 
 _lib = None
@@ -226,17 +226,18 @@ def difr_filtered_workspace_bytes(T: int, d: int, V: int) -> int:
 
 
 def difr_score_ipt_filtered(h, W, tokens, seeds, positions, temperature, top_k, top_p, out: DifrOut, stream=None,
-                            min_p=0.0):
+                            min_p=0.0, any_size=False):
     """Token-IPT-DiFR on the filtered distribution; workspace as for difr_score_gm_filtered."""
     return difr_score_gm_filtered(h, W, tokens, seeds, positions, temperature, top_k, top_p, 1, out, stream,
-                                  _fn="difr_score_ipt_filtered", min_p=min_p)
+                                  _fn="difr_score_ipt_filtered", min_p=min_p, any_size=any_size)
 
 
 def difr_score_gm_filtered(h, W, tokens, seeds, positions, temperature, top_k, top_p, s, out: DifrOut, stream=None,
-                           _fn="difr_score_gm_filtered", min_p=0.0):
+                           _fn="difr_score_gm_filtered", min_p=0.0, any_size=False):
     """Alg. Token-DiFR in full: top-k / top-p cutoff, B_i terms, s competitors; `out.workspace` must hold
     difr_filtered_workspace_bytes(T, d, V) bytes.  `top_k` (int32) and `top_p` (float32) may be device tensors
-    of T values, one per row (`min_p` likewise), and `out.temperatures` one temperature per row.
+    of T values, one per row (`min_p` likewise), and `out.temperatures` one temperature per row; `any_size`
+    lets such per-row values go beyond 128 kept ids.
     See include/difr.h."""
     import torch
 
@@ -258,7 +259,8 @@ def difr_score_gm_filtered(h, W, tokens, seeds, positions, temperature, top_k, t
     if m_rows is not None:
         _check(m_rows, torch.float32, (T,), "min_p")
     f = _CFilter(0 if k_rows is not None else int(top_k), 1.0 if p_rows is not None else float(top_p), int(s),
-                 _ptr(k_rows), _ptr(p_rows), 0.0 if m_rows is not None else float(min_p), _ptr(m_rows))
+                 _ptr(k_rows), _ptr(p_rows), 0.0 if m_rows is not None else float(min_p), _ptr(m_rows),
+                 1 if any_size else 0)
     rc = getattr(lib(), _fn)(_ptr(h), _ptr(W), _ptr(tokens), _ptr(seeds), _ptr(positions),
                              float(temperature), T, d, V, ctypes.byref(f), ctypes.byref(c), _stream(stream))
     if rc != DIFR_OK:

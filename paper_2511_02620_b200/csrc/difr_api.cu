@@ -411,12 +411,14 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
   size_t count_off, list_off, total, sel_off, logits_off;
   // One policy for the whole call whose kept set can exceed what the candidate lists resolve (a top-k above
   // 128, a nucleus or a min-p set over the whole vocabulary): the kept prefix is found by selection over the
-  // rows' logits, written out a block of rows at a time.  (Per-row policies stay within the lists' reach.)
+  // rows' logits, written out a block of rows at a time.  Per-row policies stay within the lists' reach unless
+  // the caller asks for the selection (any_size), which then resolves every row.
   const bool scalar_policy = !filter->top_k_rows && !filter->top_p_rows && !filter->min_p_rows;
   const bool whole_vocab = top_k < 1 || top_k >= V;
-  const bool select_path = scalar_policy && V > 128 &&
-                           ((!whole_vocab && top_k > 128) || (whole_vocab && top_p < 1.f) ||
-                            (ipt && whole_vocab && min_p > 0.f));
+  const bool select_path =
+      V > 128 && (scalar_policy ? ((!whole_vocab && top_k > 128) || (whole_vocab && top_p < 1.f) ||
+                                   (ipt && whole_vocab && min_p > 0.f))
+                                : filter->any_size != 0);
   // the largest number of ids any row resolves by logit rank (a nucleus without a top-k resolves 128)
   int k_max = 128;
   if (select_path) {
@@ -511,6 +513,8 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
       sp.tokens = tokens; sp.temperatures = out->temperatures; sp.temperature = temperature;
       sp.top_k = top_k; sp.top_p = top_p;
       sp.min_p = ipt ? min_p : 0.f;  // Token-DiFR takes the min-p bound itself as cutoff (exact l_max, below)
+      sp.top_k_rows = filter->top_k_rows; sp.top_p_rows = filter->top_p_rows;
+      sp.min_p_rows = ipt ? filter->min_p_rows : nullptr;
       sp.cut_id = sel_cut; sp.top_id = sel_top; sp.kept_n = sel_n;
       sp.kept_z = sel_z; sp.kept_below = sel_below; sp.kept_mine = sel_mine;
       sp.row_status = out->row_status;
@@ -703,6 +707,6 @@ const char* difr_status_string(difr_status status) {
   return "unknown status";
 }
 
-int difr_version(void) { return 220; }
+int difr_version(void) { return 221; }
 
 }  // extern "C"

@@ -176,6 +176,9 @@ struct SelectParams {
   int top_k;      // 0 or >= V: none
   float top_p;    // 1: none
   float min_p;    // 0: none
+  const int32_t* top_k_rows;  // [T], nullable: one value per row in place of the scalar; a value outside its
+  const float* top_p_rows;    //      range acts as "none" here (the finalize kernels mark such a row)
+  const float* min_p_rows;
   int* cut_id;    // [T] out: the last kept id in the order (logit descending, id ascending)
   int* top_id;    // [T] out: the id of the largest logit (lowest id among equals)
   int* kept_n;    // [T] out: how many ids are kept; negated when the min-p bound ended the prefix

@@ -77,7 +77,7 @@ __device__ __forceinline__ RowPolicy row_policy(const FilterParams& p, int row) 
   r.bad = !(r.temperature > 0.f) || isinf(r.temperature) || k < 0 || !(r.top_p > 0.f) || !(r.top_p <= 1.f) ||
           !(r.min_p >= 0.f) || !(r.min_p <= 1.f);
   if (k > p.V) k = p.V;
-  const bool selected = p.sel_cut_id != nullptr;  // one policy for the call, resolved by the selection kernel
+  const bool selected = p.sel_cut_id != nullptr;  // every row's kept prefix was resolved by the selection kernel
   if (k > kMaxK && k < p.V && !selected) r.bad = true;
   const bool whole = k < 1 || k >= p.V;  // no top-k in effect
   r.nucleus_full = (whole && r.top_p < 1.f) ? 1 : 0;
@@ -595,7 +595,9 @@ __global__ void __launch_bounds__(kFWarps * 32) ipt_select_finalize(const Filter
   const int cid = p.sel_cut_id[row], top = p.sel_top_id[row];
   const bool by_min_p = p.sel_kept_n[row] < 0;  // the min-p bound, not the rank filter, ended the kept prefix
   double cutoff = -CUDART_INF;
-  if (by_min_p && top >= 0 && top < p.V)
+  if (rp.none) {
+    // (a row of a per-row call that filters nothing: the selection kept every id)
+  } else if (by_min_p && top >= 0 && top < p.V)
     cutoff = warp_dot(hrow, p.W + (size_t)top * (size_t)p.d, p.d, lane) + (double)rp.temperature * log((double)rp.min_p);
   else if (cid >= 0 && cid < p.V)
     cutoff = warp_dot(hrow, p.W + (size_t)cid * (size_t)p.d, p.d, lane);

@@ -220,13 +220,19 @@ __global__ void __launch_bounds__(kSelThreads) select_cutoff(const SelectParams 
   const bool usable = temp > 0.f && !isinf(temp);
   if (!usable) temp = 1.f;  // (the finalize kernels mark such a row; keep the arithmetic finite here)
   const float c1 = 1.4426950408889634f / temp;
+  int top_k = p.top_k_rows != nullptr ? p.top_k_rows[row] : p.top_k;
+  float top_p = p.top_p_rows != nullptr ? p.top_p_rows[row] : p.top_p;
+  float min_p = p.min_p_rows != nullptr ? p.min_p_rows[row] : p.min_p;
+  if (top_k < 0) top_k = 0;
+  if (!(top_p > 0.f) || !(top_p <= 1.f)) top_p = 1.f;
+  if (!(min_p >= 0.f) || !(min_p <= 1.f)) min_p = 0.f;
 
   float lm = -CUDART_INF_F;
   for (int v = threadIdx.x; v < V; v += kSelThreads) lm = fmaxf(lm, lrow[v]);
   const float lmax = block_max(lm, sh);
 
   // level-0 histogram (count and mass per 1/64 of l_max - l), total mass, and how many ids reach the min-p bound
-  const float bound = p.min_p > 0.f ? lmax + temp * logf(p.min_p) : -CUDART_INF_F;
+  const float bound = min_p > 0.f ? lmax + temp * logf(min_p) : -CUDART_INF_F;
   for (int b = threadIdx.x; b < kSelBins; b += kSelThreads) { sh.cnt0[b] = 0; sh.mass0[b] = 0; }
   __syncthreads();
   unsigned long long tm = 0, tb = 0;
@@ -242,7 +248,7 @@ __global__ void __launch_bounds__(kSelThreads) select_cutoff(const SelectParams 
   const unsigned long long m_total = block_sum(tm, sh);
   const unsigned int n_minp = (unsigned int)block_sum(tb, sh);
 
-  const unsigned int k_eff = (p.top_k >= 1 && p.top_k < V) ? (unsigned int)p.top_k : (unsigned int)V;
+  const unsigned int k_eff = (top_k >= 1 && top_k < V) ? (unsigned int)top_k : (unsigned int)V;
   unsigned int n_keep = k_eff;
   Selected last;       // the selection whose position is N - 1, when one of them is
   bool have_last = false;
@@ -255,9 +261,9 @@ __global__ void __launch_bounds__(kSelThreads) select_cutoff(const SelectParams 
     m_topk = sk.m_gt + (unsigned long long)(k_eff - sk.c_gt) * e;
     last = sk; have_last = true; last_pos = k_eff - 1;
   }
-  if (p.top_p < 1.f) {
+  if (top_p < 1.f) {
     // the shortest prefix whose mass reaches top_p of the mass the top-k keeps
-    const double want = (double)p.top_p * (double)m_topk;
+    const double want = (double)top_p * (double)m_topk;
     unsigned long long target = (unsigned long long)want;
     if ((double)target < want) ++target;
     if (target < 1ull) target = 1ull;

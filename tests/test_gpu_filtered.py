@@ -423,7 +423,7 @@ def _cutoff_agrees(l_row, temperature, top_k, top_p, min_p, got_cut, want_cut, t
     """The kernel's cutoff is the oracle's, or the logit at a neighbouring position of the sorted row where the
     nucleus decision "does this prefix hold top_p of the mass" lies within tol_mass of a tie (the kernel sums
     masses of fp32 logits).  Returns (acceptable, identical)."""
-    if abs(got_cut - want_cut) <= 1e-5 or (np.isneginf(got_cut) and np.isneginf(want_cut)):
+    if (np.isneginf(got_cut) and np.isneginf(want_cut)) or abs(got_cut - want_cut) <= 1e-5:
         return True, True
     if not top_p < 1.0:
         return False, False
@@ -553,3 +553,78 @@ def test_filters_of_any_size_at_full_size_on_sampled_rows():
         assert np.all(out.row_status.cpu().numpy() & (4 | 8 | 16) == 0)
         assert np.all(np.isfinite(got)) and np.all(got <= 1e-6)
         assert np.all(np.isfinite(got_cut))
+
+
+def test_per_row_policies_of_any_size():
+    """Requests with their own sampling parameters in one batch, some of them beyond the candidate lists' reach
+    (a top-k of 700, a whole-vocabulary nucleus, min-p for the IPT estimator), some within it, some without a
+    filter: with `any_size` every row is resolved by the selection and matches the oracle run on the rows of each
+    policy by themselves."""
+    T, d, V = 60, 64, 9000
+    h, W, seeds, positions = _small(T, d, V, 131, 2.0)
+    # (top_k, top_p, min_p, temperature)
+    policies = [(700, 1.0, 0.0, 1.0), (0, 0.93, 0.0, 1.0), (40, 0.9, 0.0, 0.8), (0, 1.0, 0.0, 0.8),
+                (1500, 0.95, 0.02, 1.0), (V, 1.0, 0.0, 1.0)]
+    which = np.arange(T) % len(policies)
+    k_rows = np.array([policies[w][0] for w in which], dtype=np.int32)
+    p_rows = np.array([policies[w][1] for w in which], dtype=np.float32)
+    m_rows = np.array([policies[w][2] for w in which], dtype=np.float32)
+    t_rows = np.array([policies[w][3] for w in which], dtype=np.float32)
+    dev = Device(h, W, seeds, positions)
+    L = oracle.logits(h, W)
+    sigma, s = 0.3, 3
+
+    def call(fn, tokens, sig, s_arg=None):
+        out = difr.DifrOut.allocate(T, d, V, sig, EPS)
+        out.workspace = torch.empty(difr.difr_filtered_workspace_bytes(T, d, V), dtype=torch.uint8, device="cuda")
+        out.cutoff = torch.full((T,), float("nan"), dtype=torch.float32, device="cuda")
+        out.temperatures = to_dev(t_rows)
+        args = (dev.h, dev.W, to_dev(tokens), dev.seeds, dev.positions, 1.0, to_dev(k_rows), to_dev(p_rows))
+        if s_arg is None:
+            fn(*args, out, min_p=to_dev(m_rows), any_size=True)
+        else:
+            fn(*args, s_arg, out, min_p=to_dev(m_rows), any_size=True)
+        torch.cuda.synchronize()
+        assert int(out.device_status.item()) == 0
+        return out
+
+    # Token-DiFR
+    tokens = np.empty(T, dtype=np.int32)
+    for w, (k, p, m, t) in enumerate(policies):
+        rows = np.nonzero(which == w)[0]
+        tokens[rows] = _claims(h[rows], W, seeds[rows], positions[rows], f32(t), 140 + w)
+    out = call(difr.difr_score_gm_filtered, tokens, sigma, s)
+    got, got_cut = out.score.cpu().numpy(), out.cutoff.cpu().numpy().astype(np.float64)
+    assert np.all(out.row_status.cpu().numpy() & (4 | 8 | 16) == 0)
+    for w, (k, p, m, t) in enumerate(policies):
+        rows = np.nonzero(which == w)[0]
+        want, _, cut = filtered.score_gm_filtered(h[rows], W, tokens[rows], seeds[rows], positions[rows], f32(t),
+                                                  f32(sigma), f32(EPS), k, f32(p), s, f32(m))
+        for j, r in enumerate(rows):
+            bar = L[r].max() + f32(t) * math.log(f32(m)) if m > 0 else -np.inf
+            if m > 0 and np.isclose(cut[j], bar, atol=1e-9):
+                assert abs(got_cut[r] - cut[j]) <= 1e-5
+            else:
+                assert _cutoff_agrees(L[r], f32(t), k, f32(p), f32(m), got_cut[r], cut[j])[0], (w, r)
+        np.testing.assert_allclose(got[rows], want, rtol=0, atol=SCORE_TOL, err_msg=f"policy {w}")
+
+    # Token-IPT-DiFR on the rows' filtered distributions
+    mu = np.array([oracle.ipt_uniform(int(sd), int(ps)) for sd, ps in zip(seeds, positions)])
+    tok2 = np.array([filtered.ipt_sample_filtered(L[r], f32(t_rows[r]), int(k_rows[r]), f32(p_rows[r]), mu[r],
+                                                  f32(m_rows[r])) for r in range(T)], dtype=np.int32)
+    tok2[np.arange(T) % 7 == 2] = np.argsort(-L, axis=1)[np.arange(T) % 7 == 2, 1]
+    o2 = call(difr.difr_score_ipt_filtered, tok2, 0.1)
+    assert np.all(o2.row_status.cpu().numpy() & (8 | 16) == 0)
+    cut_ipt = o2.cutoff.cpu().numpy().astype(np.float64)
+    n_same = 0
+    for w, (k, p, m, t) in enumerate(policies):
+        rows = np.nonzero(which == w)[0]
+        want2, pt, a, _, cut2 = filtered.score_ipt_filtered(h[rows], W, tok2[rows], seeds[rows], positions[rows],
+                                                            f32(t), f32(0.1), f32(EPS), k, f32(p), f32(m))
+        same = np.isclose(cut_ipt[rows], cut2, rtol=0, atol=1e-5) | (np.isneginf(cut_ipt[rows]) & np.isneginf(cut2))
+        n_same += int(same.sum())
+        np.testing.assert_allclose(o2.score.cpu().numpy()[rows][same], want2[same], rtol=0, atol=SCORE_TOL,
+                                   err_msg=f"policy {w}")
+        np.testing.assert_allclose(o2.p_claimed.cpu().numpy()[rows][same], pt[same], rtol=2e-4, atol=1e-9)
+        np.testing.assert_allclose(o2.cdf_lo.cpu().numpy()[rows][same], a[same], rtol=0, atol=2e-5)
+    assert n_same > 0.8 * T
