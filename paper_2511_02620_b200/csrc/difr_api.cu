@@ -517,6 +517,7 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
       sp.min_p_rows = ipt ? filter->min_p_rows : nullptr;
       sp.cut_id = sel_cut; sp.top_id = sel_top; sp.kept_n = sel_n;
       sp.kept_z = sel_z; sp.kept_below = sel_below; sp.kept_mine = sel_mine;
+      sp.want_sums = ipt;
       sp.row_status = out->row_status;
       if (launch_select_cutoff(sp, s) != cudaSuccess) return DIFR_ERR_CUDA;
     }

@@ -182,6 +182,7 @@ struct SelectParams {
   int* cut_id;    // [T] out: the last kept id in the order (logit descending, id ascending)
   int* top_id;    // [T] out: the id of the largest logit (lowest id among equals)
   int* kept_n;    // [T] out: how many ids are kept; negated when the min-p bound ended the prefix
+  int want_sums;       // non-zero: also sum the kept ids' masses (one more walk over the row)
   double* kept_z;      // [T] out: mass of the kept ids, of those below the claimed id, of the claimed id if kept,
   double* kept_below;  //         all in units of 2^-40 of the row's largest term
   double* kept_mine;

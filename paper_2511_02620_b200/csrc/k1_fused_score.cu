@@ -771,9 +771,17 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
             if (MODE == kModeDump) {
               if (valid) {
                 float* dst = p.logits_out + (size_t)row * (size_t)p.V + base;
+                if ((p.V & 3) == 0 && (reinterpret_cast<unsigned long long>(p.logits_out) & 15ull) == 0ull &&
+                    base + kSub <= p.V) {
+                  // (rows start on 16-byte boundaries: four 16-byte stores, 64 contiguous bytes per thread)
 #pragma unroll
-                for (int j = 0; j < kSub; ++j)
-                  if (base + j < p.V) dst[j] = __uint_as_float(cur[j]);
+                  for (int j = 0; j < kSub; j += 4)
+                    *reinterpret_cast<uint4*>(dst + j) = make_uint4(cur[j], cur[j + 1], cur[j + 2], cur[j + 3]);
+                } else {
+#pragma unroll
+                  for (int j = 0; j < kSub; ++j)
+                    if (base + j < p.V) dst[j] = __uint_as_float(cur[j]);
+                }
               }
             } else {
               process16<MODE>(cur, base, p.V, tok, c1, neg_tl2, rn, st, cand_list, cand_count, p.cand_cap, band_list,

@@ -11,7 +11,8 @@
 // term), so sums do not depend on the order of the additions and the result is the same on every run.  One
 // walk over the row builds a histogram in bins of 1/64 of (l_max - l); each selection then scans it, gathers
 // the ids of one bin and pins the exact value by radix rounds over their key bits.  The row (V floats) is
-// walked about seven times; after the first walk it is in L2.
+// walked three times (maximum, histogram, one gather per selection) with 16-byte loads, and once more for the
+// sums over the kept ids when the IPT estimator asks for them.
 #include <cuda_runtime.h>
 #include <math_constants.h>
 
@@ -31,6 +32,27 @@ __device__ __forceinline__ uint32_t desc_key(float l) {
 
 constexpr int kSelListCap = 2048;
 
+// f(v, row[v]) for every id of the row, the CTA's threads taking turns; 16-byte loads where the row allows.
+template <class F>
+__device__ __forceinline__ void walk_row(const float* row, int V, F f) {
+  if ((reinterpret_cast<unsigned long long>(row) & 15ull) == 0ull) {
+    const int n4 = V >> 2;
+    const float4* r4 = reinterpret_cast<const float4*>(row);
+    for (int i = threadIdx.x; i < n4; i += kSelThreads) {
+      const float4 q = r4[i];
+      f(4 * i, q.x); f(4 * i + 1, q.y); f(4 * i + 2, q.z); f(4 * i + 3, q.w);
+    }
+    for (int v = (n4 << 2) + threadIdx.x; v < V; v += kSelThreads) f(v, row[v]);
+  } else {
+    for (int v = threadIdx.x; v < V; v += kSelThreads) f(v, row[v]);
+  }
+}
+
+__device__ __forceinline__ float key_to_logit(uint32_t key) {
+  const uint32_t o = ~key;
+  return __uint_as_float(o ^ ((o >> 31) ? 0x80000000u : 0xFFFFFFFFu));
+}
+
 struct SelShared {
   unsigned int cnt0[kSelBins];         // level 0: bins of 1/64 in (l_max - l), all ids of the row
   unsigned long long mass0[kSelBins];
@@ -38,6 +60,7 @@ struct SelShared {
   unsigned long long mass[kSelBins];
   int list[kSelListCap];               // the ids of that level-0 bin (when they fit)
   unsigned int list_n;
+  unsigned int list_bin;               // the level-0 bin whose ids the list holds (0xFFFFFFFF: none / overflowed)
   unsigned int warp_cnt[kSelThreads / 32];
   unsigned long long warp_mass[kSelThreads / 32];
   unsigned int found_bin;
@@ -143,15 +166,16 @@ __device__ Selected radix_select(const float* row, int V, float lmax, float c1, 
   unsigned long long m_acc = sh.m_before;
   if (threadIdx.x == 0) sh.list_n = 0u;
   __syncthreads();
-  for (int v = threadIdx.x; v < V; v += kSelThreads) {
-    if (level0_bin(row[v], lmax) == bin0) {
+  walk_row(row, V, [&](int v, float l) {
+    if (level0_bin(l, lmax) == bin0) {
       const unsigned int at = atomicAdd(&sh.list_n, 1u);
       if (at < (unsigned int)kSelListCap) sh.list[at] = v;
     }
-  }
+  });
   __syncthreads();
   const unsigned int n_sub = sh.list_n;
   const bool listed = n_sub <= (unsigned int)kSelListCap;  // else: walk the whole row in every round
+  if (threadIdx.x == 0) sh.list_bin = listed ? bin0 : 0xFFFFFFFFu;
   uint32_t prefix = 0;  // the key bits decided so far (high bits)
   int decided = 0;      // how many
   const int shifts[3] = {21, 10, 0};
@@ -227,24 +251,33 @@ __global__ void __launch_bounds__(kSelThreads) select_cutoff(const SelectParams 
   if (!(top_p > 0.f) || !(top_p <= 1.f)) top_p = 1.f;
   if (!(min_p >= 0.f) || !(min_p <= 1.f)) min_p = 0.f;
 
+  // the largest logit and its id (the lowest such id)
   float lm = -CUDART_INF_F;
-  for (int v = threadIdx.x; v < V; v += kSelThreads) lm = fmaxf(lm, lrow[v]);
+  int lm_id = 0x7fffffff;
+  walk_row(lrow, V, [&](int v, float l) {
+    if (l > lm || (l == lm && v < lm_id)) { lm = l; lm_id = v; }
+  });
   const float lmax = block_max(lm, sh);
+  if (threadIdx.x == 0) { sh.found_bin = 0x7fffffffu; sh.list_bin = 0xFFFFFFFFu; }
+  __syncthreads();
+  if (lm == lmax && lm_id != 0x7fffffff) atomicMin(&sh.found_bin, (unsigned int)lm_id);
+  __syncthreads();
+  const int top_id = sh.found_bin == 0x7fffffffu ? -1 : (int)sh.found_bin;
+  __syncthreads();
 
   // level-0 histogram (count and mass per 1/64 of l_max - l), total mass, and how many ids reach the min-p bound
   const float bound = min_p > 0.f ? lmax + temp * logf(min_p) : -CUDART_INF_F;
   for (int b = threadIdx.x; b < kSelBins; b += kSelThreads) { sh.cnt0[b] = 0; sh.mass0[b] = 0; }
   __syncthreads();
   unsigned long long tm = 0, tb = 0;
-  for (int v = threadIdx.x; v < V; v += kSelThreads) {
-    const float l = lrow[v];
+  walk_row(lrow, V, [&](int v, float l) {
     const unsigned long long q = fixed_mass(l, lmax, c1);
     const unsigned int b0 = level0_bin(l, lmax);
     atomicAdd(&sh.cnt0[b0], 1u);
     atomicAdd(&sh.mass0[b0], q);
     tm += q;
     tb += (l >= bound) ? 1u : 0u;
-  }
+  });
   const unsigned long long m_total = block_sum(tm, sh);
   const unsigned int n_minp = (unsigned int)block_sum(tb, sh);
 
@@ -294,11 +327,24 @@ __global__ void __launch_bounds__(kSelThreads) select_cutoff(const SelectParams 
   const unsigned int j = n_keep - 1u - last.c_gt;
   if (threadIdx.x == 0) sh.tie_n = 0u;
   __syncthreads();
-  for (int v = threadIdx.x; v < V; v += kSelThreads) {
-    if (desc_key(lrow[v]) == last.key) {
-      const unsigned int at = atomicAdd(&sh.tie_n, 1u);
-      if (at < (unsigned int)kSelTieCap) sh.tie_ids[at] = v;
+  const float l_last = key_to_logit(last.key);
+  if (sh.list_bin == level0_bin(l_last, lmax)) {
+    // the last selection's list holds every id of the bin the value lies in
+    const unsigned int n_list = sh.list_n;
+    for (unsigned int i = threadIdx.x; i < n_list; i += kSelThreads) {
+      const int v = sh.list[i];
+      if (desc_key(lrow[v]) == last.key) {
+        const unsigned int at = atomicAdd(&sh.tie_n, 1u);
+        if (at < (unsigned int)kSelTieCap) sh.tie_ids[at] = v;
+      }
     }
+  } else {
+    walk_row(lrow, V, [&](int v, float l) {
+      if (desc_key(l) == last.key) {
+        const unsigned int at = atomicAdd(&sh.tie_n, 1u);
+        if (at < (unsigned int)kSelTieCap) sh.tie_ids[at] = v;
+      }
+    });
   }
   __syncthreads();
   const unsigned int n_tie = sh.tie_n < (unsigned int)kSelTieCap ? sh.tie_n : (unsigned int)kSelTieCap;
@@ -315,26 +361,21 @@ __global__ void __launch_bounds__(kSelThreads) select_cutoff(const SelectParams 
   __syncthreads();
 
   // sums over the kept ids (Token-IPT-DiFR on the filtered distribution)
-  const int tok = p.tokens[row];
-  unsigned long long kz = 0, kb = 0, km = 0;
-  for (int v = threadIdx.x; v < V; v += kSelThreads) {
-    const float l = lrow[v];
-    const uint32_t k = desc_key(l);
-    if (k < last.key || (k == last.key && v <= cut_id)) {
-      const unsigned long long q = fixed_mass(l, lmax, c1);
-      kz += q;
-      if (v < tok) kb += q;
-      if (v == tok) km += q;
-    }
+  unsigned long long z = 0, below = 0, mine = 0;
+  if (p.want_sums) {
+    const int tok = p.tokens[row];
+    unsigned long long kz = 0, kb = 0, km = 0;
+    walk_row(lrow, V, [&](int v, float l) {
+      const uint32_t k = desc_key(l);
+      if (k < last.key || (k == last.key && v <= cut_id)) {
+        const unsigned long long q = fixed_mass(l, lmax, c1);
+        kz += q;
+        if (v < tok) kb += q;
+        if (v == tok) km += q;
+      }
+    });
+    z = block_sum(kz, sh); below = block_sum(kb, sh); mine = block_sum(km, sh);
   }
-  const unsigned long long z = block_sum(kz, sh), below = block_sum(kb, sh), mine = block_sum(km, sh);
-  // the id of the largest logit (the lowest such id)
-  if (threadIdx.x == 0) sh.found_bin = 0x7fffffffu;
-  __syncthreads();
-  for (int v = threadIdx.x; v < V; v += kSelThreads)
-    if (lrow[v] == lmax) atomicMin(&sh.found_bin, (unsigned int)v);
-  __syncthreads();
-  const int top_id = sh.found_bin == 0x7fffffffu ? -1 : (int)sh.found_bin;
   if (threadIdx.x == 0) {
     p.cut_id[row] = cut_id;
     p.top_id[row] = top_id;
