@@ -90,6 +90,20 @@ __device__ __forceinline__ unsigned long long fixed_mass(float l, float lmax, fl
   return (unsigned long long)__float2ull_rn(e * 1099511627776.0f);
 }
 
+// slot += q on a 64-bit shared-memory sum, as two 32-bit atomic adds: the low words wrap, and whoever sees the wrap
+// carries one into the high word (integer sums: the result does not depend on the order).  Most terms fit the low
+// word and wrap nothing, so this is one atomic where a 64-bit add would be a compare-and-swap loop.
+__device__ __forceinline__ void add_mass(unsigned long long* slot, unsigned long long q) {
+  unsigned int* w = reinterpret_cast<unsigned int*>(slot);  // (little endian: w[0] low, w[1] high)
+  const unsigned int lo = (unsigned int)q;
+  unsigned int hi = (unsigned int)(q >> 32);
+  if (lo != 0u) {
+    const unsigned int old = atomicAdd(w, lo);
+    hi += (old + lo < old) ? 1u : 0u;
+  }
+  if (hi != 0u) atomicAdd(w + 1, hi);
+}
+
 // Level-0 bin of a logit: monotone in l (larger logits in lower bins, equal logits in one bin), 1/64 wide, the
 // last bin open-ended.
 __device__ __forceinline__ unsigned int level0_bin(float l, float lmax) {
@@ -159,7 +173,7 @@ __device__ void locate(const unsigned int* cnt, const unsigned long long* mass, 
 // list (one walk over the row) and three radix rounds over their key bits (11 + 11 + 10) pin the exact value.
 // Whole CTA.
 __device__ Selected radix_select(const float* row, int V, float lmax, float c1, bool by_mass, unsigned int pos,
-                                 unsigned long long target, SelShared& sh) {
+                                 unsigned long long target, bool need_mass, SelShared& sh) {
   locate(sh.cnt0, sh.mass0, by_mass, pos, target, 0u, 0ull, sh);
   const unsigned int bin0 = sh.found_bin;
   unsigned int c_acc = sh.c_before;
@@ -194,7 +208,7 @@ __device__ Selected radix_select(const float* row, int V, float lmax, float c1, 
       if (decided == 0 || (k >> (32 - decided)) == prefix) {
         const uint32_t bin = (k >> shift) & ((1u << width) - 1u);
         atomicAdd(&sh.cnt[bin], 1u);
-        atomicAdd(&sh.mass[bin], fixed_mass(l, lmax, c1));
+        if (need_mass) add_mass(&sh.mass[bin], fixed_mass(l, lmax, c1));
       }
     }
     __syncthreads();
@@ -269,13 +283,16 @@ __global__ void __launch_bounds__(kSelThreads) select_cutoff(const SelectParams 
   const float bound = min_p > 0.f ? lmax + temp * logf(min_p) : -CUDART_INF_F;
   for (int b = threadIdx.x; b < kSelBins; b += kSelThreads) { sh.cnt0[b] = 0; sh.mass0[b] = 0; }
   __syncthreads();
+  const bool need_mass = top_p < 1.f;  // only the nucleus asks for masses
   unsigned long long tm = 0, tb = 0;
   walk_row(lrow, V, [&](int v, float l) {
-    const unsigned long long q = fixed_mass(l, lmax, c1);
     const unsigned int b0 = level0_bin(l, lmax);
     atomicAdd(&sh.cnt0[b0], 1u);
-    atomicAdd(&sh.mass0[b0], q);
-    tm += q;
+    if (need_mass) {
+      const unsigned long long q = fixed_mass(l, lmax, c1);
+      add_mass(&sh.mass0[b0], q);
+      tm += q;
+    }
     tb += (l >= bound) ? 1u : 0u;
   });
   const unsigned long long m_total = block_sum(tm, sh);
@@ -289,7 +306,7 @@ __global__ void __launch_bounds__(kSelThreads) select_cutoff(const SelectParams 
 
   unsigned long long m_topk = m_total;
   if (k_eff < (unsigned int)V) {
-    const Selected sk = radix_select(lrow, V, lmax, c1, false, k_eff - 1, 0ull, sh);
+    const Selected sk = radix_select(lrow, V, lmax, c1, false, k_eff - 1, 0ull, need_mass, sh);
     const unsigned long long e = sk.ties ? sk.m_tie / sk.ties : 0ull;
     m_topk = sk.m_gt + (unsigned long long)(k_eff - sk.c_gt) * e;
     last = sk; have_last = true; last_pos = k_eff - 1;
@@ -300,7 +317,7 @@ __global__ void __launch_bounds__(kSelThreads) select_cutoff(const SelectParams 
     unsigned long long target = (unsigned long long)want;
     if ((double)target < want) ++target;
     if (target < 1ull) target = 1ull;
-    const Selected sn = radix_select(lrow, V, lmax, c1, true, 0u, target, sh);
+    const Selected sn = radix_select(lrow, V, lmax, c1, true, 0u, target, true, sh);
     const unsigned long long e = sn.ties ? sn.m_tie / sn.ties : 0ull;
     unsigned int in_tie = sn.ties;
     if (e > 0ull && target > sn.m_gt) {
@@ -320,7 +337,7 @@ __global__ void __launch_bounds__(kSelThreads) select_cutoff(const SelectParams 
   if (n_keep < 1u) n_keep = 1u;
   if (n_keep > (unsigned int)V) n_keep = (unsigned int)V;
   if (!have_last || last_pos != n_keep - 1u || !(last.c_gt <= n_keep - 1u && n_keep - 1u < last.c_gt + last.ties)) {
-    last = radix_select(lrow, V, lmax, c1, false, n_keep - 1u, 0ull, sh);
+    last = radix_select(lrow, V, lmax, c1, false, n_keep - 1u, 0ull, false, sh);
   }
 
   // the id at position N - 1: the (N - c_gt)-th lowest id among the elements with that logit
