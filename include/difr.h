@@ -235,9 +235,9 @@ difr_status difr_score_both(const void* h, const void* W, const int32_t* tokens,
  *   filter->top_p  in (0, 1]; 1: no nucleus.  With no top-k in front of it the nucleus is the
  *                  shortest prefix that holds top_p of the whole row's softmax mass.
  *   Filters of any size: with one policy for the whole call (no *_rows arrays), a top_k above 128 or a
- *   nucleus over the whole vocabulary is resolved exactly by a selection over the rows' logits, which are
- *   written out a block of rows at a time (about 1 GiB of the workspace) by the tensor-core main loop: one
- *   more pass over the logits plus the selection (a dozen walks over each row, from L2).  Per-row policies
+ *   nucleus over the whole vocabulary is resolved exactly by a selection over the rows' logits, which the
+ *   first pass then also writes to the workspace (fp32, about 1 GiB: a call with more rows than that holds
+ *   is worked off block by block); the selection walks each row three or four times.  Per-row policies
  *   (the *_rows arrays) are by default resolved among each row's 128 largest logits: a row's top_k must be
  *   <= 128 (or >= V), and a row whose whole-vocabulary nucleus holds more than 128 ids gets row_status
  *   bit 4 and the 128th largest logit as cutoff.  The host cannot see the rows' values, so the caller says

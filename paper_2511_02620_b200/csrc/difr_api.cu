@@ -334,11 +334,13 @@ constexpr int kFilterMinStrips = 64;   // vocabularies with fewer tiles than thi
 constexpr int kFilterMaxStrips = 128;  // the bounds kernel reads at most 128 strips' records per row
 
 // Rows whose logits are written out at a time for filters of any size: about a gibibyte of fp32 logits.
-static int select_chunk_rows(int64_t T_pad, int64_t V) {
+static int64_t select_block_rows(int64_t V) {
   int64_t rows = (((int64_t)1 << 30) / (4 * V)) & ~(int64_t)255;
-  if (rows < 256) rows = 256;
-  if (rows > T_pad) rows = T_pad;
-  return (int)rows;
+  return rows < 256 ? 256 : rows;
+}
+static int select_chunk_rows(int64_t T_pad, int64_t V) {
+  const int64_t rows = select_block_rows(V);
+  return (int)(rows > T_pad ? T_pad : rows);
 }
 
 // Layout behind the ordinary workspace: per-row candidate counters, the candidate lists, and for filters of any
@@ -370,6 +372,19 @@ size_t difr_filtered_workspace_bytes(int64_t T, int64_t d, int64_t V) {
   size_t count_off, list_off, total;
   // sized for the most strips a call can ask for
   if (!filtered_layout(T, d, V, info.pairs, kFilterMaxStrips, &pl, &cap, &count_off, &list_off, &total)) return 0;
+  // a call that selects over the logits works block by block when T exceeds a block: each block is a call of
+  // its own on the same workspace
+  const int64_t block = select_block_rows(V);
+  if (T > block) {
+    size_t t2;
+    if (!filtered_layout(block, d, V, info.pairs, kFilterMaxStrips, &pl, &cap, &count_off, &list_off, &t2)) return 0;
+    if (t2 > total) total = t2;
+    if (T % block != 0) {
+      if (!filtered_layout(T % block, d, V, info.pairs, kFilterMaxStrips, &pl, &cap, &count_off, &list_off, &t2))
+        return 0;
+      if (t2 > total) total = t2;
+    }
+  }
   return total;
 }
 
@@ -419,6 +434,30 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
       V > 128 && (scalar_policy ? ((!whole_vocab && top_k > 128) || (whole_vocab && top_p < 1.f) ||
                                    (ipt && whole_vocab && min_p > 0.f))
                                 : filter->any_size != 0);
+  if (select_path && T > select_block_rows(V)) {
+    // block by block, each a call of its own on the same workspace (stream order keeps them apart): a block's
+    // logits, written by its first pass, are what its selection reads
+    if (!out->workspace || !aligned16(out->workspace) || !aligned16(h) || !aligned16(W)) {
+      return !out->workspace ? DIFR_ERR_WORKSPACE : DIFR_ERR_ALIGN;
+    }
+    if (out->workspace_bytes < difr_filtered_workspace_bytes(T, d, V)) return DIFR_ERR_WORKSPACE;
+    const int64_t block = select_block_rows(V);
+    for (int64_t r0 = 0; r0 < T; r0 += block) {
+      const int64_t rows = T - r0 < block ? T - r0 : block;
+      difr_out o = *out;
+      difr_filter f = *filter;
+      auto shift = [r0](auto*& ptr) { if (ptr != nullptr) ptr += r0; };
+      shift(o.score); shift(o.margin); shift(o.argmax); shift(o.runner_up); shift(o.lse); shift(o.p_claimed);
+      shift(o.cdf_lo); shift(o.u); shift(o.row_status); shift(o.rank); shift(o.y_max); shift(o.y_second);
+      shift(o.score_ipt); shift(o.cutoff); shift(o.temperatures);
+      shift(f.top_k_rows); shift(f.top_p_rows); shift(f.min_p_rows);
+      const difr_status rc = filtered_common(
+          ipt, static_cast<const unsigned char*>(h) + (size_t)r0 * (size_t)d * 2, W, tokens + r0, seeds + r0,
+          positions + r0, temperature, rows, d, V, &f, &o, stream);
+      if (rc != DIFR_OK) return rc;
+    }
+    return DIFR_OK;
+  }
   // the largest number of ids any row resolves by logit rank (a nucleus without a top-k resolves 128)
   int k_max = 128;
   if (select_path) {
@@ -447,7 +486,9 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
   k1.device_status = out->device_status;
   k1.temperatures = out->temperatures;
   if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
+  if (select_path) k1.logits_out = reinterpret_cast<float*>(ws + logits_off);  // for the selection below
   if (launch_k1(ipt ? 8 : 6, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;
+  k1.logits_out = nullptr;
 
   // ---- the ordinary finalize: the unfiltered outputs (and, for a row without a filter, the IPT score)
   K2Params k2;
@@ -485,7 +526,7 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
     fp.p_claimed = out->p_claimed; fp.cdf_lo = out->cdf_lo; fp.u = out->u;
   }
   if (select_path) {
-    // ---- logits of a block of rows (the fused kernel's main loop in its dump mode), then the selection
+    // ---- the selection over the rows' logits (written by the first pass; T fits one block here)
     const size_t ints = ((size_t)pl.T_pad * sizeof(int) + 255) & ~(size_t)255;
     const size_t dbls = ((size_t)pl.T_pad * sizeof(double) + 255) & ~(size_t)255;
     int* sel_cut = reinterpret_cast<int*>(ws + sel_off);
@@ -494,33 +535,19 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
     double* sel_z = reinterpret_cast<double*>(ws + sel_off + 3 * ints);
     double* sel_below = reinterpret_cast<double*>(ws + sel_off + 3 * ints + dbls);
     double* sel_mine = reinterpret_cast<double*>(ws + sel_off + 3 * ints + 2 * dbls);
-    float* logits_buf = reinterpret_cast<float*>(ws + logits_off);
-    const int chunk = select_chunk_rows(pl.T_pad, V);
-    for (int64_t r0 = 0; r0 < T; r0 += chunk) {
-      const int64_t rows = T - r0 < chunk ? T - r0 : chunk;
-      Plan pc;
-      if (!make_plan(rows, d, V, info.pairs, &pc)) return DIFR_ERR_SHAPE;
-      CUtensorMap tmap_hc;
-      const unsigned char* h_chunk = static_cast<const unsigned char*>(h) + (size_t)r0 * (size_t)d * 2;
-      if (!make_tmap(&tmap_hc, h_chunk, rows, d, kBM)) return DIFR_ERR_CUDA;
-      K1Params kd = k1_params(pc, rows, d, V, 1.f, nullptr);  // no counter: units go round robin
-      kd.logits_out = logits_buf;
-      kd.device_status = out->device_status;
-      if (launch_k1(2, tmap_hc, tmap_w, kd, k1_grid(pc, info.pairs), s) != cudaSuccess) return DIFR_ERR_CUDA;
-      SelectParams sp;
-      memset(&sp, 0, sizeof sp);
-      sp.logits = logits_buf; sp.rows = (int)rows; sp.V = (int)V; sp.row0 = (int)r0;
-      sp.tokens = tokens; sp.temperatures = out->temperatures; sp.temperature = temperature;
-      sp.top_k = top_k; sp.top_p = top_p;
-      sp.min_p = ipt ? min_p : 0.f;  // Token-DiFR takes the min-p bound itself as cutoff (exact l_max, below)
-      sp.top_k_rows = filter->top_k_rows; sp.top_p_rows = filter->top_p_rows;
-      sp.min_p_rows = ipt ? filter->min_p_rows : nullptr;
-      sp.cut_id = sel_cut; sp.top_id = sel_top; sp.kept_n = sel_n;
-      sp.kept_z = sel_z; sp.kept_below = sel_below; sp.kept_mine = sel_mine;
-      sp.want_sums = ipt;
-      sp.row_status = out->row_status;
-      if (launch_select_cutoff(sp, s) != cudaSuccess) return DIFR_ERR_CUDA;
-    }
+    SelectParams sp;
+    memset(&sp, 0, sizeof sp);
+    sp.logits = reinterpret_cast<const float*>(ws + logits_off); sp.rows = (int)T; sp.V = (int)V; sp.row0 = 0;
+    sp.tokens = tokens; sp.temperatures = out->temperatures; sp.temperature = temperature;
+    sp.top_k = top_k; sp.top_p = top_p;
+    sp.min_p = ipt ? min_p : 0.f;  // Token-DiFR takes the min-p bound itself as cutoff (exact l_max, below)
+    sp.top_k_rows = filter->top_k_rows; sp.top_p_rows = filter->top_p_rows;
+    sp.min_p_rows = ipt ? filter->min_p_rows : nullptr;
+    sp.cut_id = sel_cut; sp.top_id = sel_top; sp.kept_n = sel_n;
+    sp.kept_z = sel_z; sp.kept_below = sel_below; sp.kept_mine = sel_mine;
+    sp.want_sums = ipt;
+    sp.row_status = out->row_status;
+    if (launch_select_cutoff(sp, s) != cudaSuccess) return DIFR_ERR_CUDA;
     fp.sel_cut_id = sel_cut; fp.sel_top_id = sel_top; fp.sel_kept_n = sel_n;
     fp.sel_z = sel_z; fp.sel_below = sel_below; fp.sel_mine = sel_mine;
     if (ipt) {

@@ -768,7 +768,8 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
             const bool more = (i + 1 < kSubsPerTile) && (col0 + (i + 1) * kSub < p.V);
             if (more) tmem_ld_32x16(t0 + (uint32_t)((i + 1) * kSub), nxt);
             const int base = col0 + i * kSub;
-            if (MODE == kModeDump) {
+            if (MODE == kModeDump || (Mode<MODE>::groupmax && p.logits_out != nullptr)) {
+              // (the filters' first pass also writes the logits when a selection over them follows)
               if (valid) {
                 float* dst = p.logits_out + (size_t)row * (size_t)p.V + base;
                 if ((p.V & 3) == 0 && (reinterpret_cast<unsigned long long>(p.logits_out) & 15ull) == 0ull &&
@@ -783,7 +784,8 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
                     if (base + j < p.V) dst[j] = __uint_as_float(cur[j]);
                 }
               }
-            } else {
+            }
+            if (MODE != kModeDump) {
               process16<MODE>(cur, base, p.V, tok, c1, neg_tl2, rn, st, cand_list, cand_count, p.cand_cap, band_list,
                               band_count, p.band_cap);
             }
