@@ -38,9 +38,19 @@ __device__ __forceinline__ void walk_row(const float* row, int V, F f) {
   if ((reinterpret_cast<unsigned long long>(row) & 15ull) == 0ull) {
     const int n4 = V >> 2;
     const float4* r4 = reinterpret_cast<const float4*>(row);
-    for (int i = threadIdx.x; i < n4; i += kSelThreads) {
-      const float4 q = r4[i];
-      f(4 * i, q.x); f(4 * i + 1, q.y); f(4 * i + 2, q.z); f(4 * i + 3, q.w);
+    // four loads in flight per thread: the walks wait on memory, not on arithmetic
+    for (int i0 = threadIdx.x; i0 < n4; i0 += 4 * kSelThreads) {
+      float4 q[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * kSelThreads;
+        if (i < n4) q[u] = r4[i];
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * kSelThreads;
+        if (i < n4) { f(4 * i, q[u].x); f(4 * i + 1, q[u].y); f(4 * i + 2, q[u].z); f(4 * i + 3, q[u].w); }
+      }
     }
     for (int v = (n4 << 2) + threadIdx.x; v < V; v += kSelThreads) f(v, row[v]);
   } else {
