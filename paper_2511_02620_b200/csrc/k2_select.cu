@@ -257,7 +257,7 @@ __device__ __forceinline__ unsigned long long block_sum(unsigned long long v, Se
   return r;
 }
 
-__global__ void __launch_bounds__(kSelThreads) select_cutoff(const SelectParams p) {
+__global__ void __launch_bounds__(kSelThreads, 3) select_cutoff(const SelectParams p) {
   extern __shared__ __align__(16) unsigned char sel_smem[];
   SelShared& sh = *reinterpret_cast<SelShared*>(sel_smem);
   const int r_local = blockIdx.x;
