@@ -632,6 +632,28 @@ def run_ours(args):
         ipt_ms = a.elapsed_time(b) / n_ipt
         assert int(out.device_status.item()) == 0, "device-side wait timed out"
 
+    # ---- Alg. Token-DiFR in full under a sampling filter (top-k 50, then top-p 0.95, four competitors): two passes
+    #      of the fused kernel per call (context; the headline has no filter)
+    filt_ms = None
+    if world == 1 and temperature > 0:
+        fout = difr.DifrOut.allocate(T, d, V, sigma, 1e-12)
+        fout.workspace = torch.empty(difr.difr_filtered_workspace_bytes(T, d, V), dtype=torch.uint8, device="cuda")
+        n_f = max(1, min(args.steps, 4))
+        difr.difr_score_gm_filtered(prob.h, prob.W, prob.tokens, prob.seeds, prob.pos, temperature, 50, 0.95, 4, fout)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(n_f):
+            difr.difr_score_gm_filtered(prob.h, prob.W, prob.tokens, prob.seeds, prob.pos, temperature, 50, 0.95, 4,
+                                        fout)
+            difr.difr_detect(fout.score, prob.tau, fout.margin, None, 0, prob.seq, prob.flags, prob.stats)
+        b.record()
+        torch.cuda.synchronize()
+        filt_ms = a.elapsed_time(b) / n_f
+        assert int(fout.device_status.item()) == 0, "device-side wait timed out"
+        del fout
+        torch.cuda.empty_cache()
+
     variants = None
     if args.variants and rank == 0:
         variants = time_variants(difr, prob.h, prob.W, prob.tokens, prob.seeds, prob.pos, temperature, sigma, T, d, V)
@@ -685,6 +707,11 @@ def run_ours(args):
             "detect": {"threshold": tau_used, "calibration": "1 % of this batch's untampered rows score below it",
                        "n_flagged": n_flagged, "n_tampered": n_tampered, "n_match": int(stats_np[:, 1].sum())},
         }
+        if filt_ms is not None:
+            line["token_difr_filtered"] = {"value": T / (filt_ms * 1e-3), "unit": UNIT, "ms_per_step": filt_ms,
+                                           "filter": {"top_k": 50, "top_p": 0.95, "s": 4},
+                                           "note": "difr_score_gm_filtered + difr_detect, resident inputs; two "
+                                                   "passes of the fused kernel per call"}
         if ipt_ms is not None:
             line["token_ipt_difr"] = {"value": T / (ipt_ms * 1e-3), "unit": UNIT, "ms_per_step": ipt_ms,
                                       "tflops": flop / (ipt_ms * 1e-3) / 1e12,
