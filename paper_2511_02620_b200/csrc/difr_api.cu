@@ -211,7 +211,9 @@ difr_status score_common(int ipt, const void* h, const void* W, const int32_t* t
   k2.temperatures = out->temperatures;
   k2.sigma_ipt = out->sigma_ipt; k2.score_ipt = out->score_ipt;
   k2.rank = want_rank ? out->rank : nullptr; k2.y_max = out->y_max; k2.y_second = out->y_second;
-  k2.tok_logit_in_records = want_rank ? 0 : 1;  // (the rank mode counts in that word)
+  // (the rank mode counts in that word; the Gumbel-max score does not depend on the softmax sum, so the three
+  // fp64 transcendentals per row of the exchange are spent only where the IPT outputs are asked for)
+  k2.tok_logit_in_records = (want_rank || ipt == 0) ? 0 : 1;
   k2.band_list = k1.band_list; k2.band_count = k1.band_count; k2.band_cap = k1.band_cap;
   if (launch_k2(k2, s) != cudaSuccess) return DIFR_ERR_CUDA;
   return DIFR_OK;

@@ -58,7 +58,7 @@ __device__ __forceinline__ double normal_interval(double za, double zb) {
   return 1.0 - 0.5 * erfc(zb * r) - 0.5 * erfc(-za * r);
 }
 
-__global__ void __launch_bounds__(kK2Warps * 32) k2_finalize(const K2Params p) {
+__global__ void __launch_bounds__(kK2Warps * 32, 4) k2_finalize(const K2Params p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row = blockIdx.x * kK2Warps + warp;
   if (row >= p.T) return;  // whole warps leave together
