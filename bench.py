@@ -632,8 +632,8 @@ def run_ours(args):
         ipt_ms = a.elapsed_time(b) / n_ipt
         assert int(out.device_status.item()) == 0, "device-side wait timed out"
 
-    # ---- Alg. Token-DiFR in full under a sampling filter (top-k 50, then top-p 0.95, four competitors): two passes
-    #      of the fused kernel per call (context; the headline has no filter)
+    # ---- Alg. Token-DiFR in full under a sampling filter (top-k 50, then top-p 0.95, four competitors): the fused
+    #      kernel, storing the logits too, and a collecting pass over them (context; the headline has no filter)
     filt_ms = None
     if world == 1 and temperature > 0:
         fout = difr.DifrOut.allocate(T, d, V, sigma, 1e-12)
@@ -710,8 +710,9 @@ def run_ours(args):
         if filt_ms is not None:
             line["token_difr_filtered"] = {"value": T / (filt_ms * 1e-3), "unit": UNIT, "ms_per_step": filt_ms,
                                            "filter": {"top_k": 50, "top_p": 0.95, "s": 4},
-                                           "note": "difr_score_gm_filtered + difr_detect, resident inputs; two "
-                                                   "passes of the fused kernel per call"}
+                                           "note": "difr_score_gm_filtered + difr_detect, resident inputs; the fused "
+                                                   "kernel also stores the logits, a second kernel collects the "
+                                                   "candidates from them"}
         if ipt_ms is not None:
             line["token_ipt_difr"] = {"value": T / (ipt_ms * 1e-3), "unit": UNIT, "ms_per_step": ipt_ms,
                                       "tflops": flop / (ipt_ms * 1e-3) / 1e12,

@@ -436,9 +436,9 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
       V > 128 && (scalar_policy ? ((!whole_vocab && top_k > 128) || (whole_vocab && top_p < 1.f) ||
                                    (ipt && whole_vocab && min_p > 0.f))
                                 : filter->any_size != 0);
-  if (select_path && T > select_block_rows(V)) {
+  if (T > select_block_rows(V)) {
     // block by block, each a call of its own on the same workspace (stream order keeps them apart): a block's
-    // logits, written by its first pass, are what its selection reads
+    // logits, written by its first pass, are what its selection and its collecting pass read
     if (!out->workspace || !aligned16(out->workspace) || !aligned16(h) || !aligned16(W)) {
       return !out->workspace ? DIFR_ERR_WORKSPACE : DIFR_ERR_ALIGN;
     }
@@ -488,7 +488,7 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
   k1.device_status = out->device_status;
   k1.temperatures = out->temperatures;
   if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
-  if (select_path) k1.logits_out = reinterpret_cast<float*>(ws + logits_off);  // for the selection below
+  k1.logits_out = reinterpret_cast<float*>(ws + logits_off);  // for the selection and the collecting pass below
   if (launch_k1(ipt ? 8 : 6, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;
   k1.logits_out = nullptr;
 
@@ -560,7 +560,6 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
   }
   if (launch_filter_bounds(fp, s) != cudaSuccess) return DIFR_ERR_CUDA;
   if (cudaMemsetAsync(ws + count_off, 0, (size_t)pl.T_pad * sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
-  if (cudaMemsetAsync(k1.unit_counter, 0, sizeof(int), s) != cudaSuccess) return DIFR_ERR_CUDA;
   if (!ipt && out->rank != nullptr) {
     // the raw-logit rank of the claimed token rides on the collecting pass: claimed logits into the third
     // plane of the bounds, the counts added up in out->rank
@@ -575,7 +574,9 @@ static difr_status filtered_common(int ipt, const void* h, const void* W, const 
   k1.cand_list = ws + list_off;
   k1.cand_count = reinterpret_cast<int*>(ws + count_off);
   k1.cand_cap = cap;
-  if (launch_k1(ipt ? 9 : 7, tmap_h, tmap_w, k1, grid, s) != cudaSuccess) return DIFR_ERR_CUDA;
+  // (the collecting modes' epilogue over the stored logits: no second contraction)
+  if (launch_collect_from_logits(ipt ? 9 : 7, k1, reinterpret_cast<const float*>(ws + logits_off), s) != cudaSuccess)
+    return DIFR_ERR_CUDA;
   if ((ipt ? launch_ipt_filtered_finalize(fp, s) : launch_filtered_finalize(fp, s)) != cudaSuccess)
     return DIFR_ERR_CUDA;
   return DIFR_OK;

@@ -87,7 +87,9 @@ struct K3Params {
 // largest 16-id group maxima (word 7 of the record), 7 collect the ids that reach the row's bounds on y' / l,
 // 8 softmax statistics + group maxima, 9 collect by raw logit only.
 cudaError_t launch_k1(int mode, const CUtensorMap& tmap_h, const CUtensorMap& tmap_w, const K1Params& p, int grid,
-                      cudaStream_t stream);  // grid: number of CTAs, two per pair
+                      cudaStream_t stream);
+// The collecting modes (7, 9) over logits the first pass stored: [T][V] fp32, p as for launch_k1.
+cudaError_t launch_collect_from_logits(int mode, const K1Params& p, const float* logits, cudaStream_t stream);  // grid: number of CTAs, two per pair
 int k1_max_resident_pairs();  // CTA pairs of the fused kernel the current device keeps resident at once
 cudaError_t launch_k2(const K2Params& p, cudaStream_t stream);
 cudaError_t launch_k3(const K3Params& p, cudaStream_t stream);

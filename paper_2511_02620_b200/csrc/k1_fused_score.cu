@@ -848,6 +848,74 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
   if (threadIdx.x == 0 && *abort_flag && p.device_status != nullptr) *p.device_status = kStatusTimeout;
 }
 
+// ------------------------------------------------- the collecting pass over stored logits
+// The filters' second pass without the contraction.  Their first pass left the rows' fp32 logits in memory, bit
+// for bit what the tensor cores produce, so the collecting modes' epilogue can run over them directly: one warp
+// per row and span of columns, each lane taking 16 consecutive ids at a time (a warp reads 2 KB of the row per
+// step), with the same per-row bounds, noise and candidate lists as in the fused kernel.
+constexpr int kCflWarps = 8;
+
+template <int MODE>
+__global__ void __launch_bounds__(kCflWarps * 32) collect_from_logits(const K1Params p, const float* __restrict__ logits,
+                                                                       int span, int spans) {
+  static_assert(Mode<MODE>::collect, "collecting modes only");
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long unit = (long long)blockIdx.x * kCflWarps + warp;
+  const int row = (int)(unit / spans);
+  const int c0 = (int)(unit % spans) * span;
+  if (row >= p.T || c0 >= p.V) return;
+  const int c_end = min(p.V, c0 + span);
+  const int tok = p.tokens[row];
+  RowNoise rn;
+  RowStats st;
+  stats_init(st);
+  if (Mode<MODE>::noise) row_noise_init(rn, p.seeds[row], p.positions[row]);
+#pragma unroll
+  for (int g = 0; g < Mode<MODE>::ncnt; ++g) st.bound[g] = p.bounds[(size_t)g * (size_t)p.T_pad + row];
+  st.bw = p.bounds[(size_t)kBandPlane * (size_t)p.T_pad + row];
+  float c1 = p.c1, neg_tl2 = p.neg_tl2;
+  if (p.temperatures != nullptr) {
+    const float temp = p.temperatures[row];
+    c1 = temp > 0.f ? 1.4426950408889634f / temp : 0.f;
+    neg_tl2 = -temp * 0.6931471805599453f;
+  }
+  Candidate* cand_list = reinterpret_cast<Candidate*>(p.cand_list) + (size_t)row * (size_t)p.cand_cap;
+  int* cand_count = p.cand_count + row;
+  const float* lrow = logits + (size_t)row * (size_t)p.V;
+  const bool vec = (p.V & 3) == 0 && (reinterpret_cast<unsigned long long>(logits) & 15ull) == 0ull;
+  for (int base = c0 + lane * kSub; base < c_end; base += 32 * kSub) {
+    uint32_t cur[kSub];
+    if (vec && base + kSub <= p.V) {
+#pragma unroll
+      for (int j = 0; j < kSub; j += 4) {
+        const uint4 q = *reinterpret_cast<const uint4*>(lrow + base + j);
+        cur[j] = q.x; cur[j + 1] = q.y; cur[j + 2] = q.z; cur[j + 3] = q.w;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < kSub; ++j) cur[j] = base + j < p.V ? __float_as_uint(lrow[base + j]) : 0u;
+    }
+    process16<MODE>(cur, base, p.V, tok, c1, neg_tl2, rn, st, cand_list, cand_count, p.cand_cap, nullptr, nullptr, 0);
+  }
+  if (MODE == kModeCollect && p.rank_out != nullptr && st.cnt[2] != 0)
+    atomicAdd(p.rank_out + row, st.cnt[2]);  // this lane's share of the claimed token's raw-logit rank
+}
+
+cudaError_t launch_collect_from_logits(int mode, const K1Params& p, const float* logits, cudaStream_t stream) {
+  if (p.T <= 0) return cudaSuccess;
+  // spans of a multiple of 512 ids (a warp's step), about eight per row
+  int span = ((p.V + 7) / 8 + 511) & ~511;
+  if (span < 512) span = 512;
+  const int spans = (p.V + span - 1) / span;
+  const long long units = (long long)p.T * spans;
+  const unsigned grid = (unsigned)((units + kCflWarps - 1) / kCflWarps);
+  if (mode == kModeCollect) collect_from_logits<kModeCollect><<<grid, kCflWarps * 32, 0, stream>>>(p, logits, span, spans);
+  else if (mode == kModeCollectLogit)
+    collect_from_logits<kModeCollectLogit><<<grid, kCflWarps * 32, 0, stream>>>(p, logits, span, spans);
+  else return cudaErrorInvalidValue;
+  return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------ launcher
 template <int MODE>
 static cudaError_t launch_mode(const CUtensorMap& th, const CUtensorMap& tw, const K1Params& p, int grid,
@@ -893,9 +961,7 @@ cudaError_t launch_k1(int mode, const CUtensorMap& tmap_h, const CUtensorMap& tm
     case kModeCount1: return launch_mode<kModeCount1>(tmap_h, tmap_w, p, grid, stream);
     case kModeCount4: return launch_mode<kModeCount4>(tmap_h, tmap_w, p, grid, stream);
     case kModeGmFilter: return launch_mode<kModeGmFilter>(tmap_h, tmap_w, p, grid, stream);
-    case kModeCollect: return launch_mode<kModeCollect>(tmap_h, tmap_w, p, grid, stream);
     case kModeIptFilter: return launch_mode<kModeIptFilter>(tmap_h, tmap_w, p, grid, stream);
-    case kModeCollectLogit: return launch_mode<kModeCollectLogit>(tmap_h, tmap_w, p, grid, stream);
   }
   return cudaErrorInvalidValue;
 }
