@@ -23,7 +23,7 @@ struct K1Params {
   void* cand_list;      // collect mode: [T][cand_cap] records {int32 id, float l, float y'}
   int* cand_count;      // collect mode: [T], zeroed before the launch; may end above cand_cap (overflow)
   int cand_cap;
-  Partial* partials;  // [n_slots][T_pad]
+  Partial* partials;  // [T_pad][S]: a row's records side by side (the finalize kernels read them a row at a time)
   float* logits_out;  // dump mode only
   int32_t* device_status;
   int* row_floor;     // Gumbel-max scoring modes, nullable: [T_pad] per-row lower bounds of the second largest key

@@ -98,13 +98,19 @@ inline bool compute_plan(int64_t T, int64_t d, int64_t V, int num_pairs, Plan* o
   p.n_tiles = (int)((V + kBN - 1) / kBN);
   p.k_steps = (int)((d + kBK - 1) / kBK);
   if (num_pairs <= 0) num_pairs = 74;
-  // Measured on B200 (126 MB of L2): DRAM traffic is lowest with about 40 MB of h per raster group
-  // and strips of about eight tiles; larger groups push W out of L2 before its strip is done with it.
+  // Measured on B200 (126 MB of L2): about 40 MB of h per raster group (larger groups push W out of L2 before
+  // its strip is done with it), and strips whose W tiles hold about 12288 k-columns between them (two tiles at
+  // d = 5120, six at d = 2048).  The pairs that share a strip drift apart by up to one unit, so a shorter strip
+  // keeps fewer W tiles waiting in L2 for the last pair (at d = 5120, eight-tile strips re-read W 2.2 times per
+  // group, two-tile strips 1.2 times, and the DRAM power saved shows as clock under the power cap: 3 % at
+  // T = 65536); below that length the hand-over between units and the extra records cost more than they save.
   const double tile_bytes = 2.0 * kPairM * (double)d;  // one 256-row tile of h or of W
   const double group_bytes = (double)(ov.l2_mb > 0 ? ov.l2_mb : 40) * 1048576.0;
   int gm = (int)(group_bytes / tile_bytes);
   if (gm < 4) gm = 4;
-  int len_target = 8;
+  int len_target = (int)((12288 + d / 2) / d);
+  if (len_target < 1) len_target = 1;
+  if (len_target > 8) len_target = 8;
   if (len_target > p.n_tiles) len_target = p.n_tiles;
   // strip count: n_tiles / len_target when there are many rounds of units; otherwise the count near it
   // (or, for small problems, up to one unit per pair) whose on-demand schedule finishes first

@@ -817,7 +817,7 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
           __syncwarp();
           if (lane == 0) mbar_arrive(xch_empty_bar(quarter));
           if (valid) {
-            float4* dst = reinterpret_cast<float4*>(p.partials + (size_t)w.strip * (size_t)p.T_pad + row);
+            float4* dst = reinterpret_cast<float4*>(p.partials + (size_t)row * (size_t)p.S + w.strip);
             record_pack<MODE>(st, dst[0], dst[1]);
             // this strip's second best is a lower bound of the row's: later units of the row skip below it
             if (Mode<MODE>::skip && p.row_floor != nullptr && st.m2 > st.floor)

@@ -119,7 +119,7 @@ __device__ __forceinline__ double min_p_bound_exact(const FilterParams& p, const
 __device__ __forceinline__ double row_mass_relative(const FilterParams& p, int row, int lane, double l0, double c1) {
   double lmax = -CUDART_INF, lsum = 0.0;
   for (int slot = lane; slot < p.n_slots; slot += 32) {
-    const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * (size_t)p.T_pad + row);
+    const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)row * (size_t)p.n_slots + slot);
     const float4 b = src[1];
     const double bm = (double)b.x, bs = (double)fabsf(b.y);  // (the sign bit is the fused kernel's tie mark)
     if (bm == -CUDART_INF) continue;
@@ -195,7 +195,7 @@ __global__ void __launch_bounds__(kFWarps * 32) filter_bounds(const FilterParams
   for (int t = 0; t < 4; ++t) {
     const int slot = lane + 32 * t;
     if (slot < p.n_slots) {
-      const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * (size_t)p.T_pad + row);
+      const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)row * (size_t)p.n_slots + slot);
       const float4 a = src[0], b = src[1];
       if (__float_as_int(a.y) >= 0) yk[2 * t] = a.x;
       if (__float_as_int(a.w) >= 0) yk[2 * t + 1] = a.z;

@@ -72,7 +72,7 @@ __global__ void __launch_bounds__(kK2Warps * 32, 4) k2_finalize(const K2Params p
   acc.larger = 0;
   uint32_t tie_bits = 0u;  // bit j: this lane's record of slot lane + 32 j carries the fused kernel's tie mark
   for (int slot = lane; slot < p.n_slots; slot += 32) {
-    const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * (size_t)p.T_pad + row);
+    const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)row * (size_t)p.n_slots + slot);
     const float4 a = src[0], b = src[1];
     top2_insert(acc, a.x, __float_as_int(a.y));
     top2_insert(acc, a.z, __float_as_int(a.w));
@@ -171,7 +171,7 @@ __global__ void __launch_bounds__(kK2Warps * 32, 4) k2_finalize(const K2Params p
       float4 a = make_float4(-CUDART_INF_F, __int_as_float(-1), -CUDART_INF_F, __int_as_float(-1));
       bool tie_mark = false;
       if (slot < p.n_slots) {
-        const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * (size_t)p.T_pad + row);
+        const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)row * (size_t)p.n_slots + slot);
         a = src[0];
         tie_mark = base < 1024 ? ((tie_bits >> (base >> 5)) & 1u) != 0u : signbit(src[1].y);
       }
@@ -367,7 +367,7 @@ __global__ void __launch_bounds__(kK2Warps * 32) count_finalize(const CountParam
   if (row >= p.T) return;
   int c[4] = {0, 0, 0, 0};
   for (int slot = lane; slot < p.n_slots; slot += 32) {
-    const int4 a = *reinterpret_cast<const int4*>(p.partials + (size_t)slot * (size_t)p.T_pad + row);
+    const int4 a = *reinterpret_cast<const int4*>(p.partials + (size_t)row * (size_t)p.n_slots + slot);
     c[0] += a.x; c[1] += a.y; c[2] += a.z; c[3] += a.w;
   }
 #pragma unroll
