@@ -772,9 +772,16 @@ k1_fused_score(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
               // (the filters' first pass also writes the logits when a selection over them follows)
               if (valid) {
                 float* dst = p.logits_out + (size_t)row * (size_t)p.V + base;
-                if ((p.V & 3) == 0 && (reinterpret_cast<unsigned long long>(p.logits_out) & 15ull) == 0ull &&
+                if ((p.V & 7) == 0 && (reinterpret_cast<unsigned long long>(p.logits_out) & 31ull) == 0ull &&
                     base + kSub <= p.V) {
-                  // (rows start on 16-byte boundaries: four 16-byte stores, 64 contiguous bytes per thread)
+                  // (rows start on 32-byte boundaries and base is a multiple of 16 ids: two 32-byte stores, whole
+                  // sectors, 64 contiguous bytes per thread)
+#pragma unroll
+                  for (int j = 0; j < kSub; j += 8)
+                    st_global_v8(dst + j, cur[j], cur[j + 1], cur[j + 2], cur[j + 3], cur[j + 4], cur[j + 5],
+                                 cur[j + 6], cur[j + 7]);
+                } else if ((p.V & 3) == 0 && (reinterpret_cast<unsigned long long>(p.logits_out) & 15ull) == 0ull &&
+                           base + kSub <= p.V) {
 #pragma unroll
                   for (int j = 0; j < kSub; j += 4)
                     *reinterpret_cast<uint4*>(dst + j) = make_uint4(cur[j], cur[j + 1], cur[j + 2], cur[j + 3]);

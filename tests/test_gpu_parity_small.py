@@ -72,10 +72,13 @@ def test_library_philox_is_bit_exact():
     assert np.array_equal(got, want)
 
 
-@pytest.mark.parametrize("T,d,V", [(256, 512, 4096), (200, 72, 1000), (130, 64, 300)])
-def test_tensor_core_logits_match_fp64(T, d, V):
+# (the stores of the logits are 32, 16 or 4 bytes wide by what V and the output's address allow: every width is met)
+@pytest.mark.parametrize("T,d,V,offset", [(256, 512, 4096, 0), (200, 72, 1000, 0), (130, 64, 300, 0), (90, 64, 301, 0),
+                                          (200, 72, 1000, 4), (200, 72, 1000, 1)])
+def test_tensor_core_logits_match_fp64(T, d, V, offset):
     h, W, _, _ = _small(T, d, V, 2)
-    logits = torch.full((T, V), float("nan"), dtype=torch.float32, device="cuda")
+    flat = torch.full((T * V + 8,), float("nan"), dtype=torch.float32, device="cuda")
+    logits = flat[offset:offset + T * V].view(T, V)  # `offset` floats past an allocation boundary
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     difr.difr_logits(to_bf16(h), to_bf16(W), logits, status)
     torch.cuda.synchronize()
