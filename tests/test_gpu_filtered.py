@@ -628,3 +628,43 @@ def test_per_row_policies_of_any_size():
         np.testing.assert_allclose(o2.p_claimed.cpu().numpy()[rows][same], pt[same], rtol=2e-4, atol=1e-9)
         np.testing.assert_allclose(o2.cdf_lo.cpu().numpy()[rows][same], a[same], rtol=0, atol=2e-5)
     assert n_same > 0.8 * T
+
+
+@pytest.mark.parametrize("any_size", [False, True])
+def test_calls_beyond_a_block_of_stored_logits_equal_their_blocks(any_size):
+    """A filtered call with more rows than the workspace's block of stored logits holds (2048 rows at V = 128256)
+    is worked off block by block: every output equals, bit for bit, what separate calls on the row ranges give
+    (per-row policies, temperatures, the rank and the cutoff all travel with their rows)."""
+    T, d, V = 2048 + 700, 64, 128256
+    g = np.random.default_rng(171)
+    h = torch.from_numpy(g.standard_normal((T, d)).astype(np.float32)).cuda().to(torch.bfloat16)
+    W = torch.from_numpy((g.standard_normal((V, d)) * (2.0 / math.sqrt(d))).astype(np.float32)).cuda().to(torch.bfloat16)
+    tokens = to_dev(g.integers(0, V, size=T).astype(np.int32))
+    seeds = to_dev(g.integers(1, 2**62, size=T).astype(np.int64))
+    positions = to_dev((np.arange(T) % 512 + 1).astype(np.int32))
+    k_rows = to_dev(np.where(np.arange(T) % 3 == 0, 40, 0).astype(np.int32))
+    p_rows = to_dev(np.where(np.arange(T) % 2 == 0, 0.9, 1.0).astype(np.float32))
+    m_rows = to_dev(np.where(np.arange(T) % 5 == 0, 0.01, 0.0).astype(np.float32))
+    t_rows = to_dev(np.where(np.arange(T) % 4 == 0, 0.8, 1.0).astype(np.float32))
+
+    def run(lo, hi):
+        n = hi - lo
+        out = difr.DifrOut.allocate(n, d, V, 0.3, EPS)
+        out.workspace = torch.empty(difr.difr_filtered_workspace_bytes(n, d, V), dtype=torch.uint8, device="cuda")
+        out.cutoff = torch.full((n,), float("nan"), dtype=torch.float32, device="cuda")
+        out.rank = torch.full((n,), -7, dtype=torch.int32, device="cuda")
+        out.temperatures = t_rows[lo:hi].contiguous()
+        difr.difr_score_gm_filtered(h[lo:hi].contiguous(), W, tokens[lo:hi].contiguous(), seeds[lo:hi].contiguous(),
+                                    positions[lo:hi].contiguous(), 1.0, k_rows[lo:hi].contiguous(),
+                                    p_rows[lo:hi].contiguous(), 3, out, min_p=m_rows[lo:hi].contiguous(),
+                                    any_size=any_size)
+        torch.cuda.synchronize()
+        assert int(out.device_status.item()) == 0
+        return out
+
+    whole, first, second = run(0, T), run(0, 2048), run(2048, T)
+    for name in ("score", "cutoff", "margin", "argmax", "runner_up", "lse", "rank", "row_status"):
+        a = getattr(whole, name)
+        b = torch.cat([getattr(first, name), getattr(second, name)])
+        assert torch.equal(a.view(torch.int32), b.view(torch.int32)), name
+    assert torch.isfinite(whole.score).all()
