@@ -236,7 +236,7 @@ difr_status difr_score_both(const void* h, const void* W, const int32_t* tokens,
  *                  shortest prefix that holds top_p of the whole row's softmax mass.
  *   Filters of any size: with one policy for the whole call (no *_rows arrays), a top_k above 128 or a
  *   nucleus over the whole vocabulary is resolved exactly by a selection over the rows' logits, which the
- *   first pass then also writes to the workspace (fp32, about 1 GiB: a call with more rows than that holds
+ *   first pass then also writes to the workspace (fp32, up to 2 GiB: a call with more rows than that holds
  *   is worked off block by block); the selection walks each row three or four times.  Per-row policies
  *   (the *_rows arrays) are by default resolved among each row's 128 largest logits: a row's top_k must be
  *   <= 128 (or >= V), and a row whose whole-vocabulary nucleus holds more than 128 ids gets row_status
@@ -259,7 +259,7 @@ difr_status difr_score_both(const void* h, const void* W, const int32_t* tokens,
  * lse, y_max, y_second, and `rank`, counted during the second pass); `score` holds
  * the full estimator and out->cutoff, if given, the cutoff per row (-inf: no
  * filter).  Two passes over the logits, one contraction: the scoring pass, which
- * also stores the fp32 logits in the workspace (about 1 GiB; a call with more rows
+ * also stores the fp32 logits in the workspace (up to 2 GiB; a call with more rows
  * than that holds is worked off block by block), then a pass over the stored logits that
  * collects, per row, the ids that can be among the s + 2 best or among the top_k
  * logits (6 KB of list per row, or 12 V bytes per row for vocabularies below 16384 ids,

@@ -335,9 +335,10 @@ constexpr int kFilterFloorStrips = 32;
 constexpr int kFilterMinStrips = 64;   // vocabularies with fewer tiles than this list every id instead
 constexpr int kFilterMaxStrips = 128;  // the bounds kernel reads at most 128 strips' records per row
 
-// Rows whose logits are written out at a time for filters of any size: about a gibibyte of fp32 logits.
+// Rows whose logits the filtered calls keep at a time: two gibibytes of fp32 logits (a raster group or so of rows:
+// with fewer rows per block the first pass streams W more often and its launches get short).
 static int64_t select_block_rows(int64_t V) {
-  int64_t rows = (((int64_t)1 << 30) / (4 * V)) & ~(int64_t)255;
+  int64_t rows = (((int64_t)1 << 31) / (4 * V)) & ~(int64_t)255;
   return rows < 256 ? 256 : rows;
 }
 static int select_chunk_rows(int64_t T_pad, int64_t V) {

@@ -632,10 +632,12 @@ def test_per_row_policies_of_any_size():
 
 @pytest.mark.parametrize("any_size", [False, True])
 def test_calls_beyond_a_block_of_stored_logits_equal_their_blocks(any_size):
-    """A filtered call with more rows than the workspace's block of stored logits holds (2048 rows at V = 128256)
-    is worked off block by block: every output equals, bit for bit, what separate calls on the row ranges give
-    (per-row policies, temperatures, the rank and the cutoff all travel with their rows)."""
-    T, d, V = 2048 + 700, 64, 128256
+    """A filtered call with more rows than the workspace's block of stored logits holds (2 GiB: 4096 rows at
+    V = 128256) is worked off block by block: every output equals, bit for bit, what separate calls on the row
+    ranges give (per-row policies, temperatures, the rank and the cutoff all travel with their rows)."""
+    d, V = 64, 128256
+    block = ((2**31) // (4 * V)) & ~255
+    T = block + 700
     g = np.random.default_rng(171)
     h = torch.from_numpy(g.standard_normal((T, d)).astype(np.float32)).cuda().to(torch.bfloat16)
     W = torch.from_numpy((g.standard_normal((V, d)) * (2.0 / math.sqrt(d))).astype(np.float32)).cuda().to(torch.bfloat16)
@@ -662,7 +664,7 @@ def test_calls_beyond_a_block_of_stored_logits_equal_their_blocks(any_size):
         assert int(out.device_status.item()) == 0
         return out
 
-    whole, first, second = run(0, T), run(0, 2048), run(2048, T)
+    whole, first, second = run(0, T), run(0, block), run(block, T)
     for name in ("score", "cutoff", "margin", "argmax", "runner_up", "lse", "rank", "row_status"):
         a = getattr(whole, name)
         b = torch.cat([getattr(first, name), getattr(second, name)])
