@@ -177,6 +177,13 @@ def _check_token_ipt_difr(case):
         ref_flags, ref_stats = oracle.detect(g["score_ipt"][j].astype(np.float64), tau, None, offs)
         assert np.array_equal(flags, ref_flags), f"sigma {sigma}: {np.sum(flags != ref_flags)} decisions differ"
         assert np.array_equal(stats["n_flagged"], ref_stats["n_flagged"])
+    # the narrowest width the header states the tolerance for: the oracle's closed form on its own stored (a, p, u)
+    sigma = float(np.float32(0.01))
+    got = dev.score("ipt", tokens, temperature, sigma, eps)
+    want = np.array([oracle.ipt_score(float(a), float(a + p), float(u), sigma, eps)
+                     for a, p, u in zip(g["cdf_lo"], g["p_claimed"], g["u"])])
+    worst = np.max(np.abs(got["score"][rows] - want))
+    assert worst <= SCORE_TOL, f"sigma {sigma}: max |score - oracle| = {worst} over {n} rows"
 
 
 # case-major order: both estimators of a case run on the same resident inputs
