@@ -419,7 +419,7 @@ def strips_of(difr, w):
 
 
 def roofline_of(difr, w, k1_ms, k2_ms, k3_ms, peaks, n_seq):
-    """Roofline figures of the three kernels from their device times (see the design doc for the byte counts)."""
+    """Roofline figures of the three kernels from their device times and their algorithmic flop / bytes."""
     flop = 2.0 * w.T * w.d * w.V
     achieved = flop / (k1_ms * 1e-3) / 1e12
     traffic, traffic_src = captured_traffic(w)
