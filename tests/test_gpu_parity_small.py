@@ -99,7 +99,8 @@ def test_tiny_workload_gm(temperature, sigma):
     check_gm(dev.score("gm", tokens, temperature, sigma, EPS), ref)
 
 
-@pytest.mark.parametrize("T,d,V", [(300, 200, 1000), (129, 64, 257), (64, 328, 5000), (1, 8, 2)])
+@pytest.mark.parametrize("T,d,V", [(300, 200, 1000), (129, 64, 257), (64, 328, 5000), (1, 8, 2),
+                                   (40, 8192, 3000), (24, 16392, 1500)])  # wide heads: strips of two tiles, of one
 def test_ragged_shapes_gm(T, d, V):
     """Several tiles with ragged tails in T, d (not a multiple of 64) and V (not a multiple of 256 or 32)."""
     h, W, seeds, positions = _small(T, d, V, 3)
